@@ -1,0 +1,138 @@
+"""Pins for the CPU checker's pool / select / compact / decode-evict functions (Algorithm 2):
+library pooling routines, sort-based brute force, and numpy indexing."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import reference as ref
+
+
+def test_max_pool_matches_library_routine():
+    rng = np.random.default_rng(0)
+    s = rng.random(200).astype(np.float32)
+    for kern in (3, 5, 7):
+        lo, hi = 4, 180
+        got = ref.pool(s, lo, hi, "max", kern)
+        want = torch.nn.functional.max_pool1d(torch.from_numpy(s[lo:hi])[None, None], kern, 1, kern // 2)[0, 0].numpy()
+        assert (got[lo:hi] == want).all()
+        assert (got[:lo] == s[:lo]).all() and (got[hi:] == s[hi:]).all()
+
+
+def test_avg_pool_matches_sequential_fp32_adds_and_library():
+    rng = np.random.default_rng(1)
+    s = (rng.random(120) * 1e-3).astype(np.float32)
+    lo, hi, kern = 0, 100, 5
+    got = ref.pool(s, lo, hi, "avg", kern)
+    want = np.empty(hi - lo, np.float32)
+    for p in range(lo, hi):
+        acc = np.float32(0)
+        for t in range(p - 2, p + 3):
+            if lo <= t < hi:
+                acc = np.float32(acc + s[t])
+        want[p - lo] = np.float32(acc / np.float32(kern))
+    assert (got[lo:hi] == want).all()
+    lib = torch.nn.functional.avg_pool1d(torch.from_numpy(s[lo:hi])[None, None], kern, 1, 2,
+                                         count_include_pad=True)[0, 0].numpy()
+    np.testing.assert_allclose(got[lo:hi], lib, rtol=3e-7)
+
+
+def test_pool_none_is_identity():
+    s = np.arange(10, dtype=np.float32)
+    assert (ref.pool(s, 2, 8, "none", 1) == s).all()
+    assert (ref.pool(s, 2, 8, "max", 1) == s).all()
+
+
+def brute_select(s, budget, n_sink, n_recent):
+    N = len(s)
+    lo, hi = n_sink, N - n_recent
+    order = sorted(range(lo, hi), key=lambda p: (-float(s[p]), p))
+    keep = sorted(order[:budget - n_sink - n_recent])
+    return np.array(list(range(n_sink)) + keep + list(range(hi, N)), np.int32)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_select_matches_sort_brute_force_with_ties(seed):
+    rng = np.random.default_rng(seed)
+    N = 300
+    s = rng.integers(0, 12, N).astype(np.float32) / 8     # many exact ties
+    for budget, n_sink, n_recent in [(40, 0, 8), (64, 4, 16), (N, 0, 0), (24, 4, 20), (100, 0, 0)]:
+        got = ref.select(s, budget, n_sink, n_recent, idx_len=budget + 3)
+        want = brute_select(s, budget, n_sink, n_recent)
+        assert (got[:budget] == want).all()
+        assert (got[budget:] == -1).all()
+        assert (np.diff(got[:budget]) > 0).all()
+
+
+def test_select_agrees_with_library_topk_when_scores_are_distinct():
+    rng = np.random.default_rng(9)
+    s = rng.permutation(500).astype(np.float32)
+    got = ref.select(s, 50, 0, 10)
+    top = torch.topk(torch.from_numpy(s[:490]), 40).indices.sort().values.numpy()
+    assert (got[:40] == top).all() and (got[40:] == np.arange(490, 500)).all()
+
+
+def test_select_rejects_bad_budgets():
+    s = np.zeros(10, np.float32)
+    with pytest.raises(ValueError):
+        ref.select(s, 11, 0, 0)
+    with pytest.raises(ValueError):
+        ref.select(s, 3, 2, 2)
+
+
+def test_compact_is_a_row_gather():
+    rng = np.random.default_rng(2)
+    src = rng.integers(0, 65535, (50, 16)).astype(np.uint16)
+    idx = np.array([0, 3, 7, 49], np.int32)
+    assert (ref.compact(src, idx, 4) == src[idx]).all()
+    src32 = rng.standard_normal((50, 8)).astype(np.float32)
+    assert (ref.compact(src32, idx, 3) == src32[idx[:3]]).all()
+
+
+def test_decode_scores_match_a_single_query_prefill_problem():
+    # the live slots, in any slot order, are a W = 1 cache: same scores as the prefill scorer
+    rng = np.random.default_rng(3)
+    G, d, cap, n = 4, 16, 40, 29
+    qg = rng.standard_normal((G, d)).astype(np.float32)
+    kc = rng.standard_normal((cap, d)).astype(np.float32)
+    vc = rng.standard_normal((cap, d)).astype(np.float32)
+    pos = np.full(cap, -1, np.int32)
+    slots = rng.permutation(36)[:n]
+    pos[slots] = rng.permutation(100)[:n]
+    for var in ("V", "K", "VK", "ATTN"):
+        got = ref.decode_scores(qg, kc, vc, pos, 36, var)
+        live = np.sort(slots)
+        want = ref.score(qg[None, :, None, :], kc[live][None, None], vc[live][None, None], want=(var,))[var][0, 0]
+        np.testing.assert_allclose(got[live], want, rtol=1e-12)
+        dead = np.setdiff1d(np.arange(cap), live)
+        assert (got[dead] == 0).all()
+
+
+def test_decode_evict_brute_force():
+    rng = np.random.default_rng(4)
+    for trial in range(20):
+        cap = 30
+        pos = np.full(cap, -1, np.int32)
+        live = rng.permutation(cap)[:22]
+        pos[live] = rng.permutation(60)[:22]
+        s = (rng.integers(0, 4, cap) / 4).astype(np.float32)
+        step_pos, n_sink, n_recent = 60, 4, 10
+        cands = [p for p in range(cap) if pos[p] >= n_sink and pos[p] <= step_pos - n_recent]
+        want = min(cands, key=lambda p: (float(s[p]), -int(pos[p]))) if cands else -1
+        assert ref.decode_evict(s, pos, cap, step_pos, n_sink, n_recent) == want
+
+
+def test_decode_state_keeps_sinks_and_recents_and_respects_budget():
+    rng = np.random.default_rng(5)
+    G, d, n0, budget, n_sink, n_recent = 2, 8, 12, 12, 2, 4
+    st = ref.DecodeState(rng.standard_normal((n0, d)).astype(np.float32),
+                         rng.standard_normal((n0, d)).astype(np.float32), cap=budget + 1)
+    for t in range(30):
+        step_pos = n0 + t
+        st.append(rng.standard_normal(d).astype(np.float32), rng.standard_normal(d).astype(np.float32), step_pos)
+        st.s_acc += st.scores(rng.standard_normal((G, d)).astype(np.float32)).astype(np.float32)
+        st.evict(step_pos, budget, n_sink, n_recent)
+        assert st.live == budget
+        livepos = st.pos[st.pos >= 0]
+        assert len(set(livepos.tolist())) == budget
+        assert set(range(n_sink)) <= set(livepos.tolist())
+        assert set(range(step_pos - n_recent + 1, step_pos + 1)) <= set(livepos.tolist())
