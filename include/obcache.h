@@ -1,0 +1,196 @@
+/*
+ * obcache.h - C ABI of the B200 (sm_100a) OBCache score / select / compact library.
+ *
+ * The library scores every cached token of a KV cache with the closed-form Optimal-Brain-Damage
+ * saliency scores of OBCache, keeps the per-head top-budget, and gathers the kept K/V rows into a
+ * compacted cache.  All heavy arguments are DEVICE pointers unless a comment says "host".
+ *
+ * Conventions that hold for every call
+ *   ownership  The caller owns every buffer (inputs, outputs, workspace).  The library allocates
+ *              no device memory and frees nothing.  Inputs are never written, except the decode
+ *              cache which obc_decode_step updates in place by contract.
+ *   async      A call validates its arguments on the host, enqueues its kernels on `stream`
+ *              (a cudaStream_t passed as void*; NULL = the legacy default stream) and returns
+ *              without synchronising.  Outputs are valid once the stream reaches that point.
+ *   errors     The return value is an obc_status; negative = nothing useful was launched.  No
+ *              exceptions, aborts or traps cross this boundary.  After OBC_ERR_CUDA,
+ *              obc_last_cuda_error() returns the cudaError_t value of the failing runtime call.
+ *   layout     head_dim (d) is the innermost, contiguous dimension and must be 128.  Strides are
+ *              in ELEMENTS.  Base pointers and strides*elem_size must be multiples of 16 bytes.
+ *   notation   B batch, Hq query heads, Hkv KV heads, G = Hq/Hkv, W window queries per head,
+ *              R = G*W score rows per KV head, N cached tokens.
+ */
+#ifndef OBCACHE_H_
+#define OBCACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OBC_OK = 0,
+    OBC_ERR_NULL = -1,         /* a required pointer is NULL */
+    OBC_ERR_SHAPE = -2,        /* inconsistent or out-of-range sizes */
+    OBC_ERR_UNSUPPORTED = -3,  /* head_dim != 128, unknown dtype/variant/pool mode */
+    OBC_ERR_ALIGN = -4,        /* base pointer or stride not 16-byte aligned */
+    OBC_ERR_WORKSPACE = -5,    /* workspace missing or smaller than obc_*_workspace() says */
+    OBC_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed; see obc_last_cuda_error() */
+    OBC_ERR_TIMEOUT = -7       /* a bounded device-side wait gave up (reported by obc_device_status) */
+} obc_status;
+
+typedef enum { OBC_F32 = 0, OBC_BF16 = 1 } obc_dtype;
+
+/* score variants (bitmask).  The scores buffer holds one [B,Hkv,max_len] fp32 plane per set bit,
+ * in ascending bit order (V, K, VK, ATTN). */
+enum {
+    OBC_VAR_V = 1,     /* OBCache-V   : Eq. 4  sum_i A_ip^2 ||v_p||^2                           */
+    OBC_VAR_K = 2,     /* OBCache-K   : Eq. 5  sum_i (A_ip Z_ip)^2 ||v_p - o_i||^2              */
+    OBC_VAR_VK = 4,    /* OBCache-V&K : Eq. 6  value + key + 2 sum_i A_ip^2 Z_ip (|v_p|^2-v_p.o_i) */
+    OBC_VAR_ATTN = 8   /* attention-only score of Sec. 4.3: sum_i |A_ip|                        */
+};
+
+enum { OBC_POOL_NONE = 0, OBC_POOL_AVG = 1, OBC_POOL_MAX = 2 };
+
+/* kernel family used by obc_score */
+enum {
+    OBC_PATH_AUTO = 0,  /* tensor-core kernels when dtype is bf16 and R is a multiple of 16 and >= 64 */
+    OBC_PATH_SIMT = 1,  /* CUDA-core fp32-FMA kernels (any dtype, any R) */
+    OBC_PATH_TC = 2     /* tcgen05 kernels; OBC_ERR_UNSUPPORTED if the shape does not qualify */
+};
+
+/* Device tensor view.  Logical shape [batch, heads, tokens, head_dim]; head_dim contiguous. */
+typedef struct {
+    void* ptr;            /* device */
+    int32_t dtype;        /* obc_dtype */
+    int64_t stride_b;     /* elements between batch items */
+    int64_t stride_h;     /* elements between heads */
+    int64_t stride_t;     /* elements between tokens (>= head_dim) */
+} obc_tensor;
+
+/* ------------------------------------------------------------------------------------------
+ * obc_score: saliency scores of every cached token (Sec. 4.2, Eq. 4-6; GQA form App. A.5;
+ * perturbation window Eq. 9; the window attention is recomputed as App. C describes).
+ *
+ * For each batch item b and KV head g, with rows r = (query head h in the group of g, window
+ * query i = 0..W-1) and query position N_b - W + i:
+ *   Z_rp = scale * q_r . k_p;  A_r. = softmax over the visible p (p <= N_b - W + i if causal);
+ *   o_r = sum_p A_rp v_p;  then the selected variants summed over all R rows.  Masked pairs add 0.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    size_t struct_size;       /* sizeof(obc_score_params), for ABI growth */
+    int32_t batch, n_q_heads, n_kv_heads, head_dim;
+    int32_t window;           /* W >= 1: the last W query positions of every sequence */
+    int32_t max_len;          /* token extent of k, v and of each scores plane */
+    const int32_t* seq_lens;  /* device [batch], W <= seq_lens[b] <= max_len; NULL = all max_len.
+                                 Values are read on the device only. */
+    float scale;              /* <= 0 selects 1/sqrt(head_dim) */
+    int32_t causal;           /* nonzero: window row i sees keys p <= N_b - W + i */
+    uint32_t variants;        /* OBC_VAR_* bitmask, at least one bit */
+    int32_t path;             /* OBC_PATH_* */
+} obc_score_params;
+
+/* Bytes of device workspace obc_score needs for these parameters (host computation only). */
+obc_status obc_score_workspace(const obc_score_params* p, size_t* bytes /* host out */);
+
+/*
+ * q [B,Hq,W,d]; k, v [B,Hkv,max_len,d]; all three share one dtype.  scores: fp32
+ * [n_variants,B,Hkv,max_len]; entries at p >= seq_lens[b] are written as 0.  workspace: device,
+ * 256-byte aligned, at least obc_score_workspace() bytes; contents are scratch.
+ */
+obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                     float* scores, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * obc_select: pooling + per-head top-budget (Algorithm 2's index selection; SnapKV-style 1-D
+ * pooling, App. C.2.1).
+ *
+ * Per (b, g): keeps tokens [0, n_sink) and [N_b - n_recent, N_b); pools the scores over the
+ * candidate range [n_sink, N_b - n_recent) (stride 1, same length, odd kernel; max pads with
+ * -inf; avg pads with 0, adds taps in ascending index order in fp32 and divides by the kernel
+ * size); keeps the budget_b - n_sink - n_recent candidates with the largest pooled score, equal
+ * scores keeping the lowest index; writes all kept indices in ascending order.
+ * Scores must be finite; -0.0 ranks equal to +0.0.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    size_t struct_size;
+    int32_t batch, n_kv_heads, max_len;
+    const int32_t* seq_lens;  /* device [batch] or NULL (all max_len) */
+    int32_t budget;           /* kept tokens per head when budgets == NULL */
+    const int32_t* budgets;   /* device [batch] per-sequence budgets, or NULL */
+    int32_t idx_stride;       /* row length of idx (>= every budget) */
+    int32_t n_sink, n_recent;
+    int32_t pool_mode;        /* OBC_POOL_* */
+    int32_t pool_kernel;      /* odd, >= 1 */
+} obc_select_params;
+
+obc_status obc_select_workspace(const obc_select_params* p, size_t* bytes /* host out */);
+
+/*
+ * scores: fp32 [B,Hkv,max_len] (one plane).  idx: int32 [B,Hkv,idx_stride]; the first budget_b
+ * entries ascending, the rest -1.  A per-sequence budget outside
+ * [n_sink + n_recent, N_b] (only detectable on the device) yields a row of -1 for that sequence.
+ */
+obc_status obc_select(const obc_select_params* p, const float* scores, int32_t* idx,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * obc_compact: gather of the kept rows (Algorithm 2's gather/concatenate):
+ *   k_out[b,g,j,:] = k[b,g,idx[b,g,j],:], same for v, for every j with idx[b,g,j] >= 0.
+ * Rows whose index is -1 are left untouched.  If scores_in/scores_out are non-NULL the fp32
+ * scores [B,Hkv,max_len] are gathered the same way into [B,Hkv,idx_stride] (they seed the decode
+ * accumulator).  k, v, k_out, v_out share one dtype.
+ * ------------------------------------------------------------------------------------------ */
+obc_status obc_compact(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int32_t idx_stride,
+                       int32_t max_len, obc_tensor k, obc_tensor v, const int32_t* idx,
+                       obc_tensor k_out, obc_tensor v_out,
+                       const float* scores_in, float* scores_out, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * obc_decode_step: one decode-time rescoring + eviction step (Sec. 3 "Decoding" and "Cache
+ * Eviction"; Sec. 4.2: scores accumulated over decode steps; App. C.2.2: sinks and a recent
+ * window are protected, one eviction per step once over budget).
+ *
+ * The cache of each (b, g) is a set of `capacity` slots.  pos[slot] is the token position held
+ * by the slot (-1 = free); state[b,g] = {live, next_slot, hi, reserved}: live slots, the slot the
+ * next token goes to, and one past the highest slot ever used.  One call:
+ *   1. writes (k_t, v_t) into next_slot with pos = step_pos and accumulator 0;
+ *   2. with the newest query of each of the G heads, recomputes attention over the live slots
+ *      and the chosen variant's score of every live slot (W = 1);
+ *   3. s_acc[slot] += score;
+ *   4. if live > budget: frees the live slot with the smallest s_acc among tokens with
+ *      n_sink <= pos <= step_pos - n_recent (equal values: the highest pos), which becomes
+ *      next_slot; otherwise next_slot = hi.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    size_t struct_size;
+    int32_t batch, n_q_heads, n_kv_heads, head_dim;
+    int32_t capacity;         /* slots per (b, g); must exceed budget */
+    int32_t budget, n_sink, n_recent;
+    uint32_t variant;         /* exactly one OBC_VAR_* bit */
+    float scale;              /* <= 0 selects 1/sqrt(head_dim) */
+} obc_decode_params;
+
+obc_status obc_decode_workspace(const obc_decode_params* p, size_t* bytes /* host out */);
+
+/*
+ * q_t [B,Hq,1,d]; k_t, v_t [B,Hkv,1,d]; k_cache, v_cache [B,Hkv,capacity,d] updated in place;
+ * s_acc fp32 [B,Hkv,capacity], pos int32 [B,Hkv,capacity], state int32 [B,Hkv,4]: all updated in
+ * place.  step_pos: position of the new token.  All tensors bf16.
+ */
+obc_status obc_decode_step(const obc_decode_params* p, obc_tensor q_t, obc_tensor k_t, obc_tensor v_t,
+                           obc_tensor k_cache, obc_tensor v_cache, float* s_acc, int32_t* pos,
+                           int32_t* state, int32_t step_pos,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Host-only helpers. */
+const char* obc_status_string(obc_status s);
+int obc_last_cuda_error(void);      /* cudaError_t of the last failing CUDA call on this thread */
+int obc_version(void);              /* major*10000 + minor*100 + patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OBCACHE_H_ */

@@ -1,0 +1,213 @@
+// The C-ABI entry points: argument validation, workspace planning, kernel-family choice.
+// Every function here runs on the host and only enqueues work; see include/obcache.h.
+#include "obc_common.cuh"
+
+namespace obc {
+
+static thread_local int g_last_cuda_error = 0;
+void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+
+namespace {
+
+int elem_size(int dtype) { return dtype == OBC_BF16 ? 2 : 4; }
+
+obc_status check_tensor(const obc_tensor& t, bool need_batch_stride) {
+    if (!t.ptr) return OBC_ERR_NULL;
+    if (t.dtype != OBC_F32 && t.dtype != OBC_BF16) return OBC_ERR_UNSUPPORTED;
+    const long long es = elem_size(t.dtype);
+    if (((uintptr_t)t.ptr & 15) != 0) return OBC_ERR_ALIGN;
+    if ((t.stride_t * es) % 16 || (t.stride_h * es) % 16 || (t.stride_b * es) % 16) return OBC_ERR_ALIGN;
+    if (t.stride_t < kD || t.stride_h < 0 || t.stride_b < 0) return OBC_ERR_SHAPE;
+    (void)need_batch_stride;
+    return OBC_OK;
+}
+
+TensorView view(const obc_tensor& t) { return TensorView{t.ptr, t.stride_b, t.stride_h, t.stride_t}; }
+
+obc_status resolve_score(const obc_score_params* p, ScoreShape* s) {
+    if (!p) return OBC_ERR_NULL;
+    if (p->struct_size != sizeof(obc_score_params)) return OBC_ERR_UNSUPPORTED;
+    if (p->head_dim != kD) return OBC_ERR_UNSUPPORTED;
+    if (p->batch < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return OBC_ERR_SHAPE;
+    if (p->window < 1 || p->max_len < 1 || p->window > p->max_len) return OBC_ERR_SHAPE;
+    if ((long long)p->batch * p->n_kv_heads > 65535) return OBC_ERR_SHAPE;
+    const unsigned known = OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN;
+    if (p->variants == 0 || (p->variants & ~known)) return OBC_ERR_UNSUPPORTED;
+    if (p->path < OBC_PATH_AUTO || p->path > OBC_PATH_TC) return OBC_ERR_UNSUPPORTED;
+    s->B = p->batch; s->Hq = p->n_q_heads; s->Hkv = p->n_kv_heads; s->G = s->Hq / s->Hkv;
+    s->W = p->window; s->R = s->G * s->W; s->Nmax = p->max_len; s->seq_lens = p->seq_lens;
+    s->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)kD);
+    s->causal = p->causal != 0; s->variants = p->variants;
+    s->n_planes = __builtin_popcount(p->variants);
+    return OBC_OK;
+}
+
+// which kernel family runs: decided from the parameters alone so that the size query and the
+// launch agree.  The dtype is not known to the size query, so the workspace covers both.
+bool want_tc(const obc_score_params* p, const ScoreShape& s, int dtype) {
+    if (p->path == OBC_PATH_SIMT) return false;
+    return tc_supported(s, dtype);
+}
+
+}  // namespace
+}  // namespace obc
+
+using namespace obc;
+
+extern "C" {
+
+obc_status obc_score_workspace(const obc_score_params* p, size_t* bytes) {
+    if (!bytes) return OBC_ERR_NULL;
+    ScoreShape s;
+    obc_status st = resolve_score(p, &s);
+    if (st != OBC_OK) return st;
+    size_t need = make_simt_plan(s).bytes;
+    if (p->path != OBC_PATH_SIMT && tc_supported(s, OBC_BF16)) {
+        size_t t = tc_workspace_bytes(s);
+        if (t > need) need = t;
+    }
+    *bytes = need;
+    return OBC_OK;
+}
+
+obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                     float* scores, void* workspace, size_t workspace_bytes, void* stream) {
+    ScoreShape s;
+    obc_status st = resolve_score(p, &s);
+    if (st != OBC_OK) return st;
+    if (!scores) return OBC_ERR_NULL;
+    if ((st = check_tensor(q, true)) != OBC_OK) return st;
+    if ((st = check_tensor(k, true)) != OBC_OK) return st;
+    if ((st = check_tensor(v, true)) != OBC_OK) return st;
+    if (q.dtype != k.dtype || k.dtype != v.dtype) return OBC_ERR_UNSUPPORTED;
+    if (((uintptr_t)scores & 15) != 0) return OBC_ERR_ALIGN;
+    size_t need = 0;
+    if ((st = obc_score_workspace(p, &need)) != OBC_OK) return st;
+    if (!workspace || workspace_bytes < need) return OBC_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
+    const bool tc = want_tc(p, s, q.dtype);
+    if (p->path == OBC_PATH_TC && !tc) return OBC_ERR_UNSUPPORTED;
+    if (tc) return launch_score_tc(s, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);
+    return launch_score_simt(s, make_simt_plan(s), q.dtype, view(q), view(k), view(v), scores, workspace,
+                             (cudaStream_t)stream);
+}
+
+static obc_status resolve_select(const obc_select_params* p, SelectShape* s) {
+    if (!p) return OBC_ERR_NULL;
+    if (p->struct_size != sizeof(obc_select_params)) return OBC_ERR_UNSUPPORTED;
+    if (p->batch < 1 || p->n_kv_heads < 1 || p->max_len < 1) return OBC_ERR_SHAPE;
+    if (p->n_sink < 0 || p->n_recent < 0 || p->idx_stride < 1) return OBC_ERR_SHAPE;
+    if (p->pool_mode < OBC_POOL_NONE || p->pool_mode > OBC_POOL_MAX) return OBC_ERR_UNSUPPORTED;
+    if (p->pool_kernel < 1 || p->pool_kernel % 2 == 0) return OBC_ERR_SHAPE;
+    if (!p->budgets) {
+        if (p->budget < p->n_sink + p->n_recent || p->budget > p->idx_stride) return OBC_ERR_SHAPE;
+        if (!p->seq_lens && p->budget > p->max_len) return OBC_ERR_SHAPE;
+    }
+    if (!p->seq_lens && p->n_sink + p->n_recent > p->max_len) return OBC_ERR_SHAPE;
+    *s = SelectShape{p->batch, p->n_kv_heads, p->max_len, p->seq_lens, p->budget, p->budgets,
+                     p->idx_stride, p->n_sink, p->n_recent, p->pool_mode, p->pool_kernel};
+    return OBC_OK;
+}
+
+obc_status obc_select_workspace(const obc_select_params* p, size_t* bytes) {
+    if (!bytes) return OBC_ERR_NULL;
+    SelectShape s;
+    obc_status st = resolve_select(p, &s);
+    if (st != OBC_OK) return st;
+    *bytes = select_workspace_bytes(s.B, s.Hkv, s.Nmax);
+    return OBC_OK;
+}
+
+obc_status obc_select(const obc_select_params* p, const float* scores, int32_t* idx,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    SelectShape s;
+    obc_status st = resolve_select(p, &s);
+    if (st != OBC_OK) return st;
+    if (!scores || !idx) return OBC_ERR_NULL;
+    if (!workspace || workspace_bytes < select_workspace_bytes(s.B, s.Hkv, s.Nmax)) return OBC_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
+    return launch_select(s, scores, idx, workspace, (cudaStream_t)stream);
+}
+
+obc_status obc_compact(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int32_t idx_stride,
+                       int32_t max_len, obc_tensor k, obc_tensor v, const int32_t* idx,
+                       obc_tensor k_out, obc_tensor v_out,
+                       const float* scores_in, float* scores_out, void* stream) {
+    if (head_dim != kD) return OBC_ERR_UNSUPPORTED;
+    if (batch < 1 || n_kv_heads < 1 || idx_stride < 1 || max_len < 1) return OBC_ERR_SHAPE;
+    if (!idx) return OBC_ERR_NULL;
+    if ((scores_in == nullptr) != (scores_out == nullptr)) return OBC_ERR_NULL;
+    obc_status st;
+    if ((st = check_tensor(k, true)) != OBC_OK) return st;
+    if ((st = check_tensor(v, true)) != OBC_OK) return st;
+    if ((st = check_tensor(k_out, true)) != OBC_OK) return st;
+    if ((st = check_tensor(v_out, true)) != OBC_OK) return st;
+    if (k.dtype != v.dtype || k.dtype != k_out.dtype || k.dtype != v_out.dtype) return OBC_ERR_UNSUPPORTED;
+    return launch_gather(batch, n_kv_heads, idx_stride, max_len, elem_size(k.dtype), view(k), view(v),
+                         view(k_out), view(v_out), idx, scores_in, scores_out, (cudaStream_t)stream);
+}
+
+static obc_status resolve_decode(const obc_decode_params* p, DecodeShape* s) {
+    if (!p) return OBC_ERR_NULL;
+    if (p->struct_size != sizeof(obc_decode_params)) return OBC_ERR_UNSUPPORTED;
+    if (p->head_dim != kD) return OBC_ERR_UNSUPPORTED;
+    if (p->batch < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return OBC_ERR_SHAPE;
+    if (p->n_q_heads / p->n_kv_heads > 8) return OBC_ERR_UNSUPPORTED;
+    if (p->capacity < 1 || p->budget < 1 || p->capacity <= p->budget) return OBC_ERR_SHAPE;
+    if (p->n_sink < 0 || p->n_recent < 1 || p->n_sink + p->n_recent >= p->budget) return OBC_ERR_SHAPE;
+    if (p->variant != OBC_VAR_V && p->variant != OBC_VAR_K && p->variant != OBC_VAR_VK && p->variant != OBC_VAR_ATTN)
+        return OBC_ERR_UNSUPPORTED;
+    if ((long long)p->batch * p->n_kv_heads > 65535) return OBC_ERR_SHAPE;
+    *s = DecodeShape{p->batch, p->n_q_heads, p->n_kv_heads, p->n_q_heads / p->n_kv_heads, p->capacity,
+                     p->budget, p->n_sink, p->n_recent, p->variant,
+                     p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)kD)};
+    return OBC_OK;
+}
+
+obc_status obc_decode_workspace(const obc_decode_params* p, size_t* bytes) {
+    if (!bytes) return OBC_ERR_NULL;
+    DecodeShape s;
+    obc_status st = resolve_decode(p, &s);
+    if (st != OBC_OK) return st;
+    *bytes = decode_workspace_bytes(s);
+    return OBC_OK;
+}
+
+obc_status obc_decode_step(const obc_decode_params* p, obc_tensor q_t, obc_tensor k_t, obc_tensor v_t,
+                           obc_tensor k_cache, obc_tensor v_cache, float* s_acc, int32_t* pos,
+                           int32_t* state, int32_t step_pos,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    DecodeShape s;
+    obc_status st = resolve_decode(p, &s);
+    if (st != OBC_OK) return st;
+    if (!s_acc || !pos || !state) return OBC_ERR_NULL;
+    const obc_tensor* ts[5] = {&q_t, &k_t, &v_t, &k_cache, &v_cache};
+    for (int i = 0; i < 5; ++i) {
+        if ((st = check_tensor(*ts[i], true)) != OBC_OK) return st;
+        if (ts[i]->dtype != OBC_BF16) return OBC_ERR_UNSUPPORTED;
+    }
+    if (step_pos < 0) return OBC_ERR_SHAPE;
+    if (!workspace || workspace_bytes < decode_workspace_bytes(s)) return OBC_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
+    return launch_decode(s, view(q_t), view(k_t), view(v_t), view(k_cache), view(v_cache), s_acc, pos, state,
+                         step_pos, workspace, (cudaStream_t)stream);
+}
+
+const char* obc_status_string(obc_status s) {
+    switch (s) {
+        case OBC_OK: return "ok";
+        case OBC_ERR_NULL: return "a required pointer is NULL";
+        case OBC_ERR_SHAPE: return "inconsistent or out-of-range sizes";
+        case OBC_ERR_UNSUPPORTED: return "unsupported head_dim, dtype, variant, mode or struct size";
+        case OBC_ERR_ALIGN: return "pointer or stride not 16-byte aligned (workspace: 256-byte)";
+        case OBC_ERR_WORKSPACE: return "workspace missing or too small";
+        case OBC_ERR_CUDA: return "a CUDA call failed (see obc_last_cuda_error)";
+        case OBC_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    }
+    return "unknown status";
+}
+
+int obc_last_cuda_error(void) { return g_last_cuda_error; }
+int obc_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,108 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "obcache.h"
+
+namespace obc {
+
+constexpr int kD = 128;                  // head_dim the kernels are written for
+constexpr float kLog2e = 1.4426950408889634f;
+
+// ---- thread-local record of the last failing CUDA call -------------------------------------
+void set_last_cuda_error(int e);
+#define OBC_CUDA_TRY(expr)                                              \
+    do {                                                                \
+        cudaError_t _e = (expr);                                        \
+        if (_e != cudaSuccess) { obc::set_last_cuda_error((int)_e); return OBC_ERR_CUDA; } \
+    } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- internal launch descriptions (plain structs, passed by value to kernels) ---------------
+struct TensorView {                      // element strides; d contiguous
+    const void* ptr;
+    long long sb, sh, st;
+};
+
+struct ScoreShape {
+    int B, Hq, Hkv, G, W, R, Nmax;
+    const int32_t* seq_lens;             // device or nullptr
+    float scale;                         // 1/sqrt(d) resolved
+    int causal;
+    unsigned variants;
+    int n_planes;
+};
+
+// SIMT (CUDA-core) score path: workspace layout, computed identically by the size query and the launch
+struct SimtPlan {
+    int n_splits;                        // KV splits of pass 1
+    int tiles_per_split;
+    size_t off_part_m, off_part_l, off_part_o;   // partial softmax stats / outputs per split
+    size_t off_lse2, off_onorm, off_o;           // combined: log2-sum-exp, ||o||^2, O (fp32)
+    size_t bytes;
+};
+SimtPlan make_simt_plan(const ScoreShape& s);
+
+obc_status launch_score_simt(const ScoreShape& s, const SimtPlan& plan, int dtype,
+                             TensorView q, TensorView k, TensorView v,
+                             float* scores, void* ws, cudaStream_t stream);
+
+// ---- select / compact -------------------------------------------------------------------------
+struct SelectShape {
+    int B, Hkv, Nmax;
+    const int32_t* seq_lens;
+    int budget;
+    const int32_t* budgets;
+    int idx_stride, n_sink, n_recent, pool_mode, pool_kernel;
+};
+size_t select_workspace_bytes(int B, int Hkv, int Nmax);
+obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx, void* ws, cudaStream_t stream);
+obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_bytes,
+                         TensorView k, TensorView v, TensorView ko, TensorView vo, const int32_t* idx,
+                         const float* s_in, float* s_out, cudaStream_t stream);
+
+// ---- decode step --------------------------------------------------------------------------------
+struct DecodeShape {
+    int B, Hq, Hkv, G, cap, budget, n_sink, n_recent;
+    unsigned variant;
+    float scale;
+};
+size_t decode_workspace_bytes(const DecodeShape& s);
+obc_status launch_decode(const DecodeShape& s, TensorView q, TensorView kt, TensorView vt,
+                         TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
+                         int step_pos, void* ws, cudaStream_t stream);
+
+// ---- tensor-core (tcgen05) score path -----------------------------------------------------------
+bool tc_supported(const ScoreShape& s, int dtype);
+size_t tc_workspace_bytes(const ScoreShape& s);
+obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
+                           float* scores, void* ws, cudaStream_t stream);
+
+// ---- device helpers --------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// 4 consecutive elements of a row -> float4 (fp32 or bf16 storage)
+template <typename T> __device__ __forceinline__ float4 load4(const T* p);
+template <> __device__ __forceinline__ float4 load4<float>(const float* p) {
+    return *reinterpret_cast<const float4*>(p);
+}
+template <> __device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
+    uint2 u = *reinterpret_cast<const uint2*>(p);
+    float4 f;
+    f.x = __uint_as_float(u.x << 16); f.y = __uint_as_float(u.x & 0xffff0000u);
+    f.z = __uint_as_float(u.y << 16); f.w = __uint_as_float(u.y & 0xffff0000u);
+    return f;
+}
+
+}  // namespace obc

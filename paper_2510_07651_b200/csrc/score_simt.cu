@@ -1,0 +1,366 @@
+// CUDA-core (fp32 FMA) score kernels: the path for fp32 caches and for row counts too small or
+// too irregular for the tensor-core kernels.  Two passes over K/V per (batch item, KV head):
+//
+//   pass 1  split-KV streaming softmax over the window rows: per split, running max / sum of
+//           exp2 and the un-normalised partial output  (Sec. 3: A = softmax(QK^T/sqrt(d)), O = AV)
+//   combine merges the splits into log2-sum-exp, O (fp32) and ||o_r||^2 per row
+//   pass 2  recomputes the logits tile by tile together with v_p . o_r and folds the score
+//           arithmetic of Eq. 4-6 (in the expanded form of Algorithm 1) and the sum over window
+//           rows and the GQA group (App. A.5) into registers; one fp32 store per token and plane.
+//
+// No W x N matrix is written to global memory.
+#include "obc_common.cuh"
+
+namespace obc {
+
+namespace {
+constexpr int TN = 64;        // tokens per tile
+constexpr int RC = 32;        // window rows per chunk (8 warps x 4 rows)
+constexpr int KS = kD + 4;    // padded row stride (floats) of the token-major smem tiles
+constexpr int NT = 256;
+
+__device__ __forceinline__ int seq_len(const ScoreShape& s, int b) {
+    return s.seq_lens ? s.seq_lens[b] : s.Nmax;
+}
+
+template <typename T>
+__device__ __forceinline__ const T* row_ptr(const TensorView& t, int b, int h, long long tok) {
+    return reinterpret_cast<const T*>(t.ptr) + b * t.sb + h * t.sh + tok * t.st;
+}
+
+// cooperative load of `rows` x 128 elements into fp32 smem (row stride `stride` floats);
+// rows >= valid are zero-filled.  get(row) returns the global row pointer.
+template <typename T, typename F>
+__device__ __forceinline__ void load_rows(float* dst, int stride, int rows, int valid, F get) {
+    for (int idx = threadIdx.x; idx < rows * (kD / 4); idx += NT) {
+        int row = idx >> 5, c4 = idx & 31;
+        float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < valid) f = load4<T>(get(row) + c4 * 4);
+        *reinterpret_cast<float4*>(dst + row * stride + c4 * 4) = f;
+    }
+}
+
+__device__ __forceinline__ float dot4(float4 a, float4 b, float acc) {
+    acc = fmaf(a.x, b.x, acc); acc = fmaf(a.y, b.y, acc);
+    acc = fmaf(a.z, b.z, acc); acc = fmaf(a.w, b.w, acc);
+    return acc;
+}
+
+// acc[i][j] += sum_c A[(warp*4+i)][c] * Bt[(lane+32j)][c]   (A row stride kD, Bt row stride KS)
+__device__ __forceinline__ void tile_gemm(const float* __restrict__ sA, const float* __restrict__ sB,
+                                          int warp, int lane, float (&acc)[4][2]) {
+#pragma unroll 4
+    for (int c4 = 0; c4 < kD / 4; ++c4) {
+        float4 b0 = *reinterpret_cast<const float4*>(sB + lane * KS + c4 * 4);
+        float4 b1 = *reinterpret_cast<const float4*>(sB + (lane + 32) * KS + c4 * 4);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 a = *reinterpret_cast<const float4*>(sA + (warp * 4 + i) * kD + c4 * 4);
+            acc[i][0] = dot4(a, b0, acc[i][0]);
+            acc[i][1] = dot4(a, b1, acc[i][1]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ pass 1
+template <typename T>
+__global__ void __launch_bounds__(NT, 2)
+simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, TensorView v, float* ws) {
+    extern __shared__ __align__(16) float smem[];
+    float* sK = smem;                       // [TN][KS]
+    float* sV = sK + TN * KS;               // [TN][kD]
+    float* sQ = sV + TN * kD;               // [RC][kD]
+    float* sP = sQ + RC * kD;               // [RC][TN]
+
+    const int split = blockIdx.x, unit = blockIdx.y, r0 = blockIdx.z * RC;
+    const int b = unit / s.Hkv, g = unit % s.Hkv;
+    const int N = seq_len(s, b);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float sl2 = s.scale * kLog2e;
+
+    load_rows<T>(sQ, kD, RC, min(RC, s.R - r0), [&](int row) {
+        int r = r0 + row;
+        return row_ptr<T>(q, b, g * s.G + r / s.W, r % s.W);
+    });
+
+    float m2[4], l[4], o[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        m2[i] = -INFINITY; l[i] = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) o[i][c] = 0.f;
+    }
+    long long last[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int r = r0 + warp * 4 + i;
+        last[i] = (r < s.R) ? (s.causal ? (long long)N - s.W + (r % s.W) : (long long)N - 1) : -1;
+    }
+
+    const int tile_lo = split * plan.tiles_per_split;
+    const int tile_hi = min(tile_lo + plan.tiles_per_split, (N + TN - 1) / TN);
+    for (int tile = tile_lo; tile < tile_hi; ++tile) {
+        const int t0 = tile * TN;
+        __syncthreads();
+        load_rows<T>(sK, KS, TN, min(TN, N - t0), [&](int row) { return row_ptr<T>(k, b, g, t0 + row); });
+        load_rows<T>(sV, kD, TN, min(TN, N - t0), [&](int row) { return row_ptr<T>(v, b, g, t0 + row); });
+        __syncthreads();
+
+        float acc[4][2] = {};
+        tile_gemm(sQ, sK, warp, lane, acc);
+
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float s0 = (t0 + lane <= last[i]) ? acc[i][0] * sl2 : -INFINITY;
+            float s1 = (t0 + lane + 32 <= last[i]) ? acc[i][1] * sl2 : -INFINITY;
+            float mt = warp_max(fmaxf(s0, s1));
+            float mn = fmaxf(m2[i], mt);
+            float p0 = 0.f, p1 = 0.f, corr = 1.f;
+            if (mn != -INFINITY) {
+                corr = exp2f(m2[i] - mn);              // m2 = -inf -> 0
+                p0 = exp2f(s0 - mn); p1 = exp2f(s1 - mn);
+            }
+            float ps = warp_sum(p0 + p1);
+            l[i] = l[i] * corr + ps;
+            m2[i] = mn;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) o[i][c] *= corr;
+            sP[(warp * 4 + i) * TN + lane] = p0;
+            sP[(warp * 4 + i) * TN + lane + 32] = p1;
+        }
+        __syncwarp();
+        // O[rows of this warp][lane*4 .. +3] += P[row][p] * V[p][lane*4 .. +3]
+#pragma unroll 2
+        for (int p4 = 0; p4 < TN / 4; ++p4) {
+            float4 pr[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) pr[i] = *reinterpret_cast<const float4*>(sP + (warp * 4 + i) * TN + p4 * 4);
+#pragma unroll
+            for (int pp = 0; pp < 4; ++pp) {
+                float4 vv = *reinterpret_cast<const float4*>(sV + (p4 * 4 + pp) * kD + lane * 4);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float pw = pp == 0 ? pr[i].x : pp == 1 ? pr[i].y : pp == 2 ? pr[i].z : pr[i].w;
+                    o[i][0] = fmaf(pw, vv.x, o[i][0]); o[i][1] = fmaf(pw, vv.y, o[i][1]);
+                    o[i][2] = fmaf(pw, vv.z, o[i][2]); o[i][3] = fmaf(pw, vv.w, o[i][3]);
+                }
+            }
+        }
+        __syncwarp();
+    }
+
+    float* part_m = ws + plan.off_part_m / 4;
+    float* part_l = ws + plan.off_part_l / 4;
+    float* part_o = ws + plan.off_part_o / 4;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int r = r0 + warp * 4 + i;
+        if (r >= s.R) continue;
+        size_t row = ((size_t)unit * plan.n_splits + split) * s.R + r;
+        if (lane == 0) { part_m[row] = m2[i]; part_l[row] = l[i]; }
+        *reinterpret_cast<float4*>(part_o + row * kD + lane * 4) = make_float4(o[i][0], o[i][1], o[i][2], o[i][3]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ combine
+// one block of 128 threads per (unit, row): merge the splits
+__global__ void __launch_bounds__(128)
+simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
+    const int r = blockIdx.x % s.R, unit = blockIdx.x / s.R, c = threadIdx.x;
+    const float* part_m = ws + plan.off_part_m / 4;
+    const float* part_l = ws + plan.off_part_l / 4;
+    const float* part_o = ws + plan.off_part_o / 4;
+    float M = -INFINITY;
+    for (int sp = 0; sp < plan.n_splits; ++sp)
+        M = fmaxf(M, part_m[((size_t)unit * plan.n_splits + sp) * s.R + r]);
+    float L = 0.f, oc = 0.f;
+    for (int sp = 0; sp < plan.n_splits; ++sp) {
+        size_t row = ((size_t)unit * plan.n_splits + sp) * s.R + r;
+        float m = part_m[row];
+        if (m == -INFINITY) continue;
+        float w = exp2f(m - M);
+        L = fmaf(part_l[row], w, L);
+        oc = fmaf(part_o[row * kD + c], w, oc);
+    }
+    oc = oc / L;
+    __shared__ float red[4];
+    float sq = warp_sum(oc * oc);
+    if ((c & 31) == 0) red[c >> 5] = sq;
+    __syncthreads();
+    size_t row = (size_t)unit * s.R + r;
+    (ws + plan.off_o / 4)[row * kD + c] = oc;
+    if (c == 0) {
+        (ws + plan.off_lse2 / 4)[row] = M + log2f(L);
+        (ws + plan.off_onorm / 4)[row] = red[0] + red[1] + red[2] + red[3];
+    }
+}
+
+// ------------------------------------------------------------------------------------------ pass 2
+template <typename T>
+__global__ void __launch_bounds__(NT, 2)
+simt_pass2_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, TensorView v,
+                  const float* ws, float* scores) {
+    extern __shared__ __align__(16) float smem[];
+    float* sK = smem;                       // [TN][KS]
+    float* sV = sK + TN * KS;               // [TN][KS]
+    float* sQ = sV + TN * KS;               // [RC][kD]   (reused for the final cross-warp sum)
+    float* sO = sQ + RC * kD;               // [RC][kD]
+    float* sNv = sO + RC * kD;              // [TN]
+    float* sLse = sNv + TN;                 // [RC]
+    float* sNo = sLse + RC;                 // [RC]
+
+    const int unit = blockIdx.y, t0 = blockIdx.x * TN;
+    const int b = unit / s.Hkv, g = unit % s.Hkv;
+    const int N = seq_len(s, b);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t plane = (size_t)s.B * s.Hkv * s.Nmax;
+    float* out = scores + (size_t)unit * s.Nmax;
+
+    if (t0 >= N) {                          // padding beyond the sequence: scores are 0
+        for (int i = threadIdx.x; i < TN * s.n_planes; i += NT) {
+            int p = t0 + (i % TN);
+            if (p < s.Nmax) out[(size_t)(i / TN) * plane + p] = 0.f;
+        }
+        return;
+    }
+
+    load_rows<T>(sK, KS, TN, min(TN, N - t0), [&](int row) { return row_ptr<T>(k, b, g, t0 + row); });
+    load_rows<T>(sV, KS, TN, min(TN, N - t0), [&](int row) { return row_ptr<T>(v, b, g, t0 + row); });
+    __syncthreads();
+    // ||v_p||^2: each warp covers 8 tokens
+    for (int tkn = warp * 8; tkn < warp * 8 + 8; ++tkn) {
+        float4 f = *reinterpret_cast<const float4*>(sV + tkn * KS + lane * 4);
+        float sq = warp_sum(f.x * f.x + f.y * f.y + f.z * f.z + f.w * f.w);
+        if (lane == 0) sNv[tkn] = sq;
+    }
+
+    const float sl2 = s.scale * kLog2e;
+    const float* o_all = ws + plan.off_o / 4 + (size_t)unit * s.R * kD;
+    const float* lse_all = ws + plan.off_lse2 / 4 + (size_t)unit * s.R;
+    const float* no_all = ws + plan.off_onorm / 4 + (size_t)unit * s.R;
+
+    float sv[2] = {0.f, 0.f}, sk[2] = {0.f, 0.f}, sx[2] = {0.f, 0.f}, sa[2] = {0.f, 0.f};
+
+    for (int r0 = 0; r0 < s.R; r0 += RC) {
+        __syncthreads();
+        const int valid = min(RC, s.R - r0);
+        load_rows<T>(sQ, kD, RC, valid, [&](int row) {
+            int r = r0 + row;
+            return row_ptr<T>(q, b, g * s.G + r / s.W, r % s.W);
+        });
+        load_rows<float>(sO, kD, RC, valid, [&](int row) { return o_all + (size_t)(r0 + row) * kD; });
+        if (threadIdx.x < RC) {
+            bool ok = threadIdx.x < valid;
+            sLse[threadIdx.x] = ok ? lse_all[r0 + threadIdx.x] : 0.f;
+            sNo[threadIdx.x] = ok ? no_all[r0 + threadIdx.x] : 0.f;
+        }
+        __syncthreads();
+
+        float az[4][2] = {}, at[4][2] = {};
+        tile_gemm(sQ, sK, warp, lane, az);
+        tile_gemm(sO, sV, warp, lane, at);
+
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = r0 + warp * 4 + i;
+            if (r >= s.R) continue;
+            const long long last = s.causal ? (long long)N - s.W + (r % s.W) : (long long)N - 1;
+            const float lse = sLse[warp * 4 + i], no = sNo[warp * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int tl = lane + 32 * j;
+                if (t0 + tl > last) continue;              // masked pair: contributes 0
+                const float nv = sNv[tl];
+                const float a = exp2f(fmaf(az[i][j], sl2, -lse));
+                const float Z = az[i][j] * s.scale;
+                const float t = at[i][j];
+                const float a2 = a * a;
+                sa[j] += a;
+                sv[j] = fmaf(a2, nv, sv[j]);
+                sk[j] = fmaf(a2 * Z * Z, no + nv - 2.f * t, sk[j]);      // Alg. 1: |o|^2+|v|^2-2 v.o
+                sx[j] = fmaf(2.f * a2 * Z, nv - t, sx[j]);               // Eq. 6 cross term
+            }
+        }
+    }
+
+    // sum over the 8 warps (each warp held 4 of every 32 rows)
+    __syncthreads();
+    float* red = sQ;                        // [8][4][TN]
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const int tl = lane + 32 * j;
+        red[(warp * 4 + 0) * TN + tl] = sv[j];
+        red[(warp * 4 + 1) * TN + tl] = sk[j];
+        red[(warp * 4 + 2) * TN + tl] = sx[j];
+        red[(warp * 4 + 3) * TN + tl] = sa[j];
+    }
+    __syncthreads();
+    if (threadIdx.x < TN) {
+        const int tl = threadIdx.x, p = t0 + tl;
+        float tv = 0.f, tk = 0.f, tx = 0.f, ta = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            tv += red[(w * 4 + 0) * TN + tl]; tk += red[(w * 4 + 1) * TN + tl];
+            tx += red[(w * 4 + 2) * TN + tl]; ta += red[(w * 4 + 3) * TN + tl];
+        }
+        if (p < s.Nmax) {
+            const bool live = p < N;
+            int pl = 0;
+            if (s.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + p] = live ? tv : 0.f;
+            if (s.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + p] = live ? tk : 0.f;
+            if (s.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + p] = live ? tv + tk + tx : 0.f;
+            if (s.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + p] = live ? ta : 0.f;
+        }
+    }
+}
+
+constexpr size_t kSmemPass1 = (size_t)(TN * KS + TN * kD + RC * kD + RC * TN) * 4;
+constexpr size_t kSmemPass2 = (size_t)(2 * TN * KS + 2 * RC * kD + TN + 2 * RC) * 4;
+
+template <typename T>
+obc_status launch_typed(const ScoreShape& s, const SimtPlan& plan, TensorView q, TensorView k, TensorView v,
+                        float* scores, float* ws, cudaStream_t stream) {
+    const int units = s.B * s.Hkv, chunks = (s.R + RC - 1) / RC;
+    OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass1_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass1));
+    OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass2_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass2));
+    simt_pass1_kernel<T><<<dim3(plan.n_splits, units, chunks), NT, kSmemPass1, stream>>>(s, plan, q, k, v, ws);
+    OBC_CUDA_TRY(cudaGetLastError());
+    simt_combine_kernel<<<units * s.R, 128, 0, stream>>>(s, plan, ws);
+    OBC_CUDA_TRY(cudaGetLastError());
+    simt_pass2_kernel<T><<<dim3((s.Nmax + TN - 1) / TN, units), NT, kSmemPass2, stream>>>(s, plan, q, k, v, ws, scores);
+    OBC_CUDA_TRY(cudaGetLastError());
+    return OBC_OK;
+}
+}  // namespace
+
+SimtPlan make_simt_plan(const ScoreShape& s) {
+    SimtPlan p{};
+    const int units = s.B * s.Hkv, chunks = (s.R + RC - 1) / RC;
+    const int tiles = (s.Nmax + TN - 1) / TN;
+    // enough CTAs for ~2 waves of 148 SMs x 2 resident CTAs, at least 8 tiles per split
+    int want = (148 * 2 * 2 + units * chunks - 1) / (units * chunks);
+    int max_splits = (tiles + 7) / 8;
+    int n = want < 1 ? 1 : want;
+    if (n > max_splits) n = max_splits;
+    if (n < 1) n = 1;
+    p.tiles_per_split = (tiles + n - 1) / n;
+    p.n_splits = (tiles + p.tiles_per_split - 1) / p.tiles_per_split;
+    size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, off = 0;
+    p.off_part_m = off; off = align_up(off + prow * 4, 256);
+    p.off_part_l = off; off = align_up(off + prow * 4, 256);
+    p.off_part_o = off; off = align_up(off + prow * kD * 4, 256);
+    p.off_lse2 = off;   off = align_up(off + rows * 4, 256);
+    p.off_onorm = off;  off = align_up(off + rows * 4, 256);
+    p.off_o = off;      off = align_up(off + rows * kD * 4, 256);
+    p.bytes = off;
+    return p;
+}
+
+obc_status launch_score_simt(const ScoreShape& s, const SimtPlan& plan, int dtype,
+                             TensorView q, TensorView k, TensorView v,
+                             float* scores, void* ws, cudaStream_t stream) {
+    if (dtype == OBC_F32) return launch_typed<float>(s, plan, q, k, v, scores, (float*)ws, stream);
+    return launch_typed<__nv_bfloat16>(s, plan, q, k, v, scores, (float*)ws, stream);
+}
+
+}  // namespace obc

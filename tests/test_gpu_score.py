@@ -1,0 +1,87 @@
+"""GPU parity of obc_score against the CPU checker, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_07651_b200 import api, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(case, variants, causal=True, path="auto", tight=None):
+    want = H.oracle_scores(case, variants, causal)
+    got = H.gpu_scores(case, variants, causal, path)
+    for n in variants:
+        H.assert_scores_close(got[n], want[n], case.dtype, tight=tight, what=f"{case.name}/{n}/{path}")
+        for b in range(case.B):                      # padding beyond each sequence is written as 0
+            assert (got[n][b, :, case.seq_lens[b]:] == 0).all()
+
+
+def test_config1_fp32_all_variants():
+    case, run = synth.config(1)
+    _check(case, run["variants"] + ["ATTN"], tight=2e-5)
+
+
+@pytest.mark.parametrize("path", ["simt", "auto"])
+def test_config2_shape_reduced_length(path):
+    case, run = synth.config(2, shrink=8)            # N = 4096: several tiles per split
+    _check(case, ["V", "K", "VK"], path=path, tight=2e-2)
+
+
+@pytest.mark.parametrize("path", ["simt", "auto"])
+def test_config3_shape_reduced_length(path):
+    case, run = synth.config(3, shrink=32)           # R = 448, N = 4096
+    _check(case, run["variants"], path=path, tight=2e-2)
+
+
+@pytest.mark.parametrize("path", ["simt", "auto"])
+def test_config4_ragged_batch_reduced(path):
+    case, run = synth.config(4, shrink=16)           # lengths in [512, 4096], ragged tails
+    _check(case, run["variants"], path=path, tight=2e-2)
+
+
+@pytest.mark.parametrize("N,W,Hq,Hkv,dtype,causal", [
+    (1, 1, 1, 1, "f32", True),            # single cached token
+    (16, 16, 2, 1, "f32", True),          # window == whole cache
+    (65, 3, 7, 1, "bf16", True),          # ragged tile tail, odd group
+    (200, 1, 4, 1, "bf16", True),         # W = 1 (decode-like), R = 4
+    (333, 5, 8, 2, "f32", False),         # non-causal
+    (1000, 40, 4, 2, "bf16", True),       # R = 80: not a multiple of the row chunk
+])
+def test_small_and_degenerate_shapes(N, W, Hq, Hkv, dtype, causal):
+    case = synth.make_prefill("edge", B=2, Hq=Hq, Hkv=Hkv, d=128, W=W, N=N, dtype=dtype, seed=77 + N,
+                              hh_frac=0.05)
+    _check(case, ["V", "K", "VK", "ATTN"], causal=causal, tight=2e-2 if dtype == "bf16" else 2e-5)
+
+
+def test_peaky_attention_cancellation_case():
+    # some attention weights approach 1, so ||v_p - o_i||^2 cancels heavily
+    case = synth.make_prefill("peaky", B=1, Hq=8, Hkv=2, d=128, W=16, N=2048, dtype="bf16", seed=5,
+                              hh_frac=0.01, peaky=True)
+    _check(case, ["V", "K", "VK"], path="simt")
+    _check(case, ["V", "K", "VK"], path="auto")
+
+
+def test_strided_views_and_split_invariance():
+    # K/V given as non-contiguous views (token stride 2d) must score like their contiguous copies
+    case = synth.make_prefill("strided", B=1, Hq=4, Hkv=2, d=128, W=8, N=700, dtype="bf16", seed=9)
+    q, k, v = H.upload(case)
+    wide_k = torch.zeros((1, 2, 700, 256), dtype=torch.bfloat16, device="cuda")
+    wide_v = torch.zeros_like(wide_k)
+    wide_k[..., :128] = k
+    wide_v[..., :128] = v
+    a = api.obc_score(q, k, v, variants=["VK"])
+    b = api.obc_score(q, wide_k[..., :128], wide_v[..., :128], variants=["VK"])
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+
+
+def test_workspace_poison_does_not_leak():
+    case = synth.make_prefill("poison", B=1, Hq=4, Hkv=1, d=128, W=4, N=300, dtype="f32", seed=3)
+    q, k, v = H.upload(case)
+    p = api.score_params(q, k, variants=["VK"])
+    ws = torch.full((api.obc_score_workspace(p),), 0xFF, dtype=torch.uint8, device="cuda")   # NaN pattern
+    s = api.obc_score(q, k, v, variants=["VK"], workspace=ws)
+    want = H.oracle_scores(case, ["VK"])["VK"]
+    H.assert_scores_close(s[0].cpu().numpy(), want, "f32", tight=2e-5)
