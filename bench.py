@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the OBCache hot path (score -> pool/select -> compact) on B200.
+
+A "step" is one pass of the whole path over one Llama-3-8B-shaped layer cache (32 query heads /
+8 KV heads, head_dim 128, N = 32768 cached tokens, window W = 32, bf16, OBCache-V&K, max-pool 7,
+budget 2048 per head).  The metric is cached tokens scored+compacted per second per layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 it is launched by torch.distributed.run, one rank per GPU; every rank processes its
+own cache (the (batch, KV head) units are independent, so there is no data-path collective) and
+the reported value is the sum over ranks divided by the slowest rank's time (weak scaling).
+
+`--impl reference` times the CPU checker (oracle/) as it stands on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "cached tokens scored+compacted/sec per layer"
+UNIT = "tokens/s"
+WORKLOAD = ("llama3-8b-layer-32k: B1 Hq32 Hkv8 d128 N32768 W32 bf16, OBCache-V&K, max-pool 7, "
+            "budget 2048/head, n_recent 32")
+N_COPIES = 4            # distinct input copies rotated between steps (4 x 135 MB > 126 MB L2)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    sm_max_mhz=float(d.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, sm_max_mhz=1965.0,
+                source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons in the background."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.t0 = time.time()
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu=timestamp,{self.FIELDS}", "--format=csv,noheader,nounits",
+                                       "-lms", "50", "-i", str(device_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+        self.marks = {}
+
+    def mark(self, name):
+        self.marks[name] = time.time()
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.06)
+        self.p.terminate()
+        self.p.wait()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        from datetime import datetime
+        parsed = []
+        for r in rows:
+            try:
+                ts = datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                parsed.append((ts, float(r[1]), float(r[2]), float(r[3]), r[4:8]))
+            except (ValueError, IndexError):
+                continue
+        a, b = self.marks.get("timed_begin", self.t0), self.marks.get("timed_end", time.time())
+        inside = [x for x in parsed if a <= x[0] <= b]
+        where = "timed region"
+        if not inside:                       # region shorter than the sampling period
+            inside, where = parsed, "whole run"
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for x in inside for n, v in zip(names, x[4]) if v.strip() == "Active"})
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(x[1] for x in inside), "sm_max_mhz": inside[0][2],
+                "power_w_max": max(x[3] for x in inside), "reasons": reasons, "samples": len(inside),
+                "window": where}
+
+
+def make_case(seed):
+    from paper_2510_07651_b200 import synth
+    return synth.config(2, seed=seed)
+
+
+def run_reference(args):
+    """The CPU checker as it stands, timed on the host cores (rank 0 only).  Each step scores,
+    selects and compacts a bounded sample of the workload: the first `heads` of the 8 KV heads
+    (all 32768 tokens, all their query heads), sized so that the whole run ends within minutes."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+    from oracle import reference as ref
+    ref.build()
+    case, run = make_case(1236)
+    cores = ref.host_threads()
+    G = case.G
+
+    def step(heads):
+        s = ref.score(case.q[:, :heads * G], case.k[:, :heads], case.v[:, :heads], want=("VK",))["VK"].astype(np.float32)
+        idx = ref.select_pipeline(s, case.seq_lens, [run["budget"]], 0, run["n_recent"], run["pool_mode"],
+                                  run["pool_kernel"], run["budget"])
+        for h in range(heads):
+            ref.compact(case.k_bits[0, h], idx[0, h], run["budget"])
+            ref.compact(case.v_bits[0, h], idx[0, h], run["budget"])
+
+    t0 = time.time()
+    step(1)                                        # also the warm-up
+    t_head = time.time() - t0
+    heads = int(max(1, min(case.Hkv, 120.0 / (t_head * (args.steps + args.warmup)))))
+    for _ in range(args.warmup):
+        step(heads)
+    t0 = time.time()
+    for _ in range(args.steps):
+        step(heads)
+    dt = time.time() - t0
+    value = case.Nmax * (heads / case.Hkv) * args.steps / dt       # layer-equivalent tokens per second
+    sample = f"{heads} of {case.Hkv} KV heads (all 32768 tokens) per step, scaled to one layer"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2510_07651_b200 import api, build, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    api.lib()
+    peaks = load_peaks()
+
+    # ---- inputs: N_COPIES distinct seeded caches, resident in HBM ------------------------------
+    bf = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    cases, dev = [], []
+    for c in range(N_COPIES):
+        case, run = make_case(1236 + 100 * rank + c)
+        cases.append(case)
+        dev.append((bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)))
+    case = cases[0]
+    B, Hkv, N, d, budget = case.B, case.Hkv, case.Nmax, case.d, run["budget"]
+    tokens_per_step = int(case.seq_lens.sum())
+
+    # ---- preallocated outputs and workspaces (nothing is allocated inside the timed region) -----
+    sp = api.score_params(dev[0][0], dev[0][1], variants=run["variants"], path=args.path)
+    ws_score = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
+    scores = torch.empty((1, B, Hkv, N), dtype=torch.float32, device="cuda")
+    selp = api.select_params(scores[0], budget=budget, n_recent=run["n_recent"], pool=run["pool_mode"],
+                             pool_kernel=run["pool_kernel"])
+    ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
+    idx = torch.empty((B, Hkv, budget), dtype=torch.int32, device="cuda")
+    k_out = torch.empty((B, Hkv, budget, d), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+
+    def step(q, k, v):
+        api.obc_score(q, k, v, variants=run["variants"], path=args.path, scores=scores, workspace=ws_score)
+        api.obc_select(scores[0], budget=budget, n_recent=run["n_recent"], pool=run["pool_mode"],
+                       pool_kernel=run["pool_kernel"], idx=idx, workspace=ws_sel)
+        api.obc_compact(k, v, idx, k_out=k_out, v_out=v_out)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    for i in range(args.warmup):
+        step(*dev[i % N_COPIES])
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sampler:
+        sampler.mark("timed_begin")
+    e0.record()
+    for i in range(args.steps):
+        step(*dev[i % N_COPIES])
+    e1.record()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.mark("timed_end")
+    barrier()
+    ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms = float(ms.item())
+
+    # ---- per-kernel times (same steps again, every kernel bracketed by CUDA events) -------------
+    api.obc_profile_begin()
+    for i in range(args.steps):
+        step(*dev[i % N_COPIES])
+    torch.cuda.synchronize()
+    prof = api.obc_profile_end()
+    clocks = sampler.stop() if sampler else None
+    launches_per_step = sum(v[0] for v in prof.values()) // max(args.steps, 1)
+
+    # ---- end to end: host (pinned) inputs -> device, whole path, results back to the host -------
+    pin = lambda t: t.cpu().pin_memory()
+    host = [tuple(pin(t) for t in dev[c]) for c in range(2)]
+    dq, dk, dv = (torch.empty_like(t) for t in dev[0])
+    h_idx, h_k, h_v = pin(idx), pin(k_out), pin(v_out)
+    h2d = sum(t.numel() * t.element_size() for t in host[0])
+    d2h = sum(t.numel() * t.element_size() for t in (h_idx, h_k, h_v))
+
+    def e2e_step(i):
+        hq, hk, hv = host[i % 2]
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+        step(dq, dk, dv)
+        h_idx.copy_(idx, non_blocking=True); h_k.copy_(k_out, non_blocking=True); h_v.copy_(v_out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()          # the caller reads the result
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = torch.tensor([max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))], device="cuda")
+    if world > 1:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_value = world * tokens_per_step * e2e_steps / (float(e2e_ms.item()) * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel -----------------------------------------------------------
+    value = world * tokens_per_step * args.steps / (ms * 1e-3)
+    dom = max(prof.items(), key=lambda kv: kv[1][1])
+    dom_name, (dom_launches, dom_ms) = dom
+    dom_avg_s = dom_ms * 1e-3 / dom_launches
+    elem = 2
+    R = case.R
+    kv_bytes = B * Hkv * N * d * elem * 2                     # K and V read once
+    alg = {   # algorithmic bytes / flops per launch of each kernel on this workload
+        "pass1": (kv_bytes, 2 * 2 * R * N * d * B * Hkv),
+        "pass2": (kv_bytes + B * Hkv * N * 4, 2 * 2 * R * N * d * B * Hkv),
+    }
+    kind = "pass2" if "pass2" in dom_name else "pass1" if "pass1" in dom_name else None
+    roof = {"kernel": dom_name, "launches": dom_launches, "avg_us": dom_avg_s * 1e6, "traffic": None}
+    if kind and dom_name.startswith("simt"):
+        peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12      # fp32 FMA lanes x 2 flop x clock
+        ach = alg[kind][1] / dom_avg_s / 1e12
+        roof.update(bound="alu", achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
+                    peak_source="148 SMs x 128 fp32 lanes x 2 flop x max SM clock")
+    elif kind:
+        t_hbm = alg[kind][0] / (peaks["hbm_gbs"] * 1e9)
+        t_mma = alg[kind][1] / (peaks["bf16_tflops_sustained"] * 1e12)
+        if t_hbm >= t_mma:
+            ach = alg[kind][0] / dom_avg_s / 1e9
+            roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
+                        peak_source=f"{peaks['source']} STREAM-style copy")
+        else:
+            ach = alg[kind][1] / dom_avg_s / 1e12
+            roof.update(bound="tensor", achieved=ach, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                        frac=ach / peaks["bf16_tflops_sustained"], peak_source=f"{peaks['source']} cuBLAS bf16 sustained")
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        roof["traffic"] = json.load(open(traffic_file)).get(dom_name)
+    kernels = {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}
+
+    # ---- CPU baseline: the checker as it stands, on this machine's host cores ----------------------
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        from oracle import reference as ref
+        ref.build()
+        c0 = cases[0]
+        reps, t0 = 0, time.time()
+        while reps < 1 or (time.time() - t0 < 10.0 and reps < 8):
+            s = ref.score(c0.q, c0.k, c0.v, want=("VK",))["VK"].astype(np.float32)
+            ridx = ref.select_pipeline(s, c0.seq_lens, [budget], 0, run["n_recent"], run["pool_mode"],
+                                       run["pool_kernel"], budget)
+            for h in range(Hkv):
+                ref.compact(c0.k_bits[0, h], ridx[0, h], budget)
+                ref.compact(c0.v_bits[0, h], ridx[0, h], budget)
+            reps += 1
+        dt = time.time() - t0
+        cpu = {"value": tokens_per_step * reps / dt, "unit": UNIT, "cores": ref.host_threads(), "kind": "oracle",
+               "sample": f"the full workload (8 KV heads x 32768 tokens), {reps} repetitions, {dt:.1f} s"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "path": args.path,
+                       "l2": f"{N_COPIES} distinct input copies rotated between steps ({N_COPIES} x 135 MB > 126 MB L2)",
+                       "parallelism": f"{world} independent layer caches, one per GPU, no collective"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roof, "kernels": kernels, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

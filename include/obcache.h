@@ -38,7 +38,7 @@ typedef enum {
     OBC_ERR_ALIGN = -4,        /* base pointer or stride not 16-byte aligned */
     OBC_ERR_WORKSPACE = -5,    /* workspace missing or smaller than obc_*_workspace() says */
     OBC_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed; see obc_last_cuda_error() */
-    OBC_ERR_TIMEOUT = -7       /* a bounded device-side wait gave up (reported by obc_device_status) */
+    OBC_ERR_TIMEOUT = -7       /* a bounded device-side wait gave up */
 } obc_status;
 
 typedef enum { OBC_F32 = 0, OBC_BF16 = 1 } obc_dtype;
@@ -184,6 +184,17 @@ obc_status obc_decode_step(const obc_decode_params* p, obc_tensor q_t, obc_tenso
                            obc_tensor k_cache, obc_tensor v_cache, float* s_acc, int32_t* pos,
                            int32_t* state, int32_t step_pos,
                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Optional per-kernel timing, used by the benchmark (no counterpart in the paper).  Between
+ * obc_profile_begin() and obc_profile_end() every kernel the library enqueues from any thread
+ * is bracketed by a pair of CUDA events on its stream.  obc_profile_end() synchronises those
+ * events, sums the elapsed time per kernel name into out[0..*n_out) (host array of max_out
+ * entries) and stops recording.  Off by default; costs two event records per kernel when on.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct { char name[48]; int32_t launches; float ms_total; } obc_kernel_time;
+obc_status obc_profile_begin(void);
+obc_status obc_profile_end(obc_kernel_time* out /* host */, int32_t max_out, int32_t* n_out /* host */);
 
 /* Host-only helpers. */
 const char* obc_status_string(obc_status s);

@@ -24,8 +24,8 @@ POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
 EXPORTS = ["obc_score_workspace", "obc_score", "obc_select_workspace", "obc_select", "obc_compact",
-           "obc_decode_workspace", "obc_decode_step", "obc_status_string", "obc_last_cuda_error",
-           "obc_version"]
+           "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
+           "obc_status_string", "obc_last_cuda_error", "obc_version"]
 
 
 class ObcError(RuntimeError):
@@ -63,6 +63,10 @@ class obc_decode_params(C.Structure):
                 ("variant", C.c_uint32), ("scale", C.c_float)]
 
 
+class obc_kernel_time(C.Structure):
+    _fields_ = [("name", C.c_char * 48), ("launches", C.c_int32), ("ms_total", C.c_float)]
+
+
 _lib = None
 
 
@@ -82,6 +86,8 @@ def lib():
         L.obc_compact.argtypes = [C.c_int32] * 5 + [obc_tensor, obc_tensor, vp, obc_tensor, obc_tensor, vp, vp, vp]
         L.obc_decode_workspace.argtypes = [C.POINTER(obc_decode_params), sz]
         L.obc_decode_step.argtypes = [C.POINTER(obc_decode_params)] + [obc_tensor] * 5 + [vp, vp, vp, C.c_int32, vp, C.c_size_t, vp]
+        L.obc_profile_begin.argtypes = []
+        L.obc_profile_end.argtypes = [C.POINTER(obc_kernel_time), C.c_int32, C.POINTER(C.c_int32)]
         L.obc_status_string.argtypes = [C.c_int]
         L.obc_status_string.restype = C.c_char_p
         for n in EXPORTS:
@@ -226,6 +232,19 @@ def obc_decode_step(q_t, k_t, v_t, k_cache, v_cache, s_acc, pos, state, step_pos
                                  as_tensor4(v_cache), s_acc.data_ptr(), pos.data_ptr(), state.data_ptr(),
                                  int(step_pos), ws.data_ptr(), ws.numel(), _stream()), "obc_decode_step")
     return ws
+
+
+def obc_profile_begin():
+    """Start bracketing every library kernel with CUDA events (benchmark use)."""
+    _check(lib().obc_profile_begin(), "obc_profile_begin")
+
+
+def obc_profile_end() -> dict:
+    """Stop recording; returns {kernel name: (launches, total ms)}."""
+    buf = (obc_kernel_time * 64)()
+    n = C.c_int32(0)
+    _check(lib().obc_profile_end(buf, 64, C.byref(n)), "obc_profile_end")
+    return {buf[i].name.decode(): (buf[i].launches, buf[i].ms_total) for i in range(n.value)}
 
 
 def evict_prefill(q, k, v, *, budget=0, budgets=None, seq_lens=None, variant="VK", n_sink=0, n_recent=None,

@@ -1,11 +1,38 @@
 // The C-ABI entry points: argument validation, workspace planning, kernel-family choice.
 // Every function here runs on the host and only enqueues work; see include/obcache.h.
 #include "obc_common.cuh"
+#include <atomic>
+#include <cstring>
+#include <mutex>
+#include <vector>
 
 namespace obc {
 
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+
+// ---- optional per-kernel event timing ---------------------------------------------------------
+namespace {
+struct ProfRec { const char* name; cudaEvent_t e0, e1; };
+std::mutex g_prof_mu;
+std::vector<ProfRec> g_prof;
+std::atomic<bool> g_prof_on{false};
+}  // namespace
+
+ProfScope::ProfScope(const char* name, cudaStream_t s) : slot(-1), stream(s) {
+    if (!g_prof_on.load(std::memory_order_relaxed)) return;
+    ProfRec r{name, nullptr, nullptr};
+    if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) return;
+    cudaEventRecord(r.e0, s);
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof.push_back(r);
+    slot = (int)g_prof.size() - 1;
+}
+ProfScope::~ProfScope() {
+    if (slot < 0) return;
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    if (slot < (int)g_prof.size()) cudaEventRecord(g_prof[slot].e1, stream);
+}
 
 namespace {
 
@@ -191,6 +218,41 @@ obc_status obc_decode_step(const obc_decode_params* p, obc_tensor q_t, obc_tenso
     if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
     return launch_decode(s, view(q_t), view(k_t), view(v_t), view(k_cache), view(v_cache), s_acc, pos, state,
                          step_pos, workspace, (cudaStream_t)stream);
+}
+
+obc_status obc_profile_begin(void) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    for (auto& r : g_prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+    g_prof.clear();
+    g_prof_on.store(true);
+    return OBC_OK;
+}
+
+obc_status obc_profile_end(obc_kernel_time* out, int32_t max_out, int32_t* n_out) {
+    if (!out || !n_out || max_out < 1) return OBC_ERR_NULL;
+    g_prof_on.store(false);
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    int n = 0;
+    obc_status st = OBC_OK;
+    for (auto& r : g_prof) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(r.e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r.e0, r.e1);
+        if (e != cudaSuccess) { set_last_cuda_error((int)e); st = OBC_ERR_CUDA; }
+        int j = 0;
+        for (; j < n; ++j) if (std::strcmp(out[j].name, r.name) == 0) break;
+        if (j == n) {
+            if (n == max_out) continue;
+            std::memset(&out[n], 0, sizeof(out[n]));
+            std::strncpy(out[n].name, r.name, sizeof(out[n].name) - 1);
+            ++n;
+        }
+        out[j].launches += 1; out[j].ms_total += ms;
+        cudaEventDestroy(r.e0); cudaEventDestroy(r.e1);
+    }
+    g_prof.clear();
+    *n_out = n;
+    return st;
 }
 
 const char* obc_status_string(obc_status s) {

@@ -331,13 +331,13 @@ obc_status launch_g(const DecodeShape& s, const DecodePlan& plan, TensorView q, 
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
                     int step_pos, char* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
-    decode_pass1_kernel<G><<<dim3(plan.chunks, units), CH, 0, stream>>>(s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws);
+    { ProfScope ps("decode_pass1", stream); decode_pass1_kernel<G><<<dim3(plan.chunks, units), CH, 0, stream>>>(s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
-    decode_combine_kernel<<<units, kD, 0, stream>>>(s, plan, ws);
+    { ProfScope ps("decode_combine", stream); decode_combine_kernel<<<units, kD, 0, stream>>>(s, plan, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
-    decode_score_kernel<G><<<dim3(plan.chunks, units), CH, 0, stream>>>(s, plan, vc, s_acc, pos, state, step_pos, ws);
+    { ProfScope ps("decode_score", stream); decode_score_kernel<G><<<dim3(plan.chunks, units), CH, 0, stream>>>(s, plan, vc, s_acc, pos, state, step_pos, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
-    decode_final_kernel<<<(units + 127) / 128, 128, 0, stream>>>(s, plan, pos, state, ws);
+    { ProfScope ps("decode_final", stream); decode_final_kernel<<<(units + 127) / 128, 128, 0, stream>>>(s, plan, pos, state, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

@@ -18,6 +18,13 @@ void set_last_cuda_error(int e);
         if (_e != cudaSuccess) { obc::set_last_cuda_error((int)_e); return OBC_ERR_CUDA; } \
     } while (0)
 
+// Brackets one kernel launch with CUDA events while profiling is on (see obc_profile_begin).
+struct ProfScope {
+    ProfScope(const char* name, cudaStream_t stream);
+    ~ProfScope();
+    int slot; cudaStream_t stream;
+};
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---- internal launch descriptions (plain structs, passed by value to kernels) ---------------

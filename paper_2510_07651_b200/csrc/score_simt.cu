@@ -323,11 +323,11 @@ obc_status launch_typed(const ScoreShape& s, const SimtPlan& plan, TensorView q,
     const int units = s.B * s.Hkv, chunks = (s.R + RC - 1) / RC;
     OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass1_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass1));
     OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass2_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass2));
-    simt_pass1_kernel<T><<<dim3(plan.n_splits, units, chunks), NT, kSmemPass1, stream>>>(s, plan, q, k, v, ws);
+    { ProfScope ps("simt_pass1", stream); simt_pass1_kernel<T><<<dim3(plan.n_splits, units, chunks), NT, kSmemPass1, stream>>>(s, plan, q, k, v, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
-    simt_combine_kernel<<<units * s.R, 128, 0, stream>>>(s, plan, ws);
+    { ProfScope ps("simt_combine", stream); simt_combine_kernel<<<units * s.R, 128, 0, stream>>>(s, plan, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
-    simt_pass2_kernel<T><<<dim3((s.Nmax + TN - 1) / TN, units), NT, kSmemPass2, stream>>>(s, plan, q, k, v, ws, scores);
+    { ProfScope ps("simt_pass2", stream); simt_pass2_kernel<T><<<dim3((s.Nmax + TN - 1) / TN, units), NT, kSmemPass2, stream>>>(s, plan, q, k, v, ws, scores); }
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

@@ -188,9 +188,9 @@ size_t select_workspace_bytes(int B, int Hkv, int Nmax) { return align_up((size_
 obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx, void* ws, cudaStream_t stream) {
     uint32_t* keys = (uint32_t*)ws;
     const int units = s.B * s.Hkv;
-    pool_key_kernel<<<dim3((s.Nmax + 255) / 256, units), 256, 0, stream>>>(s, scores, keys);
+    { ProfScope ps("pool_key", stream); pool_key_kernel<<<dim3((s.Nmax + 255) / 256, units), 256, 0, stream>>>(s, scores, keys); }
     OBC_CUDA_TRY(cudaGetLastError());
-    select_kernel<<<units, SEL_NT, 0, stream>>>(s, keys, idx);
+    { ProfScope ps("select", stream); select_kernel<<<units, SEL_NT, 0, stream>>>(s, keys, idx); }
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
@@ -200,8 +200,11 @@ obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_byte
                          const float* s_in, float* s_out, cudaStream_t stream) {
     const int vecs = kD * elem_bytes / 16;
     const long long total = (long long)idx_stride * vecs;
-    gather_kernel<<<dim3((unsigned)((total + 255) / 256), B * Hkv), 256, 0, stream>>>(
-        B * Hkv, Hkv, idx_stride, vecs, elem_bytes, k, v, ko, vo, idx, s_in, s_out, Nmax);
+    {
+        ProfScope ps("gather", stream);
+        gather_kernel<<<dim3((unsigned)((total + 255) / 256), B * Hkv), 256, 0, stream>>>(
+            B * Hkv, Hkv, idx_stride, vecs, elem_bytes, k, v, ko, vo, idx, s_in, s_out, Nmax);
+    }
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

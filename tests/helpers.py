@@ -26,13 +26,17 @@ def lens_dev(case):
     return torch.from_numpy(case.seq_lens).cuda()
 
 
-def assert_scores_close(got: np.ndarray, want: np.ndarray, dtype: str, *, tight: float | None = None, what=""):
+def assert_scores_close(got: np.ndarray, want: np.ndarray, dtype: str, *, tight: float | None = None, what="",
+                        mx: float | None = None):
     """Spec tolerance, plus (tight) a relative bound normalised by the largest reference
-    score, which stays meaningful when scores are far below the absolute tolerance."""
+    score, which stays meaningful when scores are far below the absolute tolerance.  `mx` is the
+    magnitude the fp32 absolute tolerance scales with (default: the largest reference value of
+    this plane; callers pass the largest OBCache score of the case so that a plane that is
+    identically zero, e.g. the key score of a single-token cache, is judged on the same scale)."""
     want = np.asarray(want, np.float64)
     got = np.asarray(got, np.float64)
     assert np.isfinite(got).all(), what
-    mx = np.abs(want).max()
+    mx = np.abs(want).max() if mx is None else max(mx, np.abs(want).max())
     if dtype == "bf16":
         bound = BF16_ATOL + BF16_RTOL * np.abs(want)
     else:

@@ -12,8 +12,10 @@ pytestmark = pytest.mark.gpu
 def _check(case, variants, causal=True, path="auto", tight=None):
     want = H.oracle_scores(case, variants, causal)
     got = H.gpu_scores(case, variants, causal, path)
+    mx = max(np.abs(want[n]).max() for n in variants if n != "ATTN") if any(n != "ATTN" for n in variants) else None
     for n in variants:
-        H.assert_scores_close(got[n], want[n], case.dtype, tight=tight, what=f"{case.name}/{n}/{path}")
+        H.assert_scores_close(got[n], want[n], case.dtype, tight=tight, what=f"{case.name}/{n}/{path}",
+                              mx=None if n == "ATTN" else mx)
         for b in range(case.B):                      # padding beyond each sequence is written as 0
             assert (got[n][b, :, case.seq_lens[b]:] == 0).all()
 
