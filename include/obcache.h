@@ -103,6 +103,14 @@ obc_status obc_score_workspace(const obc_score_params* p, size_t* bytes /* host 
 obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
                      float* scores, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Reads the device status word that obc_score keeps in the first bytes of its workspace.  The
+ * tensor-core kernels bound every device-side wait; if one gives up, the kernel raises this word
+ * and returns early (its scores are then unspecified).  This call synchronises `stream`, copies
+ * the word to the host and returns OBC_OK or OBC_ERR_TIMEOUT.  (No counterpart in the paper.)
+ */
+obc_status obc_score_status(const void* workspace, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * obc_select: pooling + per-head top-budget (Algorithm 2's index selection; SnapKV-style 1-D
  * pooling, App. C.2.1).

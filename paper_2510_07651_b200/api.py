@@ -23,7 +23,7 @@ VARIANTS = {"V": OBC_VAR_V, "K": OBC_VAR_K, "VK": OBC_VAR_VK, "ATTN": OBC_VAR_AT
 POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
-EXPORTS = ["obc_score_workspace", "obc_score", "obc_select_workspace", "obc_select", "obc_compact",
+EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_status", "obc_select_workspace", "obc_select", "obc_compact",
            "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
            "obc_status_string", "obc_last_cuda_error", "obc_version"]
 
@@ -81,6 +81,7 @@ def lib():
         vp, sz = C.c_void_p, C.POINTER(C.c_size_t)
         L.obc_score_workspace.argtypes = [C.POINTER(obc_score_params), sz]
         L.obc_score.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, vp, vp, C.c_size_t, vp]
+        L.obc_score_status.argtypes = [vp, vp]
         L.obc_select_workspace.argtypes = [C.POINTER(obc_select_params), sz]
         L.obc_select.argtypes = [C.POINTER(obc_select_params), vp, vp, vp, C.c_size_t, vp]
         L.obc_compact.argtypes = [C.c_int32] * 5 + [obc_tensor, obc_tensor, vp, obc_tensor, obc_tensor, vp, vp, vp]
@@ -164,6 +165,11 @@ def obc_score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",
     _check(lib().obc_score(C.byref(p), as_tensor4(q), as_tensor4(k), as_tensor4(v), scores.data_ptr(),
                            ws.data_ptr(), ws.numel(), _stream()), "obc_score")
     return scores
+
+
+def obc_score_status(workspace) -> None:
+    """Synchronise and raise ObcError(OBC_ERR_TIMEOUT) if a bounded device-side wait gave up."""
+    _check(lib().obc_score_status(workspace.data_ptr(), _stream()), "obc_score_status")
 
 
 def select_params(scores, *, budget=0, budgets=None, idx_stride=None, seq_lens=None, n_sink=0, n_recent=0,

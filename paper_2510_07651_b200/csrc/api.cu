@@ -71,9 +71,9 @@ obc_status resolve_score(const obc_score_params* p, ScoreShape* s) {
 
 // which kernel family runs: decided from the parameters alone so that the size query and the
 // launch agree.  The dtype is not known to the size query, so the workspace covers both.
-bool want_tc(const obc_score_params* p, const ScoreShape& s, int dtype) {
+bool want_tc(const obc_score_params* p, const ScoreShape& s, int dtype, const TensorView& q) {
     if (p->path == OBC_PATH_SIMT) return false;
-    return tc_supported(s, dtype);
+    return tc_supported(s, dtype, q);
 }
 
 }  // namespace
@@ -88,8 +88,8 @@ obc_status obc_score_workspace(const obc_score_params* p, size_t* bytes) {
     ScoreShape s;
     obc_status st = resolve_score(p, &s);
     if (st != OBC_OK) return st;
-    size_t need = make_simt_plan(s).bytes;
-    if (p->path != OBC_PATH_SIMT && tc_supported(s, OBC_BF16)) {
+    size_t need = make_simt_plan(s, s.R, false).bytes;
+    if (p->path != OBC_PATH_SIMT && tc_shape_supported(s)) {
         size_t t = tc_workspace_bytes(s);
         if (t > need) need = t;
     }
@@ -112,11 +112,22 @@ obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_
     if ((st = obc_score_workspace(p, &need)) != OBC_OK) return st;
     if (!workspace || workspace_bytes < need) return OBC_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
-    const bool tc = want_tc(p, s, q.dtype);
+    const bool tc = want_tc(p, s, q.dtype, view(q));
     if (p->path == OBC_PATH_TC && !tc) return OBC_ERR_UNSUPPORTED;
     if (tc) return launch_score_tc(s, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);
-    return launch_score_simt(s, make_simt_plan(s), q.dtype, view(q), view(k), view(v), scores, workspace,
-                             (cudaStream_t)stream);
+    const SimtPlan plan = make_simt_plan(s, s.R, false);
+    OBC_CUDA_TRY(cudaMemsetAsync((char*)workspace + plan.off_flag, 0, 256, (cudaStream_t)stream));
+    st = launch_simt_pass1_combine(s, plan, q.dtype, view(q), view(k), view(v), workspace, (cudaStream_t)stream);
+    if (st != OBC_OK) return st;
+    return launch_simt_pass2(s, plan, q.dtype, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);
+}
+
+obc_status obc_score_status(const void* workspace, void* stream) {
+    if (!workspace) return OBC_ERR_NULL;
+    unsigned int word = 0;
+    OBC_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    OBC_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return word == 0 ? OBC_OK : OBC_ERR_TIMEOUT;
 }
 
 static obc_status resolve_select(const obc_select_params* p, SelectShape* s) {

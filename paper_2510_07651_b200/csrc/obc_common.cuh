@@ -46,13 +46,20 @@ struct ScoreShape {
 struct SimtPlan {
     int n_splits;                        // KV splits of pass 1
     int tiles_per_split;
+    int rows_out;                        // rows per unit in the combined arrays (R, or R padded)
+    int want_obf;                        // also write the bf16 copy of -2*O (tensor-core pass 2)
+    size_t off_flag;                             // 256-byte header: device status word
     size_t off_part_m, off_part_l, off_part_o;   // partial softmax stats / outputs per split
     size_t off_lse2, off_onorm, off_o;           // combined: log2-sum-exp, ||o||^2, O (fp32)
+    size_t off_obf;                              // bf16 [units][rows_out][d] = -2 * O
     size_t bytes;
 };
-SimtPlan make_simt_plan(const ScoreShape& s);
+SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf);
 
-obc_status launch_score_simt(const ScoreShape& s, const SimtPlan& plan, int dtype,
+// pass 1 + combine (window softmax statistics and outputs), then pass 2 (scores)
+obc_status launch_simt_pass1_combine(const ScoreShape& s, const SimtPlan& plan, int dtype,
+                                     TensorView q, TensorView k, TensorView v, void* ws, cudaStream_t stream);
+obc_status launch_simt_pass2(const ScoreShape& s, const SimtPlan& plan, int dtype,
                              TensorView q, TensorView k, TensorView v,
                              float* scores, void* ws, cudaStream_t stream);
 
@@ -82,7 +89,8 @@ obc_status launch_decode(const DecodeShape& s, TensorView q, TensorView kt, Tens
                          int step_pos, void* ws, cudaStream_t stream);
 
 // ---- tensor-core (tcgen05) score path -----------------------------------------------------------
-bool tc_supported(const ScoreShape& s, int dtype);
+bool tc_shape_supported(const ScoreShape& s);                       // R large enough for the MMA tiles
+bool tc_supported(const ScoreShape& s, int dtype, const TensorView& q);   // + bf16, uniformly strided Q rows
 size_t tc_workspace_bytes(const ScoreShape& s);
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
                            float* scores, void* ws, cudaStream_t stream);

@@ -163,10 +163,19 @@ simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
 }
 
 // ------------------------------------------------------------------------------------------ combine
-// one block of 128 threads per (unit, row): merge the splits
+// one block of 128 threads per (unit, output row): merge the splits.  Output rows >= R are padding
+// for the tensor-core pass: O = 0, ||o||^2 = 0 and log2-sum-exp = +inf, so that they weigh 0.
 __global__ void __launch_bounds__(128)
 simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
-    const int r = blockIdx.x % s.R, unit = blockIdx.x / s.R, c = threadIdx.x;
+    const int r = blockIdx.x % plan.rows_out, unit = blockIdx.x / plan.rows_out, c = threadIdx.x;
+    const size_t orow = (size_t)unit * plan.rows_out + r;
+    __nv_bfloat16* obf = plan.want_obf ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + plan.off_obf) : nullptr;
+    if (r >= s.R) {
+        (ws + plan.off_o / 4)[orow * kD + c] = 0.f;
+        if (obf) obf[orow * kD + c] = __float2bfloat16(0.f);
+        if (c == 0) { (ws + plan.off_lse2 / 4)[orow] = INFINITY; (ws + plan.off_onorm / 4)[orow] = 0.f; }
+        return;
+    }
     const float* part_m = ws + plan.off_part_m / 4;
     const float* part_l = ws + plan.off_part_l / 4;
     const float* part_o = ws + plan.off_part_o / 4;
@@ -187,11 +196,11 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     float sq = warp_sum(oc * oc);
     if ((c & 31) == 0) red[c >> 5] = sq;
     __syncthreads();
-    size_t row = (size_t)unit * s.R + r;
-    (ws + plan.off_o / 4)[row * kD + c] = oc;
+    (ws + plan.off_o / 4)[orow * kD + c] = oc;
+    if (obf) obf[orow * kD + c] = __float2bfloat16(-2.f * oc);
     if (c == 0) {
-        (ws + plan.off_lse2 / 4)[row] = M + log2f(L);
-        (ws + plan.off_onorm / 4)[row] = red[0] + red[1] + red[2] + red[3];
+        (ws + plan.off_lse2 / 4)[orow] = M + log2f(L);
+        (ws + plan.off_onorm / 4)[orow] = red[0] + red[1] + red[2] + red[3];
     }
 }
 
@@ -235,9 +244,9 @@ simt_pass2_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
     }
 
     const float sl2 = s.scale * kLog2e;
-    const float* o_all = ws + plan.off_o / 4 + (size_t)unit * s.R * kD;
-    const float* lse_all = ws + plan.off_lse2 / 4 + (size_t)unit * s.R;
-    const float* no_all = ws + plan.off_onorm / 4 + (size_t)unit * s.R;
+    const float* o_all = ws + plan.off_o / 4 + (size_t)unit * plan.rows_out * kD;
+    const float* lse_all = ws + plan.off_lse2 / 4 + (size_t)unit * plan.rows_out;
+    const float* no_all = ws + plan.off_onorm / 4 + (size_t)unit * plan.rows_out;
 
     float sv[2] = {0.f, 0.f}, sk[2] = {0.f, 0.f}, sx[2] = {0.f, 0.f}, sa[2] = {0.f, 0.f};
 
@@ -318,22 +327,29 @@ constexpr size_t kSmemPass1 = (size_t)(TN * KS + TN * kD + RC * kD + RC * TN) * 
 constexpr size_t kSmemPass2 = (size_t)(2 * TN * KS + 2 * RC * kD + TN + 2 * RC) * 4;
 
 template <typename T>
-obc_status launch_typed(const ScoreShape& s, const SimtPlan& plan, TensorView q, TensorView k, TensorView v,
-                        float* scores, float* ws, cudaStream_t stream) {
+obc_status launch_pass1_typed(const ScoreShape& s, const SimtPlan& plan, TensorView q, TensorView k, TensorView v,
+                              float* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv, chunks = (s.R + RC - 1) / RC;
     OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass1_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass1));
-    OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass2_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass2));
     { ProfScope ps("simt_pass1", stream); simt_pass1_kernel<T><<<dim3(plan.n_splits, units, chunks), NT, kSmemPass1, stream>>>(s, plan, q, k, v, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
-    { ProfScope ps("simt_combine", stream); simt_combine_kernel<<<units * s.R, 128, 0, stream>>>(s, plan, ws); }
+    { ProfScope ps("simt_combine", stream); simt_combine_kernel<<<units * plan.rows_out, 128, 0, stream>>>(s, plan, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
+    return OBC_OK;
+}
+
+template <typename T>
+obc_status launch_pass2_typed(const ScoreShape& s, const SimtPlan& plan, TensorView q, TensorView k, TensorView v,
+                              float* scores, float* ws, cudaStream_t stream) {
+    const int units = s.B * s.Hkv;
+    OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass2_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass2));
     { ProfScope ps("simt_pass2", stream); simt_pass2_kernel<T><<<dim3((s.Nmax + TN - 1) / TN, units), NT, kSmemPass2, stream>>>(s, plan, q, k, v, ws, scores); }
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
 }  // namespace
 
-SimtPlan make_simt_plan(const ScoreShape& s) {
+SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
     SimtPlan p{};
     const int units = s.B * s.Hkv, chunks = (s.R + RC - 1) / RC;
     const int tiles = (s.Nmax + TN - 1) / TN;
@@ -345,22 +361,32 @@ SimtPlan make_simt_plan(const ScoreShape& s) {
     if (n < 1) n = 1;
     p.tiles_per_split = (tiles + n - 1) / n;
     p.n_splits = (tiles + p.tiles_per_split - 1) / p.tiles_per_split;
-    size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, off = 0;
+    p.rows_out = rows_out;
+    p.want_obf = want_obf ? 1 : 0;
+    size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, orow = (size_t)units * rows_out, off = 0;
+    p.off_flag = off;   off = 256;
     p.off_part_m = off; off = align_up(off + prow * 4, 256);
     p.off_part_l = off; off = align_up(off + prow * 4, 256);
     p.off_part_o = off; off = align_up(off + prow * kD * 4, 256);
-    p.off_lse2 = off;   off = align_up(off + rows * 4, 256);
-    p.off_onorm = off;  off = align_up(off + rows * 4, 256);
-    p.off_o = off;      off = align_up(off + rows * kD * 4, 256);
+    p.off_lse2 = off;   off = align_up(off + orow * 4, 256);
+    p.off_onorm = off;  off = align_up(off + orow * 4, 256);
+    p.off_o = off;      off = align_up(off + orow * kD * 4, 256);
+    p.off_obf = off;    off = align_up(off + (want_obf ? orow * kD * 2 : 0), 1024);
     p.bytes = off;
     return p;
 }
 
-obc_status launch_score_simt(const ScoreShape& s, const SimtPlan& plan, int dtype,
+obc_status launch_simt_pass1_combine(const ScoreShape& s, const SimtPlan& plan, int dtype,
+                                     TensorView q, TensorView k, TensorView v, void* ws, cudaStream_t stream) {
+    if (dtype == OBC_F32) return launch_pass1_typed<float>(s, plan, q, k, v, (float*)ws, stream);
+    return launch_pass1_typed<__nv_bfloat16>(s, plan, q, k, v, (float*)ws, stream);
+}
+
+obc_status launch_simt_pass2(const ScoreShape& s, const SimtPlan& plan, int dtype,
                              TensorView q, TensorView k, TensorView v,
                              float* scores, void* ws, cudaStream_t stream) {
-    if (dtype == OBC_F32) return launch_typed<float>(s, plan, q, k, v, scores, (float*)ws, stream);
-    return launch_typed<__nv_bfloat16>(s, plan, q, k, v, scores, (float*)ws, stream);
+    if (dtype == OBC_F32) return launch_pass2_typed<float>(s, plan, q, k, v, scores, (float*)ws, stream);
+    return launch_pass2_typed<__nv_bfloat16>(s, plan, q, k, v, scores, (float*)ws, stream);
 }
 
 }  // namespace obc

@@ -58,7 +58,10 @@ def oracle_scores(case, variants, causal=True):
 def gpu_scores(case, variants, causal=True, path="auto"):
     q, k, v = upload(case)
     order = [n for n in ("V", "K", "VK", "ATTN") if n in variants]
-    s = api.obc_score(q, k, v, seq_lens=lens_dev(case), causal=causal, variants=order, path=path)
+    p = api.score_params(q, k, seq_lens=lens_dev(case), causal=causal, variants=order, path=path)
+    ws = torch.empty(api.obc_score_workspace(p), dtype=torch.uint8, device="cuda")
+    s = api.obc_score(q, k, v, seq_lens=lens_dev(case), causal=causal, variants=order, path=path, workspace=ws)
+    api.obc_score_status(ws)
     torch.cuda.synchronize()
     s = s.cpu().numpy()
     return {n: s[i] for i, n in enumerate(order)}
