@@ -59,6 +59,7 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf);
 // pass 1 + combine (window softmax statistics and outputs), then pass 2 (scores)
 obc_status launch_simt_pass1_combine(const ScoreShape& s, const SimtPlan& plan, int dtype,
                                      TensorView q, TensorView k, TensorView v, void* ws, cudaStream_t stream);
+obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream);
 obc_status launch_simt_pass2(const ScoreShape& s, const SimtPlan& plan, int dtype,
                              TensorView q, TensorView k, TensorView v,
                              float* scores, void* ws, cudaStream_t stream);

@@ -333,9 +333,7 @@ obc_status launch_pass1_typed(const ScoreShape& s, const SimtPlan& plan, TensorV
     OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass1_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass1));
     { ProfScope ps("simt_pass1", stream); simt_pass1_kernel<T><<<dim3(plan.n_splits, units, chunks), NT, kSmemPass1, stream>>>(s, plan, q, k, v, ws); }
     OBC_CUDA_TRY(cudaGetLastError());
-    { ProfScope ps("simt_combine", stream); simt_combine_kernel<<<units * plan.rows_out, 128, 0, stream>>>(s, plan, ws); }
-    OBC_CUDA_TRY(cudaGetLastError());
-    return OBC_OK;
+    return launch_combine(s, plan, ws, stream);
 }
 
 template <typename T>
@@ -374,6 +372,12 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
     p.off_obf = off;    off = align_up(off + (want_obf ? orow * kD * 2 : 0), 1024);
     p.bytes = off;
     return p;
+}
+
+obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream) {
+    { ProfScope ps("combine", stream); simt_combine_kernel<<<s.B * s.Hkv * plan.rows_out, 128, 0, stream>>>(s, plan, (float*)ws); }
+    OBC_CUDA_TRY(cudaGetLastError());
+    return OBC_OK;
 }
 
 obc_status launch_simt_pass1_combine(const ScoreShape& s, const SimtPlan& plan, int dtype,

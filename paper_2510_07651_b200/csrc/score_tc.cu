@@ -146,7 +146,8 @@ struct TcParams {
     unsigned int* status;                     // device status word (workspace header)
 };
 
-__device__ __forceinline__ int tc_seq_len(const TcParams& p, int b) { return p.seq_lens ? p.seq_lens[b] : p.Nmax; }
+__device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
+__device__ __forceinline__ int tc_seq_len(const TcParams& p, int b) { return tc_seq_len_raw(p.seq_lens, b, p.Nmax); }
 
 // VARS: variants this instantiation computes (a superset of p.variants)
 template <unsigned VARS>
@@ -409,6 +410,296 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
 }
 
+// =================================================================================================
+// Pass 1 on tensor cores: streaming softmax statistics and window outputs (Sec. 3: A = softmax(Z),
+// O = A V over the perturbation window, Eq. 9), split over the cached tokens.
+//
+// Rows of the window (one chunk of up to 128) sit on the MMA M dimension, so a TMEM lane holds one
+// row and the softmax thread that owns it reduces along the tile without cross-thread traffic:
+//     S   = Q_chunk . K_tile^T                     (tcgen05, accumulators double-buffered in TMEM)
+//     P   = exp2(S * scale*log2e - m_used)         (registers -> bf16 -> swizzled shared memory)
+//     O  += P . V_tile                             (tcgen05, V read as an MN-major B operand)
+// m_used is the exponent reference of the row; it is only moved up (and O, l rescaled) when the
+// running maximum exceeds it by more than 8 (a factor 256), which keeps P within bf16/fp32 range.
+// Each CTA writes (m_used, l, O) of its token split; the combine kernel merges the splits.
+//
+//   warp 0      TMA producer (Q chunk once, K/V tiles into a 2-stage ring)
+//   warp 1      MMA issuer
+//   warps 4-7   softmax (thread = row)
+// =================================================================================================
+constexpr int kThreadsP1 = 256;
+constexpr uint32_t P1_OFF_Q = 0;
+constexpr uint32_t P1_OFF_P = P1_OFF_Q + kOperandBytes;
+constexpr uint32_t P1_OFF_K = P1_OFF_P + kOperandBytes;
+constexpr uint32_t P1_OFF_V = P1_OFF_K + NSTAGE * kOperandBytes;
+constexpr uint32_t P1_OFF_BAR = P1_OFF_V + NSTAGE * kOperandBytes;
+enum { P1_FULL = 0, P1_EMPTY = 2, P1_QFULL = 4, P1_SFULL = 5, P1_SEMPTY = 7, P1_PFULL = 9, P1_PVDONE = 10, P1_NBARS = 11 };
+constexpr uint32_t P1_OFF_TMEM = P1_OFF_BAR + P1_NBARS * 8;
+constexpr uint32_t kSmemP1 = P1_OFF_TMEM + 16 + 1024;
+constexpr float kRescaleThreshold = 8.f;                   // log2 units
+
+struct P1Params {
+    int B, Hq, Hkv, G, W, R, Nmax;
+    const int32_t* seq_lens;
+    float scale;
+    int causal;
+    int n_chunks, chunk_rows;
+    int n_splits, tiles_per_split;
+    float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
+    unsigned int* status;
+};
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// MN-major B operand with 128-byte swizzle: 64 contiguous elements of N per 128-byte row, 8 rows of
+// K per 1024-byte group (stride byte offset), the next 64 elements of N one 16 KB block further
+// (leading byte offset).  This is the image of a [tokens][head_dim] tile loaded as two 64-wide boxes.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)(kHalfBytes >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreadsP1, 1)
+tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, P1Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + P1_OFF_BAR;
+    auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + P1_OFF_TMEM);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const int split = blockIdx.x, vu = blockIdx.y;
+    const int unit = vu / p.n_chunks, c = vu % p.n_chunks;
+    const int b = unit / p.Hkv, g = unit % p.Hkv;
+    const int N = tc_seq_len_raw(p.seq_lens, b, p.Nmax);
+    const int tile_lo = split * p.tiles_per_split;
+    const int tile_hi = min(tile_lo + p.tiles_per_split, (N + TILE - 1) / TILE);
+    const int n_tiles = max(tile_hi - tile_lo, 0);
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), 1); }
+        mbar_init(bar(P1_QFULL), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(P1_SFULL + i), 1); mbar_init(bar(P1_SEMPTY + i), 4); }
+        mbar_init(bar(P1_PFULL), 4); mbar_init(bar(P1_PVDONE), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + P1_OFF_TMEM), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base + 256u;
+    bool failed = false;
+
+    if (warp == 0) {
+        if (lane == 0 && n_tiles > 0) {
+            mbar_expect_tx(bar(P1_QFULL), (uint32_t)p.chunk_rows * 256u);
+            const int qrow = (b * p.Hq + g * p.G) * p.W + c * p.chunk_rows;
+            tma_load_2d(sbase + P1_OFF_Q, &map_q, bar(P1_QFULL), 0, qrow);
+            tma_load_2d(sbase + P1_OFF_Q + kHalfBytes, &map_q, bar(P1_QFULL), 64, qrow);
+            int issued = 0;
+            for (int i = 0; i < n_tiles; ++i) {
+                const uint32_t st = i % NSTAGE;
+                if (!mbar_wait(bar(P1_EMPTY + st), ((i / NSTAGE) & 1) ^ 1)) { failed = true; break; }
+                mbar_expect_tx(bar(P1_FULL + st), 2 * kOperandBytes);
+                const uint32_t dk = sbase + P1_OFF_K + st * kOperandBytes, dv = sbase + P1_OFF_V + st * kOperandBytes;
+                const int t0 = (tile_lo + i) * TILE;
+                tma_load_4d(dk, &map_k, bar(P1_FULL + st), 0, t0, g, b);
+                tma_load_4d(dk + kHalfBytes, &map_k, bar(P1_FULL + st), 64, t0, g, b);
+                tma_load_4d(dv, &map_v, bar(P1_FULL + st), 0, t0, g, b);
+                tma_load_4d(dv + kHalfBytes, &map_v, bar(P1_FULL + st), 64, t0, g, b);
+                ++issued;
+            }
+            for (int back = 0; back < NSTAGE && back < issued; ++back) {      // drain own copies
+                const int it = issued - 1 - back;
+                (void)mbar_wait(bar(P1_FULL + it % NSTAGE), (it / NSTAGE) & 1);
+            }
+            (void)mbar_wait(bar(P1_QFULL), 0);
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && n_tiles > 0) {
+            const uint32_t idesc_s = idesc_bf16(TILE);
+            const uint32_t idesc_pv = idesc_bf16(kD) | (1u << 16);           // B operand (V) is MN-major
+            auto issue_s = [&](int j) -> bool {
+                const uint32_t st = j % NSTAGE;
+                if (!mbar_wait(bar(P1_FULL + st), (j / NSTAGE) & 1)) return false;
+                if (!mbar_wait(bar(P1_SEMPTY + (j & 1)), ((j >> 1) & 1) ^ 1)) return false;
+                tc_fence_after();
+                const uint32_t ak = sbase + P1_OFF_K + st * kOperandBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                    tc_mma(tmem_base + (j & 1) * 128u, smem_desc_k_sw128(sbase + P1_OFF_Q + off), smem_desc_k_sw128(ak + off), idesc_s, ks > 0);
+                }
+                tc_commit(bar(P1_SFULL + (j & 1)));
+                return true;
+            };
+            failed = !mbar_wait(bar(P1_QFULL), 0);
+            if (!failed) failed = !issue_s(0);
+            for (int i = 0; i < n_tiles && !failed; ++i) {
+                if (i + 1 < n_tiles && !issue_s(i + 1)) { failed = true; break; }
+                if (!mbar_wait(bar(P1_PFULL), i & 1)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t av = sbase + P1_OFF_V + (i % NSTAGE) * kOperandBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {                             // 128 tokens = 8 steps of K = 16
+                    const uint32_t offp = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                    tc_mma(tmem_o, smem_desc_k_sw128(sbase + P1_OFF_P + offp), smem_desc_mn_sw128(av + ks * 2048), idesc_pv, (i > 0) || (ks > 0));
+                }
+                tc_commit(bar(P1_PVDONE));
+                tc_commit(bar(P1_EMPTY + (i % NSTAGE)));
+            }
+        }
+    } else if (warp >= 4) {
+        const int lane_grp = warp & 3;
+        const int row = lane_grp * 32 + lane;                                // row within the chunk
+        const int rows_valid = min(p.chunk_rows, p.R - c * p.chunk_rows);
+        const int r = c * p.chunk_rows + row;
+        const bool valid = row < rows_valid;
+        const int last = valid ? (p.causal ? N - p.W + (r % p.W) : N - 1) : -1;
+        const float sl2 = p.scale * kLog2e;
+        const uint32_t lane_addr = (uint32_t)(lane_grp * 32) << 16;
+        float m_used = -INFINITY, l = 0.f;
+        uint8_t* prow = smem + P1_OFF_P + row * 128;
+
+        for (int i = 0; i < n_tiles && !failed; ++i) {
+            const uint32_t buf = i & 1;
+            const int t0 = (tile_lo + i) * TILE;
+            if (!mbar_wait(bar(P1_SFULL + buf), (i >> 1) & 1)) { failed = true; break; }
+            tc_fence_after();
+            float sv[128];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tmem_base + lane_addr + buf * 128u + q4 * 32, reinterpret_cast<uint32_t*>(sv) + q4 * 32);
+            tc_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P1_SEMPTY + buf));
+
+            float mt = -INFINITY;
+            const int nvis = last - t0 + 1;                                  // columns j < nvis are visible
+#pragma unroll
+            for (int j = 0; j < 128; ++j) {
+                sv[j] = j < nvis ? sv[j] * sl2 : -INFINITY;
+                mt = fmaxf(mt, sv[j]);
+            }
+            const bool need = mt > m_used + kRescaleThreshold;               // also true for the first visible tile
+            const float factor = need ? fast_exp2(m_used - mt) : 1.f;        // m_used = -inf -> 0
+            if (i > 0) {
+                const bool any = __any_sync(0xffffffffu, need && m_used != -INFINITY);
+                if (!mbar_wait(bar(P1_PVDONE), (i - 1) & 1)) { failed = true; break; }   // P buffer free, O stable
+                if (any) {
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t ov[32];
+                        tc_ld32(tmem_o + lane_addr + q4 * 32, ov);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
+                        tc_st32(tmem_o + lane_addr + q4 * 32, ov);
+                    }
+                    tc_wait_st();
+                    tc_fence_before();
+                }
+            }
+            l *= factor;
+            if (need) m_used = mt;
+            const float m_eff = m_used == -INFINITY ? 0.f : m_used;
+            float lsum = 0.f;
+#pragma unroll
+            for (int ch = 0; ch < 16; ++ch) {                                // 16 chunks of 8 tokens = 16 bytes of bf16
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float p0 = fast_exp2(sv[ch * 8 + 2 * e] - m_eff), p1 = fast_exp2(sv[ch * 8 + 2 * e + 1] - m_eff);
+                    lsum += p0 + p1;
+                    w[e] = pack_bf16x2(p0, p1);
+                }
+                *reinterpret_cast<uint4*>(prow + (ch >> 3) * kHalfBytes + (((ch & 7) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            l += lsum;
+            if (t0 + TILE > N && t0 + row >= N) {                            // tail: V rows past the sequence must not reach the MMA
+                uint8_t* vrow = smem + P1_OFF_V + (i % NSTAGE) * kOperandBytes + row * 128;
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) {
+                    *reinterpret_cast<uint4*>(vrow + (ch << 4)) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(vrow + kHalfBytes + (ch << 4)) = make_uint4(0, 0, 0, 0);
+                }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(P1_PFULL));
+        }
+
+        // partial results of this split
+        const size_t prow_idx = ((size_t)unit * p.n_splits + split) * p.R + r;
+        if (n_tiles > 0 && !failed) {
+            if (!mbar_wait(bar(P1_PVDONE), (n_tiles - 1) & 1)) failed = true;
+            tc_fence_after();
+#pragma unroll 1
+            for (int q4 = 0; q4 < 4 && !failed; ++q4) {
+                uint32_t ov[32];
+                tc_ld32(tmem_o + lane_addr + q4 * 32, ov);
+                tc_wait_ld();
+                if (valid) {
+                    float4* dst = reinterpret_cast<float4*>(p.part_o + prow_idx * kD + q4 * 32);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        dst[j] = make_float4(__uint_as_float(ov[4 * j]), __uint_as_float(ov[4 * j + 1]),
+                                             __uint_as_float(ov[4 * j + 2]), __uint_as_float(ov[4 * j + 3]));
+                }
+            }
+            tc_fence_before();
+        } else if (valid) {
+            float4* dst = reinterpret_cast<float4*>(p.part_o + prow_idx * kD);
+            for (int j = 0; j < 32; ++j) dst[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (valid) { p.part_m[prow_idx] = m_used; p.part_l[prow_idx] = l; }
+    }
+
+    if (failed) atomicExch(p.status, 1u);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
 // ---- host side ----------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled get_encode() {
     static PFN_cuTensorMapEncodeTiled fn = nullptr;
@@ -463,17 +754,42 @@ bool tc_supported(const ScoreShape& s, int dtype, const TensorView& q) {
     return q.sh == (long long)s.W * q.st && q.sb == (long long)s.Hq * q.sh;
 }
 
-size_t tc_workspace_bytes(const ScoreShape& s) { return make_simt_plan(s, tc_chunks(s.R).rows_out, true).bytes; }
+// Workspace plan of the tensor-core path: the SIMT plan's layout with splits counted in 128-token tiles.
+static SimtPlan make_tc_plan(const ScoreShape& s) {
+    const TcChunks ch = tc_chunks(s.R);
+    const int units = s.B * s.Hkv, vus = units * ch.n_chunks;
+    const int tiles = (s.Nmax + TILE - 1) / TILE;
+    int n = sm_count() / vus;                          // one wave of CTAs when the sequences are equal
+    if (s.seq_lens) { const int cap = (tiles + 31) / 32; if (cap > n) n = cap; }   // ragged: bound the work per CTA
+    if (n < 1) n = 1;
+    if (n > tiles) n = tiles;
+    SimtPlan p{};
+    p.tiles_per_split = (tiles + n - 1) / n;
+    p.n_splits = (tiles + p.tiles_per_split - 1) / p.tiles_per_split;
+    p.rows_out = ch.rows_out;
+    p.want_obf = 1;
+    const size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, orow = (size_t)units * ch.rows_out;
+    size_t off = 0;
+    p.off_flag = off;   off = 256;
+    p.off_part_m = off; off = align_up(off + prow * 4, 256);
+    p.off_part_l = off; off = align_up(off + prow * 4, 256);
+    p.off_part_o = off; off = align_up(off + prow * kD * 4, 256);
+    p.off_lse2 = off;   off = align_up(off + orow * 4, 256);
+    p.off_onorm = off;  off = align_up(off + orow * 4, 256);
+    p.off_o = off;      off = align_up(off + orow * kD * 4, 256);
+    p.off_obf = off;    off = align_up(off + orow * kD * 2, 1024);
+    p.bytes = off;
+    return p;
+}
+
+size_t tc_workspace_bytes(const ScoreShape& s) { return make_tc_plan(s).bytes; }
 
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
                            float* scores, void* ws, cudaStream_t stream) {
     const TcChunks ch = tc_chunks(s.R);
-    const SimtPlan plan = make_simt_plan(s, ch.rows_out, true);
+    const SimtPlan plan = make_tc_plan(s);
     char* wsb = (char*)ws;
     OBC_CUDA_TRY(cudaMemsetAsync(wsb + plan.off_flag, 0, 256, stream));
-    obc_status st = launch_simt_pass1_combine(s, plan, OBC_BF16, q, k, v, ws, stream);
-    if (st != OBC_OK) return st;
-
     const int units = s.B * s.Hkv;
     CUtensorMap mq, mo, mk, mv;
     {
@@ -492,6 +808,22 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
             set_last_cuda_error((int)cudaErrorInvalidValue);
             return OBC_ERR_CUDA;
         }
+    }
+    {   // pass 1 + combine
+        P1Params p1{};
+        p1.B = s.B; p1.Hq = s.Hq; p1.Hkv = s.Hkv; p1.G = s.G; p1.W = s.W; p1.R = s.R; p1.Nmax = s.Nmax;
+        p1.seq_lens = s.seq_lens; p1.scale = s.scale; p1.causal = s.causal;
+        p1.n_chunks = ch.n_chunks; p1.chunk_rows = ch.chunk_rows;
+        p1.n_splits = plan.n_splits; p1.tiles_per_split = plan.tiles_per_split;
+        p1.part_m = (float*)(wsb + plan.off_part_m); p1.part_l = (float*)(wsb + plan.off_part_l);
+        p1.part_o = (float*)(wsb + plan.off_part_o);
+        p1.status = (unsigned int*)(wsb + plan.off_flag);
+        OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
+        { ProfScope ps("tc_pass1", stream);
+          tc_pass1_kernel<<<dim3(plan.n_splits, units * ch.n_chunks), kThreadsP1, kSmemP1, stream>>>(mq, mk, mv, p1); }
+        OBC_CUDA_TRY(cudaGetLastError());
+        obc_status st = launch_combine(s, plan, ws, stream);
+        if (st != OBC_OK) return st;
     }
     TcParams p{};
     p.B = s.B; p.Hkv = s.Hkv; p.G = s.G; p.W = s.W; p.R = s.R; p.Nmax = s.Nmax; p.seq_lens = s.seq_lens;
