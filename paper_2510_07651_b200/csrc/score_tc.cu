@@ -139,7 +139,6 @@ struct TcParams {
     int causal;
     unsigned variants;
     int n_chunks, chunk_rows, rows_out;       // rows_out = n_chunks * chunk_rows
-    int tiles_per_unit;
     const float* lse2;                        // [units][rows_out]
     const float* onorm;                       // [units][rows_out]
     float* scores;                            // [planes][units][Nmax]
@@ -149,12 +148,125 @@ struct TcParams {
 __device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
 __device__ __forceinline__ int tc_seq_len(const TcParams& p, int b) { return tc_seq_len_raw(p.seq_lens, b, p.Nmax); }
 
+// Walks the CTA's share of the token tiles.  All non-empty 128-token tiles of all (batch item,
+// KV head) units, in (unit, tile) order, are cut into gridDim.x contiguous, equally long runs, so
+// that a CTA stays inside one unit for as long as possible (its Q / O operands stay in shared
+// memory) and ragged batches are balanced.  Every role of the CTA runs its own copy.
+struct TileWalk {
+    int unit, tile, tiles_in_unit;            // current position
+    long long left;                           // tiles still to visit, including the current one
+    const TcParams* p;
+    __device__ __forceinline__ int tiles_of(int b) const { return (tc_seq_len(*p, b) + TILE - 1) / TILE; }
+    __device__ void init(const TcParams& prm) {
+        p = &prm;
+        long long total = 0;
+        if (p->seq_lens) { for (int b = 0; b < p->B; ++b) total += (long long)p->Hkv * tiles_of(b); }
+        else total = (long long)p->B * p->Hkv * ((p->Nmax + TILE - 1) / TILE);
+        const long long lo = total * blockIdx.x / gridDim.x, hi = total * (blockIdx.x + 1) / gridDim.x;
+        left = hi - lo;
+        unit = 0; tile = 0; tiles_in_unit = 0;
+        if (left <= 0) return;
+        long long skip = lo;
+        int b = 0;
+        for (; b < p->B; ++b) {
+            const long long blk = (long long)p->Hkv * tiles_of(b);
+            if (skip < blk) break;
+            skip -= blk;
+        }
+        tiles_in_unit = tiles_of(b);
+        unit = b * p->Hkv + (int)(skip / tiles_in_unit);
+        tile = (int)(skip % tiles_in_unit);
+    }
+    __device__ __forceinline__ bool done() const { return left <= 0; }
+    __device__ __forceinline__ void next() {
+        --left;
+        if (++tile < tiles_in_unit || left <= 0) return;
+        tile = 0;
+        do { ++unit; tiles_in_unit = tiles_of(unit / p->Hkv); } while (tiles_in_unit == 0);
+    }
+};
+
+__device__ __forceinline__ float2 bf16x2_to_f32x2(uint32_t w) {
+    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+// waits for the TMEM loads of this thread; the registers are operands so that no use is moved above it
+__device__ __forceinline__ void tc_wait_ld16x2(uint32_t (&a)[16], uint32_t (&b)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                   "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
+                   "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+                   "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15])
+                 :: "memory");
+}
+
+// Running sums of one token over the window rows, two rows per packed fp32x2 lane.  With
+// a = A_rp, u = a z (z the unscaled logit), b = a + scale u = a (1 + Z):
+//   Eq. 6   sum_r a^2 ||(1+Z) v - Z o_r||^2 = |v|^2 S1 + scale S2 + scale^2 S3
+//   Eq. 5   sum_r a^2 Z^2 ||v - o_r||^2     = scale^2 (|v|^2 S5 + S3 + S4)
+//   Eq. 4   |v|^2 S6;   attention-only: S7
+// with S1 = sum b^2, S2 = sum u b t', S3 = sum u^2 |o_r|^2, S4 = sum u^2 t', S5 = sum u^2,
+// S6 = sum a^2, S7 = sum a and t' = -2 v.o_r (the expanded norms of Algorithm 1).
+struct RowSums { float2 s1, s2, s3, s4, s5, s6, s7; };
+
+// 16 rows of one token: zr = logits, tr = -2 v.o_r, cst = per row pair (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
+template <unsigned VARS, bool MASKED>
+__device__ __forceinline__ void score_rows16(const uint32_t (&zr)[16], const uint32_t (&tr)[16], const float4* cst,
+                                             float2 sl2, float2 sc, RowSums& S, int ptok, int mask_base, int W, int& wi) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float4 cp = cst[i];
+        const float2 z = make_float2(__uint_as_float(zr[2 * i]), __uint_as_float(zr[2 * i + 1]));
+        const float2 t2 = make_float2(__uint_as_float(tr[2 * i]), __uint_as_float(tr[2 * i + 1]));
+        float2 e = __ffma2_rn(z, sl2, make_float2(cp.x, cp.y));
+        if (MASKED) {                                   // row r sees tokens p <= N - W + (r mod W)
+            if (ptok > mask_base + wi) e.x = -INFINITY;
+            wi = wi + 1 == W ? 0 : wi + 1;
+            if (ptok > mask_base + wi) e.y = -INFINITY;
+            wi = wi + 1 == W ? 0 : wi + 1;
+        }
+        const float2 a = make_float2(fast_exp2(e.x), fast_exp2(e.y));
+        const float2 u = __fmul2_rn(a, z);
+        if (VARS & OBC_VAR_VK) {
+            const float2 b = __ffma2_rn(u, sc, a);
+            S.s1 = __ffma2_rn(b, b, S.s1);
+            S.s2 = __ffma2_rn(__fmul2_rn(u, b), t2, S.s2);
+        }
+        if (VARS & (OBC_VAR_VK | OBC_VAR_K)) {
+            const float2 uu = __fmul2_rn(u, u);
+            S.s3 = __ffma2_rn(uu, make_float2(cp.z, cp.w), S.s3);
+            if (VARS & OBC_VAR_K) { S.s4 = __ffma2_rn(uu, t2, S.s4); S.s5 = __fadd2_rn(uu, S.s5); }
+        }
+        if (VARS & OBC_VAR_V) S.s6 = __ffma2_rn(a, a, S.s6);
+        if (VARS & OBC_VAR_ATTN) S.s7 = __fadd2_rn(a, S.s7);
+    }
+}
+
+// one (tile, chunk) item of one token: all rows of the chunk, TMEM loads one batch ahead of the math
+template <unsigned VARS, bool MASKED>
+__device__ __forceinline__ void score_chunk(uint32_t zt, uint32_t tt, int chunk_rows, const float4* cst,
+                                            float2 sl2, float2 sc, RowSums& S, int ptok, int mask_base, int W, int wi) {
+    uint32_t z0[16], t0[16], z1[16], t1[16];
+    tc_ld16(zt, z0);
+    tc_ld16(tt, t0);
+    for (int c0 = 0; c0 < chunk_rows; c0 += 32) {
+        tc_wait_ld16x2(z0, t0);
+        const bool second = c0 + 16 < chunk_rows;
+        if (second) { tc_ld16(zt + c0 + 16, z1); tc_ld16(tt + c0 + 16, t1); }
+        score_rows16<VARS, MASKED>(z0, t0, cst + (c0 >> 1), sl2, sc, S, ptok, mask_base, W, wi);
+        if (second) {
+            tc_wait_ld16x2(z1, t1);
+            if (c0 + 32 < chunk_rows) { tc_ld16(zt + c0 + 32, z0); tc_ld16(tt + c0 + 32, t0); }
+            score_rows16<VARS, MASKED>(z1, t1, cst + (c0 >> 1) + 8, sl2, sc, S, ptok, mask_base, W, wi);
+        }
+    }
+}
+
 // VARS: variants this instantiation computes (a superset of p.variants)
 template <unsigned VARS>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
                 const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                TcParams p) {
+                const __grid_constant__ TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -162,11 +274,10 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_TMEM);
     float* sNv = reinterpret_cast<float*>(smem + OFF_NV);
-    float2* sConst = reinterpret_cast<float2*>(smem + OFF_CONST);
+    float* sConst = reinterpret_cast<float*>(smem + OFF_CONST);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int units = p.B * p.Hkv;
-    const long long n_tiles = (long long)units * p.tiles_per_unit;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 3); }
@@ -188,19 +299,18 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const bool reload_qo_every_item = p.n_chunks > 1;
     const uint32_t qo_bytes = (uint32_t)p.chunk_rows * 128u * 2u * 2u;   // Q and O chunks, two halves each
 
-    // Every role walks the same list: tiles L = blockIdx.x + i * gridDim.x, L -> (unit, tile);
-    // for each non-empty tile, chunks c = 0 .. n_chunks-1.  `item` counts (tile, chunk) pairs that
-    // are actually processed and indexes the smem stage / TMEM buffer / constant slot rings.
+    // Every role walks the same tiles (TileWalk) and, per tile, the chunks c = 0 .. n_chunks-1.
+    // `item` counts the (tile, chunk) pairs processed so far and indexes the smem stage, TMEM
+    // buffer and constant-slot rings.
+    TileWalk tw;
+    tw.init(p);
     if (warp == 0) {
         // ===================================== TMA producer =====================================
         if (lane == 0) {
             uint32_t item = 0, qo_loads = 0;
             int qo_unit = -1;
-            for (long long L = blockIdx.x; L < n_tiles && !failed; L += gridDim.x) {
-                const int unit = (int)(L / p.tiles_per_unit), tile = (int)(L % p.tiles_per_unit);
-                const int b = unit / p.Hkv, g = unit % p.Hkv;
-                const int t0 = tile * TILE;
-                if (t0 >= tc_seq_len(p, b)) continue;
+            for (; !tw.done() && !failed; tw.next()) {
+                const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv, t0 = tw.tile * TILE;
                 for (int c = 0; c < p.n_chunks; ++c, ++item) {
                     if (reload_qo_every_item || unit != qo_unit) {
                         if (!mbar_wait(bar(BAR_QO_EMPTY), (qo_loads & 1) ^ 1)) { failed = true; break; }
@@ -236,10 +346,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const uint32_t idesc = idesc_bf16(p.chunk_rows);
             uint32_t item = 0, qo_loads = 0;
             int qo_unit = -1;
-            for (long long L = blockIdx.x; L < n_tiles && !failed; L += gridDim.x) {
-                const int unit = (int)(L / p.tiles_per_unit), tile = (int)(L % p.tiles_per_unit);
-                const int b = unit / p.Hkv;
-                if (tile * TILE >= tc_seq_len(p, b)) continue;
+            for (; !tw.done() && !failed; tw.next()) {
+                const int unit = tw.unit;
                 for (int c = 0; c < p.n_chunks; ++c, ++item) {
                     const bool new_qo = reload_qo_every_item || unit != qo_unit;
                     if (new_qo) {
@@ -265,16 +373,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     tc_commit(bar(BAR_TM_FULL + buf));             // accumulators ready for the epilogue
                     tc_commit(bar(BAR_EMPTY + st));                // K/V stage no longer read by the MMA
                     // Q / O may be overwritten once these MMAs are done, if the next item needs others
-                    bool next_needs_qo = reload_qo_every_item;
-                    if (!next_needs_qo) {
-                        long long Ln = L + gridDim.x;
-                        while (Ln < n_tiles) {
-                            const int un = (int)(Ln / p.tiles_per_unit), tn = (int)(Ln % p.tiles_per_unit);
-                            if (tn * TILE < tc_seq_len(p, un / p.Hkv)) { next_needs_qo = un != unit; break; }
-                            Ln += gridDim.x;
-                        }
-                    }
-                    if (next_needs_qo) tc_commit(bar(BAR_QO_EMPTY));
+                    const bool last_of_unit = tw.left > 1 && tw.tile + 1 == tw.tiles_in_unit && c + 1 == p.n_chunks;
+                    if (reload_qo_every_item || last_of_unit) tc_commit(bar(BAR_QO_EMPTY));
                 }
             }
         }
@@ -282,10 +382,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // ============================ ||v_p||^2 and per-row constants ===========================
         const int t64 = threadIdx.x - 64;                          // 0..63
         uint32_t item = 0;
-        for (long long L = blockIdx.x; L < n_tiles && !failed; L += gridDim.x) {
-            const int unit = (int)(L / p.tiles_per_unit), tile = (int)(L % p.tiles_per_unit);
-            const int b = unit / p.Hkv;
-            if (tile * TILE >= tc_seq_len(p, b)) continue;
+        for (; !tw.done() && !failed; tw.next()) {
+            const int unit = tw.unit;
             for (int c = 0; c < p.n_chunks; ++c, ++item) {
                 const uint32_t st = item % NSTAGE, slot = item % NSLOT;
                 // constants first (global loads overlap the wait for the tile)
@@ -294,29 +392,30 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
                     const int r = t64 + 64 * j;
-                    cst[j] = r < p.chunk_rows ? make_float2(p.lse2[crow + r], p.onorm[crow + r]) : make_float2(INFINITY, 0.f);
+                    cst[j] = r < p.chunk_rows ? make_float2(-p.lse2[crow + r], p.onorm[crow + r]) : make_float2(-INFINITY, 0.f);
                 }
                 if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; break; }
                 const uint8_t* vt = smem + OFF_V + st * kOperandBytes;
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
                     const int tok = t64 + 64 * j;
-                    float acc = 0.f;
+                    float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int ch = 0; ch < 8; ++ch) {
                             // any order of the row's 16-byte chunks gives the same sum; this one is bank-conflict free
                             const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
-                            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-                                acc = fmaf(lo, lo, acc); acc = fmaf(hi, hi, acc);
-                            }
+                            const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
+                            const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
+                            acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
+                            acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
                         }
-                    sNv[slot * TILE + tok] = acc;
-                    sConst[slot * 128 + tok] = cst[j];
+                    const float2 s = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
+                    sNv[slot * TILE + tok] = s.x + s.y;
+                    // row pair i = tok / 2 holds (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
+                    float* cdst = sConst + slot * 256 + (tok >> 1) * 4 + (tok & 1);
+                    cdst[0] = cst[j].x; cdst[2] = cst[j].y;
                 }
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(bar(BAR_NV + slot)); mbar_arrive(bar(BAR_EMPTY + st)); }
@@ -327,28 +426,21 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int wg = (warp - 4) >> 2;                            // 0: even tiles, 1: odd tiles
         const int lane_grp = warp & 3;                             // TMEM lanes 32*lane_grp .. +31
         const int tok = lane_grp * 32 + lane;                      // token within the tile
-        const float sl2 = p.scale * kLog2e;
+        const float2 sl2 = make_float2(p.scale * kLog2e, p.scale * kLog2e), sc = make_float2(p.scale, p.scale);
         const size_t plane = (size_t)units * p.Nmax;
         uint32_t item = 0, tile_seq = 0;
-        for (long long L = blockIdx.x; L < n_tiles && !failed; L += gridDim.x) {
-            const int unit = (int)(L / p.tiles_per_unit), tile = (int)(L % p.tiles_per_unit);
-            const int b = unit / p.Hkv;
-            const int N = tc_seq_len(p, b), t0 = tile * TILE;
-            float* out = p.scores + (size_t)unit * p.Nmax;
-            const int ptok = t0 + tok;
-            if (t0 >= N) {                                         // padding beyond the sequence: zeros
-                if (wg == 0 && ptok < p.Nmax) {
-                    int pl = 0;
-                    for (unsigned v = 1; v <= 8; v <<= 1) if (p.variants & v) out[(size_t)(pl++) * plane + ptok] = 0.f;
-                }
-                continue;
-            }
+        for (; !tw.done() && !failed; tw.next()) {
             const bool mine = (tile_seq & 1) == (uint32_t)wg;
             ++tile_seq;
             if (!mine) { item += p.n_chunks; continue; }
+            const int unit = tw.unit, b = unit / p.Hkv;
+            const int N = tc_seq_len(p, b), t0 = tw.tile * TILE;
+            float* out = p.scores + (size_t)unit * p.Nmax;
+            const int ptok = t0 + tok;
             // rows of the window that do not see this tile's last token need the causal mask
             const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
-            float s_a = 0.f, s_a2 = 0.f, s_k = 0.f, s_j = 0.f;
+            RowSums S;
+            S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
             float nv = 0.f;
             for (int c = 0; c < p.n_chunks && !failed; ++c, ++item) {
                 const uint32_t buf = item & 1, slot = item % NSLOT;
@@ -356,47 +448,36 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (!mbar_wait(bar(BAR_TM_FULL + buf), (item >> 1) & 1)) { failed = true; break; }
                 tc_fence_after();
                 nv = sNv[slot * TILE + tok];
-                const float nv2 = nv + nv;
-                const float2* cst = sConst + slot * 128;
+                const float4* cst = reinterpret_cast<const float4*>(sConst + slot * 256);
                 const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u, tt = zt + 128u;
-                const int rbase = c * p.chunk_rows;
-                for (int c0 = 0; c0 < p.chunk_rows; c0 += 16) {
-                    uint32_t zr[16], tr[16];
-                    tc_ld16(zt + c0, zr);
-                    tc_ld16(tt + c0, tr);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float2 cj = cst[c0 + j];                     // (log2-sum-exp, ||o_r||^2)
-                        const float z = __uint_as_float(zr[j]), t2 = __uint_as_float(tr[j]);   // t2 = -2 v.o
-                        float a = fast_exp2(fmaf(z, sl2, -cj.x));
-                        if (masked_tile) {
-                            const int r = rbase + c0 + j;
-                            if (ptok > N - p.W + (r % p.W)) a = 0.f;
-                        }
-                        const float Z = z * p.scale, a2 = a * a;
-                        if (VARS & OBC_VAR_ATTN) s_a += a;
-                        if (VARS & OBC_VAR_V) s_a2 += a2;
-                        const float vmo = (nv + cj.y) + t2;                // ||v - o||^2 = |v|^2 + |o|^2 - 2 v.o
-                        if (VARS & OBC_VAR_K) s_k = fmaf(a2 * Z * Z, vmo, s_k);
-                        if (VARS & OBC_VAR_VK) {
-                            // |v|^2 + 2 Z (|v|^2 - v.o) + Z^2 ||v - o||^2, Horner in Z
-                            const float h = fmaf(Z, vmo, nv2 + t2);
-                            s_j = fmaf(a2, fmaf(Z, h, nv), s_j);
-                        }
-                    }
-                }
+                if (masked_tile)
+                    score_chunk<VARS, true>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, N - p.W, p.W, (c * p.chunk_rows) % p.W);
+                else
+                    score_chunk<VARS, false>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, 0, 0, 0);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(BAR_TM_EMPTY + buf));
             }
             if (!failed && ptok < p.Nmax) {
                 const bool live = ptok < N;
+                const float s2 = p.scale * p.scale;
                 int pl = 0;
-                if (p.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + ptok] = live ? s_a2 * nv : 0.f;
-                if (p.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + ptok] = live ? s_k : 0.f;
-                if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] = live ? s_j : 0.f;
-                if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? s_a : 0.f;
+                if (p.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + ptok] = live ? nv * (S.s6.x + S.s6.y) : 0.f;
+                if (p.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + ptok] =
+                    live ? s2 * (fmaf(nv, S.s5.x + S.s5.y, S.s3.x + S.s3.y) + (S.s4.x + S.s4.y)) : 0.f;
+                if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] =
+                    live ? fmaf(nv, S.s1.x + S.s1.y, fmaf(p.scale, S.s2.x + S.s2.y, s2 * (S.s3.x + S.s3.y))) : 0.f;
+                if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? S.s7.x + S.s7.y : 0.f;
+            }
+        }
+        // padding beyond the last tile of a shorter sequence: zeros
+        if (p.seq_lens) {
+            const int et = threadIdx.x - 128;                      // 0..255
+            const int n_planes = __popc(p.variants);
+            for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
+                const int first = (tc_seq_len(p, unit / p.Hkv) + TILE - 1) / TILE * TILE;
+                for (int pl = 0; pl < n_planes; ++pl)
+                    for (int i = first + et; i < p.Nmax; i += 256) p.scores[(size_t)pl * plane + (size_t)unit * p.Nmax + i] = 0.f;
             }
         }
     }
@@ -829,12 +910,11 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     p.B = s.B; p.Hkv = s.Hkv; p.G = s.G; p.W = s.W; p.R = s.R; p.Nmax = s.Nmax; p.seq_lens = s.seq_lens;
     p.scale = s.scale; p.causal = s.causal; p.variants = s.variants;
     p.n_chunks = ch.n_chunks; p.chunk_rows = ch.chunk_rows; p.rows_out = ch.rows_out;
-    p.tiles_per_unit = (s.Nmax + TILE - 1) / TILE;
     p.lse2 = (const float*)(wsb + plan.off_lse2);
     p.onorm = (const float*)(wsb + plan.off_onorm);
     p.scores = scores;
     p.status = (unsigned int*)(wsb + plan.off_flag);
-    const long long n_tiles = (long long)units * p.tiles_per_unit;
+    const long long n_tiles = (long long)units * ((s.Nmax + TILE - 1) / TILE);
     const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
 
     auto launch = [&](auto kernel) -> obc_status {
