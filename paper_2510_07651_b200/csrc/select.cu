@@ -1,12 +1,19 @@
 // Pooling + per-head top-budget selection + ordered index emission (Algorithm 2's
 // "topk(S[..., :cutoff], num_hh) -> sort"), and the row gather that builds the compacted cache.
 //
-//   pool_key_kernel   pooled score of every candidate token -> order-preserving uint32 key
-//   select_kernel     one CTA per (batch item, KV head): 4 x 8-bit radix passes find the key of
-//                     the n_hh-th largest candidate and how many of its ties are kept; two
-//                     warp-segmented sweeps then emit the kept indices in ascending order
+//   select_cluster_kernel  one thread-block cluster per (batch item, KV head).  Every CTA pools
+//                     its contiguous share of the candidates into order-preserving uint32 keys
+//                     held in shared memory; three radix passes (11 + 11 + 10 bits) whose
+//                     histograms are summed in the leading CTA's shared memory find the key of
+//                     the n_hh-th largest candidate and how many of its ties are kept; the
+//                     CTAs exchange their counts and emit the kept indices in ascending order
+//   pool_key_kernel + select_kernel   the same selection with one CTA per head and the keys in
+//                     global memory: the path for sequences too long for a cluster's shared memory
 //   gather_kernel     16-byte vector copy of the kept K/V rows (and optionally their scores)
 #include "obc_common.cuh"
+
+#include <cooperative_groups.h>
+namespace cg = cooperative_groups;
 
 namespace obc {
 
@@ -160,6 +167,184 @@ select_kernel(SelectShape s, const uint32_t* __restrict__ keys_all, int32_t* __r
     }
 }
 
+// ---- cluster path ----------------------------------------------------------------------------
+constexpr int CL_NT = 512;                    // threads per CTA
+constexpr int CL_BINS = 2048;                 // 11-bit digits
+constexpr int CL_MAX_SEG = 20 * 1024;         // candidates per CTA (two 4-byte shared arrays of this size)
+
+struct ClusterShared {                        // fixed part of the CTA's shared memory
+    uint32_t hist[3][CL_BINS];                // one histogram per radix pass (summed in rank 0)
+    uint32_t bcast[3][2];                     // per pass: prefix, remaining (written by rank 0 into every CTA)
+    uint32_t rank_gt[16], rank_eq[16];        // kept-candidate counts of every CTA of the cluster
+    uint32_t warp_gt[CL_NT / 32], warp_eq[CL_NT / 32];
+    uint32_t scan[CL_NT / 32];
+};
+
+__global__ void __launch_bounds__(CL_NT)
+select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* __restrict__ idx_all, int seg_cap) {
+    extern __shared__ __align__(16) uint8_t sel_smem[];
+    ClusterShared& sh = *reinterpret_cast<ClusterShared*>(sel_smem);
+    uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(ClusterShared));
+    float* stage = reinterpret_cast<float*>(keys + seg_cap);          // seg_cap + pool_kernel - 1 floats
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const int unit = blockIdx.x / C, b = unit / s.Hkv;
+    const int N = seq_len(s, b), budget = budget_of(s, b);
+    const int lo = s.n_sink, hi = N - s.n_recent, n = hi - lo;
+    const int n_hh = budget - s.n_sink - s.n_recent;
+    int32_t* idx = idx_all + (size_t)unit * s.idx_stride;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gtid = rank * CL_NT + tid, gthreads = C * CL_NT;
+
+    // these tests depend on the unit only, so all CTAs of the cluster leave together
+    if (n_hh < 0 || n_hh > n || budget > s.idx_stride || N > s.Nmax || hi < lo) {   // bad per-sequence budget
+        for (int j = gtid; j < s.idx_stride; j += gthreads) idx[j] = -1;
+        return;
+    }
+    for (int j = gtid; j < s.n_sink; j += gthreads) idx[j] = j;
+    for (int j = gtid; j < s.n_recent; j += gthreads) idx[s.n_sink + n_hh + j] = hi + j;
+    for (int j = budget + gtid; j < s.idx_stride; j += gthreads) idx[j] = -1;
+    if (n_hh == 0) return;
+
+    // ---- this CTA's share of the candidates: [c0, c1) of [0, n) --------------------------------
+    const int seg = ((n + C - 1) / C + 31) / 32 * 32;
+    const int c0 = min(rank * seg, n), c1 = min(c0 + seg, n), m = c1 - c0;
+    for (int i = tid; i < 3 * CL_BINS; i += CL_NT) (&sh.hist[0][0])[i] = 0;
+
+    // pooled keys: stage the scores with their halo, then pool out of shared memory
+    const float* sc = scores + (size_t)unit * s.Nmax;
+    const int half = (s.pool_mode == OBC_POOL_NONE) ? 0 : s.pool_kernel / 2;
+    const float pad = s.pool_mode == OBC_POOL_MAX ? -INFINITY : 0.f;
+    for (int i = tid; i < m + 2 * half; i += CL_NT) {
+        const int p = lo + c0 + i - half;
+        stage[i] = (p >= lo && p < hi) ? sc[p] : pad;
+    }
+    __syncthreads();
+    for (int i = tid; i < m; i += CL_NT) {
+        float val;
+        if (half == 0) {
+            val = stage[i];
+        } else if (s.pool_mode == OBC_POOL_MAX) {
+            val = -INFINITY;
+            for (int t = 0; t <= 2 * half; ++t) val = fmaxf(val, stage[i + t]);
+        } else {                                   // taps in ascending index order; padding adds +0
+            val = 0.f;
+            for (int t = 0; t <= 2 * half; ++t) val = __fadd_rn(val, stage[i + t]);
+            val = __fdiv_rn(val, (float)s.pool_kernel);
+        }
+        keys[i] = float_key(val);
+    }
+    cluster.sync();                                // histograms zeroed and keys written everywhere
+
+    // ---- radix search for the key T of the n_hh-th largest candidate ---------------------------
+    uint32_t* hist0[3];                            // rank 0's histograms
+    for (int ps = 0; ps < 3; ++ps) hist0[ps] = cluster.map_shared_rank(&sh.hist[ps][0], 0);
+    uint32_t prefix = 0, mask = 0, remaining = (uint32_t)n_hh;
+    for (int ps = 0; ps < 3; ++ps) {
+        const int shift = ps == 0 ? 21 : ps == 1 ? 10 : 0;
+        const uint32_t dmask = ps == 2 ? 1023u : 2047u;
+        uint32_t* hist = sh.hist[ps];
+        for (int base = 0; base < m; base += CL_NT) {
+            const int i = base + tid;
+            const uint32_t key = i < m ? keys[i] : 0u;
+            const bool pred = i < m && ((key & mask) == prefix);
+            const unsigned act = __ballot_sync(0xffffffffu, pred);
+            if (pred) {
+                const uint32_t dgt = (key >> shift) & dmask;
+                const unsigned peers = __match_any_sync(act, dgt);
+                if (lane == __ffs(peers) - 1) atomicAdd(&hist[dgt], (uint32_t)__popc(peers));
+            }
+        }
+        __syncthreads();
+        if (rank != 0)
+            for (int bin = tid; bin < CL_BINS; bin += CL_NT) {
+                const uint32_t c = hist[bin];
+                if (c) atomicAdd(&hist0[ps][bin], c);
+            }
+        cluster.sync();                            // rank 0's histogram holds the whole unit
+        if (rank == 0) {
+            // thread t owns bins [4t, 4t+4); find the highest bin D with
+            // count(bins > D) < remaining <= count(bins >= D)
+            uint32_t loc[4], tot = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { loc[j] = hist[tid * 4 + j]; tot += loc[j]; }
+            uint32_t incl = tot;                   // suffix sum over the lanes >= lane
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_down_sync(0xffffffffu, incl, o);
+                if (lane + o < 32) incl += t;
+            }
+            if (lane == 0) sh.scan[warp] = incl;
+            __syncthreads();
+            uint32_t above = incl - tot;
+            for (int w = warp + 1; w < CL_NT / 32; ++w) above += sh.scan[w];
+            if (above < remaining && remaining <= above + tot) {
+                uint32_t run = above, found_prefix = 0, found_rem = 0;
+#pragma unroll
+                for (int j = 3; j >= 0; --j) {
+                    if (run != 0xffffffffu) {
+                        if (remaining <= run + loc[j]) {
+                            found_prefix = prefix | ((uint32_t)(tid * 4 + j) << shift);
+                            found_rem = remaining - run;
+                            run = 0xffffffffu;
+                        } else {
+                            run += loc[j];
+                        }
+                    }
+                }
+                for (int r = 0; r < C; ++r) {
+                    uint32_t* dst = cluster.map_shared_rank(&sh.bcast[ps][0], r);
+                    dst[0] = found_prefix; dst[1] = found_rem;
+                }
+            }
+        }
+        cluster.sync();                            // the search result reached every CTA
+        prefix = sh.bcast[ps][0]; remaining = sh.bcast[ps][1]; mask |= dmask << shift;
+    }
+    const uint32_t T = prefix, k_eq = remaining;   // keep all keys > T and the first k_eq keys == T
+
+    // ---- ordered emission: each warp owns a contiguous run of this CTA's candidates --------------
+    const int wseg = ((m + CL_NT / 32 - 1) / (CL_NT / 32) + 31) / 32 * 32;
+    const int s0 = min(warp * wseg, m), s1 = min(s0 + wseg, m);
+    uint32_t cgt = 0, ceq = 0;
+    for (int i = s0 + lane; i < s1; i += 32) {
+        const uint32_t key = keys[i];
+        cgt += key > T; ceq += key == T;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        cgt += __shfl_xor_sync(0xffffffffu, cgt, o);
+        ceq += __shfl_xor_sync(0xffffffffu, ceq, o);
+    }
+    if (lane == 0) { sh.warp_gt[warp] = cgt; sh.warp_eq[warp] = ceq; }
+    __syncthreads();
+    if (tid < C) {                                 // this CTA's totals into every CTA of the cluster
+        uint32_t tg = 0, te = 0;
+        for (int w = 0; w < CL_NT / 32; ++w) { tg += sh.warp_gt[w]; te += sh.warp_eq[w]; }
+        cluster.map_shared_rank(&sh.rank_gt[0], tid)[rank] = tg;
+        cluster.map_shared_rank(&sh.rank_eq[0], tid)[rank] = te;
+    }
+    cluster.sync();
+    uint32_t gt_before = 0, eq_before = 0;
+    for (int r = 0; r < rank; ++r) { gt_before += sh.rank_gt[r]; eq_before += sh.rank_eq[r]; }
+    for (int w = 0; w < warp; ++w) { gt_before += sh.warp_gt[w]; eq_before += sh.warp_eq[w]; }
+    uint32_t eq_run = eq_before;
+    uint32_t out = s.n_sink + gt_before + min(eq_before, k_eq);
+    const unsigned lt_mask = (1u << lane) - 1u;
+    for (int base = s0; base < s1; base += 32) {
+        const int i = base + lane;
+        const uint32_t key = i < s1 ? keys[i] : 0u;
+        const bool is_eq = i < s1 && key == T;
+        const unsigned beq = __ballot_sync(0xffffffffu, is_eq);
+        const bool sel = i < s1 && (key > T || (is_eq && eq_run + __popc(beq & lt_mask) < k_eq));
+        const unsigned bsel = __ballot_sync(0xffffffffu, sel);
+        if (sel) idx[out + __popc(bsel & lt_mask)] = lo + c0 + i;
+        out += __popc(bsel);
+        eq_run += __popc(beq);
+    }
+}
+
 // one 16-byte vector per thread; `vecs` vectors per row
 __global__ void __launch_bounds__(256)
 gather_kernel(int units, int Hkv, int idx_stride, int vecs, int elem_bytes,
@@ -185,9 +370,39 @@ gather_kernel(int units, int Hkv, int idx_stride, int vecs, int elem_bytes,
 
 size_t select_workspace_bytes(int B, int Hkv, int Nmax) { return align_up((size_t)B * Hkv * Nmax * 4, 256); }
 
+// Cluster size for the one-cluster-per-head path, or 0 when a head does not fit a cluster's shared memory.
+static int select_cluster_size(int Nmax, int* seg_cap) {
+    int C = 8;
+    if ((Nmax + C - 1) / C > 8192) C = 16;
+    const int seg = ((Nmax + C - 1) / C + 31) / 32 * 32;
+    if (seg > CL_MAX_SEG) return 0;
+    *seg_cap = seg;
+    return C;
+}
+
 obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx, void* ws, cudaStream_t stream) {
-    uint32_t* keys = (uint32_t*)ws;
     const int units = s.B * s.Hkv;
+    int seg_cap = 0;
+    const int C = select_cluster_size(s.Nmax, &seg_cap);
+    if (C > 0) {
+        const size_t smem = sizeof(ClusterShared) + (size_t)seg_cap * 8 + (size_t)s.pool_kernel * 4 + 16;
+        OBC_CUDA_TRY(cudaFuncSetAttribute(select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        if (C > 8) OBC_CUDA_TRY(cudaFuncSetAttribute(select_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)(units * C)); cfg.blockDim = dim3(CL_NT); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        int max_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, select_cluster_kernel, &cfg) == cudaSuccess && max_clusters > 0) {
+            { ProfScope ps("select_cluster", stream);
+              OBC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel, s, scores, idx, seg_cap)); }
+            return OBC_OK;
+        }
+        (void)cudaGetLastError();                  // the device cannot host such a cluster: one CTA per head
+    }
+    uint32_t* keys = (uint32_t*)ws;
     { ProfScope ps("pool_key", stream); pool_key_kernel<<<dim3((s.Nmax + 255) / 256, units), 256, 0, stream>>>(s, scores, keys); }
     OBC_CUDA_TRY(cudaGetLastError());
     { ProfScope ps("select", stream); select_kernel<<<units, SEL_NT, 0, stream>>>(s, keys, idx); }
