@@ -165,6 +165,16 @@ simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
 // ------------------------------------------------------------------------------------------ combine
 // one block of 128 threads per (unit, output row): merge the splits.  Output rows >= R are padding
 // for the tensor-core pass: O = 0, ||o||^2 = 0 and log2-sum-exp = +inf, so that they weigh 0.
+// The statistics of the splits are read one per thread, and the partial outputs of several splits
+// are in flight at once, so the kernel is bound by the partial-output traffic, not by load latency.
+__device__ __forceinline__ float block128_reduce(float x, bool take_max, float* red) {
+    x = take_max ? warp_max(x) : warp_sum(x);
+    __syncthreads();                                   // red may still be read from an earlier call
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
+    __syncthreads();
+    return take_max ? fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3])) : (red[0] + red[1]) + (red[2] + red[3]);
+}
+
 __global__ void __launch_bounds__(128)
 simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     const int r = blockIdx.x % plan.rows_out, unit = blockIdx.x / plan.rows_out, c = threadIdx.x;
@@ -176,31 +186,50 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
         if (c == 0) { (ws + plan.off_lse2 / 4)[orow] = INFINITY; (ws + plan.off_onorm / 4)[orow] = 0.f; }
         return;
     }
+    __shared__ float red[4];
+    __shared__ float sW[128];
     const float* part_m = ws + plan.off_part_m / 4;
     const float* part_l = ws + plan.off_part_l / 4;
     const float* part_o = ws + plan.off_part_o / 4;
+    const size_t row0 = (size_t)unit * plan.n_splits * s.R + r;          // split sp: row0 + sp * R
     float M = -INFINITY;
-    for (int sp = 0; sp < plan.n_splits; ++sp)
-        M = fmaxf(M, part_m[((size_t)unit * plan.n_splits + sp) * s.R + r]);
+    for (int sp = c; sp < plan.n_splits; sp += 128) M = fmaxf(M, part_m[row0 + (size_t)sp * s.R]);
+    M = block128_reduce(M, true, red);
     float L = 0.f, oc = 0.f;
-    for (int sp = 0; sp < plan.n_splits; ++sp) {
-        size_t row = ((size_t)unit * plan.n_splits + sp) * s.R + r;
-        float m = part_m[row];
-        if (m == -INFINITY) continue;
-        float w = exp2f(m - M);
-        L = fmaf(part_l[row], w, L);
-        oc = fmaf(part_o[row * kD + c], w, oc);
+    for (int base = 0; base < plan.n_splits; base += 128) {
+        const int sp = base + c, cnt = min(128, plan.n_splits - base);
+        float w = 0.f;
+        if (sp < plan.n_splits) {
+            const float m = part_m[row0 + (size_t)sp * s.R];
+            if (m != -INFINITY) { w = exp2f(m - M); L = fmaf(part_l[row0 + (size_t)sp * s.R], w, L); }
+        }
+        __syncthreads();
+        sW[c] = w;
+        __syncthreads();
+        const float* po = part_o + (row0 + (size_t)base * s.R) * kD + c;
+        int j = 0;
+        for (; j + 4 <= cnt; j += 4) {
+            const float w0 = sW[j], w1 = sW[j + 1], w2 = sW[j + 2], w3 = sW[j + 3];
+            // a split without visible tokens (weight 0) may hold unwritten partial outputs
+            const float o0 = w0 != 0.f ? po[(size_t)(j + 0) * s.R * kD] : 0.f;
+            const float o1 = w1 != 0.f ? po[(size_t)(j + 1) * s.R * kD] : 0.f;
+            const float o2 = w2 != 0.f ? po[(size_t)(j + 2) * s.R * kD] : 0.f;
+            const float o3 = w3 != 0.f ? po[(size_t)(j + 3) * s.R * kD] : 0.f;
+            oc = fmaf(o0, w0, oc); oc = fmaf(o1, w1, oc); oc = fmaf(o2, w2, oc); oc = fmaf(o3, w3, oc);
+        }
+        for (; j < cnt; ++j) {
+            const float w0 = sW[j];
+            if (w0 != 0.f) oc = fmaf(po[(size_t)j * s.R * kD], w0, oc);
+        }
     }
+    L = block128_reduce(L, false, red);
     oc = oc / L;
-    __shared__ float red[4];
-    float sq = warp_sum(oc * oc);
-    if ((c & 31) == 0) red[c >> 5] = sq;
-    __syncthreads();
+    const float onorm = block128_reduce(oc * oc, false, red);
     (ws + plan.off_o / 4)[orow * kD + c] = oc;
     if (obf) obf[orow * kD + c] = __float2bfloat16(-2.f * oc);
     if (c == 0) {
         (ws + plan.off_lse2 / 4)[orow] = M + log2f(L);
-        (ws + plan.off_onorm / 4)[orow] = red[0] + red[1] + red[2] + red[3];
+        (ws + plan.off_onorm / 4)[orow] = onorm;
     }
 }
 

@@ -496,25 +496,31 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 // O = A V over the perturbation window, Eq. 9), split over the cached tokens.
 //
 // Rows of the window (one chunk of up to 128) sit on the MMA M dimension, so a TMEM lane holds one
-// row and the softmax thread that owns it reduces along the tile without cross-thread traffic:
-//     S   = Q_chunk . K_tile^T                     (tcgen05, accumulators double-buffered in TMEM)
-//     P   = exp2(S * scale*log2e - m_used)         (registers -> bf16 -> swizzled shared memory)
-//     O  += P . V_tile                             (tcgen05, V read as an MN-major B operand)
-// m_used is the exponent reference of the row; it is only moved up (and O, l rescaled) when the
-// running maximum exceeds it by more than 8 (a factor 256), which keeps P within bf16/fp32 range.
-// Each CTA writes (m_used, l, O) of its token split; the combine kernel merges the splits.
+// row and the softmax thread that owns it reduces along the tile without cross-thread traffic.
+// Two softmax warpgroups take alternate token tiles; each keeps its own running statistics and its
+// own output accumulator, i.e. the CTA produces two partial results, which the combine kernel
+// merges like any other token split.  For tile t and warpgroup w = t mod 2:
+//     S_w  = Q_chunk . K_tile^T                    (tcgen05, accumulator in TMEM)
+//     P_w  = exp2(S_w * scale*log2e - m_used)      (registers -> bf16 -> TMEM, over S_w's columns)
+//     O_w += P_w . V_tile                          (tcgen05: A operand from TMEM, V as MN-major B)
+// m_used is the exponent reference of the row; it is only moved up (and O_w, l rescaled) when the
+// tile maximum exceeds it by more than 8 (a factor 256), which keeps P within bf16/fp32 range.
+// MMAs issued by one thread execute in order, so S_w of tile t+2 cannot overwrite P_w before
+// P_w . V of tile t has read it, and a commit after S_w(t) also covers P_w . V of tile t-2.
 //
-//   warp 0      TMA producer (Q chunk once, K/V tiles into a 2-stage ring)
+//   warp 0      TMA producer (Q chunk once, K/V tiles into a 3-stage ring)
 //   warp 1      MMA issuer
-//   warps 4-7   softmax (thread = row)
+//   warps 4-7   softmax warpgroup 0 (even tiles), warps 8-11 softmax warpgroup 1 (odd tiles)
+// TMEM columns: S_0 [0,128)  S_1 [128,256)  O_0 [256,384)  O_1 [384,512)
 // =================================================================================================
-constexpr int kThreadsP1 = 256;
+constexpr int kThreadsP1 = 384;
+constexpr int P1_NSTAGE = 3;
 constexpr uint32_t P1_OFF_Q = 0;
-constexpr uint32_t P1_OFF_P = P1_OFF_Q + kOperandBytes;
-constexpr uint32_t P1_OFF_K = P1_OFF_P + kOperandBytes;
-constexpr uint32_t P1_OFF_V = P1_OFF_K + NSTAGE * kOperandBytes;
-constexpr uint32_t P1_OFF_BAR = P1_OFF_V + NSTAGE * kOperandBytes;
-enum { P1_FULL = 0, P1_EMPTY = 2, P1_QFULL = 4, P1_SFULL = 5, P1_SEMPTY = 7, P1_PFULL = 9, P1_PVDONE = 10, P1_NBARS = 11 };
+constexpr uint32_t P1_OFF_K = P1_OFF_Q + kOperandBytes;
+constexpr uint32_t P1_OFF_V = P1_OFF_K + P1_NSTAGE * kOperandBytes;
+constexpr uint32_t P1_OFF_BAR = P1_OFF_V + P1_NSTAGE * kOperandBytes;
+enum { P1_FULL = 0, P1_EMPTY = P1_NSTAGE, P1_QFULL = 2 * P1_NSTAGE, P1_SFULL = 2 * P1_NSTAGE + 1,
+       P1_PFULL = 2 * P1_NSTAGE + 3, P1_ODONE = 2 * P1_NSTAGE + 5, P1_NBARS = 2 * P1_NSTAGE + 6 };
 constexpr uint32_t P1_OFF_TMEM = P1_OFF_BAR + P1_NBARS * 8;
 constexpr uint32_t kSmemP1 = P1_OFF_TMEM + 16 + 1024;
 constexpr float kRescaleThreshold = 8.f;                   // log2 units
@@ -525,8 +531,8 @@ struct P1Params {
     float scale;
     int causal;
     int n_chunks, chunk_rows;
-    int n_splits, tiles_per_split;
-    float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
+    int n_splits, tiles_per_split;                         // CTAs per (unit, chunk); each writes 2 partials
+    float* part_m; float* part_l; float* part_o;           // [units][2 * n_splits][R] (x d for part_o)
     unsigned int* status;
 };
 
@@ -539,6 +545,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
 }
+// waits for this thread's TMEM loads; the registers are operands so that no use is moved above it
+__device__ __forceinline__ void tc_wait_ld32(uint32_t* r) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
 __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
                  "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
@@ -548,8 +563,19 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
                    "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
                  : "memory");
 }
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+                 : "memory");
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (rows on lanes, K packed two bf16 per column) is read from TMEM
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 
 // MN-major B operand with 128-byte swizzle: 64 contiguous elements of N per 128-byte row, 8 rows of
 // K per 1024-byte group (stride byte offset), the next 64 elements of N one 16 KB block further
@@ -568,10 +594,15 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 
 __global__ void __launch_bounds__(kThreadsP1, 1)
 tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const __grid_constant__ CUtensorMap map_v, P1Params p) {
+                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ P1Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -589,10 +620,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int n_tiles = max(tile_hi - tile_lo, 0);
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), 1); }
-        mbar_init(bar(P1_QFULL), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(P1_SFULL + i), 1); mbar_init(bar(P1_SEMPTY + i), 4); }
-        mbar_init(bar(P1_PFULL), 4); mbar_init(bar(P1_PVDONE), 1);
+        for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), 1); }
+        mbar_init(bar(P1_QFULL), 1); mbar_init(bar(P1_ODONE), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(P1_SFULL + i), 1); mbar_init(bar(P1_PFULL + i), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -603,10 +633,10 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_o = tmem_base + 256u;
     bool failed = false;
 
     if (warp == 0) {
+        // ===================================== TMA producer =====================================
         if (lane == 0 && n_tiles > 0) {
             mbar_expect_tx(bar(P1_QFULL), (uint32_t)p.chunk_rows * 256u);
             const int qrow = (b * p.Hq + g * p.G) * p.W + c * p.chunk_rows;
@@ -614,8 +644,8 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tma_load_2d(sbase + P1_OFF_Q + kHalfBytes, &map_q, bar(P1_QFULL), 64, qrow);
             int issued = 0;
             for (int i = 0; i < n_tiles; ++i) {
-                const uint32_t st = i % NSTAGE;
-                if (!mbar_wait(bar(P1_EMPTY + st), ((i / NSTAGE) & 1) ^ 1)) { failed = true; break; }
+                const uint32_t st = i % P1_NSTAGE;
+                if (!mbar_wait(bar(P1_EMPTY + st), ((i / P1_NSTAGE) & 1) ^ 1)) { failed = true; break; }
                 mbar_expect_tx(bar(P1_FULL + st), 2 * kOperandBytes);
                 const uint32_t dk = sbase + P1_OFF_K + st * kOperandBytes, dv = sbase + P1_OFF_V + st * kOperandBytes;
                 const int t0 = (tile_lo + i) * TILE;
@@ -625,20 +655,20 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tma_load_4d(dv + kHalfBytes, &map_v, bar(P1_FULL + st), 64, t0, g, b);
                 ++issued;
             }
-            for (int back = 0; back < NSTAGE && back < issued; ++back) {      // drain own copies
+            for (int back = 0; back < P1_NSTAGE && back < issued; ++back) {   // drain own copies
                 const int it = issued - 1 - back;
-                (void)mbar_wait(bar(P1_FULL + it % NSTAGE), (it / NSTAGE) & 1);
+                (void)mbar_wait(bar(P1_FULL + it % P1_NSTAGE), (it / P1_NSTAGE) & 1);
             }
             (void)mbar_wait(bar(P1_QFULL), 0);
         }
     } else if (warp == 1) {
+        // ===================================== MMA issuer =======================================
         if (lane == 0 && n_tiles > 0) {
             const uint32_t idesc_s = idesc_bf16(TILE);
             const uint32_t idesc_pv = idesc_bf16(kD) | (1u << 16);           // B operand (V) is MN-major
-            auto issue_s = [&](int j) -> bool {
-                const uint32_t st = j % NSTAGE;
-                if (!mbar_wait(bar(P1_FULL + st), (j / NSTAGE) & 1)) return false;
-                if (!mbar_wait(bar(P1_SEMPTY + (j & 1)), ((j >> 1) & 1) ^ 1)) return false;
+            auto issue_s = [&](int j) -> bool {                              // S_w = Q . K_j^T
+                const uint32_t st = j % P1_NSTAGE;
+                if (!mbar_wait(bar(P1_FULL + st), (j / P1_NSTAGE) & 1)) return false;
                 tc_fence_after();
                 const uint32_t ak = sbase + P1_OFF_K + st * kOperandBytes;
 #pragma unroll
@@ -651,111 +681,146 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             };
             failed = !mbar_wait(bar(P1_QFULL), 0);
             if (!failed) failed = !issue_s(0);
+            if (!failed && n_tiles > 1) failed = !issue_s(1);
             for (int i = 0; i < n_tiles && !failed; ++i) {
-                if (i + 1 < n_tiles && !issue_s(i + 1)) { failed = true; break; }
-                if (!mbar_wait(bar(P1_PFULL), i & 1)) { failed = true; break; }
+                const uint32_t w = i & 1;
+                if (!mbar_wait(bar(P1_PFULL + w), (i >> 1) & 1)) { failed = true; break; }
                 tc_fence_after();
-                const uint32_t av = sbase + P1_OFF_V + (i % NSTAGE) * kOperandBytes;
+                const uint32_t av = sbase + P1_OFF_V + (i % P1_NSTAGE) * kOperandBytes;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {                             // 128 tokens = 8 steps of K = 16
-                    const uint32_t offp = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    tc_mma(tmem_o, smem_desc_k_sw128(sbase + P1_OFF_P + offp), smem_desc_mn_sw128(av + ks * 2048), idesc_pv, (i > 0) || (ks > 0));
-                }
-                tc_commit(bar(P1_PVDONE));
-                tc_commit(bar(P1_EMPTY + (i % NSTAGE)));
+                for (int ks = 0; ks < 8; ++ks)                               // 128 tokens = 8 steps of K = 16
+                    tc_mma_ts(tmem_base + 256u + w * 128u, tmem_base + w * 128u + ks * 8, smem_desc_mn_sw128(av + ks * 2048),
+                              idesc_pv, (i > 1) || (ks > 0));
+                tc_commit(bar(P1_EMPTY + (i % P1_NSTAGE)));                  // S(i) and P.V(i) have read the stage
+                if (i + 2 < n_tiles && !issue_s(i + 2)) { failed = true; break; }
             }
+            if (!failed) tc_commit(bar(P1_ODONE));
         }
     } else if (warp >= 4) {
+        // ======================================= softmax ========================================
+        const int w = (warp - 4) >> 2;                                       // warpgroup: tiles w, w+2, ...
         const int lane_grp = warp & 3;
         const int row = lane_grp * 32 + lane;                                // row within the chunk
         const int rows_valid = min(p.chunk_rows, p.R - c * p.chunk_rows);
         const int r = c * p.chunk_rows + row;
         const bool valid = row < rows_valid;
-        const int last = valid ? (p.causal ? N - p.W + (r % p.W) : N - 1) : -1;
+        const int last = valid ? (p.causal ? N - p.W + (r % p.W) : N - 1) : -1;   // last visible token
+        const int first_masked = min(p.causal ? N - p.W + 1 : N, N);         // tiles reaching it need the mask
         const float sl2 = p.scale * kLog2e;
         const uint32_t lane_addr = (uint32_t)(lane_grp * 32) << 16;
+        const uint32_t tS = tmem_base + lane_addr + w * 128u, tO = tmem_base + lane_addr + 256u + w * 128u;
         float m_used = -INFINITY, l = 0.f;
-        uint8_t* prow = smem + P1_OFF_P + row * 128;
+        int my_tiles = 0;
 
-        for (int i = 0; i < n_tiles && !failed; ++i) {
-            const uint32_t buf = i & 1;
+        for (int i = w; i < n_tiles && !failed; i += 2, ++my_tiles) {
             const int t0 = (tile_lo + i) * TILE;
-            if (!mbar_wait(bar(P1_SFULL + buf), (i >> 1) & 1)) { failed = true; break; }
+            if (!mbar_wait(bar(P1_SFULL + w), my_tiles & 1)) { failed = true; break; }
             tc_fence_after();
-            float sv[128];
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) tc_ld32(tmem_base + lane_addr + buf * 128u + q4 * 32, reinterpret_cast<uint32_t*>(sv) + q4 * 32);
-            tc_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(P1_SEMPTY + buf));
-
-            float mt = -INFINITY;
+            const bool masked = t0 + TILE > first_masked;
             const int nvis = last - t0 + 1;                                  // columns j < nvis are visible
+
+            // sweep 1: tile maximum of the row (raw logits; the scale is positive)
+            float mt = -INFINITY;
+            {
+                uint32_t sa[32], sb[32];
+                tc_ld32(tS, sa);
 #pragma unroll
-            for (int j = 0; j < 128; ++j) {
-                sv[j] = j < nvis ? sv[j] * sl2 : -INFINITY;
-                mt = fmaxf(mt, sv[j]);
+                for (int pc = 0; pc < 4; pc += 2) {
+                    tc_wait_ld32(sa);
+                    tc_ld32(tS + (pc + 1) * 32, sb);
+                    if (masked) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) if (pc * 32 + j >= nvis) sa[j] = 0xff800000u;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) mt = fmax3(mt, __uint_as_float(sa[j]), __uint_as_float(sa[j + 1]));
+                    tc_wait_ld32(sb);
+                    if (pc + 2 < 4) tc_ld32(tS + (pc + 2) * 32, sa);
+                    if (masked) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) if ((pc + 1) * 32 + j >= nvis) sb[j] = 0xff800000u;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) mt = fmax3(mt, __uint_as_float(sb[j]), __uint_as_float(sb[j + 1]));
+                }
             }
+            mt *= sl2;
             const bool need = mt > m_used + kRescaleThreshold;               // also true for the first visible tile
             const float factor = need ? fast_exp2(m_used - mt) : 1.f;        // m_used = -inf -> 0
-            if (i > 0) {
-                const bool any = __any_sync(0xffffffffu, need && m_used != -INFINITY);
-                if (!mbar_wait(bar(P1_PVDONE), (i - 1) & 1)) { failed = true; break; }   // P buffer free, O stable
-                if (any) {
-                    tc_fence_after();
+            if (my_tiles > 0 && __any_sync(0xffffffffu, valid && need && m_used != -INFINITY)) {
+                // P.V of this warpgroup's previous tile is complete (the commit that signalled S covers it)
 #pragma unroll 1
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint32_t ov[32];
-                        tc_ld32(tmem_o + lane_addr + q4 * 32, ov);
-                        tc_wait_ld();
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t ov[32];
+                    tc_ld32(tO + q4 * 32, ov);
+                    tc_wait_ld32(ov);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
-                        tc_st32(tmem_o + lane_addr + q4 * 32, ov);
-                    }
-                    tc_wait_st();
-                    tc_fence_before();
+                    for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * factor);
+                    tc_st32(tO + q4 * 32, ov);
                 }
             }
             l *= factor;
             if (need) m_used = mt;
             const float m_eff = m_used == -INFINITY ? 0.f : m_used;
-            float lsum = 0.f;
+            const float2 sl2v = make_float2(sl2, sl2), negm = make_float2(-m_eff, -m_eff);
+
+            // sweep 2: P = exp2(S * scale*log2e - m_used) as bf16 over the first 64 columns of S_w
+            float2 lsum = make_float2(0.f, 0.f);
+            {
+                uint32_t sa[32], sb[32];
+                auto piece = [&](uint32_t* sv, int pc) {
+                    uint32_t pk[16];
 #pragma unroll
-            for (int ch = 0; ch < 16; ++ch) {                                // 16 chunks of 8 tokens = 16 bytes of bf16
-                uint32_t w[4];
+                    for (int j = 0; j < 32; j += 2) {
+                        float2 x = make_float2(__uint_as_float(sv[j]), __uint_as_float(sv[j + 1]));
+                        x = __ffma2_rn(x, sl2v, negm);
+                        if (masked) {
+                            if (pc * 32 + j >= nvis) x.x = -INFINITY;
+                            if (pc * 32 + j + 1 >= nvis) x.y = -INFINITY;
+                        }
+                        const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                        lsum = __fadd2_rn(lsum, e);
+                        pk[j >> 1] = pack_bf16x2(e.x, e.y);
+                    }
+                    tc_st16(tS + pc * 16, pk);
+                };
+                tc_ld32(tS, sa);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float p0 = fast_exp2(sv[ch * 8 + 2 * e] - m_eff), p1 = fast_exp2(sv[ch * 8 + 2 * e + 1] - m_eff);
-                    lsum += p0 + p1;
-                    w[e] = pack_bf16x2(p0, p1);
+                for (int pc = 0; pc < 4; pc += 2) {
+                    tc_wait_ld32(sa);
+                    tc_ld32(tS + (pc + 1) * 32, sb);
+                    piece(sa, pc);
+                    tc_wait_ld32(sb);
+                    if (pc + 2 < 4) tc_ld32(tS + (pc + 2) * 32, sa);
+                    piece(sb, pc + 1);
                 }
-                *reinterpret_cast<uint4*>(prow + (ch >> 3) * kHalfBytes + (((ch & 7) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            l += lsum;
+            l += lsum.x + lsum.y;
+            tc_wait_st();
             if (t0 + TILE > N && t0 + row >= N) {                            // tail: V rows past the sequence must not reach the MMA
-                uint8_t* vrow = smem + P1_OFF_V + (i % NSTAGE) * kOperandBytes + row * 128;
+                uint8_t* vrow = smem + P1_OFF_V + (i % P1_NSTAGE) * kOperandBytes + row * 128;
 #pragma unroll
                 for (int ch = 0; ch < 8; ++ch) {
                     *reinterpret_cast<uint4*>(vrow + (ch << 4)) = make_uint4(0, 0, 0, 0);
                     *reinterpret_cast<uint4*>(vrow + kHalfBytes + (ch << 4)) = make_uint4(0, 0, 0, 0);
                 }
+                fence_async_smem();
             }
-            fence_async_smem();
+            tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(P1_PFULL));
+            if (lane == 0) mbar_arrive(bar(P1_PFULL + w));
         }
 
-        // partial results of this split
-        const size_t prow_idx = ((size_t)unit * p.n_splits + split) * p.R + r;
-        if (n_tiles > 0 && !failed) {
-            if (!mbar_wait(bar(P1_PVDONE), (n_tiles - 1) & 1)) failed = true;
+        // the two partial results of this CTA: slot 2*split + w
+        const size_t prow_idx = ((size_t)unit * (2 * p.n_splits) + 2 * split + w) * p.R + r;
+        if (my_tiles > 0 && !failed) {
+            if (!mbar_wait(bar(P1_ODONE), 0)) failed = true;
             tc_fence_after();
 #pragma unroll 1
             for (int q4 = 0; q4 < 4 && !failed; ++q4) {
                 uint32_t ov[32];
-                tc_ld32(tmem_o + lane_addr + q4 * 32, ov);
-                tc_wait_ld();
+                tc_ld32(tO + q4 * 32, ov);
+                tc_wait_ld32(ov);
                 if (valid) {
                     float4* dst = reinterpret_cast<float4*>(p.part_o + prow_idx * kD + q4 * 32);
 #pragma unroll
@@ -765,11 +830,8 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
             }
             tc_fence_before();
-        } else if (valid) {
-            float4* dst = reinterpret_cast<float4*>(p.part_o + prow_idx * kD);
-            for (int j = 0; j < 32; ++j) dst[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (valid) { p.part_m[prow_idx] = m_used; p.part_l[prow_idx] = l; }
+        if (valid) { p.part_m[prow_idx] = my_tiles > 0 && !failed ? m_used : -INFINITY; p.part_l[prow_idx] = l; }
     }
 
     if (failed) atomicExch(p.status, 1u);
@@ -845,8 +907,8 @@ static SimtPlan make_tc_plan(const ScoreShape& s) {
     if (n < 1) n = 1;
     if (n > tiles) n = tiles;
     SimtPlan p{};
-    p.tiles_per_split = (tiles + n - 1) / n;
-    p.n_splits = (tiles + p.tiles_per_split - 1) / p.tiles_per_split;
+    p.tiles_per_split = (tiles + n - 1) / n;                                   // per pass-1 CTA
+    p.n_splits = 2 * ((tiles + p.tiles_per_split - 1) / p.tiles_per_split);    // partial results: two per CTA
     p.rows_out = ch.rows_out;
     p.want_obf = 1;
     const size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, orow = (size_t)units * ch.rows_out;
@@ -895,13 +957,13 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.B = s.B; p1.Hq = s.Hq; p1.Hkv = s.Hkv; p1.G = s.G; p1.W = s.W; p1.R = s.R; p1.Nmax = s.Nmax;
         p1.seq_lens = s.seq_lens; p1.scale = s.scale; p1.causal = s.causal;
         p1.n_chunks = ch.n_chunks; p1.chunk_rows = ch.chunk_rows;
-        p1.n_splits = plan.n_splits; p1.tiles_per_split = plan.tiles_per_split;
+        p1.n_splits = plan.n_splits / 2; p1.tiles_per_split = plan.tiles_per_split;
         p1.part_m = (float*)(wsb + plan.off_part_m); p1.part_l = (float*)(wsb + plan.off_part_l);
         p1.part_o = (float*)(wsb + plan.off_part_o);
         p1.status = (unsigned int*)(wsb + plan.off_flag);
         OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
         { ProfScope ps("tc_pass1", stream);
-          tc_pass1_kernel<<<dim3(plan.n_splits, units * ch.n_chunks), kThreadsP1, kSmemP1, stream>>>(mq, mk, mv, p1); }
+          tc_pass1_kernel<<<dim3(plan.n_splits / 2, units * ch.n_chunks), kThreadsP1, kSmemP1, stream>>>(mq, mk, mv, p1); }
         OBC_CUDA_TRY(cudaGetLastError());
         obc_status st = launch_combine(s, plan, ws, stream);
         if (st != OBC_OK) return st;
