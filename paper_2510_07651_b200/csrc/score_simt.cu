@@ -165,8 +165,12 @@ simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
 // ------------------------------------------------------------------------------------------ combine
 // one block of 128 threads per (unit, output row): merge the splits.  Output rows >= R are padding
 // for the tensor-core pass: O = 0, ||o||^2 = 0 and log2-sum-exp = +inf, so that they weigh 0.
-// The statistics of the splits are read one per thread, and the partial outputs of several splits
-// are in flight at once, so the kernel is bound by the partial-output traffic, not by load latency.
+// Every load of a block is issued before the first one is used: thread t reads the statistics of
+// split t, warp w the float4 partial outputs of splits w, w+4, ... (pass 1 writes every partial,
+// zeros where a split saw no token), so a block costs one round trip to L2 instead of one per split.
+constexpr int CMB_NT = 128;
+constexpr int CMB_INFLIGHT = 10;                       // float4 loads in flight per thread
+
 __device__ __forceinline__ float block128_reduce(float x, bool take_max, float* red) {
     x = take_max ? warp_max(x) : warp_sum(x);
     __syncthreads();                                   // red may still be read from an earlier call
@@ -175,60 +179,70 @@ __device__ __forceinline__ float block128_reduce(float x, bool take_max, float* 
     return take_max ? fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3])) : (red[0] + red[1]) + (red[2] + red[3]);
 }
 
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(CMB_NT)
 simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
-    const int r = blockIdx.x % plan.rows_out, unit = blockIdx.x / plan.rows_out, c = threadIdx.x;
+    const int r = blockIdx.x % plan.rows_out, unit = blockIdx.x / plan.rows_out;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const size_t orow = (size_t)unit * plan.rows_out + r;
     __nv_bfloat16* obf = plan.want_obf ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + plan.off_obf) : nullptr;
     if (r >= s.R) {
-        (ws + plan.off_o / 4)[orow * kD + c] = 0.f;
-        if (obf) obf[orow * kD + c] = __float2bfloat16(0.f);
-        if (c == 0) { (ws + plan.off_lse2 / 4)[orow] = INFINITY; (ws + plan.off_onorm / 4)[orow] = 0.f; }
+        (ws + plan.off_o / 4)[orow * kD + tid] = 0.f;
+        if (obf) obf[orow * kD + tid] = __float2bfloat16(0.f);
+        if (tid == 0) { (ws + plan.off_lse2 / 4)[orow] = INFINITY; (ws + plan.off_onorm / 4)[orow] = 0.f; }
         return;
     }
     __shared__ float red[4];
-    __shared__ float sW[128];
+    __shared__ float sW[CMB_NT];
+    __shared__ __align__(16) float sAcc[4][kD];
     const float* part_m = ws + plan.off_part_m / 4;
     const float* part_l = ws + plan.off_part_l / 4;
     const float* part_o = ws + plan.off_part_o / 4;
     const size_t row0 = (size_t)unit * plan.n_splits * s.R + r;          // split sp: row0 + sp * R
-    float M = -INFINITY;
-    for (int sp = c; sp < plan.n_splits; sp += 128) M = fmaxf(M, part_m[row0 + (size_t)sp * s.R]);
-    M = block128_reduce(M, true, red);
-    float L = 0.f, oc = 0.f;
-    for (int base = 0; base < plan.n_splits; base += 128) {
-        const int sp = base + c, cnt = min(128, plan.n_splits - base);
-        float w = 0.f;
-        if (sp < plan.n_splits) {
-            const float m = part_m[row0 + (size_t)sp * s.R];
-            if (m != -INFINITY) { w = exp2f(m - M); L = fmaf(part_l[row0 + (size_t)sp * s.R], w, L); }
+    const size_t sstride = (size_t)s.R * kD;                             // floats between the outputs of two splits
+    float M = -INFINITY, L = 0.f, Mrun = -INFINITY;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = 0; base < plan.n_splits; base += CMB_NT) {
+        const int sp = base + tid, cnt = min(CMB_NT, plan.n_splits - base);
+        const float m = sp < plan.n_splits ? part_m[row0 + (size_t)sp * s.R] : -INFINITY;
+        const float l = sp < plan.n_splits ? part_l[row0 + (size_t)sp * s.R] : 0.f;
+        const float* po = part_o + (row0 + (size_t)base * s.R) * kD + lane * 4;
+        for (int j0 = warp; j0 < cnt || j0 == warp; j0 += 4 * CMB_INFLIGHT) {
+            float4 o4[CMB_INFLIGHT];
+#pragma unroll
+            for (int u = 0; u < CMB_INFLIGHT; ++u) {
+                const int j = j0 + 4 * u;
+                o4[u] = j < cnt ? *reinterpret_cast<const float4*>(po + (size_t)j * sstride) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (j0 == warp) {                          // first round: weights of this batch of splits
+                M = block128_reduce(m, true, red);
+                if (M > Mrun) {                        // (only with more than 128 splits) rescale what was summed
+                    const float f = Mrun == -INFINITY ? 0.f : exp2f(Mrun - M);
+                    L *= f; acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
+                    Mrun = M;
+                }
+                const float w = m == -INFINITY ? 0.f : exp2f(m - Mrun);
+                L = fmaf(l, w, L);
+                sW[tid] = w;
+                __syncthreads();
+            }
+#pragma unroll
+            for (int u = 0; u < CMB_INFLIGHT; ++u) {
+                const int j = j0 + 4 * u;
+                const float w = j < cnt ? sW[j] : 0.f;
+                acc.x = fmaf(o4[u].x, w, acc.x); acc.y = fmaf(o4[u].y, w, acc.y);
+                acc.z = fmaf(o4[u].z, w, acc.z); acc.w = fmaf(o4[u].w, w, acc.w);
+            }
         }
-        __syncthreads();
-        sW[c] = w;
-        __syncthreads();
-        const float* po = part_o + (row0 + (size_t)base * s.R) * kD + c;
-        int j = 0;
-        for (; j + 4 <= cnt; j += 4) {
-            const float w0 = sW[j], w1 = sW[j + 1], w2 = sW[j + 2], w3 = sW[j + 3];
-            // a split without visible tokens (weight 0) may hold unwritten partial outputs
-            const float o0 = w0 != 0.f ? po[(size_t)(j + 0) * s.R * kD] : 0.f;
-            const float o1 = w1 != 0.f ? po[(size_t)(j + 1) * s.R * kD] : 0.f;
-            const float o2 = w2 != 0.f ? po[(size_t)(j + 2) * s.R * kD] : 0.f;
-            const float o3 = w3 != 0.f ? po[(size_t)(j + 3) * s.R * kD] : 0.f;
-            oc = fmaf(o0, w0, oc); oc = fmaf(o1, w1, oc); oc = fmaf(o2, w2, oc); oc = fmaf(o3, w3, oc);
-        }
-        for (; j < cnt; ++j) {
-            const float w0 = sW[j];
-            if (w0 != 0.f) oc = fmaf(po[(size_t)j * s.R * kD], w0, oc);
-        }
+        __syncthreads();                               // sW is rewritten by the next batch
     }
-    L = block128_reduce(L, false, red);
-    oc = oc / L;
+    *reinterpret_cast<float4*>(&sAcc[warp][lane * 4]) = acc;
+    L = block128_reduce(L, false, red);                // its barriers also publish sAcc
+    const float oc = ((sAcc[0][tid] + sAcc[1][tid]) + (sAcc[2][tid] + sAcc[3][tid])) / L;
     const float onorm = block128_reduce(oc * oc, false, red);
-    (ws + plan.off_o / 4)[orow * kD + c] = oc;
-    if (obf) obf[orow * kD + c] = __float2bfloat16(-2.f * oc);
-    if (c == 0) {
-        (ws + plan.off_lse2 / 4)[orow] = M + log2f(L);
+    (ws + plan.off_o / 4)[orow * kD + tid] = oc;
+    if (obf) obf[orow * kD + tid] = __float2bfloat16(-2.f * oc);
+    if (tid == 0) {
+        (ws + plan.off_lse2 / 4)[orow] = Mrun + log2f(L);
         (ws + plan.off_onorm / 4)[orow] = onorm;
     }
 }
@@ -404,7 +418,7 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
 }
 
 obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream) {
-    { ProfScope ps("combine", stream); simt_combine_kernel<<<s.B * s.Hkv * plan.rows_out, 128, 0, stream>>>(s, plan, (float*)ws); }
+    { ProfScope ps("combine", stream); simt_combine_kernel<<<s.B * s.Hkv * plan.rows_out, CMB_NT, 0, stream>>>(s, plan, (float*)ws); }
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

@@ -831,6 +831,10 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             tc_fence_before();
         }
+        if (my_tiles == 0 && valid) {                                        // no tile for this warpgroup: an all-zero partial
+            float4* dst = reinterpret_cast<float4*>(p.part_o + prow_idx * kD);
+            for (int j = 0; j < kD / 4; ++j) dst[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         if (valid) { p.part_m[prow_idx] = my_tiles > 0 && !failed ? m_used : -INFINITY; p.part_l[prow_idx] = l; }
     }
 
