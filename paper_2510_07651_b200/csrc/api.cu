@@ -116,7 +116,6 @@ obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_
     if (p->path == OBC_PATH_TC && !tc) return OBC_ERR_UNSUPPORTED;
     if (tc) return launch_score_tc(s, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);
     const SimtPlan plan = make_simt_plan(s, s.R, false);
-    OBC_CUDA_TRY(cudaMemsetAsync((char*)workspace + plan.off_flag, 0, 256, (cudaStream_t)stream));
     st = launch_simt_pass1_combine(s, plan, q.dtype, view(q), view(k), view(v), workspace, (cudaStream_t)stream);
     if (st != OBC_OK) return st;
     return launch_simt_pass2(s, plan, q.dtype, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);

@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(CH)
 decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt, TensorView vt,
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, const int32_t* state,
                     int step_pos, char* ws) {
+    pdl_wait();
     __shared__ __align__(16) float sQ[G][kD];
     __shared__ float sP[G][CH];
     __shared__ __align__(16) float sO[8][G][kD];
@@ -177,6 +178,7 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
 // one block of 128 threads per (b, g): merge the chunk partials
 __global__ void __launch_bounds__(kD)
 decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
+    pdl_wait();
     const int unit = blockIdx.x, c = threadIdx.x, G = s.G;
     __shared__ float red[4];
     for (int r = 0; r < G; ++r) {
@@ -210,6 +212,7 @@ template <int G>
 __global__ void __launch_bounds__(CH)
 decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc, const int32_t* pos,
                     const int32_t* state, int step_pos, char* ws) {
+    pdl_wait();
     __shared__ __align__(16) float sO[G][kD];
     __shared__ float sLse[G], sNo[G];
     __shared__ MinCand sMin[8];
@@ -299,6 +302,7 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
 
 __global__ void __launch_bounds__(128)
 decode_final_kernel(DecodeShape s, DecodePlan plan, int32_t* pos, int32_t* state, const char* ws) {
+    pdl_wait();
     const int unit = blockIdx.x * blockDim.x + threadIdx.x;
     if (unit >= s.B * s.Hkv) return;
     int live = state[unit * 4 + 0];
@@ -331,14 +335,10 @@ obc_status launch_g(const DecodeShape& s, const DecodePlan& plan, TensorView q, 
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
                     int step_pos, char* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
-    { ProfScope ps("decode_pass1", stream); decode_pass1_kernel<G><<<dim3(plan.chunks, units), CH, 0, stream>>>(s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws); }
-    OBC_CUDA_TRY(cudaGetLastError());
-    { ProfScope ps("decode_combine", stream); decode_combine_kernel<<<units, kD, 0, stream>>>(s, plan, ws); }
-    OBC_CUDA_TRY(cudaGetLastError());
-    { ProfScope ps("decode_score", stream); decode_score_kernel<G><<<dim3(plan.chunks, units), CH, 0, stream>>>(s, plan, vc, s_acc, pos, state, step_pos, ws); }
-    OBC_CUDA_TRY(cudaGetLastError());
-    { ProfScope ps("decode_final", stream); decode_final_kernel<<<(units + 127) / 128, 128, 0, stream>>>(s, plan, pos, state, ws); }
-    OBC_CUDA_TRY(cudaGetLastError());
+    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), 0, stream, 1, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
+    { ProfScope ps("decode_combine", stream); OBC_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(units), dim3(kD), 0, stream, 1, s, plan, ws)); }
+    { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G>, dim3(plan.chunks, units), dim3(CH), 0, stream, 1, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
+    { ProfScope ps("decode_final", stream); OBC_CUDA_TRY(launch_pdl(decode_final_kernel, dim3((units + 127) / 128), dim3(128), 0, stream, 1, s, plan, pos, state, ws)); }
     return OBC_OK;
 }
 

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <utility>
 #include "obcache.h"
 
 namespace obc {
@@ -95,6 +96,31 @@ bool tc_supported(const ScoreShape& s, int dtype, const TensorView& q);   // + b
 size_t tc_workspace_bytes(const ScoreShape& s);
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
                            float* scores, void* ws, cudaStream_t stream);
+
+// ---- programmatic dependent launch ------------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialization: its CTAs may
+// become resident while the preceding kernel of the stream is still draining.  A kernel executes
+// pdl_wait() before its first access to memory that an earlier kernel may have written (or may
+// still read, for its own writes); what precedes the wait is set-up that touches no such memory.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              int cluster_x, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 1;
+    if (cluster_x > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cluster_x; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    cfg.attrs = attr;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
 
 // ---- device helpers --------------------------------------------------------------------------
 __device__ __forceinline__ float warp_max(float x) {

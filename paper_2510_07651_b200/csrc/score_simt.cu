@@ -66,6 +66,7 @@ __device__ __forceinline__ void tile_gemm(const float* __restrict__ sA, const fl
 template <typename T>
 __global__ void __launch_bounds__(NT, 2)
 simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, TensorView v, float* ws) {
+    pdl_wait();
     extern __shared__ __align__(16) float smem[];
     float* sK = smem;                       // [TN][KS]
     float* sV = sK + TN * KS;               // [TN][kD]
@@ -77,6 +78,9 @@ simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
     const int N = seq_len(s, b);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float sl2 = s.scale * kLog2e;
+    // the status word of the workspace header is only raised by the tensor-core kernels
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0)
+        *reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(ws) + plan.off_flag) = 0u;
 
     load_rows<T>(sQ, kD, RC, min(RC, s.R - r0), [&](int row) {
         int r = r0 + row;
@@ -181,6 +185,7 @@ __device__ __forceinline__ float block128_reduce(float x, bool take_max, float* 
 
 __global__ void __launch_bounds__(CMB_NT)
 simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
+    pdl_wait();
     const int r = blockIdx.x % plan.rows_out, unit = blockIdx.x / plan.rows_out;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const size_t orow = (size_t)unit * plan.rows_out + r;
@@ -252,6 +257,7 @@ template <typename T>
 __global__ void __launch_bounds__(NT, 2)
 simt_pass2_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, TensorView v,
                   const float* ws, float* scores) {
+    pdl_wait();
     extern __shared__ __align__(16) float smem[];
     float* sK = smem;                       // [TN][KS]
     float* sV = sK + TN * KS;               // [TN][KS]
@@ -374,8 +380,7 @@ obc_status launch_pass1_typed(const ScoreShape& s, const SimtPlan& plan, TensorV
                               float* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv, chunks = (s.R + RC - 1) / RC;
     OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass1_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass1));
-    { ProfScope ps("simt_pass1", stream); simt_pass1_kernel<T><<<dim3(plan.n_splits, units, chunks), NT, kSmemPass1, stream>>>(s, plan, q, k, v, ws); }
-    OBC_CUDA_TRY(cudaGetLastError());
+    { ProfScope ps("simt_pass1", stream); OBC_CUDA_TRY(launch_pdl(simt_pass1_kernel<T>, dim3(plan.n_splits, units, chunks), dim3(NT), kSmemPass1, stream, 1, s, plan, q, k, v, ws)); }
     return launch_combine(s, plan, ws, stream);
 }
 
@@ -384,8 +389,7 @@ obc_status launch_pass2_typed(const ScoreShape& s, const SimtPlan& plan, TensorV
                               float* scores, float* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
     OBC_CUDA_TRY(cudaFuncSetAttribute(simt_pass2_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemPass2));
-    { ProfScope ps("simt_pass2", stream); simt_pass2_kernel<T><<<dim3((s.Nmax + TN - 1) / TN, units), NT, kSmemPass2, stream>>>(s, plan, q, k, v, ws, scores); }
-    OBC_CUDA_TRY(cudaGetLastError());
+    { ProfScope ps("simt_pass2", stream); OBC_CUDA_TRY(launch_pdl(simt_pass2_kernel<T>, dim3((s.Nmax + TN - 1) / TN, units), dim3(NT), kSmemPass2, stream, 1, s, plan, q, k, v, ws, scores)); }
     return OBC_OK;
 }
 }  // namespace
@@ -418,8 +422,7 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
 }
 
 obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream) {
-    { ProfScope ps("combine", stream); simt_combine_kernel<<<s.B * s.Hkv * plan.rows_out, CMB_NT, 0, stream>>>(s, plan, (float*)ws); }
-    OBC_CUDA_TRY(cudaGetLastError());
+    { ProfScope ps("combine", stream); OBC_CUDA_TRY(launch_pdl(simt_combine_kernel, dim3(s.B * s.Hkv * plan.rows_out), dim3(CMB_NT), 0, stream, 1, s, plan, (float*)ws)); }
     return OBC_OK;
 }
 

@@ -304,6 +304,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // buffer and constant-slot rings.
     TileWalk tw;
     tw.init(p);
+    if (!(warp == 0 && lane == 0)) pdl_wait();       // the producer thread waits after its first K/V copies
     if (warp == 0) {
         // ===================================== TMA producer =====================================
         if (lane == 0) {
@@ -312,6 +313,17 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (; !tw.done() && !failed; tw.next()) {
                 const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv, t0 = tw.tile * TILE;
                 for (int c = 0; c < p.n_chunks; ++c, ++item) {
+                    const uint32_t st = item % NSTAGE, use = item / NSTAGE;
+                    if (!mbar_wait(bar(BAR_EMPTY + st), (use & 1) ^ 1)) { failed = true; break; }
+                    mbar_expect_tx(bar(BAR_FULL + st), 2 * kOperandBytes);
+                    const uint32_t dk = sbase + OFF_K + st * kOperandBytes, dv = sbase + OFF_V + st * kOperandBytes;
+                    tma_load_4d(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b);
+                    tma_load_4d(dk + kHalfBytes, &map_k, bar(BAR_FULL + st), 64, t0, g, b);
+                    tma_load_4d(dv, &map_v, bar(BAR_FULL + st), 0, t0, g, b);
+                    tma_load_4d(dv + kHalfBytes, &map_v, bar(BAR_FULL + st), 64, t0, g, b);
+                    // K, V and the sequence lengths were read by pass 1 of this call, so the first tile
+                    // may be fetched while the preceding kernel drains; -2 O is that kernel's output
+                    if (item == 0) pdl_wait();
                     if (reload_qo_every_item || unit != qo_unit) {
                         if (!mbar_wait(bar(BAR_QO_EMPTY), (qo_loads & 1) ^ 1)) { failed = true; break; }
                         mbar_expect_tx(bar(BAR_QO_FULL), qo_bytes);
@@ -323,14 +335,6 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         tma_load_2d(sbase + OFF_O + kHalfBytes, &map_o, bar(BAR_QO_FULL), 64, orow);
                         qo_unit = unit; ++qo_loads;
                     }
-                    const uint32_t st = item % NSTAGE, use = item / NSTAGE;
-                    if (!mbar_wait(bar(BAR_EMPTY + st), (use & 1) ^ 1)) { failed = true; break; }
-                    mbar_expect_tx(bar(BAR_FULL + st), 2 * kOperandBytes);
-                    const uint32_t dk = sbase + OFF_K + st * kOperandBytes, dv = sbase + OFF_V + st * kOperandBytes;
-                    tma_load_4d(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b);
-                    tma_load_4d(dk + kHalfBytes, &map_k, bar(BAR_FULL + st), 64, t0, g, b);
-                    tma_load_4d(dv, &map_v, bar(BAR_FULL + st), 0, t0, g, b);
-                    tma_load_4d(dv + kHalfBytes, &map_v, bar(BAR_FULL + st), 64, t0, g, b);
                 }
             }
             // drain: every copy this thread issued must have landed before the CTA may exit
@@ -614,10 +618,6 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int split = blockIdx.x, vu = blockIdx.y;
     const int unit = vu / p.n_chunks, c = vu % p.n_chunks;
     const int b = unit / p.Hkv, g = unit % p.Hkv;
-    const int N = tc_seq_len_raw(p.seq_lens, b, p.Nmax);
-    const int tile_lo = split * p.tiles_per_split;
-    const int tile_hi = min(tile_lo + p.tiles_per_split, (N + TILE - 1) / TILE);
-    const int n_tiles = max(tile_hi - tile_lo, 0);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), 1); }
@@ -634,6 +634,13 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    pdl_wait();                                    // nothing above reads or writes global memory
+    // the status word starts at 0: no wait of this call can have given up yet (each lasts seconds)
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.status = 0u;
+    const int N = tc_seq_len_raw(p.seq_lens, b, p.Nmax);
+    const int tile_lo = split * p.tiles_per_split;
+    const int tile_hi = min(tile_lo + p.tiles_per_split, (N + TILE - 1) / TILE);
+    const int n_tiles = max(tile_hi - tile_lo, 0);
 
     if (warp == 0) {
         // ===================================== TMA producer =====================================
@@ -936,7 +943,6 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     const TcChunks ch = tc_chunks(s.R);
     const SimtPlan plan = make_tc_plan(s);
     char* wsb = (char*)ws;
-    OBC_CUDA_TRY(cudaMemsetAsync(wsb + plan.off_flag, 0, 256, stream));
     const int units = s.B * s.Hkv;
     CUtensorMap mq, mo, mk, mv;
     {
@@ -967,8 +973,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.status = (unsigned int*)(wsb + plan.off_flag);
         OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
         { ProfScope ps("tc_pass1", stream);
-          tc_pass1_kernel<<<dim3(plan.n_splits / 2, units * ch.n_chunks), kThreadsP1, kSmemP1, stream>>>(mq, mk, mv, p1); }
-        OBC_CUDA_TRY(cudaGetLastError());
+          OBC_CUDA_TRY(launch_pdl(tc_pass1_kernel, dim3(plan.n_splits / 2, units * ch.n_chunks), dim3(kThreadsP1), kSmemP1, stream, 1, mq, mk, mv, p1)); }
         obc_status st = launch_combine(s, plan, ws, stream);
         if (st != OBC_OK) return st;
     }
@@ -985,8 +990,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
 
     auto launch = [&](auto kernel) -> obc_status {
         OBC_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-        { ProfScope ps("tc_pass2", stream); kernel<<<grid, kThreads, kSmemBytes, stream>>>(mq, mo, mk, mv, p); }
-        OBC_CUDA_TRY(cudaGetLastError());
+        { ProfScope ps("tc_pass2", stream); OBC_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mq, mo, mk, mv, p)); }
         return OBC_OK;
     };
     if (s.variants == OBC_VAR_VK) return launch(tc_pass2_kernel<OBC_VAR_VK>);

@@ -30,6 +30,7 @@ __device__ __forceinline__ int budget_of(const SelectShape& s, int b) { return s
 
 __global__ void __launch_bounds__(256)
 pool_key_kernel(SelectShape s, const float* __restrict__ scores, uint32_t* __restrict__ keys) {
+    pdl_wait();
     const int unit = blockIdx.y, b = unit / s.Hkv;
     const int N = seq_len(s, b), lo = s.n_sink, hi = N - s.n_recent;
     const int p = blockIdx.x * blockDim.x + threadIdx.x;
@@ -60,6 +61,7 @@ constexpr int SEL_NT = 1024;
 
 __global__ void __launch_bounds__(SEL_NT)
 select_kernel(SelectShape s, const uint32_t* __restrict__ keys_all, int32_t* __restrict__ idx_all) {
+    pdl_wait();
     __shared__ uint32_t hist[256];
     __shared__ uint32_t sh_prefix, sh_remaining;
     __shared__ uint32_t warp_gt[32], warp_eq[32];
@@ -187,6 +189,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(ClusterShared));
     float* stage = reinterpret_cast<float*>(keys + seg_cap);          // seg_cap + pool_kernel - 1 floats
 
+    pdl_wait();
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
     const int unit = blockIdx.x / C, b = unit / s.Hkv;
@@ -350,6 +353,7 @@ __global__ void __launch_bounds__(256)
 gather_kernel(int units, int Hkv, int idx_stride, int vecs, int elem_bytes,
               TensorView k, TensorView v, TensorView ko, TensorView vo,
               const int32_t* __restrict__ idx, const float* __restrict__ s_in, float* __restrict__ s_out, int Nmax) {
+    pdl_wait();
     const int unit = blockIdx.y, b = unit / Hkv, g = unit % Hkv;
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     const int j = e / vecs, c = e % vecs;
@@ -397,16 +401,14 @@ obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx
         int max_clusters = 0;
         if (cudaOccupancyMaxActiveClusters(&max_clusters, select_cluster_kernel, &cfg) == cudaSuccess && max_clusters > 0) {
             { ProfScope ps("select_cluster", stream);
-              OBC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel, s, scores, idx, seg_cap)); }
+              OBC_CUDA_TRY(launch_pdl(select_cluster_kernel, dim3((unsigned)(units * C)), dim3(CL_NT), smem, stream, C, s, scores, idx, seg_cap)); }
             return OBC_OK;
         }
         (void)cudaGetLastError();                  // the device cannot host such a cluster: one CTA per head
     }
     uint32_t* keys = (uint32_t*)ws;
-    { ProfScope ps("pool_key", stream); pool_key_kernel<<<dim3((s.Nmax + 255) / 256, units), 256, 0, stream>>>(s, scores, keys); }
-    OBC_CUDA_TRY(cudaGetLastError());
-    { ProfScope ps("select", stream); select_kernel<<<units, SEL_NT, 0, stream>>>(s, keys, idx); }
-    OBC_CUDA_TRY(cudaGetLastError());
+    { ProfScope ps("pool_key", stream); OBC_CUDA_TRY(launch_pdl(pool_key_kernel, dim3((s.Nmax + 255) / 256, units), dim3(256), 0, stream, 1, s, scores, keys)); }
+    { ProfScope ps("select", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(units), dim3(SEL_NT), 0, stream, 1, s, (const uint32_t*)keys, idx)); }
     return OBC_OK;
 }
 
@@ -417,10 +419,9 @@ obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_byte
     const long long total = (long long)idx_stride * vecs;
     {
         ProfScope ps("gather", stream);
-        gather_kernel<<<dim3((unsigned)((total + 255) / 256), B * Hkv), 256, 0, stream>>>(
-            B * Hkv, Hkv, idx_stride, vecs, elem_bytes, k, v, ko, vo, idx, s_in, s_out, Nmax);
+        OBC_CUDA_TRY(launch_pdl(gather_kernel, dim3((unsigned)((total + 255) / 256), B * Hkv), dim3(256), 0, stream, 1,
+                                B * Hkv, Hkv, idx_stride, vecs, elem_bytes, k, v, ko, vo, idx, s_in, s_out, Nmax));
     }
-    OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
 
