@@ -502,8 +502,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 // Rows of the window (one chunk of up to 128) sit on the MMA M dimension, so a TMEM lane holds one
 // row and the softmax thread that owns it reduces along the tile without cross-thread traffic.
 // Two softmax warpgroups take alternate token tiles; each keeps its own running statistics and its
-// own output accumulator, i.e. the CTA produces two partial results, which the combine kernel
-// merges like any other token split.  For tile t and warpgroup w = t mod 2:
+// own output accumulator; at the end the CTA merges the two and writes one partial result per
+// token split, which the combine kernel merges across splits.  For tile t and warpgroup w = t mod 2:
 //     S_w  = Q_chunk . K_tile^T                    (tcgen05, accumulator in TMEM)
 //     P_w  = exp2(S_w * scale*log2e - m_used)      (registers -> bf16 -> TMEM, over S_w's columns)
 //     O_w += P_w . V_tile                          (tcgen05: A operand from TMEM, V as MN-major B)
@@ -535,8 +535,8 @@ struct P1Params {
     float scale;
     int causal;
     int n_chunks, chunk_rows;
-    int n_splits, tiles_per_split;                         // CTAs per (unit, chunk); each writes 2 partials
-    float* part_m; float* part_l; float* part_o;           // [units][2 * n_splits][R] (x d for part_o)
+    int n_splits, tiles_per_split;                         // CTAs per (unit, chunk); each writes one partial
+    float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
     unsigned int* status;
 };
 
@@ -818,31 +818,68 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (lane == 0) mbar_arrive(bar(P1_PFULL + w));
         }
 
-        // the two partial results of this CTA: slot 2*split + w
-        const size_t prow_idx = ((size_t)unit * (2 * p.n_splits) + 2 * split + w) * p.R + r;
-        if (my_tiles > 0 && !failed) {
-            if (!mbar_wait(bar(P1_ODONE), 0)) failed = true;
+        // ---- the CTA's partial result: merge the two warpgroups, then store whole 512-byte rows ----
+        // Exchange buffers in shared memory that the MMAs no longer read: statistics in the Q region,
+        // a [128 rows][32 x 16 B] tile in the first K/V stage, 16-byte chunks XOR-swizzled by the row.
+        float* xm = reinterpret_cast<float*>(smem + P1_OFF_Q);
+        float* xl = xm + 128;
+        uint8_t* xo = smem + P1_OFF_K;
+        bool have = my_tiles > 0 && !failed;
+        if (n_tiles > 0) {                                                   // all MMAs done: accumulators final, smem free
+            if (!mbar_wait(bar(P1_ODONE), 0)) { failed = true; have = false; }
             tc_fence_after();
+        }
+        if (w == 1) {
+            xm[row] = have ? m_used : -INFINITY;
+            xl[row] = l;
+            if (have) {
 #pragma unroll 1
-            for (int q4 = 0; q4 < 4 && !failed; ++q4) {
-                uint32_t ov[32];
-                tc_ld32(tO + q4 * 32, ov);
-                tc_wait_ld32(ov);
-                if (valid) {
-                    float4* dst = reinterpret_cast<float4*>(p.part_o + prow_idx * kD + q4 * 32);
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t ov[32];
+                    tc_ld32(tO + q4 * 32, ov);
+                    tc_wait_ld32(ov);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        dst[j] = make_float4(__uint_as_float(ov[4 * j]), __uint_as_float(ov[4 * j + 1]),
-                                             __uint_as_float(ov[4 * j + 2]), __uint_as_float(ov[4 * j + 3]));
+                        *reinterpret_cast<uint4*>(xo + row * 512 + (((q4 * 8 + j) ^ (row & 31)) << 4)) =
+                            make_uint4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
                 }
             }
-            tc_fence_before();
         }
-        if (my_tiles == 0 && valid) {                                        // no tile for this warpgroup: an all-zero partial
-            float4* dst = reinterpret_cast<float4*>(p.part_o + prow_idx * kD);
-            for (int j = 0; j < kD / 4; ++j) dst[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        asm volatile("bar.sync 1, 256;" ::: "memory");                       // both softmax warpgroups
+        if (w == 0) {
+            const float ma = have ? m_used : -INFINITY, mb = xm[row];
+            const float M = fmaxf(ma, mb);
+            const float fa = ma == -INFINITY ? 0.f : fast_exp2(ma - M), fb = mb == -INFINITY ? 0.f : fast_exp2(mb - M);
+#pragma unroll 1
+            for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t ov[32];
+                if (have) { tc_ld32(tO + q4 * 32, ov); tc_wait_ld32(ov); }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint4* cell = reinterpret_cast<uint4*>(xo + row * 512 + (((q4 * 8 + j) ^ (row & 31)) << 4));
+                    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (mb != -INFINITY) {
+                        const uint4 u = *cell;
+                        o = make_float4(__uint_as_float(u.x) * fb, __uint_as_float(u.y) * fb, __uint_as_float(u.z) * fb, __uint_as_float(u.w) * fb);
+                    }
+                    if (have) {
+                        o.x = fmaf(__uint_as_float(ov[4 * j]), fa, o.x);     o.y = fmaf(__uint_as_float(ov[4 * j + 1]), fa, o.y);
+                        o.z = fmaf(__uint_as_float(ov[4 * j + 2]), fa, o.z); o.w = fmaf(__uint_as_float(ov[4 * j + 3]), fa, o.w);
+                    }
+                    *cell = make_uint4(__float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z), __float_as_uint(o.w));
+                }
+            }
+            const size_t prow0 = ((size_t)unit * p.n_splits + split) * p.R + (size_t)c * p.chunk_rows;   // row 0 of the chunk
+            if (valid) { p.part_m[prow0 + row] = M; p.part_l[prow0 + row] = fmaf(l, fa, xl[row] * fb); }
+            asm volatile("bar.sync 2, 128;" ::: "memory");                   // warpgroup 0: the merged tile is complete
+            for (int rr = 0; rr < 32; ++rr) {                                // one coalesced 512-byte row per instruction
+                const int orow = lane_grp * 32 + rr;
+                if (orow < rows_valid)
+                    *reinterpret_cast<uint4*>(p.part_o + (prow0 + orow) * kD + lane * 4) =
+                        *reinterpret_cast<const uint4*>(xo + orow * 512 + ((lane ^ (orow & 31)) << 4));
+            }
         }
-        if (valid) { p.part_m[prow_idx] = my_tiles > 0 && !failed ? m_used : -INFINITY; p.part_l[prow_idx] = l; }
+        tc_fence_before();
     }
 
     if (failed) atomicExch(p.status, 1u);
@@ -919,7 +956,7 @@ static SimtPlan make_tc_plan(const ScoreShape& s) {
     if (n > tiles) n = tiles;
     SimtPlan p{};
     p.tiles_per_split = (tiles + n - 1) / n;                                   // per pass-1 CTA
-    p.n_splits = 2 * ((tiles + p.tiles_per_split - 1) / p.tiles_per_split);    // partial results: two per CTA
+    p.n_splits = (tiles + p.tiles_per_split - 1) / p.tiles_per_split;          // CTAs, and partial results, per unit
     p.rows_out = ch.rows_out;
     p.want_obf = 1;
     const size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, orow = (size_t)units * ch.rows_out;
@@ -967,13 +1004,13 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.B = s.B; p1.Hq = s.Hq; p1.Hkv = s.Hkv; p1.G = s.G; p1.W = s.W; p1.R = s.R; p1.Nmax = s.Nmax;
         p1.seq_lens = s.seq_lens; p1.scale = s.scale; p1.causal = s.causal;
         p1.n_chunks = ch.n_chunks; p1.chunk_rows = ch.chunk_rows;
-        p1.n_splits = plan.n_splits / 2; p1.tiles_per_split = plan.tiles_per_split;
+        p1.n_splits = plan.n_splits; p1.tiles_per_split = plan.tiles_per_split;
         p1.part_m = (float*)(wsb + plan.off_part_m); p1.part_l = (float*)(wsb + plan.off_part_l);
         p1.part_o = (float*)(wsb + plan.off_part_o);
         p1.status = (unsigned int*)(wsb + plan.off_flag);
         OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
         { ProfScope ps("tc_pass1", stream);
-          OBC_CUDA_TRY(launch_pdl(tc_pass1_kernel, dim3(plan.n_splits / 2, units * ch.n_chunks), dim3(kThreadsP1), kSmemP1, stream, 1, mq, mk, mv, p1)); }
+          OBC_CUDA_TRY(launch_pdl(tc_pass1_kernel, dim3(plan.n_splits, units * ch.n_chunks), dim3(kThreadsP1), kSmemP1, stream, 1, mq, mk, mv, p1)); }
         obc_status st = launch_combine(s, plan, ws, stream);
         if (st != OBC_OK) return st;
     }
