@@ -38,7 +38,8 @@ typedef enum {
     OBC_ERR_ALIGN = -4,        /* base pointer or stride not 16-byte aligned */
     OBC_ERR_WORKSPACE = -5,    /* workspace missing or smaller than obc_*_workspace() says */
     OBC_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed; see obc_last_cuda_error() */
-    OBC_ERR_TIMEOUT = -7       /* a bounded device-side wait gave up */
+    OBC_ERR_TIMEOUT = -7,      /* a bounded device-side wait gave up */
+    OBC_ERR_CAPACITY = -8      /* the problem exceeds the fixed capacity of an allocation-free entry point */
 } obc_status;
 
 typedef enum { OBC_F32 = 0, OBC_BF16 = 1 } obc_dtype;
@@ -143,6 +144,32 @@ obc_status obc_select_workspace(const obc_select_params* p, size_t* bytes /* hos
  */
 obc_status obc_select(const obc_select_params* p, const float* scores, int32_t* idx,
                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * obc_select_noalloc: obc_select for callers that have no device memory to give as workspace and
+ * may not allocate any.  (The paper has no counterpart: this is a packaging variant of obc_select.)
+ *
+ * Typical callers: a plug-in inside an inference engine that owns the whole device heap and hands
+ * out no allocator; a serving loop whose memory budget was fixed at start-up, where cudaMalloc
+ * would also stall every stream of the device; code that runs after start-up under a policy of
+ * "no allocation on the hot path".  Such callers still pass the scores and the index buffer; only
+ * the scratch memory is the library's own.
+ *
+ * The scratch (one 32-bit key per score) lives in a fixed array inside the library image,
+ * OBC_SELECT_NOALLOC_MAX_KEYS keys = 4 MiB, which every GPU that loads the library holds until the
+ * process exits.  Problems with batch * n_kv_heads * max_len > OBC_SELECT_NOALLOC_MAX_KEYS are
+ * rejected with OBC_ERR_CAPACITY and nothing is launched; use obc_select with a caller-owned
+ * workspace for those.  The call runs the one-CTA-per-head kernels and gives the same idx, bit
+ * for bit, as obc_select; it calls neither cudaMalloc nor cudaFree nor any allocating routine.
+ *
+ * First call on a device: looks up the device address of the scratch array (a host-side runtime
+ * query, done once per device with that device current).  Make that first call outside any stream
+ * capture.  All calls on one device share the one array and leave their keys in it: no part of it
+ * needs to start at zero (every key that is read was written by the same call), but two calls
+ * whose kernels may overlap on the GPU (different streams) race on it; serialise them.
+ */
+#define OBC_SELECT_NOALLOC_MAX_KEYS (1 << 20)
+obc_status obc_select_noalloc(const obc_select_params* p, const float* scores, int32_t* idx, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * obc_compact: gather of the kept rows (Algorithm 2's gather/concatenate):

@@ -23,7 +23,8 @@ VARIANTS = {"V": OBC_VAR_V, "K": OBC_VAR_K, "VK": OBC_VAR_VK, "ATTN": OBC_VAR_AT
 POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
-EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_status", "obc_select_workspace", "obc_select", "obc_compact",
+EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_status", "obc_select_workspace", "obc_select",
+           "obc_select_noalloc", "obc_compact",
            "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
            "obc_status_string", "obc_last_cuda_error", "obc_version"]
 
@@ -84,6 +85,7 @@ def lib():
         L.obc_score_status.argtypes = [vp, vp]
         L.obc_select_workspace.argtypes = [C.POINTER(obc_select_params), sz]
         L.obc_select.argtypes = [C.POINTER(obc_select_params), vp, vp, vp, C.c_size_t, vp]
+        L.obc_select_noalloc.argtypes = [C.POINTER(obc_select_params), vp, vp, vp]
         L.obc_compact.argtypes = [C.c_int32] * 5 + [obc_tensor, obc_tensor, vp, obc_tensor, obc_tensor, vp, vp, vp]
         L.obc_decode_workspace.argtypes = [C.POINTER(obc_decode_params), sz]
         L.obc_decode_step.argtypes = [C.POINTER(obc_decode_params)] + [obc_tensor] * 5 + [vp, vp, vp, C.c_int32, vp, C.c_size_t, vp]
@@ -198,6 +200,23 @@ def obc_select(scores, *, budget=0, budgets=None, idx_stride=None, seq_lens=None
     ws = _workspace(obc_select_workspace(p), scores, workspace)
     _check(lib().obc_select(C.byref(p), scores.data_ptr(), idx.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
            "obc_select")
+    return idx
+
+
+SELECT_NOALLOC_MAX_KEYS = 1 << 20
+
+
+def obc_select_noalloc(scores, idx, *, budget=0, budgets=None, seq_lens=None, n_sink=0, n_recent=0,
+                       pool="none", pool_kernel=1):
+    """obc_select without a workspace, for callers that may not allocate device memory (an engine
+    plug-in without an allocator, a serving loop with a fixed memory budget): the key scratch is a
+    fixed 4 MiB array inside the library.  `idx` [B,Hkv,idx_stride] int32 is the caller's buffer;
+    this wrapper allocates nothing either.  Raises ObcError(OBC_ERR_CAPACITY) when
+    B*Hkv*Nmax > SELECT_NOALLOC_MAX_KEYS.  Calls on one device share the scratch: do not let two
+    of them overlap on the GPU; make the first call on a device outside stream capture."""
+    p = select_params(scores, budget=budget, budgets=budgets, idx_stride=idx.shape[2], seq_lens=seq_lens,
+                      n_sink=n_sink, n_recent=n_recent, pool=pool, pool_kernel=pool_kernel)
+    _check(lib().obc_select_noalloc(C.byref(p), scores.data_ptr(), idx.data_ptr(), _stream()), "obc_select_noalloc")
     return idx
 
 

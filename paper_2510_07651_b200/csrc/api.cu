@@ -166,6 +166,14 @@ obc_status obc_select(const obc_select_params* p, const float* scores, int32_t* 
     return launch_select(s, scores, idx, workspace, (cudaStream_t)stream);
 }
 
+obc_status obc_select_noalloc(const obc_select_params* p, const float* scores, int32_t* idx, void* stream) {
+    SelectShape s;
+    obc_status st = resolve_select(p, &s);
+    if (st != OBC_OK) return st;
+    if (!scores || !idx) return OBC_ERR_NULL;
+    return launch_select_static(s, scores, idx, (cudaStream_t)stream);
+}
+
 obc_status obc_compact(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int32_t idx_stride,
                        int32_t max_len, obc_tensor k, obc_tensor v, const int32_t* idx,
                        obc_tensor k_out, obc_tensor v_out,
@@ -275,6 +283,7 @@ const char* obc_status_string(obc_status s) {
         case OBC_ERR_WORKSPACE: return "workspace missing or too small";
         case OBC_ERR_CUDA: return "a CUDA call failed (see obc_last_cuda_error)";
         case OBC_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case OBC_ERR_CAPACITY: return "problem larger than the fixed capacity of the allocation-free entry point";
     }
     return "unknown status";
 }

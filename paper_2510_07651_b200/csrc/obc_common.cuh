@@ -75,6 +75,7 @@ struct SelectShape {
 };
 size_t select_workspace_bytes(int B, int Hkv, int Nmax);
 obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx, void* ws, cudaStream_t stream);
+obc_status launch_select_static(const SelectShape& s, const float* scores, int32_t* idx, cudaStream_t stream);
 obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_bytes,
                          TensorView k, TensorView v, TensorView ko, TensorView vo, const int32_t* idx,
                          const float* s_in, float* s_out, cudaStream_t stream);

@@ -13,6 +13,7 @@
 #include "obc_common.cuh"
 
 #include <cooperative_groups.h>
+#include <mutex>
 namespace cg = cooperative_groups;
 
 namespace obc {
@@ -407,6 +408,42 @@ obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx
         (void)cudaGetLastError();                  // the device cannot host such a cluster: one CTA per head
     }
     uint32_t* keys = (uint32_t*)ws;
+    { ProfScope ps("pool_key", stream); OBC_CUDA_TRY(launch_pdl(pool_key_kernel, dim3((s.Nmax + 255) / 256, units), dim3(256), 0, stream, 1, s, scores, keys)); }
+    { ProfScope ps("select", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(units), dim3(SEL_NT), 0, stream, 1, s, (const uint32_t*)keys, idx)); }
+    return OBC_OK;
+}
+
+// ---- allocation-free variant: the key scratch is part of the library image -----------------------
+// One key per score, shared by every call on the device (see obc_select_noalloc in obcache.h).
+static __device__ __align__(256) uint32_t g_select_keys[OBC_SELECT_NOALLOC_MAX_KEYS];
+
+// Device address of g_select_keys on the current device.  In host code the array's name only
+// stands for the symbol; the address a kernel can use comes from the runtime, per device.
+static obc_status select_static_keys(uint32_t** out) {
+    constexpr int kMaxDev = 64;
+    static std::mutex mu;
+    static uint32_t* ptrs[kMaxDev] = {};
+    int dev = 0;
+    OBC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDev) return OBC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!ptrs[dev]) {
+        uint32_t* ptr = nullptr;
+        OBC_CUDA_TRY(cudaGetSymbolAddress((void**)&ptr, g_select_keys));
+        if (!ptr) return OBC_ERR_CUDA;
+        ptrs[dev] = ptr;
+    }
+    *out = ptrs[dev];
+    return OBC_OK;
+}
+
+obc_status launch_select_static(const SelectShape& s, const float* scores, int32_t* idx, cudaStream_t stream) {
+    const int units = s.B * s.Hkv;
+    if ((long long)units * s.Nmax > (long long)OBC_SELECT_NOALLOC_MAX_KEYS) return OBC_ERR_CAPACITY;
+    uint32_t* keys = nullptr;
+    obc_status st = select_static_keys(&keys);
+    if (st != OBC_OK) return st;
+    // every key a head reads is written by pool_key_kernel of this call: nothing has to be cleared
     { ProfScope ps("pool_key", stream); OBC_CUDA_TRY(launch_pdl(pool_key_kernel, dim3((s.Nmax + 255) / 256, units), dim3(256), 0, stream, 1, s, scores, keys)); }
     { ProfScope ps("select", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(units), dim3(SEL_NT), 0, stream, 1, s, (const uint32_t*)keys, idx)); }
     return OBC_OK;
