@@ -95,6 +95,20 @@ class ClockSampler:
                 "window": where}
 
 
+def ncu_traffic(kernel):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary, or None when there is no
+    capture or the kernel source has changed since it was taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "traffic.txt")
+    if not os.path.exists(path):
+        return None
+    rec = dict(l.split() for l in open(path) if l.strip() and not l.startswith("#"))
+    src = os.path.join(ROOT, "paper_2510_07651_b200", "csrc", "score_tc.cu")
+    if rec.get("source_sha256") != hashlib.sha256(open(src, "rb").read()).hexdigest():
+        return None
+    return float(rec[kernel]) if kernel in rec else None
+
+
 def make_case(seed):
     from paper_2510_07651_b200 import synth
     return synth.config(2, seed=seed)
@@ -314,9 +328,7 @@ def run_ours(args):
             ach = alg[kind][1] / dom_avg_s / 1e12
             roof.update(bound="tensor", achieved=ach, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
                         frac=ach / peaks["bf16_tflops_sustained"], peak_source=f"{peaks['source']} cuBLAS bf16 sustained")
-    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_file):
-        roof["traffic"] = json.load(open(traffic_file)).get(dom_name)
+    roof["traffic"] = ncu_traffic(dom_name)
     kernels = {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}
 
     # ---- CPU baseline: the checker as it stands, on this machine's host cores ----------------------
