@@ -819,61 +819,55 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
 
         // ---- the CTA's partial result: merge the two warpgroups, then store whole 512-byte rows ----
-        // Exchange buffers in shared memory that the MMAs no longer read: statistics in the Q region,
-        // a [128 rows][32 x 16 B] tile in the first K/V stage, 16-byte chunks XOR-swizzled by the row.
-        float* xm = reinterpret_cast<float*>(smem + P1_OFF_Q);
-        float* xl = xm + 128;
+        // A warp may read its 32 TMEM lanes in any column, so the thread of row r in either
+        // warpgroup can read both accumulators of that row.  The warpgroups exchange (m, l) through
+        // shared memory (the Q region, which the MMAs no longer read), then warpgroup w merges
+        // head-dim columns [64 w, 64 w + 64) into a [128 rows][32 x 16 B] tile in the first K/V stage
+        // (16-byte chunks XOR-swizzled by the row), and all eight warps store 512-byte rows.
+        float* xm = reinterpret_cast<float*>(smem + P1_OFF_Q);               // [2][128]
+        float* xl = xm + 256;                                                // [2][128]
         uint8_t* xo = smem + P1_OFF_K;
         bool have = my_tiles > 0 && !failed;
         if (n_tiles > 0) {                                                   // all MMAs done: accumulators final, smem free
             if (!mbar_wait(bar(P1_ODONE), 0)) { failed = true; have = false; }
             tc_fence_after();
         }
-        if (w == 1) {
-            xm[row] = have ? m_used : -INFINITY;
-            xl[row] = l;
-            if (have) {
-#pragma unroll 1
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint32_t ov[32];
-                    tc_ld32(tO + q4 * 32, ov);
-                    tc_wait_ld32(ov);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        *reinterpret_cast<uint4*>(xo + row * 512 + (((q4 * 8 + j) ^ (row & 31)) << 4)) =
-                            make_uint4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
-                }
-            }
-        }
+        xm[w * 128 + row] = have ? m_used : -INFINITY;
+        xl[w * 128 + row] = l;
         asm volatile("bar.sync 1, 256;" ::: "memory");                       // both softmax warpgroups
-        if (w == 0) {
-            const float ma = have ? m_used : -INFINITY, mb = xm[row];
-            const float M = fmaxf(ma, mb);
-            const float fa = ma == -INFINITY ? 0.f : fast_exp2(ma - M), fb = mb == -INFINITY ? 0.f : fast_exp2(mb - M);
+        {
+            const float m0 = xm[row], m1 = xm[128 + row];
+            const float M = fmaxf(m0, m1);
+            const float f0 = m0 == -INFINITY ? 0.f : fast_exp2(m0 - M), f1 = m1 == -INFINITY ? 0.f : fast_exp2(m1 - M);
+            const uint32_t tO0 = tmem_base + lane_addr + 256u + w * 64u, tO1 = tO0 + 128u;   // this half of O_0 and O_1
+            const size_t prow0 = ((size_t)unit * p.n_splits + split) * p.R + (size_t)c * p.chunk_rows;   // row 0 of the chunk
+            if (w == 0 && valid) { p.part_m[prow0 + row] = M; p.part_l[prow0 + row] = fmaf(xl[row], f0, xl[128 + row] * f1); }
 #pragma unroll 1
-            for (int q4 = 0; q4 < 4; ++q4) {
-                uint32_t ov[32];
-                if (have) { tc_ld32(tO + q4 * 32, ov); tc_wait_ld32(ov); }
+            for (int q = 0; q < 2; ++q) {
+                // CTA-uniform: warpgroup 0 owns tiles iff the split has any, warpgroup 1 iff it has two or more
+                // (an accumulator that no MMA wrote is never read; one whose row saw no token holds zeros)
+                uint32_t oa[32], ob[32];
+                if (n_tiles > 0) { tc_ld32(tO0 + q * 32, oa); tc_wait_ld32(oa); }
+                if (n_tiles > 1) { tc_ld32(tO1 + q * 32, ob); tc_wait_ld32(ob); }
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    uint4* cell = reinterpret_cast<uint4*>(xo + row * 512 + (((q4 * 8 + j) ^ (row & 31)) << 4));
                     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (mb != -INFINITY) {
-                        const uint4 u = *cell;
-                        o = make_float4(__uint_as_float(u.x) * fb, __uint_as_float(u.y) * fb, __uint_as_float(u.z) * fb, __uint_as_float(u.w) * fb);
+                    if (n_tiles > 0)
+                        o = make_float4(__uint_as_float(oa[4 * j]) * f0, __uint_as_float(oa[4 * j + 1]) * f0,
+                                        __uint_as_float(oa[4 * j + 2]) * f0, __uint_as_float(oa[4 * j + 3]) * f0);
+                    if (n_tiles > 1) {
+                        o.x = fmaf(__uint_as_float(ob[4 * j]), f1, o.x);     o.y = fmaf(__uint_as_float(ob[4 * j + 1]), f1, o.y);
+                        o.z = fmaf(__uint_as_float(ob[4 * j + 2]), f1, o.z); o.w = fmaf(__uint_as_float(ob[4 * j + 3]), f1, o.w);
                     }
-                    if (have) {
-                        o.x = fmaf(__uint_as_float(ov[4 * j]), fa, o.x);     o.y = fmaf(__uint_as_float(ov[4 * j + 1]), fa, o.y);
-                        o.z = fmaf(__uint_as_float(ov[4 * j + 2]), fa, o.z); o.w = fmaf(__uint_as_float(ov[4 * j + 3]), fa, o.w);
-                    }
-                    *cell = make_uint4(__float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z), __float_as_uint(o.w));
+                    const int chunk = w * 16 + q * 8 + j;
+                    *reinterpret_cast<uint4*>(xo + row * 512 + ((chunk ^ (row & 31)) << 4)) =
+                        make_uint4(__float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z), __float_as_uint(o.w));
                 }
             }
-            const size_t prow0 = ((size_t)unit * p.n_splits + split) * p.R + (size_t)c * p.chunk_rows;   // row 0 of the chunk
-            if (valid) { p.part_m[prow0 + row] = M; p.part_l[prow0 + row] = fmaf(l, fa, xl[row] * fb); }
-            asm volatile("bar.sync 2, 128;" ::: "memory");                   // warpgroup 0: the merged tile is complete
-            for (int rr = 0; rr < 32; ++rr) {                                // one coalesced 512-byte row per instruction
-                const int orow = lane_grp * 32 + rr;
+            asm volatile("bar.sync 2, 256;" ::: "memory");                   // the merged tile is complete
+            const int row_lo = (warp - 4) * 16;                              // 8 warps x 16 rows
+            for (int rr = 0; rr < 16; ++rr) {                                // one coalesced 512-byte row per instruction
+                const int orow = row_lo + rr;
                 if (orow < rows_valid)
                     *reinterpret_cast<uint4*>(p.part_o + (prow0 + orow) * kD + lane * 4) =
                         *reinterpret_cast<const uint4*>(xo + orow * 512 + ((lane ^ (orow & 31)) << 4));
