@@ -93,6 +93,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                  ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -280,6 +283,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int units = p.B * p.Hkv;
 
     if (threadIdx.x == 0) {
+        prefetch_tmap(&map_k); prefetch_tmap(&map_v); prefetch_tmap(&map_q); prefetch_tmap(&map_o);
         for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 3); }
         mbar_init(bar(BAR_QO_FULL), 1); mbar_init(bar(BAR_QO_EMPTY), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_TM_FULL + i), 1); mbar_init(bar(BAR_TM_EMPTY + i), 4); }
@@ -620,6 +624,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int b = unit / p.Hkv, g = unit % p.Hkv;
 
     if (threadIdx.x == 0) {
+        prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
         for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), 1); }
         mbar_init(bar(P1_QFULL), 1); mbar_init(bar(P1_ODONE), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(bar(P1_SFULL + i), 1); mbar_init(bar(P1_PFULL + i), 4); }
@@ -866,11 +871,16 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             asm volatile("bar.sync 2, 256;" ::: "memory");                   // the merged tile is complete
             const int row_lo = (warp - 4) * 16;                              // 8 warps x 16 rows
+            uint4 rowv[16];
+#pragma unroll
+            for (int rr = 0; rr < 16; ++rr) {
+                const int orow = row_lo + rr;
+                rowv[rr] = *reinterpret_cast<const uint4*>(xo + orow * 512 + ((lane ^ (orow & 31)) << 4));
+            }
+#pragma unroll
             for (int rr = 0; rr < 16; ++rr) {                                // one coalesced 512-byte row per instruction
                 const int orow = row_lo + rr;
-                if (orow < rows_valid)
-                    *reinterpret_cast<uint4*>(p.part_o + (prow0 + orow) * kD + lane * 4) =
-                        *reinterpret_cast<const uint4*>(xo + orow * 512 + ((lane ^ (orow & 31)) << 4));
+                if (orow < rows_valid) *reinterpret_cast<uint4*>(p.part_o + (prow0 + orow) * kD + lane * 4) = rowv[rr];
             }
         }
         tc_fence_before();

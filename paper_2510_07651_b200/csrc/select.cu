@@ -176,8 +176,10 @@ constexpr int CL_BINS = 2048;                 // 11-bit digits
 constexpr int CL_MAX_SEG = 20 * 1024;         // candidates per CTA (two 4-byte shared arrays of this size)
 
 struct ClusterShared {                        // fixed part of the CTA's shared memory
-    uint32_t hist[3][CL_BINS];                // one histogram per radix pass (summed in rank 0)
-    uint32_t bcast[3][2];                     // per pass: prefix, remaining (written by rank 0 into every CTA)
+    uint32_t sum[3][CL_BINS];                 // per radix pass: histogram of the whole head (every CTA adds into every copy)
+    uint32_t local[CL_BINS];                  // this CTA's histogram of the current pass
+    uint32_t found[2];                        // result of a pass: prefix, remaining
+    uint32_t n_list;                          // candidates of this CTA that survive the first pass
     uint32_t rank_gt[16], rank_eq[16];        // kept-candidate counts of every CTA of the cluster
     uint32_t warp_gt[CL_NT / 32], warp_eq[CL_NT / 32];
     uint32_t scan[CL_NT / 32];
@@ -214,7 +216,8 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     // ---- this CTA's share of the candidates: [c0, c1) of [0, n) --------------------------------
     const int seg = ((n + C - 1) / C + 31) / 32 * 32;
     const int c0 = min(rank * seg, n), c1 = min(c0 + seg, n), m = c1 - c0;
-    for (int i = tid; i < 3 * CL_BINS; i += CL_NT) (&sh.hist[0][0])[i] = 0;
+    for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;   // sum[3][] and local[]
+    if (tid == 0) sh.n_list = 0;
 
     // pooled keys: stage the scores with their halo, then pool out of shared memory
     const float* sc = scores + (size_t)unit * s.Nmax;
@@ -242,37 +245,42 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     cluster.sync();                                // histograms zeroed and keys written everywhere
 
     // ---- radix search for the key T of the n_hh-th largest candidate ---------------------------
-    uint32_t* hist0[3];                            // rank 0's histograms
-    for (int ps = 0; ps < 3; ++ps) hist0[ps] = cluster.map_shared_rank(&sh.hist[ps][0], 0);
+    // Pass 0 histograms the top 11 bits of all keys of the CTA; the keys that fall into the bin
+    // of the n_hh-th largest are copied to a list (in the staging buffer, free by now), and passes
+    // 1 and 2 only walk that list.  Every CTA adds its non-empty bins into the `sum` copy of every
+    // CTA of the cluster, so that after one cluster barrier each CTA finds the bin by itself.
+    uint32_t* list = reinterpret_cast<uint32_t*>(stage);
     uint32_t prefix = 0, mask = 0, remaining = (uint32_t)n_hh;
     for (int ps = 0; ps < 3; ++ps) {
         const int shift = ps == 0 ? 21 : ps == 1 ? 10 : 0;
         const uint32_t dmask = ps == 2 ? 1023u : 2047u;
-        uint32_t* hist = sh.hist[ps];
-        for (int base = 0; base < m; base += CL_NT) {
+        const uint32_t* src = ps == 0 ? keys : list;
+        const int cnt = ps == 0 ? m : (int)sh.n_list;
+        for (int base = 0; base < cnt; base += CL_NT) {
             const int i = base + tid;
-            const uint32_t key = i < m ? keys[i] : 0u;
-            const bool pred = i < m && ((key & mask) == prefix);
+            const bool pred = i < cnt && (ps < 2 || (src[i] & mask) == prefix);   // the list holds pass 0's bin only
             const unsigned act = __ballot_sync(0xffffffffu, pred);
             if (pred) {
-                const uint32_t dgt = (key >> shift) & dmask;
+                const uint32_t dgt = (src[i] >> shift) & dmask;
                 const unsigned peers = __match_any_sync(act, dgt);
-                if (lane == __ffs(peers) - 1) atomicAdd(&hist[dgt], (uint32_t)__popc(peers));
+                if (lane == __ffs(peers) - 1) atomicAdd(&sh.local[dgt], (uint32_t)__popc(peers));
             }
         }
         __syncthreads();
-        if (rank != 0)
-            for (int bin = tid; bin < CL_BINS; bin += CL_NT) {
-                const uint32_t c = hist[bin];
-                if (c) atomicAdd(&hist0[ps][bin], c);
+        for (int bin = tid; bin < CL_BINS; bin += CL_NT) {
+            const uint32_t c = sh.local[bin];
+            if (c) {
+                for (int r = 0; r < C; ++r) atomicAdd(cluster.map_shared_rank(&sh.sum[ps][bin], r), c);
+                sh.local[bin] = 0;
             }
-        cluster.sync();                            // rank 0's histogram holds the whole unit
-        if (rank == 0) {
+        }
+        cluster.sync();                            // every copy of sum[ps] holds the whole head
+        {
             // thread t owns bins [4t, 4t+4); find the highest bin D with
             // count(bins > D) < remaining <= count(bins >= D)
             uint32_t loc[4], tot = 0;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { loc[j] = hist[tid * 4 + j]; tot += loc[j]; }
+            for (int j = 0; j < 4; ++j) { loc[j] = sh.sum[ps][tid * 4 + j]; tot += loc[j]; }
             uint32_t incl = tot;                   // suffix sum over the lanes >= lane
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -284,27 +292,36 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
             uint32_t above = incl - tot;
             for (int w = warp + 1; w < CL_NT / 32; ++w) above += sh.scan[w];
             if (above < remaining && remaining <= above + tot) {
-                uint32_t run = above, found_prefix = 0, found_rem = 0;
+                uint32_t run = above;
 #pragma unroll
                 for (int j = 3; j >= 0; --j) {
                     if (run != 0xffffffffu) {
                         if (remaining <= run + loc[j]) {
-                            found_prefix = prefix | ((uint32_t)(tid * 4 + j) << shift);
-                            found_rem = remaining - run;
+                            sh.found[0] = prefix | ((uint32_t)(tid * 4 + j) << shift);
+                            sh.found[1] = remaining - run;
                             run = 0xffffffffu;
                         } else {
                             run += loc[j];
                         }
                     }
                 }
-                for (int r = 0; r < C; ++r) {
-                    uint32_t* dst = cluster.map_shared_rank(&sh.bcast[ps][0], r);
-                    dst[0] = found_prefix; dst[1] = found_rem;
-                }
+            }
+            __syncthreads();
+        }
+        prefix = sh.found[0]; remaining = sh.found[1]; mask |= dmask << shift;
+        if (ps == 0) {                             // survivors of the first pass -> list (any order)
+            for (int base = 0; base < m; base += CL_NT) {
+                const int i = base + tid;
+                const uint32_t key = i < m ? keys[i] : 0u;
+                const bool pred = i < m && (key & mask) == prefix;
+                const unsigned act = __ballot_sync(0xffffffffu, pred);
+                uint32_t at = 0;
+                if (lane == 0 && act) at = atomicAdd(&sh.n_list, (uint32_t)__popc(act));
+                at = __shfl_sync(0xffffffffu, at, 0);
+                if (pred) list[at + __popc(act & ((1u << lane) - 1u))] = key;
             }
         }
-        cluster.sync();                            // the search result reached every CTA
-        prefix = sh.bcast[ps][0]; remaining = sh.bcast[ps][1]; mask |= dmask << shift;
+        __syncthreads();                           // found[] may be rewritten, the list is complete
     }
     const uint32_t T = prefix, k_eq = remaining;   // keep all keys > T and the first k_eq keys == T
 
