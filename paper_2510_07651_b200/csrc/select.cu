@@ -223,19 +223,42 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     const float* sc = scores + (size_t)unit * s.Nmax;
     const int half = (s.pool_mode == OBC_POOL_NONE) ? 0 : s.pool_kernel / 2;
     const float pad = s.pool_mode == OBC_POOL_MAX ? -INFINITY : 0.f;
-    for (int i = tid; i < m + 2 * half; i += CL_NT) {
-        const int p = lo + c0 + i - half;
-        stage[i] = (p >= lo && p < hi) ? sc[p] : pad;
+    for (int base = 0; base < m + 2 * half; base += 8 * CL_NT) {      // eight loads in flight per thread
+        float val[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + u * CL_NT + tid, p = lo + c0 + i - half;
+            val[u] = (i < m + 2 * half && p >= lo && p < hi) ? sc[p] : pad;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + u * CL_NT + tid;
+            if (i < m + 2 * half) stage[i] = val[u];
+        }
     }
     __syncthreads();
     for (int i = tid; i < m; i += CL_NT) {
         float val;
         if (half == 0) {
             val = stage[i];
+        } else if (half <= 3) {                    // kernels up to 7: all taps read before they are combined
+            float tap[7];
+#pragma unroll
+            for (int t = 0; t < 7; ++t) tap[t] = t <= 2 * half ? stage[i + t] : pad;
+            if (s.pool_mode == OBC_POOL_MAX) {
+                val = -INFINITY;
+#pragma unroll
+                for (int t = 0; t < 7; ++t) val = fmaxf(val, tap[t]);      // padding taps are -inf
+            } else {                               // taps in ascending index order; padding adds +0
+                val = 0.f;
+#pragma unroll
+                for (int t = 0; t < 7; ++t) if (t <= 2 * half) val = __fadd_rn(val, tap[t]);
+                val = __fdiv_rn(val, (float)s.pool_kernel);
+            }
         } else if (s.pool_mode == OBC_POOL_MAX) {
             val = -INFINITY;
             for (int t = 0; t <= 2 * half; ++t) val = fmaxf(val, stage[i + t]);
-        } else {                                   // taps in ascending index order; padding adds +0
+        } else {
             val = 0.f;
             for (int t = 0; t <= 2 * half; ++t) val = __fadd_rn(val, stage[i + t]);
             val = __fdiv_rn(val, (float)s.pool_kernel);
@@ -259,12 +282,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
         for (int base = 0; base < cnt; base += CL_NT) {
             const int i = base + tid;
             const bool pred = i < cnt && (ps < 2 || (src[i] & mask) == prefix);   // the list holds pass 0's bin only
-            const unsigned act = __ballot_sync(0xffffffffu, pred);
-            if (pred) {
-                const uint32_t dgt = (src[i] >> shift) & dmask;
-                const unsigned peers = __match_any_sync(act, dgt);
-                if (lane == __ffs(peers) - 1) atomicAdd(&sh.local[dgt], (uint32_t)__popc(peers));
-            }
+            if (pred) atomicAdd(&sh.local[(src[i] >> shift) & dmask], 1u);
         }
         __syncthreads();
         for (int bin = tid; bin < CL_BINS; bin += CL_NT) {
@@ -289,8 +307,14 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
             }
             if (lane == 0) sh.scan[warp] = incl;
             __syncthreads();
-            uint32_t above = incl - tot;
-            for (int w = warp + 1; w < CL_NT / 32; ++w) above += sh.scan[w];
+            uint32_t wsum = lane < CL_NT / 32 ? sh.scan[lane] : 0u;      // suffix sum over the warps > warp
+#pragma unroll
+            for (int o = 1; o < CL_NT / 32; o <<= 1) {
+                const uint32_t t = __shfl_down_sync(0xffffffffu, wsum, o);
+                if (lane + o < CL_NT / 32) wsum += t;
+            }
+            const uint32_t above_warps = __shfl_sync(0xffffffffu, wsum, min(warp + 1, 31));
+            uint32_t above = incl - tot + (warp + 1 < CL_NT / 32 ? above_warps : 0u);
             if (above < remaining && remaining <= above + tot) {
                 uint32_t run = above;
 #pragma unroll
