@@ -108,7 +108,9 @@ obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_
  * Reads the device status word that obc_score keeps in the first bytes of its workspace.  The
  * tensor-core kernels bound every device-side wait; if one gives up, the kernel raises this word
  * and returns early (its scores are then unspecified).  This call synchronises `stream`, copies
- * the word to the host and returns OBC_OK or OBC_ERR_TIMEOUT.  (No counterpart in the paper.)
+ * the word to the host and returns OBC_OK or OBC_ERR_TIMEOUT.  The word itself (the first 4 bytes
+ * of the workspace) holds the source line of the wait that gave up first, for bug reports.
+ * (No counterpart in the paper.)
  */
 obc_status obc_score_status(const void* workspace, void* stream);
 

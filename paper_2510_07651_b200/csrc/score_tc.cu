@@ -41,12 +41,14 @@ constexpr uint32_t OFF_V = OFF_K + NSTAGE * kOperandBytes;        // NSTAGE x 32
 constexpr uint32_t OFF_NV = OFF_V + NSTAGE * kOperandBytes;       // NSLOT x 128 floats
 constexpr uint32_t OFF_CONST = OFF_NV + NSLOT * TILE * 4;         // NSLOT x 128 float2 (lse2, ||o||^2)
 constexpr uint32_t OFF_BAR = OFF_CONST + NSLOT * 128 * 8;
-constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + NSLOT;
+constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + 2 + 2 * NSLOT;
 constexpr uint32_t OFF_TMEM = OFF_BAR + kNumBars * 8;
 constexpr uint32_t kSmemBytes = OFF_TMEM + 16 + 1024;             // + alignment slack
 
 enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_QO_FULL = 2 * NSTAGE, BAR_QO_EMPTY = 2 * NSTAGE + 1,
-       BAR_TM_FULL = 2 * NSTAGE + 2, BAR_TM_EMPTY = 2 * NSTAGE + 4, BAR_NV = 2 * NSTAGE + 6 };
+       BAR_TM_FULL = 2 * NSTAGE + 2,      // [epilogue group][TMEM buffer]
+       BAR_TM_EMPTY = 2 * NSTAGE + 6,     // [TMEM buffer]
+       BAR_NV = 2 * NSTAGE + 8 };         // [epilogue group][slot]
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -286,8 +288,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         prefetch_tmap(&map_k); prefetch_tmap(&map_v); prefetch_tmap(&map_q); prefetch_tmap(&map_o);
         for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 3); }
         mbar_init(bar(BAR_QO_FULL), 1); mbar_init(bar(BAR_QO_EMPTY), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_TM_FULL + i), 1); mbar_init(bar(BAR_TM_EMPTY + i), 4); }
-        for (int i = 0; i < NSLOT; ++i) mbar_init(bar(BAR_NV + i), 2);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_TM_FULL + i), 1);
+        for (int i = 0; i < 2; ++i) mbar_init(bar(BAR_TM_EMPTY + i), 4);
+        for (int i = 0; i < 2 * NSLOT; ++i) mbar_init(bar(BAR_NV + i), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -300,10 +303,14 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
 
     bool failed = false;
+    int fail_site = 0;                             // source line of the wait that gave up (status word)
     const bool reload_qo_every_item = p.n_chunks > 1;
     const uint32_t qo_bytes = (uint32_t)p.chunk_rows * 128u * 2u * 2u;   // Q and O chunks, two halves each
 
     // Every role walks the same tiles (TileWalk) and, per tile, the chunks c = 0 .. n_chunks-1.
+    // Tiles go to the two epilogue groups alternately.  What an epilogue group waits for (accumulators
+    // ready, norms and constants ready) is signalled on barriers of its own, so that each waiter sees
+    // every phase of the barriers it uses; a parity wait must never fall two phases behind.
     // `item` counts the (tile, chunk) pairs processed so far and indexes the smem stage, TMEM
     // buffer and constant-slot rings.
     TileWalk tw;
@@ -318,7 +325,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv, t0 = tw.tile * TILE;
                 for (int c = 0; c < p.n_chunks; ++c, ++item) {
                     const uint32_t st = item % NSTAGE, use = item / NSTAGE;
-                    if (!mbar_wait(bar(BAR_EMPTY + st), (use & 1) ^ 1)) { failed = true; break; }
+                    if (!mbar_wait(bar(BAR_EMPTY + st), (use & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                     mbar_expect_tx(bar(BAR_FULL + st), 2 * kOperandBytes);
                     const uint32_t dk = sbase + OFF_K + st * kOperandBytes, dv = sbase + OFF_V + st * kOperandBytes;
                     tma_load_4d(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b);
@@ -329,7 +336,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     // may be fetched while the preceding kernel drains; -2 O is that kernel's output
                     if (item == 0) pdl_wait();
                     if (reload_qo_every_item || unit != qo_unit) {
-                        if (!mbar_wait(bar(BAR_QO_EMPTY), (qo_loads & 1) ^ 1)) { failed = true; break; }
+                        if (!mbar_wait(bar(BAR_QO_EMPTY), (qo_loads & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                         mbar_expect_tx(bar(BAR_QO_FULL), qo_bytes);
                         const int qrow = (b * p.Hkv * p.G + g * p.G) * p.W + c * p.chunk_rows;
                         const int orow = unit * p.rows_out + c * p.chunk_rows;
@@ -352,19 +359,20 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // ===================================== MMA issuer =======================================
         if (lane == 0) {
             const uint32_t idesc = idesc_bf16(p.chunk_rows);
-            uint32_t item = 0, qo_loads = 0;
+            uint32_t item = 0, qo_loads = 0, tile_seq = 0;
             int qo_unit = -1;
-            for (; !tw.done() && !failed; tw.next()) {
+            for (; !tw.done() && !failed; tw.next(), ++tile_seq) {
                 const int unit = tw.unit;
+                const uint32_t owner = tile_seq & 1;               // epilogue group of this tile
                 for (int c = 0; c < p.n_chunks; ++c, ++item) {
                     const bool new_qo = reload_qo_every_item || unit != qo_unit;
                     if (new_qo) {
-                        if (!mbar_wait(bar(BAR_QO_FULL), qo_loads & 1)) { failed = true; break; }
+                        if (!mbar_wait(bar(BAR_QO_FULL), qo_loads & 1)) { failed = true; fail_site = __LINE__; break; }
                         qo_unit = unit; ++qo_loads;
                     }
                     const uint32_t st = item % NSTAGE, buf = item & 1;
-                    if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; break; }
-                    if (!mbar_wait(bar(BAR_TM_EMPTY + buf), ((item >> 1) & 1) ^ 1)) { failed = true; break; }
+                    if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
+                    if (!mbar_wait(bar(BAR_TM_EMPTY + buf), ((item >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                     tc_fence_after();
                     const uint32_t zt = tmem_base + buf * 256u, tt = zt + 128u;
                     const uint32_t ak = sbase + OFF_K + st * kOperandBytes, av = sbase + OFF_V + st * kOperandBytes;
@@ -378,7 +386,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
                         tc_mma(tt, smem_desc_k_sw128(av + off), smem_desc_k_sw128(sbase + OFF_O + off), idesc, ks > 0);
                     }
-                    tc_commit(bar(BAR_TM_FULL + buf));             // accumulators ready for the epilogue
+                    tc_commit(bar(BAR_TM_FULL + owner * 2 + buf)); // accumulators ready for the tile's epilogue group
                     tc_commit(bar(BAR_EMPTY + st));                // K/V stage no longer read by the MMA
                     // Q / O may be overwritten once these MMAs are done, if the next item needs others
                     const bool last_of_unit = tw.left > 1 && tw.tile + 1 == tw.tiles_in_unit && c + 1 == p.n_chunks;
@@ -389,9 +397,10 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     } else if (warp < 4) {
         // ============================ ||v_p||^2 and per-row constants ===========================
         const int t64 = threadIdx.x - 64;                          // 0..63
-        uint32_t item = 0;
-        for (; !tw.done() && !failed; tw.next()) {
+        uint32_t item = 0, tile_seq = 0;
+        for (; !tw.done() && !failed; tw.next(), ++tile_seq) {
             const int unit = tw.unit;
+            const uint32_t owner = tile_seq & 1;                   // epilogue group of this tile
             for (int c = 0; c < p.n_chunks; ++c, ++item) {
                 const uint32_t st = item % NSTAGE, slot = item % NSLOT;
                 // constants first (global loads overlap the wait for the tile)
@@ -402,7 +411,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     const int r = t64 + 64 * j;
                     cst[j] = r < p.chunk_rows ? make_float2(-p.lse2[crow + r], p.onorm[crow + r]) : make_float2(-INFINITY, 0.f);
                 }
-                if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; break; }
+                if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
                 const uint8_t* vt = smem + OFF_V + st * kOperandBytes;
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
@@ -426,7 +435,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     cdst[0] = cst[j].x; cdst[2] = cst[j].y;
                 }
                 __syncwarp();
-                if (lane == 0) { mbar_arrive(bar(BAR_NV + slot)); mbar_arrive(bar(BAR_EMPTY + st)); }
+                if (lane == 0) { mbar_arrive(bar(BAR_NV + owner * NSLOT + slot)); mbar_arrive(bar(BAR_EMPTY + st)); }
             }
         }
     } else {
@@ -437,6 +446,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float2 sl2 = make_float2(p.scale * kLog2e, p.scale * kLog2e), sc = make_float2(p.scale, p.scale);
         const size_t plane = (size_t)units * p.Nmax;
         uint32_t item = 0, tile_seq = 0;
+        uint32_t full_par = 0, nv_par = 0;                         // phase parity of this group's barriers, one bit each
         for (; !tw.done() && !failed; tw.next()) {
             const bool mine = (tile_seq & 1) == (uint32_t)wg;
             ++tile_seq;
@@ -452,8 +462,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             float nv = 0.f;
             for (int c = 0; c < p.n_chunks && !failed; ++c, ++item) {
                 const uint32_t buf = item & 1, slot = item % NSLOT;
-                if (!mbar_wait(bar(BAR_NV + slot), (item / NSLOT) & 1)) { failed = true; break; }
-                if (!mbar_wait(bar(BAR_TM_FULL + buf), (item >> 1) & 1)) { failed = true; break; }
+                if (!mbar_wait(bar(BAR_NV + wg * NSLOT + slot), (nv_par >> slot) & 1)) { failed = true; fail_site = __LINE__; break; }
+                if (!mbar_wait(bar(BAR_TM_FULL + wg * 2 + buf), (full_par >> buf) & 1)) { failed = true; fail_site = __LINE__; break; }
+                nv_par ^= 1u << slot; full_par ^= 1u << buf;
                 tc_fence_after();
                 nv = sNv[slot * TILE + tok];
                 const float4* cst = reinterpret_cast<const float4*>(sConst + slot * 256);
@@ -490,7 +501,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     }
 
-    if (failed) atomicExch(p.status, 1u);
+    if (failed) atomicCAS(p.status, 0u, (unsigned)(fail_site > 0 ? fail_site : 1));   // the first failure is kept
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -639,6 +650,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    int fail_site = 0;                             // source line of the wait that gave up (status word)
     pdl_wait();                                    // nothing above reads or writes global memory
     // the status word starts at 0: no wait of this call can have given up yet (each lasts seconds)
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.status = 0u;
@@ -657,7 +669,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             int issued = 0;
             for (int i = 0; i < n_tiles; ++i) {
                 const uint32_t st = i % P1_NSTAGE;
-                if (!mbar_wait(bar(P1_EMPTY + st), ((i / P1_NSTAGE) & 1) ^ 1)) { failed = true; break; }
+                if (!mbar_wait(bar(P1_EMPTY + st), ((i / P1_NSTAGE) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                 mbar_expect_tx(bar(P1_FULL + st), 2 * kOperandBytes);
                 const uint32_t dk = sbase + P1_OFF_K + st * kOperandBytes, dv = sbase + P1_OFF_V + st * kOperandBytes;
                 const int t0 = (tile_lo + i) * TILE;
@@ -694,9 +706,10 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             failed = !mbar_wait(bar(P1_QFULL), 0);
             if (!failed) failed = !issue_s(0);
             if (!failed && n_tiles > 1) failed = !issue_s(1);
+            if (failed) fail_site = __LINE__;
             for (int i = 0; i < n_tiles && !failed; ++i) {
                 const uint32_t w = i & 1;
-                if (!mbar_wait(bar(P1_PFULL + w), (i >> 1) & 1)) { failed = true; break; }
+                if (!mbar_wait(bar(P1_PFULL + w), (i >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
                 tc_fence_after();
                 const uint32_t av = sbase + P1_OFF_V + (i % P1_NSTAGE) * kOperandBytes;
 #pragma unroll
@@ -704,7 +717,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     tc_mma_ts(tmem_base + 256u + w * 128u, tmem_base + w * 128u + ks * 8, smem_desc_mn_sw128(av + ks * 2048),
                               idesc_pv, (i > 1) || (ks > 0));
                 tc_commit(bar(P1_EMPTY + (i % P1_NSTAGE)));                  // S(i) and P.V(i) have read the stage
-                if (i + 2 < n_tiles && !issue_s(i + 2)) { failed = true; break; }
+                if (i + 2 < n_tiles && !issue_s(i + 2)) { failed = true; fail_site = __LINE__; break; }
             }
             if (!failed) tc_commit(bar(P1_ODONE));
         }
@@ -726,7 +739,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
         for (int i = w; i < n_tiles && !failed; i += 2, ++my_tiles) {
             const int t0 = (tile_lo + i) * TILE;
-            if (!mbar_wait(bar(P1_SFULL + w), my_tiles & 1)) { failed = true; break; }
+            if (!mbar_wait(bar(P1_SFULL + w), my_tiles & 1)) { failed = true; fail_site = __LINE__; break; }
             tc_fence_after();
             const bool masked = t0 + TILE > first_masked;
             const int nvis = last - t0 + 1;                                  // columns j < nvis are visible
@@ -834,7 +847,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         uint8_t* xo = smem + P1_OFF_K;
         bool have = my_tiles > 0 && !failed;
         if (n_tiles > 0) {                                                   // all MMAs done: accumulators final, smem free
-            if (!mbar_wait(bar(P1_ODONE), 0)) { failed = true; have = false; }
+            if (!mbar_wait(bar(P1_ODONE), 0)) { failed = true; fail_site = __LINE__; have = false; }
             tc_fence_after();
         }
         xm[w * 128 + row] = have ? m_used : -INFINITY;
@@ -886,7 +899,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         tc_fence_before();
     }
 
-    if (failed) atomicExch(p.status, 1u);
+    if (failed) atomicCAS(p.status, 0u, (unsigned)(fail_site > 0 ? fail_site : 1));   // the first failure is kept
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
