@@ -168,7 +168,7 @@ def run_ours(args):
     import numpy as np
     import torch
     import torch.distributed as dist
-    from paper_2510_07651_b200 import api, build, synth
+    from paper_2510_07651_b200 import api, build, multirank, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -248,10 +248,7 @@ def run_ours(args):
     if sampler:
         sampler.mark("timed_end")
     barrier()
-    ms = torch.tensor([e0.elapsed_time(e1)], device="cuda")
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms = float(ms.item())
+    ms = multirank.max_over_ranks(e0.elapsed_time(e1), "cuda")
 
     # ---- per-kernel times (same steps again, every kernel bracketed by CUDA events) -------------
     prof_steps = min(args.steps, 200)
@@ -367,6 +364,118 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_other(args):
+    """The other workloads (parity-test cases, not the headline): one JSON line each with the step
+    time from CUDA events and the per-kernel event times.  Single GPU."""
+    import numpy as np
+    import torch
+    from paper_2510_07651_b200 import api, build, synth
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    build.build()
+    api.lib()
+    bf = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    if args.workload == "decode":
+        # Llama-3-8B shapes, batch 32: a 16384-token context already reduced to the 4096-token budget;
+        # every step appends one token, rescores all 4097 live slots (W = 1) and evicts one.
+        B, Hq, Hkv, n0, budget, n_sink, n_recent = 32, 32, 8, 4096, 4096, 4, 256
+        total = warmup + steps
+        dc = synth.make_decode(B=B, Hq=Hq, Hkv=Hkv, d=128, n0=n0, steps=min(total, 64), seed=1239)
+        cap = budget + 1
+        kc = torch.zeros((B, Hkv, cap, 128), dtype=torch.bfloat16, device="cuda")
+        vc = torch.zeros_like(kc)
+        kc[:, :, :n0] = bf(dc.k0_bits); vc[:, :, :n0] = bf(dc.v0_bits)
+        pos = torch.full((B, Hkv, cap), -1, dtype=torch.int32, device="cuda")
+        pos[:, :, :n0] = torch.arange(n0, dtype=torch.int32, device="cuda")
+        s_acc = torch.zeros((B, Hkv, cap), dtype=torch.float32, device="cuda")
+        state = torch.zeros((B, Hkv, 4), dtype=torch.int32, device="cuda")
+        state[..., 0] = n0; state[..., 1] = n0; state[..., 2] = n0
+        qd, kd, vd = bf(dc.q_t_bits), bf(dc.k_t_bits), bf(dc.v_t_bits)
+        ns = qd.shape[0]
+        q_t = [qd[t].unsqueeze(2) for t in range(ns)]; k_t = [kd[t].unsqueeze(2) for t in range(ns)]
+        v_t = [vd[t].unsqueeze(2) for t in range(ns)]
+        p = api.decode_params(q_t[0], kc, budget=budget, n_sink=n_sink, n_recent=n_recent)
+        ws = torch.empty(api.obc_decode_workspace(p), dtype=torch.uint8, device="cuda")
+
+        def step(t):
+            api.obc_decode_step(q_t[t % ns], k_t[t % ns], v_t[t % ns], kc, vc, s_acc, pos, state, n0 + t,
+                                budget=budget, n_sink=n_sink, n_recent=n_recent, variant="VK", workspace=ws)
+        for t in range(warmup):
+            step(t)
+        torch.cuda.synchronize()
+        e0.record()
+        for t in range(warmup, total):
+            step(t)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        api.obc_profile_begin()
+        for t in range(total, total + min(steps, 100)):
+            step(t)
+        torch.cuda.synchronize()
+        prof = api.obc_profile_end()
+        live_bytes = B * Hkv * (n0 + 1) * 128 * 2 * 3            # K once, V twice per step
+        line = {"metric": "decode rescoring steps/sec", "value": steps / (ms * 1e-3), "unit": "steps/s",
+                "ms_per_step": ms / steps, "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "decode: B32 Hq32 Hkv8 d128, live 4096 -> 4097 -> 4096 per step, W1, OBCache-V&K, "
+                                       "4 sinks, 256 recent, one eviction per head per step"},
+                "hbm_gbs_algorithmic": live_bytes / (ms / steps * 1e-3) / 1e9,
+                "kernels": {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}}
+        print(json.dumps(line))
+        return
+
+    idx_cfg = {"qwen128k": 3, "ragged": 4}[args.workload]
+    case, run = synth.config(idx_cfg)
+    q, k, v = bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)
+    lens = None if (case.seq_lens == case.Nmax).all() else torch.from_numpy(case.seq_lens).cuda()
+    order = [n for n in ("V", "K", "VK") if n in run["variants"]]
+    budgets = np.asarray(run["budget"] if isinstance(run["budget"], list) else [run["budget"]] * case.B, np.int32)
+    uniform = bool((budgets == budgets[0]).all())
+    bud_d = None if uniform else torch.from_numpy(budgets).cuda()
+    stride = int(budgets.max())
+    sp = api.score_params(q, k, seq_lens=lens, variants=order)
+    ws_score = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
+    scores = torch.empty((len(order), case.B, case.Hkv, case.Nmax), dtype=torch.float32, device="cuda")
+    selp = api.select_params(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
+                             seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"])
+    ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
+    idx = torch.empty((case.B, case.Hkv, stride), dtype=torch.int32, device="cuda")
+    k_out = torch.empty((case.B, case.Hkv, stride, 128), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+
+    def step():
+        api.obc_score(q, k, v, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
+        api.obc_select(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
+                       seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
+                       idx=idx, workspace=ws_sel)
+        api.obc_compact(k, v, idx, k_out=k_out, v_out=v_out)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    api.obc_profile_begin()
+    for _ in range(min(steps, 50)):
+        step()
+    torch.cuda.synchronize()
+    prof = api.obc_profile_end()
+    tokens = int(case.seq_lens.sum())
+    line = {"metric": METRIC, "value": tokens * steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps,
+            "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{case.name}: B{case.B} Hq{case.Hq} Hkv{case.Hkv} d128 Nmax{case.Nmax} W{case.W} bf16, "
+                                   f"variants {order}, pool {run['pool_mode']} {run['pool_kernel']}, tokens/step {tokens}",
+                       "l2": "inputs (K+V) larger than L2" if tokens * case.Hkv * 512 > 126e6 else "single input copy"},
+            "kernels": {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -376,16 +485,20 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--eager", action="store_true", help="time plain library calls instead of replaying CUDA graphs")
+    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode"],
+                    help="llama32k is the headline benchmark; the others print a shorter line (1 GPU)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"
     if args.steps is None:
-        args.steps = 3 if ref_arm else 2000
+        args.steps = 3 if ref_arm else (2000 if args.workload == "llama32k" else 200)
     if args.warmup is None:
         args.warmup = 1 if ref_arm else 20
     if not ref_arm:
         args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload != "llama32k":
+        run_other(args)
     else:
         run_ours(args)
 
