@@ -18,6 +18,7 @@ namespace obc {
 namespace {
 
 constexpr int CH = 256;                  // slots per chunk = threads per block
+constexpr size_t kStageBytes = (size_t)CH * 256;   // one chunk of 256-byte rows in shared memory
 
 struct DecodePlan {
     int chunks;
@@ -54,12 +55,35 @@ __device__ __forceinline__ const __nv_bfloat16* bf_row(const TensorView& t, int 
     return reinterpret_cast<const __nv_bfloat16*>(t.ptr) + b * t.sb + h * t.sh + tok * t.st;
 }
 
+// Cooperative copy of the 256-byte rows [c0, c0 + CH) of one cache into shared memory, in two steps so
+// that the caller can put work between them: load_rows issues all 16 loads of a thread before any
+// use (a warp reads two whole rows per instruction, coalesced; rows at or beyond `hi` are not
+// read), store_rows puts the 16-byte chunk c of row r at chunk c ^ (r & 15), so that the thread
+// that owns row r later reads its row without bank conflicts.
+__device__ __forceinline__ void load_rows(uint4 (&v)[16], const TensorView& t, int b, int g, int c0, int hi) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const int i = threadIdx.x + k * CH, r = i >> 4, c = i & 15;
+        // plain loads: the new token's row was stored by this CTA just before
+        v[k] = c0 + r < hi ? reinterpret_cast<const uint4*>(bf_row(t, b, g, c0 + r))[c] : make_uint4(0, 0, 0, 0);
+    }
+}
+__device__ __forceinline__ void store_rows(uint4* dst, const uint4 (&v)[16]) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const int i = threadIdx.x + k * CH, r = i >> 4, c = i & 15;
+        dst[r * 16 + (c ^ (r & 15))] = v[k];
+    }
+}
+__device__ __forceinline__ uint4 staged_chunk(const uint4* src, int r, int c) { return src[r * 16 + (c ^ (r & 15))]; }
+
 template <int G>
 __global__ void __launch_bounds__(CH)
 decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt, TensorView vt,
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, const int32_t* state,
                     int step_pos, char* ws) {
     pdl_wait();
+    extern __shared__ __align__(16) uint4 sRows[];                      // [CH][16]: the chunk's K rows
     __shared__ __align__(16) float sQ[G][kD];
     __shared__ float sP[G][CH];
     __shared__ __align__(16) float sO[8][G][kD];
@@ -90,7 +114,12 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         else if (tid < 32) reinterpret_cast<uint4*>(vdst)[tid - 16] = reinterpret_cast<const uint4*>(bf_row(vt, b, g, 0))[tid - 16];
         else if (tid == 32) { pos[(size_t)unit * s.cap + next] = step_pos; s_acc[(size_t)unit * s.cap + next] = 0.f; }
     }
+    __syncthreads();                                       // the new token's row is in place
+    uint4 stage[16];
+    load_rows(stage, kc, b, g, c0, hi);
+    store_rows(sRows, stage);
     __syncthreads();
+    load_rows(stage, vc, b, g, c0, hi);                    // V rows travel while the logits are computed
 
     const int slot = c0 + tid;
     const bool live = slot < hi && ((valid && slot == next) || pos[(size_t)unit * s.cap + slot] >= 0);
@@ -99,11 +128,10 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
 #pragma unroll
     for (int r = 0; r < G; ++r) z2[r] = 0.f;
     if (live) {
-        const uint4* krow = reinterpret_cast<const uint4*>(bf_row(kc, b, g, slot));
 #pragma unroll 4
         for (int c = 0; c < 16; ++c) {
             float kf[8];
-            unpack8(krow[c], kf);
+            unpack8(staged_chunk(sRows, tid, c), kf);
 #pragma unroll
             for (int r = 0; r < G; ++r) {
                 const float4 qa = *reinterpret_cast<const float4*>(&sQ[r][c * 8]);
@@ -137,7 +165,8 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         sP[r][tid] = p;
         lsum[r] = warp_sum(p);
     }
-    __syncthreads();                                       // sRed reads done, sP complete
+    __syncthreads();                                       // sRed reads done, sP complete, K rows no longer read
+    store_rows(sRows, stage);
 #pragma unroll
     for (int r = 0; r < G; ++r) if (lane == 0) sRed[warp][r] = lsum[r];
 
@@ -146,9 +175,15 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
     float o[G][4];
 #pragma unroll
     for (int r = 0; r < G; ++r) { o[r][0] = o[r][1] = o[r][2] = o[r][3] = 0.f; }
+    __syncthreads();                                       // V rows staged
     for (int t = 0; t < 32; ++t) {
         if (!((live_mask >> t) & 1u)) continue;
-        const float4 vv = load4<__nv_bfloat16>(bf_row(vc, b, g, c0 + warp * 32 + t) + lane * 4);
+        // channels 4*lane .. +3 of slot row: half (lane & 1) of the 16-byte chunk lane / 2
+        const int row = warp * 32 + t;
+        const uint2 raw = reinterpret_cast<const uint2*>(&sRows[row * 16 + ((lane >> 1) ^ (row & 15))])[lane & 1];
+        float4 vv;
+        vv.x = __uint_as_float(raw.x << 16); vv.y = __uint_as_float(raw.x & 0xffff0000u);
+        vv.z = __uint_as_float(raw.y << 16); vv.w = __uint_as_float(raw.y & 0xffff0000u);
 #pragma unroll
         for (int r = 0; r < G; ++r) {
             const float p = sP[r][warp * 32 + t];
@@ -175,36 +210,58 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
     }
 }
 
-// one block of 128 threads per (b, g): merge the chunk partials
+// one block of 128 threads per (b, g, row): merge the chunk partials.  The statistics of the chunks
+// are read one per thread and the partial outputs eight at a time, so the block costs a couple of
+// round trips to L2 however many chunks there are.
+__device__ __forceinline__ float decode_block_reduce(float x, bool take_max, float* red) {
+    x = take_max ? warp_max(x) : warp_sum(x);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
+    __syncthreads();
+    return take_max ? fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3])) : (red[0] + red[1]) + (red[2] + red[3]);
+}
+
 __global__ void __launch_bounds__(kD)
 decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
     pdl_wait();
-    const int unit = blockIdx.x, c = threadIdx.x, G = s.G;
+    const int G = s.G, unit = blockIdx.x / G, r = blockIdx.x % G, c = threadIdx.x;
     __shared__ float red[4];
-    for (int r = 0; r < G; ++r) {
-        const float* pm = (const float*)(ws + plan.off_pm) + (size_t)unit * plan.chunks * G + r;
-        const float* pl = (const float*)(ws + plan.off_pl) + (size_t)unit * plan.chunks * G + r;
-        const float* po = (const float*)(ws + plan.off_po) + ((size_t)unit * plan.chunks * G + r) * kD + c;
-        float M = -INFINITY;
-        for (int ch = 0; ch < plan.chunks; ++ch) M = fmaxf(M, pm[(size_t)ch * G]);
-        float L = 0.f, oc = 0.f;
-        for (int ch = 0; ch < plan.chunks; ++ch) {
+    __shared__ float sW[kD];
+    const float* pm = (const float*)(ws + plan.off_pm) + (size_t)unit * plan.chunks * G + r;
+    const float* pl = (const float*)(ws + plan.off_pl) + (size_t)unit * plan.chunks * G + r;
+    const float* po = (const float*)(ws + plan.off_po) + ((size_t)unit * plan.chunks * G + r) * kD + c;
+    float M = -INFINITY;
+    for (int ch = c; ch < plan.chunks; ch += kD) M = fmaxf(M, pm[(size_t)ch * G]);
+    M = decode_block_reduce(M, true, red);
+    float L = 0.f, oc = 0.f;
+    for (int base = 0; base < plan.chunks; base += kD) {
+        const int ch = base + c, cnt = min(kD, plan.chunks - base);
+        float w = 0.f;
+        if (ch < plan.chunks) {
             const float m = pm[(size_t)ch * G];
-            if (m == -INFINITY) continue;
-            const float w = exp2f(m - M);
-            L = fmaf(pl[(size_t)ch * G], w, L);
-            oc = fmaf(po[(size_t)ch * G * kD], w, oc);
+            if (m != -INFINITY) { w = exp2f(m - M); L = fmaf(pl[(size_t)ch * G], w, L); }
         }
-        oc = L > 0.f ? oc / L : 0.f;
-        const float sq = warp_sum(oc * oc);
         __syncthreads();
-        if ((c & 31) == 0) red[c >> 5] = sq;
+        sW[c] = w;
         __syncthreads();
-        ((float*)(ws + plan.off_o))[((size_t)unit * G + r) * kD + c] = oc;
-        if (c == 0) {
-            ((float*)(ws + plan.off_lse))[(size_t)unit * G + r] = M + log2f(L);
-            ((float*)(ws + plan.off_no))[(size_t)unit * G + r] = red[0] + red[1] + red[2] + red[3];
+        for (int j0 = 0; j0 < cnt; j0 += 8) {
+            float o8[8], w8[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {                  // chunks without a live slot hold no partial output
+                w8[u] = j0 + u < cnt ? sW[j0 + u] : 0.f;
+                o8[u] = w8[u] != 0.f ? po[(size_t)(base + j0 + u) * G * kD] : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) oc = fmaf(o8[u], w8[u], oc);
         }
+    }
+    L = decode_block_reduce(L, false, red);
+    oc = L > 0.f ? oc / L : 0.f;
+    const float sq = decode_block_reduce(oc * oc, false, red);
+    ((float*)(ws + plan.off_o))[((size_t)unit * G + r) * kD + c] = oc;
+    if (c == 0) {
+        ((float*)(ws + plan.off_lse))[(size_t)unit * G + r] = M + log2f(L);
+        ((float*)(ws + plan.off_no))[(size_t)unit * G + r] = sq;
     }
 }
 
@@ -213,6 +270,7 @@ __global__ void __launch_bounds__(CH)
 decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc, const int32_t* pos,
                     const int32_t* state, int step_pos, char* ws) {
     pdl_wait();
+    extern __shared__ __align__(16) uint4 sRows[];                      // [CH][16]: the chunk's V rows
     __shared__ __align__(16) float sO[G][kD];
     __shared__ float sLse[G], sNo[G];
     __shared__ MinCand sMin[8];
@@ -233,6 +291,11 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
         sLse[tid] = ((const float*)(ws + plan.off_lse))[(size_t)unit * G + tid];
         sNo[tid] = ((const float*)(ws + plan.off_no))[(size_t)unit * G + tid];
     }
+    {
+        uint4 stage[16];
+        load_rows(stage, vc, b, g, c0, hi);
+        store_rows(sRows, stage);
+    }
     __syncthreads();
 
     const int slot = c0 + tid;
@@ -240,14 +303,13 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
     const bool live = my_pos >= 0;
     MinCand cand{INFINITY, -1, -1, 0};
     if (live) {
-        const uint4* vrow = reinterpret_cast<const uint4*>(bf_row(vc, b, g, slot));
         float nv = 0.f, t[G];
 #pragma unroll
         for (int r = 0; r < G; ++r) t[r] = 0.f;
 #pragma unroll 4
         for (int c = 0; c < 16; ++c) {
             float vf[8];
-            unpack8(vrow[c], vf);
+            unpack8(staged_chunk(sRows, tid, c), vf);
 #pragma unroll
             for (int j = 0; j < 8; ++j) nv = fmaf(vf[j], vf[j], nv);
 #pragma unroll
@@ -335,9 +397,11 @@ obc_status launch_g(const DecodeShape& s, const DecodePlan& plan, TensorView q, 
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
                     int step_pos, char* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
-    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), 0, stream, 1, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
-    { ProfScope ps("decode_combine", stream); OBC_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(units), dim3(kD), 0, stream, 1, s, plan, ws)); }
-    { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G>, dim3(plan.chunks, units), dim3(CH), 0, stream, 1, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
+    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_pass1_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageBytes));
+      OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), kStageBytes, stream, 1, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
+    { ProfScope ps("decode_combine", stream); OBC_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(units * s.G), dim3(kD), 0, stream, 1, s, plan, ws)); }
+    { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_score_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageBytes));
+      OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G>, dim3(plan.chunks, units), dim3(CH), kStageBytes, stream, 1, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
     { ProfScope ps("decode_final", stream); OBC_CUDA_TRY(launch_pdl(decode_final_kernel, dim3((units + 127) / 128), dim3(128), 0, stream, 1, s, plan, pos, state, ws)); }
     return OBC_OK;
 }
