@@ -511,6 +511,280 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 }
 
 // =================================================================================================
+// Pass 2 for more than 128 window rows per KV head (e.g. GQA 7 x W 64 = 448).  The rows are cut
+// into chunks of 64; a K/V tile is fetched ONCE and stays in shared memory while its chunks pass:
+//     per tile    K/V through the 2-stage ring, ||v_p||^2
+//     per chunk   Q / -2 O chunk into one of two buffers, one pair of MMAs with N = 64 into one of
+//                 four TMEM buffers (Z 64 + T' 64 columns), per-row constants into one of four slots
+// The two epilogue warpgroups take alternate chunks (so each owns two TMEM buffers and the MMAs of
+// its next chunk run while it sums the current one) and keep partial sums of the same 128 tokens;
+// after the tile's last chunk warpgroup 1 hands its sums to warpgroup 0 through shared memory.
+// =================================================================================================
+constexpr int MC_ROWS = 64;
+constexpr uint32_t kHalfB64 = 64 * 128;                           // B operand block: [64 rows][64 bf16]                                       // window rows per chunk
+constexpr uint32_t kQoBuf = 4 * kHalfB64;                         // Q chunk (2 x 8 KB) + -2 O chunk (2 x 8 KB)
+constexpr uint32_t MC_OFF_QO = 0;                                 // 2 buffers x 32 KB
+constexpr uint32_t MC_OFF_K = MC_OFF_QO + 2 * kQoBuf;             // NSTAGE x 32 KB
+constexpr uint32_t MC_OFF_V = MC_OFF_K + NSTAGE * kOperandBytes;
+constexpr uint32_t MC_OFF_NV = MC_OFF_V + NSTAGE * kOperandBytes; // NSLOT x 128 floats (per tile)
+constexpr uint32_t MC_OFF_CONST = MC_OFF_NV + NSLOT * TILE * 4;   // 4 slots x 32 float4 (per chunk)
+constexpr uint32_t MC_OFF_X = MC_OFF_CONST + 4 * 32 * 16;         // 2 x 128 tokens x 8 floats (exchange)
+constexpr uint32_t MC_OFF_BAR = MC_OFF_X + 2 * TILE * 8 * 4;
+enum { MC_FULL = 0, MC_EMPTY = 2, MC_QO_FULL = 4, MC_QO_EMPTY = 6, MC_TM_FULL = 8, MC_TM_EMPTY = 12,
+       MC_NV = 16, MC_CONST = 16 + NSLOT, MC_XCHG = 20 + NSLOT, MC_NBARS = 22 + NSLOT };
+constexpr uint32_t MC_OFF_TMEM = MC_OFF_BAR + MC_NBARS * 8;
+constexpr uint32_t kSmemMulti = MC_OFF_TMEM + 16 + 1024;
+
+template <unsigned VARS>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
+                      const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                      const __grid_constant__ TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + MC_OFF_BAR;
+    auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + MC_OFF_TMEM);
+    float* sNv = reinterpret_cast<float*>(smem + MC_OFF_NV);
+    float* sConst = reinterpret_cast<float*>(smem + MC_OFF_CONST);
+    float* sX = reinterpret_cast<float*>(smem + MC_OFF_X);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int units = p.B * p.Hkv;
+    const int nc = p.n_chunks;                                   // chunks of MC_ROWS rows per tile
+
+    if (threadIdx.x == 0) {
+        prefetch_tmap(&map_k); prefetch_tmap(&map_v); prefetch_tmap(&map_q); prefetch_tmap(&map_o);
+        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(MC_FULL + i), 1); mbar_init(bar(MC_EMPTY + i), 3); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(MC_QO_FULL + i), 1); mbar_init(bar(MC_QO_EMPTY + i), 1); }
+        for (int i = 0; i < 4; ++i) { mbar_init(bar(MC_TM_FULL + i), 1); mbar_init(bar(MC_TM_EMPTY + i), 4); }
+        for (int i = 0; i < NSLOT; ++i) mbar_init(bar(MC_NV + i), 2);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(MC_CONST + i), 2);
+        for (int i = 0; i < 2; ++i) mbar_init(bar(MC_XCHG + i), 4);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + MC_OFF_TMEM), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    bool failed = false;
+    int fail_site = 0;                             // source line of the wait that gave up (status word)
+    const uint32_t qo_bytes = MC_ROWS * 128u * 2u * 2u;
+
+    // `titem` counts tiles, `item` (tile, chunk) pairs.  Rings: K/V stage and norm slot by titem;
+    // Q/O buffer by item & 1, TMEM buffer and constant slot by item & 3.  Items go to the epilogue
+    // groups alternately, so a group always sees the same TMEM buffers and constant slots.
+    TileWalk tw;
+    tw.init(p);
+    if (!(warp == 0 && lane == 0)) pdl_wait();       // the producer thread waits after its first K/V copies
+    if (warp == 0) {
+        // ===================================== TMA producer =====================================
+        if (lane == 0) {
+            uint32_t item = 0, titem = 0, kv_issued = 0;
+            TileWalk ahead = tw;                                   // position of the next K/V tile to fetch
+            auto fetch_kv = [&]() -> bool {                        // next tile of the walk into its stage
+                if (ahead.done()) return true;
+                const uint32_t st = kv_issued % NSTAGE;
+                if (!mbar_wait(bar(MC_EMPTY + st), ((kv_issued / NSTAGE) & 1) ^ 1)) return false;
+                const int unit = ahead.unit, b = unit / p.Hkv, g = unit % p.Hkv, t0 = ahead.tile * TILE;
+                mbar_expect_tx(bar(MC_FULL + st), 2 * kOperandBytes);
+                const uint32_t dk = sbase + MC_OFF_K + st * kOperandBytes, dv = sbase + MC_OFF_V + st * kOperandBytes;
+                tma_load_4d(dk, &map_k, bar(MC_FULL + st), 0, t0, g, b);
+                tma_load_4d(dk + kHalfBytes, &map_k, bar(MC_FULL + st), 64, t0, g, b);
+                tma_load_4d(dv, &map_v, bar(MC_FULL + st), 0, t0, g, b);
+                tma_load_4d(dv + kHalfBytes, &map_v, bar(MC_FULL + st), 64, t0, g, b);
+                ++kv_issued; ahead.next();
+                return true;
+            };
+            if (!fetch_kv()) { failed = true; fail_site = __LINE__; }
+            pdl_wait();                                            // K and V were read by pass 1; -2 O is the preceding kernel's output
+            for (; !tw.done() && !failed; tw.next(), ++titem) {
+                const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv;
+                for (int c = 0; c < nc; ++c, ++item) {
+                    const uint32_t qb = item & 1;
+                    if (!mbar_wait(bar(MC_QO_EMPTY + qb), ((item >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                    mbar_expect_tx(bar(MC_QO_FULL + qb), qo_bytes);
+                    const int qrow = (b * p.Hkv * p.G + g * p.G) * p.W + c * MC_ROWS;
+                    const int orow = unit * p.rows_out + c * MC_ROWS;
+                    const uint32_t dq = sbase + MC_OFF_QO + qb * kQoBuf, dob = dq + 2 * kHalfB64;
+                    tma_load_2d(dq, &map_q, bar(MC_QO_FULL + qb), 0, qrow);
+                    tma_load_2d(dq + kHalfB64, &map_q, bar(MC_QO_FULL + qb), 64, qrow);
+                    tma_load_2d(dob, &map_o, bar(MC_QO_FULL + qb), 0, orow);
+                    tma_load_2d(dob + kHalfB64, &map_o, bar(MC_QO_FULL + qb), 64, orow);
+                    // the next tile's K/V once this tile's first two chunks are on their way
+                    if (c == (nc > 1 ? 1 : 0) && !fetch_kv()) { failed = true; fail_site = __LINE__; break; }
+                }
+            }
+            // drain: every copy this thread issued must have landed before the CTA may exit
+            for (uint32_t back = 0; back < NSTAGE && back < kv_issued; ++back) {
+                const uint32_t it = kv_issued - 1 - back;
+                (void)mbar_wait(bar(MC_FULL + it % NSTAGE), (it / NSTAGE) & 1);
+            }
+            for (uint32_t back = 0; back < 2 && back < item; ++back) {
+                const uint32_t it = item - 1 - back;
+                (void)mbar_wait(bar(MC_QO_FULL + (it & 1)), (it >> 1) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        // ===================================== MMA issuer =======================================
+        if (lane == 0) {
+            const uint32_t idesc = idesc_bf16(MC_ROWS);
+            uint32_t item = 0, titem = 0;
+            for (; !tw.done() && !failed; tw.next(), ++titem) {
+                const uint32_t st = titem % NSTAGE;
+                if (!mbar_wait(bar(MC_FULL + st), (titem / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
+                const uint32_t ak = sbase + MC_OFF_K + st * kOperandBytes, av = sbase + MC_OFF_V + st * kOperandBytes;
+                for (int c = 0; c < nc; ++c, ++item) {
+                    const uint32_t qb = item & 1, buf = item & 3;
+                    if (!mbar_wait(bar(MC_QO_FULL + qb), (item >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
+                    if (!mbar_wait(bar(MC_TM_EMPTY + buf), ((item >> 2) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                    tc_fence_after();
+                    const uint32_t zt = tmem_base + buf * 128u, tt = zt + 64u;
+                    const uint32_t bq = sbase + MC_OFF_QO + qb * kQoBuf, bo = bq + 2 * kHalfB64;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {               // d = 128 = 8 steps of K = 16
+                        const uint32_t offa = (ks >> 2) * kHalfBytes + (ks & 3) * 32, offb = (ks >> 2) * kHalfB64 + (ks & 3) * 32;
+                        tc_mma(zt, smem_desc_k_sw128(ak + offa), smem_desc_k_sw128(bq + offb), idesc, ks > 0);
+                    }
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t offa = (ks >> 2) * kHalfBytes + (ks & 3) * 32, offb = (ks >> 2) * kHalfB64 + (ks & 3) * 32;
+                        tc_mma(tt, smem_desc_k_sw128(av + offa), smem_desc_k_sw128(bo + offb), idesc, ks > 0);
+                    }
+                    tc_commit(bar(MC_TM_FULL + buf));              // accumulators ready for the chunk's epilogue group
+                    tc_commit(bar(MC_QO_EMPTY + qb));              // this Q / O buffer may be refilled
+                }
+                if (!failed) tc_commit(bar(MC_EMPTY + st));        // K/V stage no longer read by the MMAs
+            }
+        }
+    } else if (warp < 4) {
+        // ==================== ||v_p||^2 per tile, per-row constants per chunk ===================
+        const int t64 = threadIdx.x - 64;                          // 0..63
+        uint32_t item = 0, titem = 0;
+        for (; !tw.done() && !failed; tw.next(), ++titem) {
+            const int unit = tw.unit;
+            const uint32_t st = titem % NSTAGE, slot = titem % NSLOT;
+            if (!mbar_wait(bar(MC_FULL + st), (titem / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
+            const uint8_t* vt = smem + MC_OFF_V + st * kOperandBytes;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int tok = t64 + 64 * j;
+                float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
+                        const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
+                        const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
+                        acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
+                        acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
+                    }
+                const float2 sum = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
+                sNv[slot * TILE + tok] = sum.x + sum.y;
+            }
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(bar(MC_NV + slot)); mbar_arrive(bar(MC_EMPTY + st)); }
+            for (int c = 0; c < nc; ++c, ++item) {
+                const uint32_t cs = item & 3;
+                const size_t crow = (size_t)unit * p.rows_out + (size_t)c * MC_ROWS + t64;
+                const float2 cst = make_float2(-p.lse2[crow], p.onorm[crow]);
+                // slot cs is free once the chunk that used it four items ago has been summed
+                if (!mbar_wait(bar(MC_TM_EMPTY + cs), ((item >> 2) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                float* cdst = sConst + cs * 128 + (t64 >> 1) * 4 + (t64 & 1);      // row pair: (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
+                cdst[0] = cst.x; cdst[2] = cst.y;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(MC_CONST + cs));
+            }
+        }
+    } else {
+        // ======================================= epilogue =======================================
+        const int wg = (warp - 4) >> 2;                            // takes the items with item & 1 == wg
+        const int lane_grp = warp & 3;                             // TMEM lanes 32*lane_grp .. +31
+        const int tok = lane_grp * 32 + lane;                      // token within the tile
+        const float2 sl2 = make_float2(p.scale * kLog2e, p.scale * kLog2e), sc = make_float2(p.scale, p.scale);
+        const size_t plane = (size_t)units * p.Nmax;
+        uint32_t item = 0, titem = 0;
+        for (; !tw.done() && !failed; tw.next(), ++titem) {
+            const int unit = tw.unit, b = unit / p.Hkv;
+            const int N = tc_seq_len(p, b), t0 = tw.tile * TILE;
+            const int ptok = t0 + tok;
+            const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
+            RowSums S;
+            S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
+            for (int c = 0; c < nc && !failed; ++c, ++item) {
+                if ((item & 1) != (uint32_t)wg) continue;
+                const uint32_t buf = item & 3;
+                if (!mbar_wait(bar(MC_CONST + buf), (item >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
+                if (!mbar_wait(bar(MC_TM_FULL + buf), (item >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
+                tc_fence_after();
+                const float4* cst = reinterpret_cast<const float4*>(sConst + buf * 128);
+                const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 128u, tt = zt + 64u;
+                if (masked_tile)
+                    score_chunk<VARS, true>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, N - p.W, p.W, (c * MC_ROWS) % p.W);
+                else
+                    score_chunk<VARS, false>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, 0, 0, 0);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(MC_TM_EMPTY + buf));
+            }
+            if (failed) break;
+            // the tile's sums: group 1 hands its part to group 0 (buffers alternate with the tile)
+            float* xs = sX + (titem & 1) * (TILE * 8) + tok * 8;
+            float q[7] = {S.s1.x + S.s1.y, S.s2.x + S.s2.y, S.s3.x + S.s3.y, S.s4.x + S.s4.y,
+                          S.s5.x + S.s5.y, S.s6.x + S.s6.y, S.s7.x + S.s7.y};
+            if (wg == 1) {
+                *reinterpret_cast<float4*>(xs) = make_float4(q[0], q[1], q[2], q[3]);
+                *reinterpret_cast<float4*>(xs + 4) = make_float4(q[4], q[5], q[6], 0.f);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(MC_XCHG + (titem & 1)));
+            } else {
+                const uint32_t slot = titem % NSLOT;
+                if (!mbar_wait(bar(MC_NV + slot), (titem / NSLOT) & 1)) { failed = true; fail_site = __LINE__; break; }
+                const float nv = sNv[slot * TILE + tok];
+                if (!mbar_wait(bar(MC_XCHG + (titem & 1)), (titem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
+                const float4 xa = *reinterpret_cast<const float4*>(xs), xb = *reinterpret_cast<const float4*>(xs + 4);
+                q[0] += xa.x; q[1] += xa.y; q[2] += xa.z; q[3] += xa.w; q[4] += xb.x; q[5] += xb.y; q[6] += xb.z;
+                if (ptok < p.Nmax) {
+                    float* out = p.scores + (size_t)unit * p.Nmax;
+                    const bool live = ptok < N;
+                    const float s2 = p.scale * p.scale;
+                    int pl = 0;
+                    if (p.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + ptok] = live ? nv * q[5] : 0.f;
+                    if (p.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + ptok] = live ? s2 * (fmaf(nv, q[4], q[2]) + q[3]) : 0.f;
+                    if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] = live ? fmaf(nv, q[0], fmaf(p.scale, q[1], s2 * q[2])) : 0.f;
+                    if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? q[6] : 0.f;
+                }
+            }
+        }
+        // padding beyond the last tile of a shorter sequence: zeros
+        if (p.seq_lens) {
+            const int et = threadIdx.x - 128;                      // 0..255
+            const int n_planes = __popc(p.variants);
+            for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
+                const int first = (tc_seq_len(p, unit / p.Hkv) + TILE - 1) / TILE * TILE;
+                for (int pl = 0; pl < n_planes; ++pl)
+                    for (int i = first + et; i < p.Nmax; i += 256) p.scores[(size_t)pl * plane + (size_t)unit * p.Nmax + i] = 0.f;
+            }
+        }
+    }
+
+    if (failed) atomicCAS(p.status, 0u, (unsigned)(fail_site > 0 ? fail_site : 1));   // the first failure is kept
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// =================================================================================================
 // Pass 1 on tensor cores: streaming softmax statistics and window outputs (Sec. 3: A = softmax(Z),
 // O = A V over the perturbation window, Eq. 9), split over the cached tokens.
 //
@@ -934,12 +1208,15 @@ bool make_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row chunks.  Pass 1 cuts the R window rows into n_chunks pieces of chunk_rows <= 128 (its MMA M
+// dimension).  Pass 2 takes the rows whole when R <= 128 and in pieces of 64 otherwise; rows_out is
+// the padded row count of the combined arrays it reads.
 struct TcChunks { int n_chunks, chunk_rows, rows_out; };
 TcChunks tc_chunks(int R) {
     TcChunks c;
     c.n_chunks = (R + 127) / 128;
     c.chunk_rows = ((R + c.n_chunks - 1) / c.n_chunks + 15) / 16 * 16;
-    c.rows_out = c.n_chunks * c.chunk_rows;
+    c.rows_out = c.n_chunks > 1 ? (R + MC_ROWS - 1) / MC_ROWS * MC_ROWS : c.chunk_rows;
     return c;
 }
 
@@ -1041,6 +1318,27 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     p.status = (unsigned int*)(wsb + plan.off_flag);
     const long long n_tiles = (long long)units * ((s.Nmax + TILE - 1) / TILE);
     const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
+
+    if (ch.n_chunks > 1) {                               // more than 128 window rows: chunks of 64, K/V tile kept
+        CUtensorMap mq64, mo64;
+        const uint64_t qd[2] = {(uint64_t)kD, (uint64_t)s.B * s.Hq * s.W};
+        const uint64_t qs[1] = {(uint64_t)q.st * 2};
+        const uint64_t od[2] = {(uint64_t)kD, (uint64_t)units * ch.rows_out};
+        const uint64_t os[1] = {(uint64_t)kD * 2};
+        if (!make_map(&mq64, q.ptr, 2, qd, qs, MC_ROWS) || !make_map(&mo64, wsb + plan.off_obf, 2, od, os, MC_ROWS)) {
+            set_last_cuda_error((int)cudaErrorInvalidValue);
+            return OBC_ERR_CUDA;
+        }
+        p.n_chunks = ch.rows_out / MC_ROWS; p.chunk_rows = MC_ROWS;
+        auto launch_multi = [&](auto kernel) -> obc_status {
+            OBC_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMulti));
+            { ProfScope ps("tc_pass2", stream); OBC_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmemMulti, stream, 1, mq64, mo64, mk, mv, p)); }
+            return OBC_OK;
+        };
+        if (s.variants == OBC_VAR_VK) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_VK>);
+        if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_K | OBC_VAR_VK>);
+        return launch_multi(tc_pass2_multi_kernel<OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN>);
+    }
 
     auto launch = [&](auto kernel) -> obc_status {
         OBC_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
