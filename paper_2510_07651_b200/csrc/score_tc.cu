@@ -121,16 +121,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 64 bf16 (128 B),
-// 8-row groups 1024 B apart (the image a swizzle-128B TMA box of 64 elements x rows leaves)
-__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);           // start address >> 4
-    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset: 8 rows x 128 B
-    d |= (uint64_t)1 << 46;                          // descriptor version (sm_100)
-    d |= (uint64_t)2 << 61;                          // layout: 128-byte swizzle
+// Shared-memory matrix descriptors: K-major operand with 128-byte swizzle = rows of 64 bf16 (128 B),
+// 8-row groups 1024 B apart (the image a swizzle-128B TMA box of 64 elements x rows leaves).
+// The MMA thread builds two descriptors per instruction, so they are kept cheap: the high word of a
+// descriptor is a constant and the low word is (address >> 4) plus constant fields; shared memory
+// addresses are below 256 KB, so adding a byte offset / 16 to the low word cannot carry out of the
+// 14-bit address field.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);       // SBO 1024 B, version 1, 128-byte swizzle
+__device__ __forceinline__ uint32_t desc_lo_k(uint32_t addr) { return (addr >> 4) | (1u << 16); }                     // K-major
+__device__ __forceinline__ uint32_t desc_lo_mn(uint32_t addr) { return (addr >> 4) | ((kHalfBytes >> 4) << 16); }     // MN-major, LBO 16 KB
+__device__ __forceinline__ uint64_t desc_make(uint32_t lo) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(kDescHi));
     return d;
+}
+__device__ __forceinline__ constexpr uint32_t desc_kstep(int ks, uint32_t half_bytes) {   // K step ks of a [rows][2 x 64] operand
+    return (uint32_t)(ks >> 2) * (half_bytes >> 4) + (uint32_t)(ks & 3) * 2u;
 }
 // kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128
 __host__ __device__ constexpr uint32_t idesc_bf16(int n) {
@@ -159,14 +165,17 @@ __device__ __forceinline__ int tc_seq_len(const TcParams& p, int b) { return tc_
 // memory) and ragged batches are balanced.  Every role of the CTA runs its own copy.
 struct TileWalk {
     int unit, tile, tiles_in_unit;            // current position
-    long long left;                           // tiles still to visit, including the current one
+    long long left;                           // positions still to visit, including the current one
     const TcParams* p;
-    __device__ __forceinline__ int tiles_of(int b) const { return (tc_seq_len(*p, b) + TILE - 1) / TILE; }
-    __device__ void init(const TcParams& prm) {
-        p = &prm;
+    int span;                                 // consecutive tiles of a unit that one position stands for
+    __device__ __forceinline__ int tiles_of(int b) const {
+        return ((tc_seq_len(*p, b) + TILE - 1) / TILE + span - 1) / span;
+    }
+    __device__ void init(const TcParams& prm, int tiles_per_position = 1) {
+        p = &prm; span = tiles_per_position;
         long long total = 0;
         if (p->seq_lens) { for (int b = 0; b < p->B; ++b) total += (long long)p->Hkv * tiles_of(b); }
-        else total = (long long)p->B * p->Hkv * ((p->Nmax + TILE - 1) / TILE);
+        else total = (long long)p->B * p->Hkv * tiles_of(0);
         const long long lo = total * blockIdx.x / gridDim.x, hi = total * (blockIdx.x + 1) / gridDim.x;
         left = hi - lo;
         unit = 0; tile = 0; tiles_in_unit = 0;
@@ -375,17 +384,14 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     if (!mbar_wait(bar(BAR_TM_EMPTY + buf), ((item >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                     tc_fence_after();
                     const uint32_t zt = tmem_base + buf * 256u, tt = zt + 128u;
-                    const uint32_t ak = sbase + OFF_K + st * kOperandBytes, av = sbase + OFF_V + st * kOperandBytes;
+                    const uint32_t ak = desc_lo_k(sbase + OFF_K + st * kOperandBytes), av = desc_lo_k(sbase + OFF_V + st * kOperandBytes);
+                    const uint32_t bq = desc_lo_k(sbase + OFF_Q), bo = desc_lo_k(sbase + OFF_O);
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {               // d = 128 = 8 steps of K = 16
-                        const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        tc_mma(zt, smem_desc_k_sw128(ak + off), smem_desc_k_sw128(sbase + OFF_Q + off), idesc, ks > 0);
-                    }
+                    for (int ks = 0; ks < 8; ++ks)                 // d = 128 = 8 steps of K = 16
+                        tc_mma(zt, desc_make(ak + desc_kstep(ks, kHalfBytes)), desc_make(bq + desc_kstep(ks, kHalfBytes)), idesc, ks > 0);
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        tc_mma(tt, smem_desc_k_sw128(av + off), smem_desc_k_sw128(sbase + OFF_O + off), idesc, ks > 0);
-                    }
+                    for (int ks = 0; ks < 8; ++ks)
+                        tc_mma(tt, desc_make(av + desc_kstep(ks, kHalfBytes)), desc_make(bo + desc_kstep(ks, kHalfBytes)), idesc, ks > 0);
                     tc_commit(bar(BAR_TM_FULL + owner * 2 + buf)); // accumulators ready for the tile's epilogue group
                     tc_commit(bar(BAR_EMPTY + st));                // K/V stage no longer read by the MMA
                     // Q / O may be overwritten once these MMAs are done, if the next item needs others
@@ -512,26 +518,23 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
 // =================================================================================================
 // Pass 2 for more than 128 window rows per KV head (e.g. GQA 7 x W 64 = 448).  The rows are cut
-// into chunks of 64; a K/V tile is fetched ONCE and stays in shared memory while its chunks pass:
-//     per tile    K/V through the 2-stage ring, ||v_p||^2
-//     per chunk   Q / -2 O chunk into one of two buffers, one pair of MMAs with N = 64 into one of
-//                 four TMEM buffers (Z 64 + T' 64 columns), per-row constants into one of four slots
-// The two epilogue warpgroups take alternate chunks (so each owns two TMEM buffers and the MMAs of
-// its next chunk run while it sums the current one) and keep partial sums of the same 128 tokens;
-// after the tile's last chunk warpgroup 1 hands its sums to warpgroup 0 through shared memory.
+// into chunks of 64.  A CTA holds TWO consecutive token tiles of a unit in its two K/V stages and
+// sweeps the row chunks over both: every Q / -2 O chunk (two buffers) is fetched once per tile pair
+// and used by two MMA pairs with N = 64 (four TMEM buffers of Z 64 + T' 64 columns), so the fetch
+// of the next chunk hides behind twice the tensor work.  Epilogue warpgroup j owns tile j of the
+// pair: it sums all chunks of its 128 tokens in registers and stores their scores itself.
 // =================================================================================================
-constexpr int MC_ROWS = 64;
-constexpr uint32_t kHalfB64 = 64 * 128;                           // B operand block: [64 rows][64 bf16]                                       // window rows per chunk
+constexpr int MC_ROWS = 64;                                       // window rows per chunk
+constexpr uint32_t kHalfB64 = 64 * 128;                           // B operand block: [64 rows][64 bf16]
 constexpr uint32_t kQoBuf = 4 * kHalfB64;                         // Q chunk (2 x 8 KB) + -2 O chunk (2 x 8 KB)
 constexpr uint32_t MC_OFF_QO = 0;                                 // 2 buffers x 32 KB
-constexpr uint32_t MC_OFF_K = MC_OFF_QO + 2 * kQoBuf;             // NSTAGE x 32 KB
-constexpr uint32_t MC_OFF_V = MC_OFF_K + NSTAGE * kOperandBytes;
-constexpr uint32_t MC_OFF_NV = MC_OFF_V + NSTAGE * kOperandBytes; // NSLOT x 128 floats (per tile)
-constexpr uint32_t MC_OFF_CONST = MC_OFF_NV + NSLOT * TILE * 4;   // 4 slots x 32 float4 (per chunk)
-constexpr uint32_t MC_OFF_X = MC_OFF_CONST + 4 * 32 * 16;         // 2 x 128 tokens x 8 floats (exchange)
-constexpr uint32_t MC_OFF_BAR = MC_OFF_X + 2 * TILE * 8 * 4;
+constexpr uint32_t MC_OFF_K = MC_OFF_QO + 2 * kQoBuf;             // 2 tiles x 32 KB
+constexpr uint32_t MC_OFF_V = MC_OFF_K + 2 * kOperandBytes;
+constexpr uint32_t MC_OFF_NV = MC_OFF_V + 2 * kOperandBytes;      // [pair parity][tile of the pair][128] floats
+constexpr uint32_t MC_OFF_CONST = MC_OFF_NV + 4 * TILE * 4;       // 4 slots x 32 float4 (per chunk)
+constexpr uint32_t MC_OFF_BAR = MC_OFF_CONST + 4 * 32 * 16;
 enum { MC_FULL = 0, MC_EMPTY = 2, MC_QO_FULL = 4, MC_QO_EMPTY = 6, MC_TM_FULL = 8, MC_TM_EMPTY = 12,
-       MC_NV = 16, MC_CONST = 16 + NSLOT, MC_XCHG = 20 + NSLOT, MC_NBARS = 22 + NSLOT };
+       MC_NV = 16, MC_CONST = 18, MC_NBARS = 22 };
 constexpr uint32_t MC_OFF_TMEM = MC_OFF_BAR + MC_NBARS * 8;
 constexpr uint32_t kSmemMulti = MC_OFF_TMEM + 16 + 1024;
 
@@ -548,20 +551,18 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + MC_OFF_TMEM);
     float* sNv = reinterpret_cast<float*>(smem + MC_OFF_NV);
     float* sConst = reinterpret_cast<float*>(smem + MC_OFF_CONST);
-    float* sX = reinterpret_cast<float*>(smem + MC_OFF_X);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int units = p.B * p.Hkv;
-    const int nc = p.n_chunks;                                   // chunks of MC_ROWS rows per tile
+    const int nc = p.n_chunks;                                   // chunks of MC_ROWS rows
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_k); prefetch_tmap(&map_v); prefetch_tmap(&map_q); prefetch_tmap(&map_o);
-        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(MC_FULL + i), 1); mbar_init(bar(MC_EMPTY + i), 3); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(MC_FULL + i), 1); mbar_init(bar(MC_EMPTY + i), 3); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(MC_QO_FULL + i), 1); mbar_init(bar(MC_QO_EMPTY + i), 1); }
         for (int i = 0; i < 4; ++i) { mbar_init(bar(MC_TM_FULL + i), 1); mbar_init(bar(MC_TM_EMPTY + i), 4); }
-        for (int i = 0; i < NSLOT; ++i) mbar_init(bar(MC_NV + i), 2);
+        for (int i = 0; i < 2; ++i) mbar_init(bar(MC_NV + i), 2);
         for (int i = 0; i < 4; ++i) mbar_init(bar(MC_CONST + i), 2);
-        for (int i = 0; i < 2; ++i) mbar_init(bar(MC_XCHG + i), 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -577,38 +578,34 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     int fail_site = 0;                             // source line of the wait that gave up (status word)
     const uint32_t qo_bytes = MC_ROWS * 128u * 2u * 2u;
 
-    // `titem` counts tiles, `item` (tile, chunk) pairs.  Rings: K/V stage and norm slot by titem;
-    // Q/O buffer by item & 1, TMEM buffer and constant slot by item & 3.  Items go to the epilogue
-    // groups alternately, so a group always sees the same TMEM buffers and constant slots.
+    // A position of the walk is a pair of tiles (2 * tw.tile + j, j = 0, 1; the second one may lie past
+    // the end of a unit with an odd tile count: it is computed all the same and stores only zeros).
+    // `pitem` counts positions, `citem` row chunks over all positions; the chunk's two MMA pairs are
+    // items 2 * citem + j.  Rings: K/V stage j; Q/O buffer citem & 1; constant slot citem & 3; TMEM
+    // buffer item & 3, so that epilogue group j always sees buffers j and j + 2.
     TileWalk tw;
-    tw.init(p);
+    tw.init(p, 2);
     if (!(warp == 0 && lane == 0)) pdl_wait();       // the producer thread waits after its first K/V copies
     if (warp == 0) {
         // ===================================== TMA producer =====================================
         if (lane == 0) {
-            uint32_t item = 0, titem = 0, kv_issued = 0;
-            TileWalk ahead = tw;                                   // position of the next K/V tile to fetch
-            auto fetch_kv = [&]() -> bool {                        // next tile of the walk into its stage
-                if (ahead.done()) return true;
-                const uint32_t st = kv_issued % NSTAGE;
-                if (!mbar_wait(bar(MC_EMPTY + st), ((kv_issued / NSTAGE) & 1) ^ 1)) return false;
-                const int unit = ahead.unit, b = unit / p.Hkv, g = unit % p.Hkv, t0 = ahead.tile * TILE;
-                mbar_expect_tx(bar(MC_FULL + st), 2 * kOperandBytes);
-                const uint32_t dk = sbase + MC_OFF_K + st * kOperandBytes, dv = sbase + MC_OFF_V + st * kOperandBytes;
-                tma_load_4d(dk, &map_k, bar(MC_FULL + st), 0, t0, g, b);
-                tma_load_4d(dk + kHalfBytes, &map_k, bar(MC_FULL + st), 64, t0, g, b);
-                tma_load_4d(dv, &map_v, bar(MC_FULL + st), 0, t0, g, b);
-                tma_load_4d(dv + kHalfBytes, &map_v, bar(MC_FULL + st), 64, t0, g, b);
-                ++kv_issued; ahead.next();
-                return true;
-            };
-            if (!fetch_kv()) { failed = true; fail_site = __LINE__; }
-            pdl_wait();                                            // K and V were read by pass 1; -2 O is the preceding kernel's output
-            for (; !tw.done() && !failed; tw.next(), ++titem) {
+            uint32_t pitem = 0, citem = 0;
+            for (; !tw.done() && !failed; tw.next(), ++pitem) {
                 const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv;
-                for (int c = 0; c < nc; ++c, ++item) {
-                    const uint32_t qb = item & 1;
-                    if (!mbar_wait(bar(MC_QO_EMPTY + qb), ((item >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                for (int j = 0; j < 2 && !failed; ++j) {
+                    if (!mbar_wait(bar(MC_EMPTY + j), (pitem & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                    const int t0 = (tw.tile * 2 + j) * TILE;
+                    mbar_expect_tx(bar(MC_FULL + j), 2 * kOperandBytes);
+                    const uint32_t dk = sbase + MC_OFF_K + j * kOperandBytes, dv = sbase + MC_OFF_V + j * kOperandBytes;
+                    tma_load_4d(dk, &map_k, bar(MC_FULL + j), 0, t0, g, b);
+                    tma_load_4d(dk + kHalfBytes, &map_k, bar(MC_FULL + j), 64, t0, g, b);
+                    tma_load_4d(dv, &map_v, bar(MC_FULL + j), 0, t0, g, b);
+                    tma_load_4d(dv + kHalfBytes, &map_v, bar(MC_FULL + j), 64, t0, g, b);
+                }
+                if (pitem == 0) pdl_wait();                        // K and V were read by pass 1; -2 O is the preceding kernel's output
+                for (int c = 0; c < nc && !failed; ++c, ++citem) {
+                    const uint32_t qb = citem & 1;
+                    if (!mbar_wait(bar(MC_QO_EMPTY + qb), ((citem >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                     mbar_expect_tx(bar(MC_QO_FULL + qb), qo_bytes);
                     const int qrow = (b * p.Hkv * p.G + g * p.G) * p.W + c * MC_ROWS;
                     const int orow = unit * p.rows_out + c * MC_ROWS;
@@ -617,17 +614,15 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     tma_load_2d(dq + kHalfB64, &map_q, bar(MC_QO_FULL + qb), 64, qrow);
                     tma_load_2d(dob, &map_o, bar(MC_QO_FULL + qb), 0, orow);
                     tma_load_2d(dob + kHalfB64, &map_o, bar(MC_QO_FULL + qb), 64, orow);
-                    // the next tile's K/V once this tile's first two chunks are on their way
-                    if (c == (nc > 1 ? 1 : 0) && !fetch_kv()) { failed = true; fail_site = __LINE__; break; }
                 }
             }
             // drain: every copy this thread issued must have landed before the CTA may exit
-            for (uint32_t back = 0; back < NSTAGE && back < kv_issued; ++back) {
-                const uint32_t it = kv_issued - 1 - back;
-                (void)mbar_wait(bar(MC_FULL + it % NSTAGE), (it / NSTAGE) & 1);
+            if (pitem > 0) {
+                (void)mbar_wait(bar(MC_FULL + 0), (pitem - 1) & 1);
+                (void)mbar_wait(bar(MC_FULL + 1), (pitem - 1) & 1);
             }
-            for (uint32_t back = 0; back < 2 && back < item; ++back) {
-                const uint32_t it = item - 1 - back;
+            for (uint32_t back = 0; back < 2 && back < citem; ++back) {
+                const uint32_t it = citem - 1 - back;
                 (void)mbar_wait(bar(MC_QO_FULL + (it & 1)), (it >> 1) & 1);
             }
         }
@@ -635,68 +630,74 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         // ===================================== MMA issuer =======================================
         if (lane == 0) {
             const uint32_t idesc = idesc_bf16(MC_ROWS);
-            uint32_t item = 0, titem = 0;
-            for (; !tw.done() && !failed; tw.next(), ++titem) {
-                const uint32_t st = titem % NSTAGE;
-                if (!mbar_wait(bar(MC_FULL + st), (titem / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
-                const uint32_t ak = sbase + MC_OFF_K + st * kOperandBytes, av = sbase + MC_OFF_V + st * kOperandBytes;
-                for (int c = 0; c < nc; ++c, ++item) {
-                    const uint32_t qb = item & 1, buf = item & 3;
-                    if (!mbar_wait(bar(MC_QO_FULL + qb), (item >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
-                    if (!mbar_wait(bar(MC_TM_EMPTY + buf), ((item >> 2) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
-                    tc_fence_after();
-                    const uint32_t zt = tmem_base + buf * 128u, tt = zt + 64u;
-                    const uint32_t bq = sbase + MC_OFF_QO + qb * kQoBuf, bo = bq + 2 * kHalfB64;
+            uint32_t pitem = 0, citem = 0;
+            for (; !tw.done() && !failed; tw.next(), ++pitem) {
+                if (!mbar_wait(bar(MC_FULL + 0), pitem & 1) || !mbar_wait(bar(MC_FULL + 1), pitem & 1)) { failed = true; fail_site = __LINE__; break; }
+                for (int c = 0; c < nc && !failed; ++c, ++citem) {
+                    const uint32_t qb = citem & 1;
+                    if (!mbar_wait(bar(MC_QO_FULL + qb), (citem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
+                    const uint32_t bq = desc_lo_k(sbase + MC_OFF_QO + qb * kQoBuf), bo = bq + ((2 * kHalfB64) >> 4);
+                    for (int j = 0; j < 2; ++j) {
+                        const uint32_t item = 2 * citem + j, buf = item & 3;
+                        if (!mbar_wait(bar(MC_TM_EMPTY + buf), ((item >> 2) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                        tc_fence_after();
+                        const uint32_t zt = tmem_base + buf * 128u, tt = zt + 64u;
+                        const uint32_t ak = desc_lo_k(sbase + MC_OFF_K + j * kOperandBytes), av = desc_lo_k(sbase + MC_OFF_V + j * kOperandBytes);
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {               // d = 128 = 8 steps of K = 16
-                        const uint32_t offa = (ks >> 2) * kHalfBytes + (ks & 3) * 32, offb = (ks >> 2) * kHalfB64 + (ks & 3) * 32;
-                        tc_mma(zt, smem_desc_k_sw128(ak + offa), smem_desc_k_sw128(bq + offb), idesc, ks > 0);
-                    }
+                        for (int ks = 0; ks < 8; ++ks)             // d = 128 = 8 steps of K = 16
+                            tc_mma(zt, desc_make(ak + desc_kstep(ks, kHalfBytes)), desc_make(bq + desc_kstep(ks, kHalfB64)), idesc, ks > 0);
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t offa = (ks >> 2) * kHalfBytes + (ks & 3) * 32, offb = (ks >> 2) * kHalfB64 + (ks & 3) * 32;
-                        tc_mma(tt, smem_desc_k_sw128(av + offa), smem_desc_k_sw128(bo + offb), idesc, ks > 0);
+                        for (int ks = 0; ks < 8; ++ks)
+                            tc_mma(tt, desc_make(av + desc_kstep(ks, kHalfBytes)), desc_make(bo + desc_kstep(ks, kHalfB64)), idesc, ks > 0);
+                        tc_commit(bar(MC_TM_FULL + buf));          // accumulators ready for epilogue group j
                     }
-                    tc_commit(bar(MC_TM_FULL + buf));              // accumulators ready for the chunk's epilogue group
+                    if (failed) break;
                     tc_commit(bar(MC_QO_EMPTY + qb));              // this Q / O buffer may be refilled
                 }
-                if (!failed) tc_commit(bar(MC_EMPTY + st));        // K/V stage no longer read by the MMAs
+                if (!failed) { tc_commit(bar(MC_EMPTY + 0)); tc_commit(bar(MC_EMPTY + 1)); }   // both tiles no longer read
             }
         }
     } else if (warp < 4) {
         // ==================== ||v_p||^2 per tile, per-row constants per chunk ===================
         const int t64 = threadIdx.x - 64;                          // 0..63
-        uint32_t item = 0, titem = 0;
-        for (; !tw.done() && !failed; tw.next(), ++titem) {
+        uint32_t pitem = 0, citem = 0;
+        for (; !tw.done() && !failed; tw.next(), ++pitem) {
             const int unit = tw.unit;
-            const uint32_t st = titem % NSTAGE, slot = titem % NSLOT;
-            if (!mbar_wait(bar(MC_FULL + st), (titem / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
-            const uint8_t* vt = smem + MC_OFF_V + st * kOperandBytes;
+            for (int j = 0; j < 2 && !failed; ++j) {
+                if (!mbar_wait(bar(MC_FULL + j), pitem & 1)) { failed = true; fail_site = __LINE__; break; }
+                const uint8_t* vt = smem + MC_OFF_V + j * kOperandBytes;
+                float* nvdst = sNv + ((pitem & 1) * 2 + j) * TILE;
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int tok = t64 + 64 * j;
-                float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int tok = t64 + 64 * jj;
+                    float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
-                        const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
-                        const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
-                        acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
-                        acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
-                    }
-                const float2 sum = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
-                sNv[slot * TILE + tok] = sum.x + sum.y;
+                        for (int ch = 0; ch < 8; ++ch) {
+                            const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
+                            const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
+                            const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
+                            acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
+                            acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
+                        }
+                    const float2 sum = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
+                    nvdst[tok] = sum.x + sum.y;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(MC_EMPTY + j));
             }
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(bar(MC_NV + slot)); mbar_arrive(bar(MC_EMPTY + st)); }
-            for (int c = 0; c < nc; ++c, ++item) {
-                const uint32_t cs = item & 3;
+            if (failed) break;
+            if (lane == 0) mbar_arrive(bar(MC_NV + (pitem & 1)));
+            for (int c = 0; c < nc; ++c, ++citem) {
+                const uint32_t cs = citem & 3;
                 const size_t crow = (size_t)unit * p.rows_out + (size_t)c * MC_ROWS + t64;
                 const float2 cst = make_float2(-p.lse2[crow], p.onorm[crow]);
-                // slot cs is free once the chunk that used it four items ago has been summed
-                if (!mbar_wait(bar(MC_TM_EMPTY + cs), ((item >> 2) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                // slot cs was last read by the chunk four back; the chunk two back has been summed once
+                // the TMEM buffers this chunk is going to use are free again
+                const uint32_t i0 = 2 * citem, i1 = i0 + 1;
+                if (!mbar_wait(bar(MC_TM_EMPTY + (i0 & 3)), ((i0 >> 2) & 1) ^ 1) ||
+                    !mbar_wait(bar(MC_TM_EMPTY + (i1 & 3)), ((i1 >> 2) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                 float* cdst = sConst + cs * 128 + (t64 >> 1) * 4 + (t64 & 1);      // row pair: (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
                 cdst[0] = cst.x; cdst[2] = cst.y;
                 __syncwarp();
@@ -705,26 +706,25 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         }
     } else {
         // ======================================= epilogue =======================================
-        const int wg = (warp - 4) >> 2;                            // takes the items with item & 1 == wg
+        const int wg = (warp - 4) >> 2;                            // owns tile wg of every pair
         const int lane_grp = warp & 3;                             // TMEM lanes 32*lane_grp .. +31
         const int tok = lane_grp * 32 + lane;                      // token within the tile
         const float2 sl2 = make_float2(p.scale * kLog2e, p.scale * kLog2e), sc = make_float2(p.scale, p.scale);
         const size_t plane = (size_t)units * p.Nmax;
-        uint32_t item = 0, titem = 0;
-        for (; !tw.done() && !failed; tw.next(), ++titem) {
+        uint32_t pitem = 0, citem = 0;
+        for (; !tw.done() && !failed; tw.next(), ++pitem) {
             const int unit = tw.unit, b = unit / p.Hkv;
-            const int N = tc_seq_len(p, b), t0 = tw.tile * TILE;
+            const int N = tc_seq_len(p, b), t0 = (tw.tile * 2 + wg) * TILE;
             const int ptok = t0 + tok;
             const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
-            for (int c = 0; c < nc && !failed; ++c, ++item) {
-                if ((item & 1) != (uint32_t)wg) continue;
-                const uint32_t buf = item & 3;
-                if (!mbar_wait(bar(MC_CONST + buf), (item >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
+            for (int c = 0; c < nc; ++c, ++citem) {
+                const uint32_t item = 2 * citem + wg, buf = item & 3, cs = citem & 3;
+                if (!mbar_wait(bar(MC_CONST + cs), (citem >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
                 if (!mbar_wait(bar(MC_TM_FULL + buf), (item >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
                 tc_fence_after();
-                const float4* cst = reinterpret_cast<const float4*>(sConst + buf * 128);
+                const float4* cst = reinterpret_cast<const float4*>(sConst + cs * 128);
                 const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 128u, tt = zt + 64u;
                 if (masked_tile)
                     score_chunk<VARS, true>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, N - p.W, p.W, (c * MC_ROWS) % p.W);
@@ -735,32 +735,19 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 if (lane == 0) mbar_arrive(bar(MC_TM_EMPTY + buf));
             }
             if (failed) break;
-            // the tile's sums: group 1 hands its part to group 0 (buffers alternate with the tile)
-            float* xs = sX + (titem & 1) * (TILE * 8) + tok * 8;
-            float q[7] = {S.s1.x + S.s1.y, S.s2.x + S.s2.y, S.s3.x + S.s3.y, S.s4.x + S.s4.y,
-                          S.s5.x + S.s5.y, S.s6.x + S.s6.y, S.s7.x + S.s7.y};
-            if (wg == 1) {
-                *reinterpret_cast<float4*>(xs) = make_float4(q[0], q[1], q[2], q[3]);
-                *reinterpret_cast<float4*>(xs + 4) = make_float4(q[4], q[5], q[6], 0.f);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(MC_XCHG + (titem & 1)));
-            } else {
-                const uint32_t slot = titem % NSLOT;
-                if (!mbar_wait(bar(MC_NV + slot), (titem / NSLOT) & 1)) { failed = true; fail_site = __LINE__; break; }
-                const float nv = sNv[slot * TILE + tok];
-                if (!mbar_wait(bar(MC_XCHG + (titem & 1)), (titem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
-                const float4 xa = *reinterpret_cast<const float4*>(xs), xb = *reinterpret_cast<const float4*>(xs + 4);
-                q[0] += xa.x; q[1] += xa.y; q[2] += xa.z; q[3] += xa.w; q[4] += xb.x; q[5] += xb.y; q[6] += xb.z;
-                if (ptok < p.Nmax) {
-                    float* out = p.scores + (size_t)unit * p.Nmax;
-                    const bool live = ptok < N;
-                    const float s2 = p.scale * p.scale;
-                    int pl = 0;
-                    if (p.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + ptok] = live ? nv * q[5] : 0.f;
-                    if (p.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + ptok] = live ? s2 * (fmaf(nv, q[4], q[2]) + q[3]) : 0.f;
-                    if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] = live ? fmaf(nv, q[0], fmaf(p.scale, q[1], s2 * q[2])) : 0.f;
-                    if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? q[6] : 0.f;
-                }
+            if (!mbar_wait(bar(MC_NV + (pitem & 1)), (pitem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
+            const float nv = sNv[((pitem & 1) * 2 + wg) * TILE + tok];
+            if (ptok < p.Nmax) {
+                float* out = p.scores + (size_t)unit * p.Nmax;
+                const bool live = ptok < N;
+                const float s2 = p.scale * p.scale;
+                int pl = 0;
+                if (p.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + ptok] = live ? nv * (S.s6.x + S.s6.y) : 0.f;
+                if (p.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + ptok] =
+                    live ? s2 * (fmaf(nv, S.s5.x + S.s5.y, S.s3.x + S.s3.y) + (S.s4.x + S.s4.y)) : 0.f;
+                if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] =
+                    live ? fmaf(nv, S.s1.x + S.s1.y, fmaf(p.scale, S.s2.x + S.s2.y, s2 * (S.s3.x + S.s3.y))) : 0.f;
+                if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? S.s7.x + S.s7.y : 0.f;
             }
         }
         // padding beyond the last tile of a shorter sequence: zeros
@@ -870,18 +857,9 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
                  ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-// MN-major B operand with 128-byte swizzle: 64 contiguous elements of N per 128-byte row, 8 rows of
-// K per 1024-byte group (stride byte offset), the next 64 elements of N one 16 KB block further
-// (leading byte offset).  This is the image of a [tokens][head_dim] tile loaded as two 64-wide boxes.
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)(kHalfBytes >> 4) << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
+// (V as the MN-major B operand of P.V: 64 contiguous head-dim elements per 128-byte row, 8 tokens per
+// 1024-byte group = stride byte offset, the next 64 head-dim elements one 16 KB block further = leading
+// byte offset: the image of a [tokens][head_dim] tile loaded as two 64-wide boxes; see desc_lo_mn.)
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -968,12 +946,10 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const uint32_t st = j % P1_NSTAGE;
                 if (!mbar_wait(bar(P1_FULL + st), (j / P1_NSTAGE) & 1)) return false;
                 tc_fence_after();
-                const uint32_t ak = sbase + P1_OFF_K + st * kOperandBytes;
+                const uint32_t ak = desc_lo_k(sbase + P1_OFF_K + st * kOperandBytes), aq = desc_lo_k(sbase + P1_OFF_Q);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    tc_mma(tmem_base + (j & 1) * 128u, smem_desc_k_sw128(sbase + P1_OFF_Q + off), smem_desc_k_sw128(ak + off), idesc_s, ks > 0);
-                }
+                for (int ks = 0; ks < 8; ++ks)
+                    tc_mma(tmem_base + (j & 1) * 128u, desc_make(aq + desc_kstep(ks, kHalfBytes)), desc_make(ak + desc_kstep(ks, kHalfBytes)), idesc_s, ks > 0);
                 tc_commit(bar(P1_SFULL + (j & 1)));
                 return true;
             };
@@ -985,11 +961,12 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const uint32_t w = i & 1;
                 if (!mbar_wait(bar(P1_PFULL + w), (i >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
                 tc_fence_after();
-                const uint32_t av = sbase + P1_OFF_V + (i % P1_NSTAGE) * kOperandBytes;
+                const uint32_t av = desc_lo_mn(sbase + P1_OFF_V + (i % P1_NSTAGE) * kOperandBytes);
+                const uint32_t first = i > 1;                                // the warpgroup's first tile initialises O_w
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)                               // 128 tokens = 8 steps of K = 16
-                    tc_mma_ts(tmem_base + 256u + w * 128u, tmem_base + w * 128u + ks * 8, smem_desc_mn_sw128(av + ks * 2048),
-                              idesc_pv, (i > 1) || (ks > 0));
+                for (int ks = 0; ks < 8; ++ks)                               // 128 tokens = 8 steps of K = 16 (2048 bytes of V each)
+                    tc_mma_ts(tmem_base + 256u + w * 128u, tmem_base + w * 128u + ks * 8, desc_make(av + ks * (2048 >> 4)),
+                              idesc_pv, ks > 0 ? 1u : first);
                 tc_commit(bar(P1_EMPTY + (i % P1_NSTAGE)));                  // S(i) and P.V(i) have read the stage
                 if (i + 2 < n_tiles && !issue_s(i + 2)) { failed = true; fail_site = __LINE__; break; }
             }
