@@ -313,10 +313,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     bool failed = false;
     int fail_site = 0;                             // source line of the wait that gave up (status word)
-    const bool reload_qo_every_item = p.n_chunks > 1;
     const uint32_t qo_bytes = (uint32_t)p.chunk_rows * 128u * 2u * 2u;   // Q and O chunks, two halves each
 
-    // Every role walks the same tiles (TileWalk) and, per tile, the chunks c = 0 .. n_chunks-1.
+    // Every role walks the same tiles (TileWalk); all window rows of a unit (at most 128) are one chunk.
     // Tiles go to the two epilogue groups alternately.  What an epilogue group waits for (accumulators
     // ready, norms and constants ready) is signalled on barriers of its own, so that each waiter sees
     // every phase of the barriers it uses; a parity wait must never fall two phases behind.
@@ -332,30 +331,29 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             int qo_unit = -1;
             for (; !tw.done() && !failed; tw.next()) {
                 const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv, t0 = tw.tile * TILE;
-                for (int c = 0; c < p.n_chunks; ++c, ++item) {
-                    const uint32_t st = item % NSTAGE, use = item / NSTAGE;
-                    if (!mbar_wait(bar(BAR_EMPTY + st), (use & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
-                    mbar_expect_tx(bar(BAR_FULL + st), 2 * kOperandBytes);
-                    const uint32_t dk = sbase + OFF_K + st * kOperandBytes, dv = sbase + OFF_V + st * kOperandBytes;
-                    tma_load_4d(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b);
-                    tma_load_4d(dk + kHalfBytes, &map_k, bar(BAR_FULL + st), 64, t0, g, b);
-                    tma_load_4d(dv, &map_v, bar(BAR_FULL + st), 0, t0, g, b);
-                    tma_load_4d(dv + kHalfBytes, &map_v, bar(BAR_FULL + st), 64, t0, g, b);
-                    // K, V and the sequence lengths were read by pass 1 of this call, so the first tile
-                    // may be fetched while the preceding kernel drains; -2 O is that kernel's output
-                    if (item == 0) pdl_wait();
-                    if (reload_qo_every_item || unit != qo_unit) {
-                        if (!mbar_wait(bar(BAR_QO_EMPTY), (qo_loads & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
-                        mbar_expect_tx(bar(BAR_QO_FULL), qo_bytes);
-                        const int qrow = (b * p.Hkv * p.G + g * p.G) * p.W + c * p.chunk_rows;
-                        const int orow = unit * p.rows_out + c * p.chunk_rows;
-                        tma_load_2d(sbase + OFF_Q, &map_q, bar(BAR_QO_FULL), 0, qrow);
-                        tma_load_2d(sbase + OFF_Q + kHalfBytes, &map_q, bar(BAR_QO_FULL), 64, qrow);
-                        tma_load_2d(sbase + OFF_O, &map_o, bar(BAR_QO_FULL), 0, orow);
-                        tma_load_2d(sbase + OFF_O + kHalfBytes, &map_o, bar(BAR_QO_FULL), 64, orow);
-                        qo_unit = unit; ++qo_loads;
-                    }
+                const uint32_t st = item % NSTAGE, use = item / NSTAGE;
+                if (!mbar_wait(bar(BAR_EMPTY + st), (use & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                mbar_expect_tx(bar(BAR_FULL + st), 2 * kOperandBytes);
+                const uint32_t dk = sbase + OFF_K + st * kOperandBytes, dv = sbase + OFF_V + st * kOperandBytes;
+                tma_load_4d(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b);
+                tma_load_4d(dk + kHalfBytes, &map_k, bar(BAR_FULL + st), 64, t0, g, b);
+                tma_load_4d(dv, &map_v, bar(BAR_FULL + st), 0, t0, g, b);
+                tma_load_4d(dv + kHalfBytes, &map_v, bar(BAR_FULL + st), 64, t0, g, b);
+                // K, V and the sequence lengths were read by pass 1 of this call, so the first tile
+                // may be fetched while the preceding kernel drains; -2 O is that kernel's output
+                if (item == 0) pdl_wait();
+                if (unit != qo_unit) {
+                    if (!mbar_wait(bar(BAR_QO_EMPTY), (qo_loads & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                    mbar_expect_tx(bar(BAR_QO_FULL), qo_bytes);
+                    const int qrow = (b * p.Hkv * p.G + g * p.G) * p.W;
+                    const int orow = unit * p.rows_out;
+                    tma_load_2d(sbase + OFF_Q, &map_q, bar(BAR_QO_FULL), 0, qrow);
+                    tma_load_2d(sbase + OFF_Q + kHalfBytes, &map_q, bar(BAR_QO_FULL), 64, qrow);
+                    tma_load_2d(sbase + OFF_O, &map_o, bar(BAR_QO_FULL), 0, orow);
+                    tma_load_2d(sbase + OFF_O + kHalfBytes, &map_o, bar(BAR_QO_FULL), 64, orow);
+                    qo_unit = unit; ++qo_loads;
                 }
+                ++item;
             }
             // drain: every copy this thread issued must have landed before the CTA may exit
             for (uint32_t back = 0; back < NSTAGE && back < item; ++back) {
@@ -373,31 +371,30 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             for (; !tw.done() && !failed; tw.next(), ++tile_seq) {
                 const int unit = tw.unit;
                 const uint32_t owner = tile_seq & 1;               // epilogue group of this tile
-                for (int c = 0; c < p.n_chunks; ++c, ++item) {
-                    const bool new_qo = reload_qo_every_item || unit != qo_unit;
-                    if (new_qo) {
-                        if (!mbar_wait(bar(BAR_QO_FULL), qo_loads & 1)) { failed = true; fail_site = __LINE__; break; }
-                        qo_unit = unit; ++qo_loads;
-                    }
-                    const uint32_t st = item % NSTAGE, buf = item & 1;
-                    if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
-                    if (!mbar_wait(bar(BAR_TM_EMPTY + buf), ((item >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
-                    tc_fence_after();
-                    const uint32_t zt = tmem_base + buf * 256u, tt = zt + 128u;
-                    const uint32_t ak = desc_lo_k(sbase + OFF_K + st * kOperandBytes), av = desc_lo_k(sbase + OFF_V + st * kOperandBytes);
-                    const uint32_t bq = desc_lo_k(sbase + OFF_Q), bo = desc_lo_k(sbase + OFF_O);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)                 // d = 128 = 8 steps of K = 16
-                        tc_mma(zt, desc_make(ak + desc_kstep(ks, kHalfBytes)), desc_make(bq + desc_kstep(ks, kHalfBytes)), idesc, ks > 0);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        tc_mma(tt, desc_make(av + desc_kstep(ks, kHalfBytes)), desc_make(bo + desc_kstep(ks, kHalfBytes)), idesc, ks > 0);
-                    tc_commit(bar(BAR_TM_FULL + owner * 2 + buf)); // accumulators ready for the tile's epilogue group
-                    tc_commit(bar(BAR_EMPTY + st));                // K/V stage no longer read by the MMA
-                    // Q / O may be overwritten once these MMAs are done, if the next item needs others
-                    const bool last_of_unit = tw.left > 1 && tw.tile + 1 == tw.tiles_in_unit && c + 1 == p.n_chunks;
-                    if (reload_qo_every_item || last_of_unit) tc_commit(bar(BAR_QO_EMPTY));
+                const bool new_qo = unit != qo_unit;
+                if (new_qo) {
+                    if (!mbar_wait(bar(BAR_QO_FULL), qo_loads & 1)) { failed = true; fail_site = __LINE__; break; }
+                    qo_unit = unit; ++qo_loads;
                 }
+                const uint32_t st = item % NSTAGE, buf = item & 1;
+                if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
+                if (!mbar_wait(bar(BAR_TM_EMPTY + buf), ((item >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
+                tc_fence_after();
+                const uint32_t zt = tmem_base + buf * 256u, tt = zt + 128u;
+                const uint32_t ak = desc_lo_k(sbase + OFF_K + st * kOperandBytes), av = desc_lo_k(sbase + OFF_V + st * kOperandBytes);
+                const uint32_t bq = desc_lo_k(sbase + OFF_Q), bo = desc_lo_k(sbase + OFF_O);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)                 // d = 128 = 8 steps of K = 16
+                    tc_mma(zt, desc_make(ak + desc_kstep(ks, kHalfBytes)), desc_make(bq + desc_kstep(ks, kHalfBytes)), idesc, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    tc_mma(tt, desc_make(av + desc_kstep(ks, kHalfBytes)), desc_make(bo + desc_kstep(ks, kHalfBytes)), idesc, ks > 0);
+                tc_commit(bar(BAR_TM_FULL + owner * 2 + buf)); // accumulators ready for the tile's epilogue group
+                tc_commit(bar(BAR_EMPTY + st));                // K/V stage no longer read by the MMA
+                // Q / O may be overwritten once these MMAs are done, if the next item needs others
+                const bool last_of_unit = tw.left > 1 && tw.tile + 1 == tw.tiles_in_unit;
+                if (last_of_unit) tc_commit(bar(BAR_QO_EMPTY));
+                ++item;
             }
         }
     } else if (warp < 4) {
@@ -407,42 +404,41 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (; !tw.done() && !failed; tw.next(), ++tile_seq) {
             const int unit = tw.unit;
             const uint32_t owner = tile_seq & 1;                   // epilogue group of this tile
-            for (int c = 0; c < p.n_chunks; ++c, ++item) {
-                const uint32_t st = item % NSTAGE, slot = item % NSLOT;
-                // constants first (global loads overlap the wait for the tile)
-                const size_t crow = (size_t)unit * p.rows_out + (size_t)c * p.chunk_rows;
-                float2 cst[2];
+            const uint32_t st = item % NSTAGE, slot = item % NSLOT;
+            // constants first (global loads overlap the wait for the tile)
+            const size_t crow = (size_t)unit * p.rows_out;
+            float2 cst[2];
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int r = t64 + 64 * j;
-                    cst[j] = r < p.chunk_rows ? make_float2(-p.lse2[crow + r], p.onorm[crow + r]) : make_float2(-INFINITY, 0.f);
-                }
-                if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
-                const uint8_t* vt = smem + OFF_V + st * kOperandBytes;
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int tok = t64 + 64 * j;
-                    float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int ch = 0; ch < 8; ++ch) {
-                            // any order of the row's 16-byte chunks gives the same sum; this one is bank-conflict free
-                            const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
-                            const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
-                            const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
-                            acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
-                            acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
-                        }
-                    const float2 s = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
-                    sNv[slot * TILE + tok] = s.x + s.y;
-                    // row pair i = tok / 2 holds (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
-                    float* cdst = sConst + slot * 256 + (tok >> 1) * 4 + (tok & 1);
-                    cdst[0] = cst[j].x; cdst[2] = cst[j].y;
-                }
-                __syncwarp();
-                if (lane == 0) { mbar_arrive(bar(BAR_NV + owner * NSLOT + slot)); mbar_arrive(bar(BAR_EMPTY + st)); }
+            for (int j = 0; j < 2; ++j) {
+                const int r = t64 + 64 * j;
+                cst[j] = r < p.chunk_rows ? make_float2(-p.lse2[crow + r], p.onorm[crow + r]) : make_float2(-INFINITY, 0.f);
             }
+            if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
+            const uint8_t* vt = smem + OFF_V + st * kOperandBytes;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int tok = t64 + 64 * j;
+                float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        // any order of the row's 16-byte chunks gives the same sum; this one is bank-conflict free
+                        const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
+                        const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
+                        const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
+                        acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
+                        acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
+                    }
+                const float2 s = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
+                sNv[slot * TILE + tok] = s.x + s.y;
+                // row pair i = tok / 2 holds (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
+                float* cdst = sConst + slot * 256 + (tok >> 1) * 4 + (tok & 1);
+                cdst[0] = cst[j].x; cdst[2] = cst[j].y;
+            }
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(bar(BAR_NV + owner * NSLOT + slot)); mbar_arrive(bar(BAR_EMPTY + st)); }
+            ++item;
         }
     } else {
         // ======================================= epilogue =======================================
@@ -456,7 +452,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (; !tw.done() && !failed; tw.next()) {
             const bool mine = (tile_seq & 1) == (uint32_t)wg;
             ++tile_seq;
-            if (!mine) { item += p.n_chunks; continue; }
+            if (!mine) { ++item; continue; }
             const int unit = tw.unit, b = unit / p.Hkv;
             const int N = tc_seq_len(p, b), t0 = tw.tile * TILE;
             float* out = p.scores + (size_t)unit * p.Nmax;
@@ -466,23 +462,22 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
             float nv = 0.f;
-            for (int c = 0; c < p.n_chunks && !failed; ++c, ++item) {
-                const uint32_t buf = item & 1, slot = item % NSLOT;
-                if (!mbar_wait(bar(BAR_NV + wg * NSLOT + slot), (nv_par >> slot) & 1)) { failed = true; fail_site = __LINE__; break; }
-                if (!mbar_wait(bar(BAR_TM_FULL + wg * 2 + buf), (full_par >> buf) & 1)) { failed = true; fail_site = __LINE__; break; }
-                nv_par ^= 1u << slot; full_par ^= 1u << buf;
-                tc_fence_after();
-                nv = sNv[slot * TILE + tok];
-                const float4* cst = reinterpret_cast<const float4*>(sConst + slot * 256);
-                const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u, tt = zt + 128u;
-                if (masked_tile)
-                    score_chunk<VARS, true>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, N - p.W, p.W, (c * p.chunk_rows) % p.W);
-                else
-                    score_chunk<VARS, false>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, 0, 0, 0);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_TM_EMPTY + buf));
-            }
+            const uint32_t buf = item & 1, slot = item % NSLOT;
+            if (!mbar_wait(bar(BAR_NV + wg * NSLOT + slot), (nv_par >> slot) & 1)) { failed = true; fail_site = __LINE__; break; }
+            if (!mbar_wait(bar(BAR_TM_FULL + wg * 2 + buf), (full_par >> buf) & 1)) { failed = true; fail_site = __LINE__; break; }
+            nv_par ^= 1u << slot; full_par ^= 1u << buf;
+            tc_fence_after();
+            nv = sNv[slot * TILE + tok];
+            const float4* cst = reinterpret_cast<const float4*>(sConst + slot * 256);
+            const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u, tt = zt + 128u;
+            if (masked_tile)
+                score_chunk<VARS, true>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, N - p.W, p.W, 0);
+            else
+                score_chunk<VARS, false>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, 0, 0, 0);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_TM_EMPTY + buf));
+            ++item;
             if (!failed && ptok < p.Nmax) {
                 const bool live = ptok < N;
                 const float s2 = p.scale * p.scale;
