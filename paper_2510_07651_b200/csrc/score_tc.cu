@@ -222,7 +222,8 @@ __device__ __forceinline__ void tc_wait_ld16x2(uint32_t (&a)[16], uint32_t (&b)[
 // S6 = sum a^2, S7 = sum a and t' = -2 v.o_r (the expanded norms of Algorithm 1).
 struct RowSums { float2 s1, s2, s3, s4, s5, s6, s7; };
 
-// 16 rows of one token: zr = logits, tr = -2 v.o_r, cst = per row pair (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
+// 16 rows of one token: zr = logits, tr = -2 v.o_r, cst = per row pair (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2);
+// when only the joint score is computed (VARS == OBC_VAR_VK) the |o|^2 entries arrive multiplied by scale
 template <unsigned VARS, bool MASKED>
 __device__ __forceinline__ void score_rows16(const uint32_t (&zr)[16], const uint32_t (&tr)[16], const float4* cst,
                                              float2 sl2, float2 sc, RowSums& S, int ptok, int mask_base, int W, int& wi) {
@@ -240,12 +241,18 @@ __device__ __forceinline__ void score_rows16(const uint32_t (&zr)[16], const uin
         }
         const float2 a = make_float2(fast_exp2(e.x), fast_exp2(e.y));
         const float2 u = __fmul2_rn(a, z);
-        if (VARS & OBC_VAR_VK) {
+        if (VARS == OBC_VAR_VK) {
+            // joint score alone: the constants hold scale |o_r|^2, and s2 collects u (b t' + u scale |o_r|^2),
+            // i.e. S2 + scale S3 of the general form below, with one packed instruction less
+            const float2 b = __ffma2_rn(u, sc, a);
+            S.s1 = __ffma2_rn(b, b, S.s1);
+            S.s2 = __ffma2_rn(u, __ffma2_rn(u, make_float2(cp.z, cp.w), __fmul2_rn(b, t2)), S.s2);
+        } else if (VARS & OBC_VAR_VK) {
             const float2 b = __ffma2_rn(u, sc, a);
             S.s1 = __ffma2_rn(b, b, S.s1);
             S.s2 = __ffma2_rn(__fmul2_rn(u, b), t2, S.s2);
         }
-        if (VARS & (OBC_VAR_VK | OBC_VAR_K)) {
+        if ((VARS & (OBC_VAR_VK | OBC_VAR_K)) && VARS != OBC_VAR_VK) {
             const float2 uu = __fmul2_rn(u, u);
             S.s3 = __ffma2_rn(uu, make_float2(cp.z, cp.w), S.s3);
             if (VARS & OBC_VAR_K) { S.s4 = __ffma2_rn(uu, t2, S.s4); S.s5 = __fadd2_rn(uu, S.s5); }
@@ -411,7 +418,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int r = t64 + 64 * j;
-                cst[j] = r < p.chunk_rows ? make_float2(-p.lse2[crow + r], p.onorm[crow + r]) : make_float2(-INFINITY, 0.f);
+                cst[j] = r < p.chunk_rows ? make_float2(-p.lse2[crow + r], p.onorm[crow + r] * (VARS == OBC_VAR_VK ? p.scale : 1.f))
+                                          : make_float2(-INFINITY, 0.f);
             }
             if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
             const uint8_t* vt = smem + OFF_V + st * kOperandBytes;
@@ -687,7 +695,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             for (int c = 0; c < nc; ++c, ++citem) {
                 const uint32_t cs = citem & 3;
                 const size_t crow = (size_t)unit * p.rows_out + (size_t)c * MC_ROWS + t64;
-                const float2 cst = make_float2(-p.lse2[crow], p.onorm[crow]);
+                const float2 cst = make_float2(-p.lse2[crow], p.onorm[crow] * (VARS == OBC_VAR_VK ? p.scale : 1.f));
                 // slot cs was last read by the chunk four back; the chunk two back has been summed once
                 // the TMEM buffers this chunk is going to use are free again
                 const uint32_t i0 = 2 * citem, i1 = i0 + 1;
