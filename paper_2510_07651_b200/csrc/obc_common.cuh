@@ -53,6 +53,8 @@ struct SimtPlan {
     size_t off_part_m, off_part_l, off_part_o;   // partial softmax stats / outputs per split
     size_t off_lse2, off_onorm, off_o;           // combined: log2-sum-exp, ||o||^2, O (fp32)
     size_t off_obf;                              // bf16 [units][rows_out][d] = -2 * O
+    size_t off_cpair;                            // float4 per row pair: (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
+    size_t off_nv;                               // fp32 [units][Nmax]: ||v_p||^2 (written by tensor-core pass 1)
     size_t bytes;
 };
 SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf);

@@ -190,10 +190,14 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const size_t orow = (size_t)unit * plan.rows_out + r;
     __nv_bfloat16* obf = plan.want_obf ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + plan.off_obf) : nullptr;
+    float* cpair = plan.want_obf ? ws + plan.off_cpair / 4 + (orow >> 1) * 4 + (orow & 1) : nullptr;
     if (r >= s.R) {
         (ws + plan.off_o / 4)[orow * kD + tid] = 0.f;
         if (obf) obf[orow * kD + tid] = __float2bfloat16(0.f);
-        if (tid == 0) { (ws + plan.off_lse2 / 4)[orow] = INFINITY; (ws + plan.off_onorm / 4)[orow] = 0.f; }
+        if (tid == 0) {
+            (ws + plan.off_lse2 / 4)[orow] = INFINITY; (ws + plan.off_onorm / 4)[orow] = 0.f;
+            if (cpair) { cpair[0] = -INFINITY; cpair[2] = 0.f; }
+        }
         return;
     }
     __shared__ float red[4];
@@ -247,8 +251,10 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     (ws + plan.off_o / 4)[orow * kD + tid] = oc;
     if (obf) obf[orow * kD + tid] = __float2bfloat16(-2.f * oc);
     if (tid == 0) {
-        (ws + plan.off_lse2 / 4)[orow] = Mrun + log2f(L);
+        const float lse2 = Mrun + log2f(L);
+        (ws + plan.off_lse2 / 4)[orow] = lse2;
         (ws + plan.off_onorm / 4)[orow] = onorm;
+        if (cpair) { cpair[0] = -lse2; cpair[2] = onorm; }
     }
 }
 
@@ -417,6 +423,7 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
     p.off_onorm = off;  off = align_up(off + orow * 4, 256);
     p.off_o = off;      off = align_up(off + orow * kD * 4, 256);
     p.off_obf = off;    off = align_up(off + (want_obf ? orow * kD * 2 : 0), 1024);
+    p.off_cpair = off; p.off_nv = off;             // tensor-core plan only
     p.bytes = off;
     return p;
 }

@@ -10,9 +10,9 @@
 // W x N matrix ever leaves the SM.
 //
 // Warp roles of the 384-thread CTA (persistent, one CTA per SM):
-//   warp 0      TMA producer: K/V tiles into a 2-stage ring, Q / -2O chunks when they change
+//   warp 0      TMA producer: K/V tiles into a 2-stage ring, Q / -2O when the unit changes
 //   warp 1      MMA issuer (one elected lane), double-buffered TMEM accumulators (2 x 256 columns)
-//   warps 2-3   ||v_p||^2 of the tile from shared memory, per-row constants into shared memory
+//   warps 2-3   idle here (||v_p||^2 is computed by pass 1, whose two spare warps have the V tile at hand)
 //   warps 4-7   epilogue group 0 (even tiles), warps 8-11 epilogue group 1 (odd tiles)
 //
 // Every mbarrier wait is bounded: on a timeout the kernel raises the status word in the workspace
@@ -27,7 +27,6 @@ namespace {
 
 constexpr int TILE = 128;                       // tokens per tile = MMA M
 constexpr int NSTAGE = 2;
-constexpr int NSLOT = 4;                        // ring depth of the per-tile constants / norms
 constexpr uint32_t kHalfBytes = 128 * 128;      // [128 rows][64 bf16] = 16 KB, one swizzle-128B block
 constexpr uint32_t kOperandBytes = 2 * kHalfBytes;
 constexpr int kThreads = 384;
@@ -38,17 +37,15 @@ constexpr uint32_t OFF_Q = 0;
 constexpr uint32_t OFF_O = OFF_Q + kOperandBytes;
 constexpr uint32_t OFF_K = OFF_O + kOperandBytes;                 // NSTAGE x 32 KB
 constexpr uint32_t OFF_V = OFF_K + NSTAGE * kOperandBytes;        // NSTAGE x 32 KB
-constexpr uint32_t OFF_NV = OFF_V + NSTAGE * kOperandBytes;       // NSLOT x 128 floats
-constexpr uint32_t OFF_CONST = OFF_NV + NSLOT * TILE * 4;         // NSLOT x 128 float2 (lse2, ||o||^2)
-constexpr uint32_t OFF_BAR = OFF_CONST + NSLOT * 128 * 8;
-constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + 2 + 2 * NSLOT;
+constexpr uint32_t OFF_CONST = OFF_V + NSTAGE * kOperandBytes;    // 8 epilogue warps x 64 float4 (row-pair constants)
+constexpr uint32_t OFF_BAR = OFF_CONST + 8 * 64 * 16;
+constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + 2;
 constexpr uint32_t OFF_TMEM = OFF_BAR + kNumBars * 8;
 constexpr uint32_t kSmemBytes = OFF_TMEM + 16 + 1024;             // + alignment slack
 
 enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_QO_FULL = 2 * NSTAGE, BAR_QO_EMPTY = 2 * NSTAGE + 1,
        BAR_TM_FULL = 2 * NSTAGE + 2,      // [epilogue group][TMEM buffer]
-       BAR_TM_EMPTY = 2 * NSTAGE + 6,     // [TMEM buffer]
-       BAR_NV = 2 * NSTAGE + 8 };         // [epilogue group][slot]
+       BAR_TM_EMPTY = 2 * NSTAGE + 6 };   // [TMEM buffer]
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -151,6 +148,8 @@ struct TcParams {
     unsigned variants;
     int n_chunks, chunk_rows, rows_out;       // rows_out = n_chunks * chunk_rows
     const float* lse2;                        // [units][rows_out]
+    const float4* cpair;                      // [units][rows_out / 2]: (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2) per row pair
+    const float* nv;                          // [units][Nmax]: ||v_p||^2 from pass 1
     const float* onorm;                       // [units][rows_out]
     float* scores;                            // [planes][units][Nmax]
     unsigned int* status;                     // device status word (workspace header)
@@ -294,19 +293,17 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const uint32_t bars = sbase + OFF_BAR;
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_TMEM);
-    float* sNv = reinterpret_cast<float*>(smem + OFF_NV);
-    float* sConst = reinterpret_cast<float*>(smem + OFF_CONST);
+    float4* sConst = reinterpret_cast<float4*>(smem + OFF_CONST);   // [8 epilogue warps][64 row pairs]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int units = p.B * p.Hkv;
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_k); prefetch_tmap(&map_v); prefetch_tmap(&map_q); prefetch_tmap(&map_o);
-        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 3); }
+        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
         mbar_init(bar(BAR_QO_FULL), 1); mbar_init(bar(BAR_QO_EMPTY), 1);
         for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_TM_FULL + i), 1);
         for (int i = 0; i < 2; ++i) mbar_init(bar(BAR_TM_EMPTY + i), 4);
-        for (int i = 0; i < 2 * NSLOT; ++i) mbar_init(bar(BAR_NV + i), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -324,8 +321,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     // Every role walks the same tiles (TileWalk); all window rows of a unit (at most 128) are one chunk.
     // Tiles go to the two epilogue groups alternately.  What an epilogue group waits for (accumulators
-    // ready, norms and constants ready) is signalled on barriers of its own, so that each waiter sees
-    // every phase of the barriers it uses; a parity wait must never fall two phases behind.
+    // ready) is signalled on barriers of its own, so that each waiter sees every phase of the barriers
+    // it uses; a parity wait must never fall two phases behind.  ||v_p||^2 comes from pass 1 and the
+    // per-row constants from the combine kernel, so no warp here reads the K/V tiles.
     // `item` counts the (tile, chunk) pairs processed so far and indexes the smem stage, TMEM
     // buffer and constant-slot rings.
     TileWalk tw;
@@ -404,51 +402,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 ++item;
             }
         }
-    } else if (warp < 4) {
-        // ============================ ||v_p||^2 and per-row constants ===========================
-        const int t64 = threadIdx.x - 64;                          // 0..63
-        uint32_t item = 0, tile_seq = 0;
-        for (; !tw.done() && !failed; tw.next(), ++tile_seq) {
-            const int unit = tw.unit;
-            const uint32_t owner = tile_seq & 1;                   // epilogue group of this tile
-            const uint32_t st = item % NSTAGE, slot = item % NSLOT;
-            // constants first (global loads overlap the wait for the tile)
-            const size_t crow = (size_t)unit * p.rows_out;
-            float2 cst[2];
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int r = t64 + 64 * j;
-                cst[j] = r < p.chunk_rows ? make_float2(-p.lse2[crow + r], p.onorm[crow + r] * (VARS == OBC_VAR_VK ? p.scale : 1.f))
-                                          : make_float2(-INFINITY, 0.f);
-            }
-            if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
-            const uint8_t* vt = smem + OFF_V + st * kOperandBytes;
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int tok = t64 + 64 * j;
-                float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        // any order of the row's 16-byte chunks gives the same sum; this one is bank-conflict free
-                        const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
-                        const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
-                        const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
-                        acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
-                        acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
-                    }
-                const float2 s = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
-                sNv[slot * TILE + tok] = s.x + s.y;
-                // row pair i = tok / 2 holds (-lse2_0, -lse2_1, |o_0|^2, |o_1|^2)
-                float* cdst = sConst + slot * 256 + (tok >> 1) * 4 + (tok & 1);
-                cdst[0] = cst[j].x; cdst[2] = cst[j].y;
-            }
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(bar(BAR_NV + owner * NSLOT + slot)); mbar_arrive(bar(BAR_EMPTY + st)); }
-            ++item;
-        }
-    } else {
+    } else if (warp >= 4) {
         // ======================================= epilogue =======================================
         const int wg = (warp - 4) >> 2;                            // 0: even tiles, 1: odd tiles
         const int lane_grp = warp & 3;                             // TMEM lanes 32*lane_grp .. +31
@@ -456,7 +410,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float2 sl2 = make_float2(p.scale * kLog2e, p.scale * kLog2e), sc = make_float2(p.scale, p.scale);
         const size_t plane = (size_t)units * p.Nmax;
         uint32_t item = 0, tile_seq = 0;
-        uint32_t full_par = 0, nv_par = 0;                         // phase parity of this group's barriers, one bit each
+        uint32_t full_par = 0;                                     // phase parity of this group's barriers, one bit each
+        float4* my_const = sConst + (warp - 4) * 64;               // this warp's copy of the unit's row constants
+        int const_unit = -1;
         for (; !tw.done() && !failed; tw.next()) {
             const bool mine = (tile_seq & 1) == (uint32_t)wg;
             ++tile_seq;
@@ -469,14 +425,22 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
-            float nv = 0.f;
-            const uint32_t buf = item & 1, slot = item % NSLOT;
-            if (!mbar_wait(bar(BAR_NV + wg * NSLOT + slot), (nv_par >> slot) & 1)) { failed = true; fail_site = __LINE__; break; }
+            const uint32_t buf = item & 1;
+            const float nv = ptok < N ? p.nv[(size_t)unit * p.Nmax + ptok] : 0.f;      // used after the row loop
+            if (unit != const_unit) {                              // at most once per unit: (-lse2, |o|^2) of every row pair
+                __syncwarp();
+                for (int i = lane; i < 64; i += 32) {
+                    float4 c4 = i * 2 < p.chunk_rows ? p.cpair[(((size_t)unit * p.rows_out) >> 1) + i] : make_float4(-INFINITY, -INFINITY, 0.f, 0.f);
+                    if (VARS == OBC_VAR_VK) { c4.z *= p.scale; c4.w *= p.scale; }
+                    my_const[i] = c4;
+                }
+                __syncwarp();
+                const_unit = unit;
+            }
             if (!mbar_wait(bar(BAR_TM_FULL + wg * 2 + buf), (full_par >> buf) & 1)) { failed = true; fail_site = __LINE__; break; }
-            nv_par ^= 1u << slot; full_par ^= 1u << buf;
+            full_par ^= 1u << buf;
             tc_fence_after();
-            nv = sNv[slot * TILE + tok];
-            const float4* cst = reinterpret_cast<const float4*>(sConst + slot * 256);
+            const float4* cst = my_const;
             const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u, tt = zt + 128u;
             if (masked_tile)
                 score_chunk<VARS, true>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, N - p.W, p.W, 0);
@@ -816,6 +780,7 @@ struct P1Params {
     int n_chunks, chunk_rows;
     int n_splits, tiles_per_split;                         // CTAs per (unit, chunk); each writes one partial
     float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
+    float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the chunk-0 CTAs
     unsigned int* status;
 };
 
@@ -891,7 +856,8 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
-        for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), 1); }
+        // a K/V stage is released by the MMA commit and, in chunk-0 CTAs, by the two ||v||^2 warps
+        for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), c == 0 ? 3 : 1); }
         mbar_init(bar(P1_QFULL), 1); mbar_init(bar(P1_ODONE), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(bar(P1_SFULL + i), 1); mbar_init(bar(P1_PFULL + i), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -975,7 +941,40 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             }
             if (!failed) tc_commit(bar(P1_ODONE));
         }
-    } else if (warp >= 4) {
+    } else if (warp < 4) {
+        // ====================== ||v_p||^2 of every cached token (chunk-0 CTAs) ===================
+        // Pass 2 needs it per token; the V tile is in shared memory here anyway, and these two warps
+        // have nothing else to do, whereas in pass 2 every issue slot next to the epilogue counts.
+        if (c == 0) {
+            const int t64 = threadIdx.x - 64;                                // 0..63
+            for (int i = 0; i < n_tiles && !failed; ++i) {
+                const uint32_t st = i % P1_NSTAGE;
+                if (!mbar_wait(bar(P1_FULL + st), (i / P1_NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
+                const uint8_t* vt = smem + P1_OFF_V + st * kOperandBytes;
+                const int t0 = (tile_lo + i) * TILE;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int tok = t64 + 64 * j;
+                    float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch) {
+                            // any order of the row's 16-byte chunks gives the same sum; this one is bank-conflict free
+                            const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
+                            const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
+                            const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
+                            acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
+                            acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
+                        }
+                    const float2 sum = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
+                    if (t0 + tok < p.Nmax) p.nv[(size_t)unit * p.Nmax + t0 + tok] = sum.x + sum.y;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(P1_EMPTY + st));
+            }
+        }
+    } else {
         // ======================================= softmax ========================================
         const int w = (warp - 4) >> 2;                                       // warpgroup: tiles w, w+2, ...
         const int lane_grp = warp & 3;
@@ -1243,6 +1242,8 @@ static SimtPlan make_tc_plan(const ScoreShape& s) {
     p.off_onorm = off;  off = align_up(off + orow * 4, 256);
     p.off_o = off;      off = align_up(off + orow * kD * 4, 256);
     p.off_obf = off;    off = align_up(off + orow * kD * 2, 1024);
+    p.off_cpair = off;  off = align_up(off + orow * 8, 256);
+    p.off_nv = off;     off = align_up(off + (size_t)units * s.Nmax * 4, 256);
     p.bytes = off;
     return p;
 }
@@ -1281,6 +1282,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.n_splits = plan.n_splits; p1.tiles_per_split = plan.tiles_per_split;
         p1.part_m = (float*)(wsb + plan.off_part_m); p1.part_l = (float*)(wsb + plan.off_part_l);
         p1.part_o = (float*)(wsb + plan.off_part_o);
+        p1.nv = (float*)(wsb + plan.off_nv);
         p1.status = (unsigned int*)(wsb + plan.off_flag);
         OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
         { ProfScope ps("tc_pass1", stream);
@@ -1296,6 +1298,8 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     p.onorm = (const float*)(wsb + plan.off_onorm);
     p.scores = scores;
     p.status = (unsigned int*)(wsb + plan.off_flag);
+    p.cpair = (const float4*)(wsb + plan.off_cpair);
+    p.nv = (const float*)(wsb + plan.off_nv);
     const long long n_tiles = (long long)units * ((s.Nmax + TILE - 1) / TILE);
     const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
 
