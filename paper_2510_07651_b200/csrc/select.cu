@@ -390,26 +390,43 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     }
 }
 
-// one 16-byte vector per thread; `vecs` vectors per row
+// four 16-byte vectors of K and of V per thread, all loads issued before the first store (`vecs`
+// vectors per row; a thread's vectors are a quarter of the unit's vectors apart)
 __global__ void __launch_bounds__(256)
 gather_kernel(int units, int Hkv, int idx_stride, int vecs, int elem_bytes,
               TensorView k, TensorView v, TensorView ko, TensorView vo,
               const int32_t* __restrict__ idx, const float* __restrict__ s_in, float* __restrict__ s_out, int Nmax) {
     pdl_wait();
     const int unit = blockIdx.y, b = unit / Hkv, g = unit % Hkv;
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
-    const int j = e / vecs, c = e % vecs;
-    if (j >= idx_stride) return;
-    const int src = idx[(size_t)unit * idx_stride + j];
-    if (src < 0) return;
+    const int total = idx_stride * vecs, quarter = (total + 3) / 4;
+    const int e0 = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e0 >= quarter) return;
     const size_t eb = (size_t)elem_bytes;
-    const char* kp = (const char*)k.ptr + ((size_t)b * k.sb + (size_t)g * k.sh + (size_t)src * k.st) * eb;
-    const char* vp = (const char*)v.ptr + ((size_t)b * v.sb + (size_t)g * v.sh + (size_t)src * v.st) * eb;
-    char* kop = (char*)ko.ptr + ((size_t)b * ko.sb + (size_t)g * ko.sh + (size_t)j * ko.st) * eb;
-    char* vop = (char*)vo.ptr + ((size_t)b * vo.sb + (size_t)g * vo.sh + (size_t)j * vo.st) * eb;
-    reinterpret_cast<uint4*>(kop)[c] = __ldg(reinterpret_cast<const uint4*>(kp) + c);
-    reinterpret_cast<uint4*>(vop)[c] = __ldg(reinterpret_cast<const uint4*>(vp) + c);
-    if (s_in && c == 0) s_out[(size_t)unit * idx_stride + j] = s_in[(size_t)unit * Nmax + src];
+    const char* kb = (const char*)k.ptr + ((size_t)b * k.sb + (size_t)g * k.sh) * eb;
+    const char* vb = (const char*)v.ptr + ((size_t)b * v.sb + (size_t)g * v.sh) * eb;
+    char* kob = (char*)ko.ptr + ((size_t)b * ko.sb + (size_t)g * ko.sh) * eb;
+    char* vob = (char*)vo.ptr + ((size_t)b * vo.sb + (size_t)g * vo.sh) * eb;
+    int src[4], j[4], c[4];
+    uint4 kv[4], vv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * quarter;
+        j[u] = e / vecs; c[u] = e % vecs;
+        src[u] = e < total ? idx[(size_t)unit * idx_stride + j[u]] : -1;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        if (src[u] >= 0) {
+            kv[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)src[u] * k.st * eb) + c[u]);
+            vv[u] = __ldg(reinterpret_cast<const uint4*>(vb + (size_t)src[u] * v.st * eb) + c[u]);
+        }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        if (src[u] >= 0) {
+            reinterpret_cast<uint4*>(kob + (size_t)j[u] * ko.st * eb)[c[u]] = kv[u];
+            reinterpret_cast<uint4*>(vob + (size_t)j[u] * vo.st * eb)[c[u]] = vv[u];
+            if (s_in && c[u] == 0) s_out[(size_t)unit * idx_stride + j[u]] = s_in[(size_t)unit * Nmax + src[u]];
+        }
 }
 
 }  // namespace
@@ -494,7 +511,7 @@ obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_byte
                          TensorView k, TensorView v, TensorView ko, TensorView vo, const int32_t* idx,
                          const float* s_in, float* s_out, cudaStream_t stream) {
     const int vecs = kD * elem_bytes / 16;
-    const long long total = (long long)idx_stride * vecs;
+    const long long total = ((long long)idx_stride * vecs + 3) / 4;    // four vectors per thread
     {
         ProfScope ps("gather", stream);
         OBC_CUDA_TRY(launch_pdl(gather_kernel, dim3((unsigned)((total + 255) / 256), B * Hkv), dim3(256), 0, stream, 1,

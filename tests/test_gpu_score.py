@@ -57,6 +57,27 @@ def test_small_and_degenerate_shapes(N, W, Hq, Hkv, dtype, causal):
     _check(case, ["V", "K", "VK", "ATTN"], causal=causal, tight=2e-2 if dtype == "bf16" else None)
 
 
+@pytest.mark.parametrize("lens,W,Hq,Hkv", [
+    ([1100, 333], 64, 14, 2),      # R = 448 (row chunks of 64), odd tile counts: the second tile of the last pair is past the end
+    ([2900], 40, 5, 1),            # R = 200: padded to 256 rows, 23 tiles
+    ([129, 4000, 640], 48, 12, 3), # R = 192, ragged, a unit with two tiles of which the second holds one token
+])
+def test_more_than_128_window_rows(lens, W, Hq, Hkv):
+    case = synth.make_prefill("rows", B=len(lens), Hq=Hq, Hkv=Hkv, d=128, W=W, N=lens, dtype="bf16", seed=101 + W,
+                              hh_frac=0.02)
+    _check(case, ["V", "K", "VK", "ATTN"], tight=2e-2)
+    _check(case, ["K", "VK"], tight=2e-2)
+    _check(case, ["VK"], tight=2e-2)
+
+
+@pytest.mark.parametrize("N,W,Hq,Hkv", [(5000, 64, 1, 1), (3001, 16, 8, 2), (257, 128, 1, 1), (4224, 24, 4, 1)])
+def test_tensor_core_row_counts(N, W, Hq, Hkv):
+    # R = 64, 64, 128, 96 (chunks of 64 / 64 / 128 / 96 rows), token counts with and without a ragged last tile
+    case = synth.make_prefill("tc", B=1, Hq=Hq, Hkv=Hkv, d=128, W=W, N=N, dtype="bf16", seed=7 + N, hh_frac=0.02)
+    _check(case, ["VK"], path="tc", tight=2e-2)
+    _check(case, ["V", "K", "VK", "ATTN"], path="tc", tight=2e-2)
+
+
 def test_peaky_attention_cancellation_case():
     # some attention weights approach 1, so ||v_p - o_i||^2 cancels heavily
     case = synth.make_prefill("peaky", B=1, Hq=8, Hkv=2, d=128, W=16, N=2048, dtype="bf16", seed=5,
