@@ -51,6 +51,14 @@ __device__ __forceinline__ void unpack8(uint4 u, float (&f)[8]) {
     f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
 }
 
+// four packed pairs (lo, hi) of the eight bf16 of a 16-byte chunk
+__device__ __forceinline__ void unpack8x2(uint4 u, float2 (&f)[4]) {
+    f[0] = make_float2(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+    f[1] = make_float2(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+    f[2] = make_float2(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+    f[3] = make_float2(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
+}
+
 __device__ __forceinline__ const __nv_bfloat16* bf_row(const TensorView& t, int b, int h, long long tok) {
     return reinterpret_cast<const __nv_bfloat16*>(t.ptr) + b * t.sb + h * t.sh + tok * t.st;
 }
@@ -128,20 +136,23 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
 #pragma unroll
     for (int r = 0; r < G; ++r) z2[r] = 0.f;
     if (live) {
+        float2 zz[G];                                      // two partial dot products per row (packed fp32x2)
+#pragma unroll
+        for (int r = 0; r < G; ++r) zz[r] = make_float2(0.f, 0.f);
 #pragma unroll 4
         for (int c = 0; c < 16; ++c) {
-            float kf[8];
-            unpack8(staged_chunk(sRows, tid, c), kf);
+            float2 kf[4];
+            unpack8x2(staged_chunk(sRows, tid, c), kf);
 #pragma unroll
             for (int r = 0; r < G; ++r) {
                 const float4 qa = *reinterpret_cast<const float4*>(&sQ[r][c * 8]);
                 const float4 qb = *reinterpret_cast<const float4*>(&sQ[r][c * 8 + 4]);
-                z2[r] = fmaf(qa.x, kf[0], z2[r]); z2[r] = fmaf(qa.y, kf[1], z2[r]);
-                z2[r] = fmaf(qa.z, kf[2], z2[r]); z2[r] = fmaf(qa.w, kf[3], z2[r]);
-                z2[r] = fmaf(qb.x, kf[4], z2[r]); z2[r] = fmaf(qb.y, kf[5], z2[r]);
-                z2[r] = fmaf(qb.z, kf[6], z2[r]); z2[r] = fmaf(qb.w, kf[7], z2[r]);
+                zz[r] = __ffma2_rn(make_float2(qa.x, qa.y), kf[0], zz[r]); zz[r] = __ffma2_rn(make_float2(qa.z, qa.w), kf[1], zz[r]);
+                zz[r] = __ffma2_rn(make_float2(qb.x, qb.y), kf[2], zz[r]); zz[r] = __ffma2_rn(make_float2(qb.z, qb.w), kf[3], zz[r]);
             }
         }
+#pragma unroll
+        for (int r = 0; r < G; ++r) z2[r] = zz[r].x + zz[r].y;
     }
     float* zbuf = (float*)(ws + plan.off_z) + (size_t)unit * G * s.cap;
 #pragma unroll
@@ -303,25 +314,27 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
     const bool live = my_pos >= 0;
     MinCand cand{INFINITY, -1, -1, 0};
     if (live) {
-        float nv = 0.f, t[G];
+        float nv, t[G];
+        float2 nn = make_float2(0.f, 0.f), tt[G];          // packed fp32x2 partial sums
 #pragma unroll
-        for (int r = 0; r < G; ++r) t[r] = 0.f;
+        for (int r = 0; r < G; ++r) tt[r] = make_float2(0.f, 0.f);
 #pragma unroll 4
         for (int c = 0; c < 16; ++c) {
-            float vf[8];
-            unpack8(staged_chunk(sRows, tid, c), vf);
+            float2 vf[4];
+            unpack8x2(staged_chunk(sRows, tid, c), vf);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) nv = fmaf(vf[j], vf[j], nv);
+            for (int j = 0; j < 4; ++j) nn = __ffma2_rn(vf[j], vf[j], nn);
 #pragma unroll
             for (int r = 0; r < G; ++r) {
                 const float4 oa = *reinterpret_cast<const float4*>(&sO[r][c * 8]);
                 const float4 ob = *reinterpret_cast<const float4*>(&sO[r][c * 8 + 4]);
-                t[r] = fmaf(oa.x, vf[0], t[r]); t[r] = fmaf(oa.y, vf[1], t[r]);
-                t[r] = fmaf(oa.z, vf[2], t[r]); t[r] = fmaf(oa.w, vf[3], t[r]);
-                t[r] = fmaf(ob.x, vf[4], t[r]); t[r] = fmaf(ob.y, vf[5], t[r]);
-                t[r] = fmaf(ob.z, vf[6], t[r]); t[r] = fmaf(ob.w, vf[7], t[r]);
+                tt[r] = __ffma2_rn(make_float2(oa.x, oa.y), vf[0], tt[r]); tt[r] = __ffma2_rn(make_float2(oa.z, oa.w), vf[1], tt[r]);
+                tt[r] = __ffma2_rn(make_float2(ob.x, ob.y), vf[2], tt[r]); tt[r] = __ffma2_rn(make_float2(ob.z, ob.w), vf[3], tt[r]);
             }
         }
+        nv = nn.x + nn.y;
+#pragma unroll
+        for (int r = 0; r < G; ++r) t[r] = tt[r].x + tt[r].y;
         const float* zbuf = (const float*)(ws + plan.off_z) + (size_t)unit * G * s.cap;
         float sc = 0.f;
 #pragma unroll
