@@ -44,13 +44,6 @@ DecodePlan make_plan(const DecodeShape& s) {
 
 struct MinCand { float val; int pos; int slot; int pad; };
 
-__device__ __forceinline__ void unpack8(uint4 u, float (&f)[8]) {
-    f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
-    f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
-    f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
-    f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
-}
-
 // four packed pairs (lo, hi) of the eight bf16 of a 16-byte chunk
 __device__ __forceinline__ void unpack8x2(uint4 u, float2 (&f)[4]) {
     f[0] = make_float2(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));

@@ -116,7 +116,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptors: K-major operand with 128-byte swizzle = rows of 64 bf16 (128 B),
 // 8-row groups 1024 B apart (the image a swizzle-128B TMA box of 64 elements x rows leaves).
