@@ -114,6 +114,19 @@ obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_
  */
 obc_status obc_score_status(const void* workspace, void* stream);
 
+/*
+ * Device-side extent of the two tensor-core kernels of obc_score, for measurement.  Every CTA of
+ * the window-statistics kernel and of the fused score kernel folds its first and its last reading
+ * of the GPU's nanosecond timer into four words of the workspace header; this call synchronises
+ * `stream`, returns latest end - earliest start of each kernel in microseconds (host pointers;
+ * 0 when nothing was recorded, e.g. on the CUDA-core path) and zeroes the words.  The figures
+ * cover the launches since the words were last zero, so zero the workspace header (or call this
+ * once) before the obc_score call to be measured, and measure one call at a time.  Unlike an event
+ * pair around the launch, the span leaves out launch latency and keeps the overlap of consecutive
+ * kernels' prologues intact.  (No counterpart in the paper.)
+ */
+obc_status obc_score_kernel_spans(void* workspace, void* stream, double* pass1_us, double* pass2_us);
+
 /* ------------------------------------------------------------------------------------------
  * obc_select: pooling + per-head top-budget (Algorithm 2's index selection; SnapKV-style 1-D
  * pooling, App. C.2.1).

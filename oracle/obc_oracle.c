@@ -15,6 +15,10 @@
  *   joint score                Eq. 6  (App. A.4 boxed form)
  *   "alg1" formulation         Algorithm 1 (expanded norms: |o|^2 + |v|^2 - 2 v.o, |v|^2 - v.o)
  *   attention-only score       Sec. 4.3 (sum_i |A_ip|)
+ *   value-aware l1 score       remark after Eq. 4 and App. C.2 "VATP": Eq. 4 with l1 norms,
+ *                              sum_i |A_ip| * ||v_p||_1
+ *   scores from a given O/LSE  Eq. 4-6 with A = exp(Z - lse) and o_i as supplied by the caller
+ *                              (the attention kernel's own outputs instead of a recompute)
  *   GQA reduction              App. A.5 (sum over the query heads of a KV head's group)
  *   pool / select / compact    Algorithm 2 (top-k below the cutoff, indices sorted ascending,
  *                              gather, recent tail appended) with SnapKV-style 1-D pooling
@@ -90,7 +94,7 @@ typedef struct {
     double scale; int causal; int formulation;
     /* per (b, g, r): softmax statistics and window outputs */
     double *m, *l, *o;                 /* [B*Hkv*R], [B*Hkv*R], [B*Hkv*R*d] */
-    double *s_value, *s_key, *s_joint, *s_attn;   /* [B,Hkv,Nmax], any may be NULL */
+    double *s_value, *s_key, *s_joint, *s_attn, *s_vatp;   /* [B,Hkv,Nmax], any may be NULL */
     long chunk;                        /* tokens per phase-2 item */
     long chunks_per_unit;
 } score_ctx;
@@ -148,6 +152,8 @@ static void phase2_item(void* vctx, long item) {
     for (long p = p0; p < p1; ++p) {
         const float* kp = K + p * d; const float* vp = V + p * d;
         double nv = dot_fd(vp, vp, d);                       /* ||v_p||^2 */
+        double nv1 = 0.0;                                    /* ||v_p||_1 */
+        for (int cc = 0; cc < d; ++cc) nv1 += fabs((double)vp[cc]);
         double sv = 0.0, sk = 0.0, sj = 0.0, sa = 0.0;
         for (int r = 0; r < R; ++r) {
             if (p > last_visible(c, N, r)) continue;         /* masked pair: contributes 0 */
@@ -183,6 +189,7 @@ static void phase2_item(void* vctx, long item) {
         if (c->s_key)   c->s_key[idx]   = sk;
         if (c->s_joint) c->s_joint[idx] = sj;
         if (c->s_attn)  c->s_attn[idx]  = sa;
+        if (c->s_vatp)  c->s_vatp[idx]  = sa * nv1;          /* remark after Eq. 4: l1 norms */
     }
 }
 
@@ -195,12 +202,14 @@ static void phase2_item(void* vctx, long item) {
  *   o_out [B,Hkv,R,d], m_out, l_out [B,Hkv,R]: optional copies of the window outputs / stats.
  * Returns 0, or -1 on a bad argument / allocation failure.
  */
-int obc_oracle_score(const float* q, const float* k, const float* v,
+static int score_run(const float* q, const float* k, const float* v,
+                     const float* o_given, const float* lse_given,
                      int B, int Hq, int Hkv, int d, int W, int Nmax, const int32_t* seq_lens,
                      double scale, int causal, int formulation,
-                     double* s_value, double* s_key, double* s_joint, double* s_attn,
+                     double* s_value, double* s_key, double* s_joint, double* s_attn, double* s_vatp,
                      double* o_out, double* m_out, double* l_out, int n_threads) {
     if (!q || !k || !v || B < 1 || Hkv < 1 || Hq % Hkv || d < 1 || W < 1 || Nmax < 1) return -1;
+    if ((o_given == NULL) != (lse_given == NULL)) return -1;
     for (int b = 0; b < B; ++b) { int n = seq_lens ? seq_lens[b] : Nmax; if (n < W || n > Nmax) return -1; }
     score_ctx c; memset(&c, 0, sizeof c);
     c.q = q; c.k = k; c.v = v; c.B = B; c.Hq = Hq; c.Hkv = Hkv; c.d = d; c.W = W; c.Nmax = Nmax;
@@ -211,10 +220,17 @@ int obc_oracle_score(const float* q, const float* k, const float* v,
     c.l = (double*)malloc(sizeof(double) * units * R);
     c.o = (double*)malloc(sizeof(double) * units * R * d);
     if (!c.m || !c.l || !c.o) { free(c.m); free(c.l); free(c.o); return -1; }
-    c.s_value = s_value; c.s_key = s_key; c.s_joint = s_joint; c.s_attn = s_attn;
-    double* outs[4] = { s_value, s_key, s_joint, s_attn };
-    for (int i = 0; i < 4; ++i) if (outs[i]) memset(outs[i], 0, sizeof(double) * units * Nmax);
-    run_items(phase1_item, &c, units * R, n_threads);
+    c.s_value = s_value; c.s_key = s_key; c.s_joint = s_joint; c.s_attn = s_attn; c.s_vatp = s_vatp;
+    double* outs[5] = { s_value, s_key, s_joint, s_attn, s_vatp };
+    for (int i = 0; i < 5; ++i) if (outs[i]) memset(outs[i], 0, sizeof(double) * units * Nmax);
+    if (o_given) {
+        /* Row r of KV head g is (query head g*G + r / W, window index r % W), so [B,Hq,W,d] and
+         * [B,Hkv,R,d] are the same memory order.  A_ip = exp(z_ip - lse_i): m = lse, l = 1. */
+        for (long i = 0; i < units * R; ++i) { c.m[i] = (double)lse_given[i]; c.l[i] = 1.0; }
+        for (long i = 0; i < units * R * d; ++i) c.o[i] = (double)o_given[i];
+    } else {
+        run_items(phase1_item, &c, units * R, n_threads);
+    }
     c.chunk = 256; c.chunks_per_unit = (Nmax + c.chunk - 1) / c.chunk;
     run_items(phase2_item, &c, units * c.chunks_per_unit, n_threads);
     if (o_out) memcpy(o_out, c.o, sizeof(double) * units * R * d);
@@ -222,6 +238,34 @@ int obc_oracle_score(const float* q, const float* k, const float* v,
     if (l_out) memcpy(l_out, c.l, sizeof(double) * units * R);
     free(c.m); free(c.l); free(c.o);
     return 0;
+}
+
+int obc_oracle_score(const float* q, const float* k, const float* v,
+                     int B, int Hq, int Hkv, int d, int W, int Nmax, const int32_t* seq_lens,
+                     double scale, int causal, int formulation,
+                     double* s_value, double* s_key, double* s_joint, double* s_attn, double* s_vatp,
+                     double* o_out, double* m_out, double* l_out, int n_threads) {
+    return score_run(q, k, v, NULL, NULL, B, Hq, Hkv, d, W, Nmax, seq_lens, scale, causal, formulation,
+                     s_value, s_key, s_joint, s_attn, s_vatp, o_out, m_out, l_out, n_threads);
+}
+
+/*
+ * The same scores from attention outputs the caller already has (what a fused attention kernel
+ * returns for the window rows) instead of a recompute:
+ *   o_given   [B,Hq,W,d]  host float, the window rows of O = A V
+ *   lse_given [B,Hq,W]    host float, natural-log log-sum-exp of the scaled logits of each row
+ * Eq. 4-6 are evaluated with A_ip = exp(z_ip - lse_i) and o_i = o_given row i.  Other arguments
+ * and outputs as obc_oracle_score.
+ */
+int obc_oracle_score_given(const float* q, const float* k, const float* v,
+                           const float* o_given, const float* lse_given,
+                           int B, int Hq, int Hkv, int d, int W, int Nmax, const int32_t* seq_lens,
+                           double scale, int causal, int formulation,
+                           double* s_value, double* s_key, double* s_joint, double* s_attn, double* s_vatp,
+                           int n_threads) {
+    if (!o_given || !lse_given) return -1;
+    return score_run(q, k, v, o_given, lse_given, B, Hq, Hkv, d, W, Nmax, seq_lens, scale, causal, formulation,
+                     s_value, s_key, s_joint, s_attn, s_vatp, NULL, NULL, NULL, n_threads);
 }
 
 /* ------------------------------------------------------------------ pool */

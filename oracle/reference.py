@@ -15,7 +15,7 @@ _SRC = os.path.join(_HERE, "obc_oracle.c")
 _LIB = os.path.join(_HERE, "libobc_oracle.so")
 _lib = None
 
-VARIANT_BITS = {"V": 1, "K": 2, "VK": 4, "ATTN": 8}
+VARIANT_BITS = {"V": 1, "K": 2, "VK": 4, "ATTN": 8, "VATP": 16}
 
 
 def build(force: bool = False) -> str:
@@ -40,7 +40,9 @@ def lib():
         L = C.CDLL(_LIB)
         fp, dp, ip = C.POINTER(C.c_float), C.POINTER(C.c_double), C.POINTER(C.c_int32)
         L.obc_oracle_score.argtypes = [fp, fp, fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, ip,
-                                       C.c_double, C.c_int, C.c_int, dp, dp, dp, dp, dp, dp, dp, C.c_int]
+                                       C.c_double, C.c_int, C.c_int, dp, dp, dp, dp, dp, dp, dp, dp, C.c_int]
+        L.obc_oracle_score_given.argtypes = [fp, fp, fp, fp, fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, ip,
+                                             C.c_double, C.c_int, C.c_int, dp, dp, dp, dp, dp, C.c_int]
         L.obc_oracle_pool.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, fp]
         L.obc_oracle_select.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, ip, C.c_int]
         L.obc_oracle_compact.argtypes = [C.c_void_p, C.c_int, C.c_int, ip, C.c_int, C.c_void_p]
@@ -66,11 +68,13 @@ def _d(a):
 
 
 def score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, formulation="eq",
-          want=("V", "K", "VK"), return_attention=False, n_threads=None):
+          want=("V", "K", "VK"), return_attention=False, n_threads=None, given=None):
     """Scores for q [B,Hq,W,d], k/v [B,Hkv,Nmax,d] -> dict name -> float64 [B,Hkv,Nmax].
 
     formulation "eq" follows Eq. 4-6, "alg1" follows Algorithm 1's expanded norms.
     With return_attention the dict also holds "O" [B,Hkv,R,d], "m" and "l" [B,Hkv,R].
+    given = (o [B,Hq,W,d], lse [B,Hq,W]) evaluates the formulas with the caller's attention outputs
+    (A = exp(Z - lse), natural log) instead of recomputing the window attention.
     """
     q, qp = _f(q); k, kp = _f(k); v, vp = _f(v)
     B, Hq, W, d = q.shape
@@ -87,9 +91,20 @@ def score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, formulation="eq",
     if return_attention:
         o = np.zeros((B, Hkv, R, d)); m = np.zeros((B, Hkv, R)); l = np.zeros((B, Hkv, R))
         op, mp, lp = _d(o), _d(m), _d(l)
-    rc = lib().obc_oracle_score(qp, kp, vp, B, Hq, Hkv, d, W, Nmax, slp, float(scale), int(bool(causal)),
-                                {"eq": 0, "alg1": 1}[formulation], ptr("V"), ptr("K"), ptr("VK"),
-                                ptr("ATTN"), op, mp, lp, n_threads or host_threads())
+    form = {"eq": 0, "alg1": 1}[formulation]
+    if given is not None:
+        if return_attention:
+            raise ValueError("return_attention has nothing to return when O and LSE are given")
+        og, ogp = _f(given[0]); lg, lgp = _f(given[1])
+        if og.shape != (B, Hq, W, d) or lg.shape != (B, Hq, W):
+            raise ValueError("given O must be [B,Hq,W,d] and LSE [B,Hq,W]")
+        rc = lib().obc_oracle_score_given(qp, kp, vp, ogp, lgp, B, Hq, Hkv, d, W, Nmax, slp, float(scale),
+                                          int(bool(causal)), form, ptr("V"), ptr("K"), ptr("VK"), ptr("ATTN"),
+                                          ptr("VATP"), n_threads or host_threads())
+    else:
+        rc = lib().obc_oracle_score(qp, kp, vp, B, Hq, Hkv, d, W, Nmax, slp, float(scale), int(bool(causal)),
+                                    form, ptr("V"), ptr("K"), ptr("VK"), ptr("ATTN"), ptr("VATP"),
+                                    op, mp, lp, n_threads or host_threads())
     if rc != 0:
         raise ValueError("obc_oracle_score rejected its arguments")
     if return_attention:

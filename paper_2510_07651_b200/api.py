@@ -23,7 +23,7 @@ VARIANTS = {"V": OBC_VAR_V, "K": OBC_VAR_K, "VK": OBC_VAR_VK, "ATTN": OBC_VAR_AT
 POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
-EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_status", "obc_select_workspace", "obc_select",
+EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
            "obc_select_noalloc", "obc_compact",
            "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
            "obc_status_string", "obc_last_cuda_error", "obc_version"]
@@ -83,6 +83,7 @@ def lib():
         L.obc_score_workspace.argtypes = [C.POINTER(obc_score_params), sz]
         L.obc_score.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, vp, vp, C.c_size_t, vp]
         L.obc_score_status.argtypes = [vp, vp]
+        L.obc_score_kernel_spans.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.obc_select_workspace.argtypes = [C.POINTER(obc_select_params), sz]
         L.obc_select.argtypes = [C.POINTER(obc_select_params), vp, vp, vp, C.c_size_t, vp]
         L.obc_select_noalloc.argtypes = [C.POINTER(obc_select_params), vp, vp, vp]
@@ -172,6 +173,15 @@ def obc_score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",
 def obc_score_status(workspace) -> None:
     """Synchronise and raise ObcError(OBC_ERR_TIMEOUT) if a bounded device-side wait gave up."""
     _check(lib().obc_score_status(workspace.data_ptr(), _stream()), "obc_score_status")
+
+
+def obc_score_kernel_spans(workspace) -> tuple[float, float]:
+    """Synchronise; return the device-side extents (us) of the window-statistics kernel and of the fused
+    score kernel since the header words were last zero, and zero them.  (0, 0) on the CUDA-core path."""
+    p1, p2 = C.c_double(0), C.c_double(0)
+    _check(lib().obc_score_kernel_spans(workspace.data_ptr(), _stream(), C.byref(p1), C.byref(p2)),
+           "obc_score_kernel_spans")
+    return p1.value, p2.value
 
 
 def select_params(scores, *, budget=0, budgets=None, idx_stride=None, seq_lens=None, n_sink=0, n_recent=0,

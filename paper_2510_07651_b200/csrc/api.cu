@@ -129,6 +129,22 @@ obc_status obc_score_status(const void* workspace, void* stream) {
     return word == 0 ? OBC_OK : OBC_ERR_TIMEOUT;
 }
 
+obc_status obc_score_kernel_spans(void* workspace, void* stream, double* pass1_us, double* pass2_us) {
+    if (!workspace || !pass1_us || !pass2_us) return OBC_ERR_NULL;
+    unsigned long long w[4] = {0, 0, 0, 0};
+    char* at = static_cast<char*>(workspace) + kSpanOffset;
+    OBC_CUDA_TRY(cudaMemcpyAsync(w, at, sizeof(w), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    OBC_CUDA_TRY(cudaMemsetAsync(at, 0, sizeof(w), (cudaStream_t)stream));
+    OBC_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    auto span_us = [](unsigned long long not_start, unsigned long long end) {
+        const unsigned long long start = ~not_start;
+        return (not_start == 0 || end == 0 || end < start) ? 0.0 : (double)(end - start) * 1e-3;
+    };
+    *pass1_us = span_us(w[0], w[1]);
+    *pass2_us = span_us(w[2], w[3]);
+    return OBC_OK;
+}
+
 static obc_status resolve_select(const obc_select_params* p, SelectShape* s) {
     if (!p) return OBC_ERR_NULL;
     if (p->struct_size != sizeof(obc_select_params)) return OBC_ERR_UNSUPPORTED;

@@ -43,13 +43,15 @@ struct ScoreShape {
     int n_planes;
 };
 
+constexpr size_t kSpanOffset = 64;   // byte offset, in the workspace header, of the four kernel-span words
+
 // SIMT (CUDA-core) score path: workspace layout, computed identically by the size query and the launch
 struct SimtPlan {
     int n_splits;                        // KV splits of pass 1
     int tiles_per_split;
     int rows_out;                        // rows per unit in the combined arrays (R, or R padded)
     int want_obf;                        // also write the bf16 copy of -2*O (tensor-core pass 2)
-    size_t off_flag;                             // 256-byte header: device status word
+    size_t off_flag;                             // 256-byte header: device status word, kernel spans at kSpanOffset
     size_t off_part_m, off_part_l, off_part_o;   // partial softmax stats / outputs per split
     size_t off_lse2, off_onorm, off_o;           // combined: log2-sum-exp, ||o||^2, O (fp32)
     size_t off_obf;                              // bf16 [units][rows_out][d] = -2 * O

@@ -70,6 +70,15 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+// Device-side extent of a kernel: every CTA folds its first and last clock reading into two words of
+// the workspace header (both by atomicMax, the start as its complement, so that zeros mean "no
+// reading").  obc_score_kernel_spans() reads and zeroes them.
+__device__ __forceinline__ void span_begin(unsigned long long* span) {
+    if (threadIdx.x == 0) atomicMax(span, ~global_ns());
+}
+__device__ __forceinline__ void span_end(unsigned long long* span) {
+    if (threadIdx.x == 0) atomicMax(span + 1, global_ns());
+}
 // bounded wait: false after kWaitNs without completion
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (mbar_try(bar, parity)) return true;
@@ -152,6 +161,7 @@ struct TcParams {
     const float* onorm;                       // [units][rows_out]
     float* scores;                            // [planes][units][Nmax]
     unsigned int* status;                     // device status word (workspace header)
+    unsigned long long* span;                 // [2]: ~(earliest CTA start), latest CTA end, in globaltimer ns
 };
 
 __device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
@@ -295,6 +305,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     float4* sConst = reinterpret_cast<float4*>(smem + OFF_CONST);   // [8 epilogue warps][64 row pairs]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    span_begin(p.span);
     const int units = p.B * p.Hkv;
 
     if (threadIdx.x == 0) {
@@ -476,6 +487,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (failed) atomicCAS(p.status, 0u, (unsigned)(fail_site > 0 ? fail_site : 1));   // the first failure is kept
     tc_fence_before();
     __syncthreads();
+    span_end(p.span);
     if (warp == 0) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -519,6 +531,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     float* sConst = reinterpret_cast<float*>(smem + MC_OFF_CONST);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    span_begin(p.span);
     const int units = p.B * p.Hkv;
     const int nc = p.n_chunks;                                   // chunks of MC_ROWS rows
 
@@ -731,6 +744,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     if (failed) atomicCAS(p.status, 0u, (unsigned)(fail_site > 0 ? fail_site : 1));   // the first failure is kept
     tc_fence_before();
     __syncthreads();
+    span_end(p.span);
     if (warp == 0) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -781,6 +795,7 @@ struct P1Params {
     float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
     float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the chunk-0 CTAs
     unsigned int* status;
+    unsigned long long* span;                              // [2]: ~(earliest CTA start), latest CTA end, in globaltimer ns
 };
 
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
@@ -848,6 +863,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + P1_OFF_TMEM);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    span_begin(p.span);
 
     const int split = blockIdx.x, vu = blockIdx.y;
     const int unit = vu / p.n_chunks, c = vu % p.n_chunks;
@@ -1154,6 +1170,7 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (failed) atomicCAS(p.status, 0u, (unsigned)(fail_site > 0 ? fail_site : 1));   // the first failure is kept
     tc_fence_before();
     __syncthreads();
+    span_end(p.span);
     if (warp == 0) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -1283,6 +1300,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.part_o = (float*)(wsb + plan.off_part_o);
         p1.nv = (float*)(wsb + plan.off_nv);
         p1.status = (unsigned int*)(wsb + plan.off_flag);
+        p1.span = (unsigned long long*)(wsb + plan.off_flag + kSpanOffset);
         OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
         { ProfScope ps("tc_pass1", stream);
           OBC_CUDA_TRY(launch_pdl(tc_pass1_kernel, dim3(plan.n_splits, units * ch.n_chunks), dim3(kThreadsP1), kSmemP1, stream, 1, mq, mk, mv, p1)); }
@@ -1297,6 +1315,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     p.onorm = (const float*)(wsb + plan.off_onorm);
     p.scores = scores;
     p.status = (unsigned int*)(wsb + plan.off_flag);
+    p.span = (unsigned long long*)(wsb + plan.off_flag + kSpanOffset) + 2;
     p.cpair = (const float4*)(wsb + plan.off_cpair);
     p.nv = (const float*)(wsb + plan.off_nv);
     const long long n_tiles = (long long)units * ((s.Nmax + TILE - 1) / TILE);

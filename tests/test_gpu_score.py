@@ -108,3 +108,20 @@ def test_workspace_poison_does_not_leak():
     s = api.obc_score(q, k, v, variants=["VK"], workspace=ws)
     want = H.oracle_scores(case, ["VK"])["VK"]
     H.assert_scores_close(s[0].cpu().numpy(), want, "f32", tight=2e-5)
+
+
+def test_kernel_spans_are_recorded_and_cleared():
+    """Both tensor-core kernels leave a plausible device-side extent in the workspace header; reading
+    it zeroes it; the CUDA-core path leaves nothing."""
+    case, run = synth.config(2, shrink=8)
+    q, k, v = H.upload(case)
+    p = api.score_params(q, k, variants=["VK"])
+    ws = torch.zeros(api.obc_score_workspace(p), dtype=torch.uint8, device="cuda")
+    api.obc_score(q, k, v, variants=["VK"], workspace=ws)
+    p1, p2 = api.obc_score_kernel_spans(ws)
+    assert 1.0 < p1 < 1e4 and 1.0 < p2 < 1e4
+    assert api.obc_score_kernel_spans(ws) == (0.0, 0.0)
+    ps = api.score_params(q, k, variants=["VK"], path="simt")
+    ws2 = torch.zeros(api.obc_score_workspace(ps), dtype=torch.uint8, device="cuda")
+    api.obc_score(q, k, v, variants=["VK"], path="simt", workspace=ws2)
+    assert api.obc_score_kernel_spans(ws2) == (0.0, 0.0)

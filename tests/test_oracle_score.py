@@ -242,3 +242,64 @@ def test_peaky_attention_is_finite_and_nonnegative():
     out = ref.score(c.q, c.k, c.v)
     for n in ("V", "K", "VK"):
         assert np.isfinite(out[n]).all() and (out[n] >= 0).all()
+
+
+# ---- scores from attention outputs the caller supplies; the l1 value-aware variant -------------
+def test_given_attention_outputs_reproduce_the_recompute():
+    # O and LSE from the independent numpy attention above, laid out [B,Hq,W,d] / [B,Hq,W] with two KV
+    # heads of two query heads each: the given-statistics path must land on the recomputed scores
+    rng = np.random.default_rng(21)
+    Hkv, G, W, N, d = 2, 2, 3, 19, 8
+    q = rng.standard_normal((1, Hkv * G, W, d)).astype(np.float32)
+    k = rng.standard_normal((1, Hkv, N, d)).astype(np.float32)
+    v = rng.standard_normal((1, Hkv, N, d)).astype(np.float32)
+    o = np.zeros((1, Hkv * G, W, d)); lse = np.zeros((1, Hkv * G, W))
+    for g in range(Hkv):
+        A, Z, O = window_outputs(q[0, g * G:(g + 1) * G].astype(float), k[0, g].astype(float),
+                                 v[0, g].astype(float), 1 / np.sqrt(d))
+        o[0, g * G:(g + 1) * G] = O
+        lse[0, g * G:(g + 1) * G] = np.log(np.where(A > 0, np.exp(Z), 0.0).sum(-1))
+    names = ("V", "K", "VK", "ATTN", "VATP")
+    want = ref.score(q, k, v, want=names)
+    got = ref.score(q, k, v, want=names, given=(o, lse))
+    for n in names:      # O and LSE pass through fp32 on the way in
+        np.testing.assert_allclose(got[n], want[n], rtol=2e-5, atol=1e-7 * want[n].max())
+
+
+def test_given_statistics_are_used_as_supplied():
+    # one query, one key: z = q.k/sqrt(d); lse = z - ln a forces A = a whatever softmax would say, and
+    # the supplied o (not the true output v) enters the key and cross terms
+    d, a = 4, 0.3
+    q = np.array([[[[1.0, 2.0, 0.0, -1.0]]]], np.float32)
+    k = np.array([[[[0.5, -1.0, 3.0, 2.0]]]], np.float32)
+    v = np.array([[[[3.0, -4.0, 0.0, 1.0]]]], np.float32)
+    o = np.array([[[[1.0, 1.0, -2.0, 0.5]]]], np.float32)
+    z = (1.0 * 0.5 - 2.0 * 1.0 - 1.0 * 2.0) / 2.0                     # = -1.75
+    lse = np.array([[[z - np.log(a)]]])
+    s = ref.score(q, k, v, want=("V", "K", "VK", "ATTN", "VATP"), given=(o, lse))
+    nv, vo, dvo = 26.0, 3.0 - 4.0 + 0.5, 4.0 + 25.0 + 4.0 + 0.25       # |v|^2, v.o, |v-o|^2
+    tol = dict(rtol=1e-6)                                              # lse is rounded to fp32
+    np.testing.assert_allclose(s["ATTN"].ravel(), [a], **tol)
+    np.testing.assert_allclose(s["V"].ravel(), [a * a * nv], **tol)
+    np.testing.assert_allclose(s["K"].ravel(), [(a * z) ** 2 * dvo], **tol)
+    np.testing.assert_allclose(s["VK"].ravel(), [a * a * nv + (a * z) ** 2 * dvo + 2 * a * a * z * (nv - vo)], **tol)
+    np.testing.assert_allclose(s["VATP"].ravel(), [a * 8.0], **tol)   # |v|_1 = 8, not |v|^2 = 26
+    # doubling exp(lse) halves every A: value score / 4, attention / 2
+    s2 = ref.score(q, k, v, want=("V", "ATTN"), given=(o, lse + np.log(2.0)))
+    np.testing.assert_allclose(s2["V"].ravel(), [a * a * nv / 4], **tol)
+    np.testing.assert_allclose(s2["ATTN"].ravel(), [a / 2], **tol)
+
+
+def test_l1_value_aware_score():
+    # sum_i |A_ip| ||v_p||_1: the attention-only score (pinned above by its row sums) times the l1 norm;
+    # unchanged by flipping signs of value channels, linear (not quadratic) in the value scale
+    q, k, v = tiny(31)
+    s = run_oracle(q, k, v, want=("ATTN", "VATP"))
+    np.testing.assert_allclose(s["VATP"], s["ATTN"] * np.abs(v.astype(float)).sum(-1), rtol=1e-12)
+    flip = v * np.where(np.arange(v.shape[1]) % 2, -1.0, 1.0).astype(np.float32)
+    np.testing.assert_allclose(run_oracle(q, k, flip, want=("VATP",))["VATP"], s["VATP"], rtol=1e-12)
+    np.testing.assert_allclose(run_oracle(q, k, 2 * v, want=("VATP",))["VATP"], 2 * s["VATP"], rtol=1e-12)
+    # uniform attention (q = 0, non-causal): every token gets R / N times its l1 norm
+    G, W, N = 2, 3, k.shape[0]
+    u = run_oracle(np.zeros((G, W, k.shape[1]), np.float32), k, v, want=("VATP",), causal=False)
+    np.testing.assert_allclose(u["VATP"], G * W / N * np.abs(v.astype(float)).sum(-1), rtol=1e-12)
