@@ -449,7 +449,8 @@ def run_other(args):
         print(json.dumps(line))
         return
 
-    idx_cfg = {"qwen128k": 3, "ragged": 4}[args.workload]
+    given = args.workload.endswith("-given")     # the caller's attention outputs instead of a recompute
+    idx_cfg = {"llama32k": 2, "qwen128k": 3, "ragged": 4}[args.workload.replace("-given", "")]
     case, run = synth.config(idx_cfg)
     q, k, v = bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)
     lens = None if (case.seq_lens == case.Nmax).all() else torch.from_numpy(case.seq_lens).cuda()
@@ -468,21 +469,53 @@ def run_other(args):
     k_out = torch.empty((case.B, case.Hkv, stride, 128), dtype=torch.bfloat16, device="cuda")
     v_out = torch.empty_like(k_out)
 
+    o_win = lse_win = None
+    if given:
+        # what the model's attention kernel would hand over for the window rows, made here (untimed set-up)
+        # with plain tensor ops: O = softmax(scale * Q K^T) V and the natural-log LSE, causal over the window
+        G, W, scale = case.G, case.W, 1.0 / np.sqrt(128.0)
+        o_win = torch.empty((case.B, case.Hq, W, 128), dtype=torch.bfloat16, device="cuda")
+        lse_win = torch.empty((case.B, case.Hq, W), dtype=torch.float32, device="cuda")
+        for b_ in range(case.B):
+            n = int(case.seq_lens[b_])
+            vis = torch.arange(n, device="cuda")[None, :] <= (n - W + torch.arange(W, device="cuda"))[:, None]
+            for g_ in range(case.Hkv):
+                qg = q[b_, g_ * G:(g_ + 1) * G].float()                          # [G, W, d]
+                z = torch.einsum("gwd,nd->gwn", qg, k[b_, g_, :n].float()) * scale
+                z = z.masked_fill(~vis[None], float("-inf"))
+                lse_win[b_, g_ * G:(g_ + 1) * G] = torch.logsumexp(z, dim=-1)
+                o_win[b_, g_ * G:(g_ + 1) * G] = (torch.softmax(z, dim=-1) @ v[b_, g_, :n].float()).to(torch.bfloat16)
+                del z
+        torch.cuda.synchronize()
+
     def step():
-        api.obc_score(q, k, v, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
+        if given:
+            api.obc_score_given(q, k, v, o_win, lse_win, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
+        else:
+            api.obc_score(q, k, v, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
         api.obc_select(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
                        seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
                        idx=idx, workspace=ws_sel)
         api.obc_compact(k, v, idx, k_out=k_out, v_out=v_out)
-    for _ in range(warmup):
+    for _ in range(3):
         step()
     torch.cuda.synchronize()
-    e0.record()
-    for _ in range(steps):
+    graph = torch.cuda.CUDAGraph()               # the library allocates nothing and only enqueues: a step can be captured
+    with torch.cuda.graph(graph):
         step()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
+
+    def timed(run):
+        for _ in range(warmup):
+            run()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+    ms_by_mode = {"plain library calls": timed(step), "one captured CUDA graph per step, replayed": timed(graph.replay)}
+    launch_mode, ms = min(ms_by_mode.items(), key=lambda kv: kv[1])
     api.obc_profile_begin()
     for _ in range(min(steps, 50)):
         step()
@@ -492,7 +525,9 @@ def run_other(args):
     line = {"metric": METRIC, "value": tokens * steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps,
             "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{case.name}: B{case.B} Hq{case.Hq} Hkv{case.Hkv} d128 Nmax{case.Nmax} W{case.W} bf16, "
-                                   f"variants {order}, pool {run['pool_mode']} {run['pool_kernel']}, tokens/step {tokens}",
+                                   f"variants {order}, pool {run['pool_mode']} {run['pool_kernel']}, tokens/step {tokens}"
+                                   + (", window O and LSE supplied by the caller (no recompute)" if given else ""),
+                       "launch": launch_mode, "ms_per_step_by_launch": {k_: v_ / steps for k_, v_ in ms_by_mode.items()},
                        "l2": "inputs (K+V) larger than L2" if tokens * case.Hkv * 512 > 126e6 else "single input copy"},
             "kernels": {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}}
     print(json.dumps(line))
@@ -507,7 +542,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--eager", action="store_true", help="time plain library calls instead of replaying CUDA graphs")
-    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode"],
+    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given"],
                     help="llama32k is the headline benchmark; the others print a shorter line (1 GPU)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"

@@ -45,12 +45,13 @@ typedef enum {
 typedef enum { OBC_F32 = 0, OBC_BF16 = 1 } obc_dtype;
 
 /* score variants (bitmask).  The scores buffer holds one [B,Hkv,max_len] fp32 plane per set bit,
- * in ascending bit order (V, K, VK, ATTN). */
+ * in ascending bit order (V, K, VK, ATTN, VATP). */
 enum {
     OBC_VAR_V = 1,     /* OBCache-V   : Eq. 4  sum_i A_ip^2 ||v_p||^2                           */
     OBC_VAR_K = 2,     /* OBCache-K   : Eq. 5  sum_i (A_ip Z_ip)^2 ||v_p - o_i||^2              */
     OBC_VAR_VK = 4,    /* OBCache-V&K : Eq. 6  value + key + 2 sum_i A_ip^2 Z_ip (|v_p|^2-v_p.o_i) */
-    OBC_VAR_ATTN = 8   /* attention-only score of Sec. 4.3: sum_i |A_ip|                        */
+    OBC_VAR_ATTN = 8,  /* attention-only score of Sec. 4.3: sum_i |A_ip|                        */
+    OBC_VAR_VATP = 16  /* Eq. 4 with l1 norms (remark after Eq. 4; App. C.2): sum_i |A_ip| ||v_p||_1 */
 };
 
 enum { OBC_POOL_NONE = 0, OBC_POOL_AVG = 1, OBC_POOL_MAX = 2 };
@@ -103,6 +104,22 @@ obc_status obc_score_workspace(const obc_score_params* p, size_t* bytes /* host 
  */
 obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
                      float* scores, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same scores from attention outputs the caller already has, instead of recomputing the window
+ * attention: the window rows of O = A V and their log-sum-exp, as the model's own (fused)
+ * attention kernel returns them.  Eq. 4-6 are evaluated with A_rp = exp(Z_rp - lse_r) and o_r as
+ * given; K and V are then read once instead of twice.  (The paper recomputes the window attention,
+ * App. C, because its attention kernel does not expose these; this entry point is the integration
+ * the recompute stands in for.)
+ *   o    [B,Hq,W,d], device, f32 or bf16 (need not match q), strided like any obc_tensor
+ *   lse  device fp32 [B,Hq,W] contiguous: natural log of sum_p exp(scale * q_r . k_p) over the
+ *        positions row r sees
+ * Everything else as obc_score, including the workspace size (obc_score_workspace).
+ */
+obc_status obc_score_given(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                           obc_tensor o, const float* lse,
+                           float* scores, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Reads the device status word that obc_score keeps in the first bytes of its workspace.  The

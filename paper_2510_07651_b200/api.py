@@ -16,14 +16,14 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libobcache.so")
 
 OBC_F32, OBC_BF16 = 0, 1
-OBC_VAR_V, OBC_VAR_K, OBC_VAR_VK, OBC_VAR_ATTN = 1, 2, 4, 8
+OBC_VAR_V, OBC_VAR_K, OBC_VAR_VK, OBC_VAR_ATTN, OBC_VAR_VATP = 1, 2, 4, 8, 16
 OBC_POOL_NONE, OBC_POOL_AVG, OBC_POOL_MAX = 0, 1, 2
 OBC_PATH_AUTO, OBC_PATH_SIMT, OBC_PATH_TC = 0, 1, 2
-VARIANTS = {"V": OBC_VAR_V, "K": OBC_VAR_K, "VK": OBC_VAR_VK, "ATTN": OBC_VAR_ATTN}
+VARIANTS = {"V": OBC_VAR_V, "K": OBC_VAR_K, "VK": OBC_VAR_VK, "ATTN": OBC_VAR_ATTN, "VATP": OBC_VAR_VATP}
 POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
-EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
+EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_given", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
            "obc_select_noalloc", "obc_compact",
            "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
            "obc_status_string", "obc_last_cuda_error", "obc_version"]
@@ -82,6 +82,7 @@ def lib():
         vp, sz = C.c_void_p, C.POINTER(C.c_size_t)
         L.obc_score_workspace.argtypes = [C.POINTER(obc_score_params), sz]
         L.obc_score.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, vp, vp, C.c_size_t, vp]
+        L.obc_score_given.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, obc_tensor, vp, vp, vp, C.c_size_t, vp]
         L.obc_score_status.argtypes = [vp, vp]
         L.obc_score_kernel_spans.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.obc_select_workspace.argtypes = [C.POINTER(obc_select_params), sz]
@@ -158,7 +159,7 @@ def obc_score_workspace(p: obc_score_params) -> int:
 def obc_score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",), path="auto",
               scores=None, workspace=None):
     """q [B,Hq,W,d], k/v [B,Hkv,Nmax,d] CUDA tensors -> fp32 scores [n_variants,B,Hkv,Nmax]
-    (planes in V, K, VK, ATTN order).  Enqueued on the current stream."""
+    (planes in V, K, VK, ATTN, VATP order).  Enqueued on the current stream."""
     p = score_params(q, k, seq_lens=seq_lens, scale=scale, causal=causal, variants=variants, path=path)
     B, Hkv, Nmax = k.shape[0], k.shape[1], k.shape[2]
     n_planes = bin(p.variants).count("1")
@@ -167,6 +168,26 @@ def obc_score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",
     ws = _workspace(obc_score_workspace(p), k, workspace)
     _check(lib().obc_score(C.byref(p), as_tensor4(q), as_tensor4(k), as_tensor4(v), scores.data_ptr(),
                            ws.data_ptr(), ws.numel(), _stream()), "obc_score")
+    return scores
+
+
+def obc_score_given(q, k, v, o, lse, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",), path="auto",
+                    scores=None, workspace=None):
+    """obc_score from attention outputs the caller already has: o [B,Hq,W,d] (f32 or bf16) and lse
+    fp32 [B,Hq,W] (natural log, contiguous) of the window rows; no window attention is recomputed."""
+    p = score_params(q, k, seq_lens=seq_lens, scale=scale, causal=causal, variants=variants, path=path)
+    B, Hkv, Nmax = k.shape[0], k.shape[1], k.shape[2]
+    if tuple(o.shape) != tuple(q.shape) or tuple(lse.shape) != tuple(q.shape[:3]):
+        raise ValueError("o must be shaped like q and lse like q without its last axis")
+    if lse.dtype != torch.float32 or not lse.is_contiguous():
+        raise ValueError("lse must be a contiguous float32 tensor")
+    n_planes = bin(p.variants).count("1")
+    if scores is None:
+        scores = torch.empty((n_planes, B, Hkv, Nmax), dtype=torch.float32, device=k.device)
+    ws = _workspace(obc_score_workspace(p), k, workspace)
+    _check(lib().obc_score_given(C.byref(p), as_tensor4(q), as_tensor4(k), as_tensor4(v), as_tensor4(o),
+                                 lse.data_ptr(), scores.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "obc_score_given")
     return scores
 
 

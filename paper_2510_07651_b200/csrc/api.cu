@@ -58,7 +58,7 @@ obc_status resolve_score(const obc_score_params* p, ScoreShape* s) {
     if (p->batch < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return OBC_ERR_SHAPE;
     if (p->window < 1 || p->max_len < 1 || p->window > p->max_len) return OBC_ERR_SHAPE;
     if ((long long)p->batch * p->n_kv_heads > 65535) return OBC_ERR_SHAPE;
-    const unsigned known = OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN;
+    const unsigned known = OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN | OBC_VAR_VATP;
     if (p->variants == 0 || (p->variants & ~known)) return OBC_ERR_UNSUPPORTED;
     if (p->path < OBC_PATH_AUTO || p->path > OBC_PATH_TC) return OBC_ERR_UNSUPPORTED;
     s->B = p->batch; s->Hq = p->n_q_heads; s->Hkv = p->n_kv_heads; s->G = s->Hq / s->Hkv;
@@ -97,8 +97,9 @@ obc_status obc_score_workspace(const obc_score_params* p, size_t* bytes) {
     return OBC_OK;
 }
 
-obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
-                     float* scores, void* workspace, size_t workspace_bytes, void* stream) {
+static obc_status score_impl(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                             const obc_tensor* o, const float* lse,
+                             float* scores, void* workspace, size_t workspace_bytes, void* stream) {
     ScoreShape s;
     obc_status st = resolve_score(p, &s);
     if (st != OBC_OK) return st;
@@ -108,17 +109,37 @@ obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_
     if ((st = check_tensor(v, true)) != OBC_OK) return st;
     if (q.dtype != k.dtype || k.dtype != v.dtype) return OBC_ERR_UNSUPPORTED;
     if (((uintptr_t)scores & 15) != 0) return OBC_ERR_ALIGN;
+    GivenAttention given{};
+    if (o) {
+        if (!lse) return OBC_ERR_NULL;
+        if ((st = check_tensor(*o, true)) != OBC_OK) return st;
+        if (((uintptr_t)lse & 3) != 0) return OBC_ERR_ALIGN;
+        given = GivenAttention{view(*o), o->dtype, lse};
+    }
     size_t need = 0;
     if ((st = obc_score_workspace(p, &need)) != OBC_OK) return st;
     if (!workspace || workspace_bytes < need) return OBC_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
     const bool tc = want_tc(p, s, q.dtype, view(q));
     if (p->path == OBC_PATH_TC && !tc) return OBC_ERR_UNSUPPORTED;
-    if (tc) return launch_score_tc(s, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);
+    if (tc) return launch_score_tc(s, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream, o ? &given : nullptr);
     const SimtPlan plan = make_simt_plan(s, s.R, false);
-    st = launch_simt_pass1_combine(s, plan, q.dtype, view(q), view(k), view(v), workspace, (cudaStream_t)stream);
+    st = o ? launch_given_prep(s, plan, given, workspace, (cudaStream_t)stream)
+           : launch_simt_pass1_combine(s, plan, q.dtype, view(q), view(k), view(v), workspace, (cudaStream_t)stream);
     if (st != OBC_OK) return st;
     return launch_simt_pass2(s, plan, q.dtype, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);
+}
+
+obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                     float* scores, void* workspace, size_t workspace_bytes, void* stream) {
+    return score_impl(p, q, k, v, nullptr, nullptr, scores, workspace, workspace_bytes, stream);
+}
+
+obc_status obc_score_given(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                           obc_tensor o, const float* lse,
+                           float* scores, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!lse) return OBC_ERR_NULL;
+    return score_impl(p, q, k, v, &o, lse, scores, workspace, workspace_bytes, stream);
 }
 
 obc_status obc_score_status(const void* workspace, void* stream) {

@@ -61,6 +61,18 @@ struct SimtPlan {
 };
 SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf);
 
+// Attention outputs supplied by the caller instead of a recompute: o [B,Hq,W,d] (any dtype, strided),
+// lse fp32 [B,Hq,W] contiguous, natural log of the row's sum of exp(scaled logit).
+struct GivenAttention {
+    TensorView o;
+    int o_dtype;
+    const float* lse;
+};
+// writes what the combine kernel would have written (log2-sum-exp, ||o||^2, O, -2 O in bf16, row-pair
+// constants) from the caller's arrays, and clears the status word
+obc_status launch_given_prep(const ScoreShape& s, const SimtPlan& plan, const GivenAttention& given,
+                             void* ws, cudaStream_t stream);
+
 // pass 1 + combine (window softmax statistics and outputs), then pass 2 (scores)
 obc_status launch_simt_pass1_combine(const ScoreShape& s, const SimtPlan& plan, int dtype,
                                      TensorView q, TensorView k, TensorView v, void* ws, cudaStream_t stream);
@@ -100,7 +112,7 @@ bool tc_shape_supported(const ScoreShape& s);                       // R large e
 bool tc_supported(const ScoreShape& s, int dtype, const TensorView& q);   // + bf16, uniformly strided Q rows
 size_t tc_workspace_bytes(const ScoreShape& s);
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
-                           float* scores, void* ws, cudaStream_t stream);
+                           float* scores, void* ws, cudaStream_t stream, const GivenAttention* given = nullptr);
 
 // ---- programmatic dependent launch ------------------------------------------------------------
 // Every kernel of the library is launched with programmatic stream serialization: its CTAs may

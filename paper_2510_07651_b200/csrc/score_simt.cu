@@ -28,6 +28,9 @@ __device__ __forceinline__ const T* row_ptr(const TensorView& t, int b, int h, l
     return reinterpret_cast<const T*>(t.ptr) + b * t.sb + h * t.sh + tok * t.st;
 }
 
+__device__ __forceinline__ float elem_to_float(float x) { return x; }
+__device__ __forceinline__ float elem_to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
 // cooperative load of `rows` x 128 elements into fp32 smem (row stride `stride` floats);
 // rows >= valid are zero-filled.  get(row) returns the global row pointer.
 template <typename T, typename F>
@@ -258,6 +261,37 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     }
 }
 
+// One block of 128 threads per (unit, output row), like the combine kernel, but the row comes from the
+// caller: o [B,Hq,W,d] and the natural-log LSE [B,Hq,W] of an attention kernel that already ran.
+// Row r of KV head g is (query head g*G + r / W, window query r % W).
+template <typename T>
+__global__ void __launch_bounds__(CMB_NT)
+given_prep_kernel(ScoreShape s, SimtPlan plan, TensorView o, const float* lse, float* ws) {
+    pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0)     // no wait of this call can have given up yet
+        *reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(ws) + plan.off_flag) = 0u;
+    const int r = blockIdx.x % plan.rows_out, unit = blockIdx.x / plan.rows_out;
+    const int tid = threadIdx.x;
+    const size_t orow = (size_t)unit * plan.rows_out + r;
+    __nv_bfloat16* obf = plan.want_obf ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + plan.off_obf) : nullptr;
+    float* cpair = plan.want_obf ? ws + plan.off_cpair / 4 + (orow >> 1) * 4 + (orow & 1) : nullptr;
+    __shared__ float red[4];
+    float oc = 0.f, lse2 = INFINITY;             // padding rows weigh 0
+    if (r < s.R) {
+        const int b = unit / s.Hkv, g = unit % s.Hkv, h = g * s.G + r / s.W, i = r % s.W;
+        oc = elem_to_float(row_ptr<T>(o, b, h, i)[tid]);
+        lse2 = lse[((size_t)b * s.Hq + h) * s.W + i] * kLog2e;
+    }
+    const float onorm = block128_reduce(oc * oc, false, red);
+    (ws + plan.off_o / 4)[orow * kD + tid] = oc;
+    if (obf) obf[orow * kD + tid] = __float2bfloat16(-2.f * oc);
+    if (tid == 0) {
+        (ws + plan.off_lse2 / 4)[orow] = lse2;
+        (ws + plan.off_onorm / 4)[orow] = onorm;
+        if (cpair) { cpair[0] = -lse2; cpair[2] = onorm; }
+    }
+}
+
 // ------------------------------------------------------------------------------------------ pass 2
 template <typename T>
 __global__ void __launch_bounds__(NT, 2)
@@ -270,7 +304,8 @@ simt_pass2_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
     float* sQ = sV + TN * KS;               // [RC][kD]   (reused for the final cross-warp sum)
     float* sO = sQ + RC * kD;               // [RC][kD]
     float* sNv = sO + RC * kD;              // [TN]
-    float* sLse = sNv + TN;                 // [RC]
+    float* sNv1 = sNv + TN;                 // [TN]
+    float* sLse = sNv1 + TN;                // [RC]
     float* sNo = sLse + RC;                 // [RC]
 
     const int unit = blockIdx.y, t0 = blockIdx.x * TN;
@@ -295,7 +330,8 @@ simt_pass2_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
     for (int tkn = warp * 8; tkn < warp * 8 + 8; ++tkn) {
         float4 f = *reinterpret_cast<const float4*>(sV + tkn * KS + lane * 4);
         float sq = warp_sum(f.x * f.x + f.y * f.y + f.z * f.z + f.w * f.w);
-        if (lane == 0) sNv[tkn] = sq;
+        float ab = warp_sum((fabsf(f.x) + fabsf(f.y)) + (fabsf(f.z) + fabsf(f.w)));
+        if (lane == 0) { sNv[tkn] = sq; sNv1[tkn] = ab; }
     }
 
     const float sl2 = s.scale * kLog2e;
@@ -374,12 +410,13 @@ simt_pass2_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
             if (s.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + p] = live ? tk : 0.f;
             if (s.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + p] = live ? tv + tk + tx : 0.f;
             if (s.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + p] = live ? ta : 0.f;
+            if (s.variants & OBC_VAR_VATP) out[(size_t)(pl++) * plane + p] = live ? ta * sNv1[tl] : 0.f;
         }
     }
 }
 
 constexpr size_t kSmemPass1 = (size_t)(TN * KS + TN * kD + RC * kD + RC * TN) * 4;
-constexpr size_t kSmemPass2 = (size_t)(2 * TN * KS + 2 * RC * kD + TN + 2 * RC) * 4;
+constexpr size_t kSmemPass2 = (size_t)(2 * TN * KS + 2 * RC * kD + 2 * TN + 2 * RC) * 4;
 
 template <typename T>
 obc_status launch_pass1_typed(const ScoreShape& s, const SimtPlan& plan, TensorView q, TensorView k, TensorView v,
@@ -430,6 +467,17 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
 
 obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream) {
     { ProfScope ps("combine", stream); OBC_CUDA_TRY(launch_pdl(simt_combine_kernel, dim3(s.B * s.Hkv * plan.rows_out), dim3(CMB_NT), 0, stream, 1, s, plan, (float*)ws)); }
+    return OBC_OK;
+}
+
+obc_status launch_given_prep(const ScoreShape& s, const SimtPlan& plan, const GivenAttention& given,
+                             void* ws, cudaStream_t stream) {
+    const dim3 grid(s.B * s.Hkv * plan.rows_out), block(CMB_NT);
+    ProfScope ps("given_prep", stream);
+    if (given.o_dtype == OBC_F32)
+        OBC_CUDA_TRY(launch_pdl(given_prep_kernel<float>, grid, block, 0, stream, 1, s, plan, given.o, given.lse, (float*)ws));
+    else
+        OBC_CUDA_TRY(launch_pdl(given_prep_kernel<__nv_bfloat16>, grid, block, 0, stream, 1, s, plan, given.o, given.lse, (float*)ws));
     return OBC_OK;
 }
 

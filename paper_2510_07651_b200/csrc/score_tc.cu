@@ -12,7 +12,8 @@
 // Warp roles of the 384-thread CTA (persistent, one CTA per SM):
 //   warp 0      TMA producer: K/V tiles into a 2-stage ring, Q / -2O when the unit changes
 //   warp 1      MMA issuer (one elected lane), double-buffered TMEM accumulators (2 x 256 columns)
-//   warps 2-3   idle here (||v_p||^2 is computed by pass 1, whose two spare warps have the V tile at hand)
+//   warps 2-3   idle when pass 1 ran (its two spare warps computed ||v_p||^2 with the V tile at hand);
+//               otherwise (attention outputs supplied by the caller, or the l1 variant) the value norms of every tile
 //   warps 4-7   epilogue group 0 (even tiles), warps 8-11 epilogue group 1 (odd tiles)
 //
 // Every mbarrier wait is bounded: on a timeout the kernel raises the status word in the workspace
@@ -26,6 +27,7 @@ namespace obc {
 namespace {
 
 constexpr int TILE = 128;                       // tokens per tile = MMA M
+constexpr unsigned kAllVariants = OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN | OBC_VAR_VATP;
 constexpr int NSTAGE = 2;
 constexpr uint32_t kHalfBytes = 128 * 128;      // [128 rows][64 bf16] = 16 KB, one swizzle-128B block
 constexpr uint32_t kOperandBytes = 2 * kHalfBytes;
@@ -38,14 +40,17 @@ constexpr uint32_t OFF_O = OFF_Q + kOperandBytes;
 constexpr uint32_t OFF_K = OFF_O + kOperandBytes;                 // NSTAGE x 32 KB
 constexpr uint32_t OFF_V = OFF_K + NSTAGE * kOperandBytes;        // NSTAGE x 32 KB
 constexpr uint32_t OFF_CONST = OFF_V + NSTAGE * kOperandBytes;    // 8 epilogue warps x 64 float4 (row-pair constants)
-constexpr uint32_t OFF_BAR = OFF_CONST + 8 * 64 * 16;
-constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + 2;
+constexpr int NSLOT = 4;                                          // ring depth of the per-tile value norms
+constexpr uint32_t OFF_NV = OFF_CONST + 8 * 64 * 16;              // NSLOT x 128 x (||v||^2, ||v||_1), own-norm kernels only
+constexpr uint32_t OFF_BAR = OFF_NV + NSLOT * TILE * 8;
+constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + 2 + 2 * NSLOT;
 constexpr uint32_t OFF_TMEM = OFF_BAR + kNumBars * 8;
 constexpr uint32_t kSmemBytes = OFF_TMEM + 16 + 1024;             // + alignment slack
 
 enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_QO_FULL = 2 * NSTAGE, BAR_QO_EMPTY = 2 * NSTAGE + 1,
        BAR_TM_FULL = 2 * NSTAGE + 2,      // [epilogue group][TMEM buffer]
-       BAR_TM_EMPTY = 2 * NSTAGE + 6 };   // [TMEM buffer]
+       BAR_TM_EMPTY = 2 * NSTAGE + 6,     // [TMEM buffer]
+       BAR_NV = 2 * NSTAGE + 8 };         // [epilogue group][slot], own-norm kernels only
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -73,11 +78,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Device-side extent of a kernel: every CTA folds its first and last clock reading into two words of
 // the workspace header (both by atomicMax, the start as its complement, so that zeros mean "no
 // reading").  obc_score_kernel_spans() reads and zeroes them.
+// (Taken by a thread that has nothing urgent to do at either end: thread 0 issues the first copies.)
 __device__ __forceinline__ void span_begin(unsigned long long* span) {
-    if (threadIdx.x == 0) atomicMax(span, ~global_ns());
+    if (threadIdx.x == 96) atomicMax(span, ~global_ns());
 }
 __device__ __forceinline__ void span_end(unsigned long long* span) {
-    if (threadIdx.x == 0) atomicMax(span + 1, global_ns());
+    if (threadIdx.x == 96) atomicMax(span + 1, global_ns());
 }
 // bounded wait: false after kWaitNs without completion
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -221,6 +227,32 @@ __device__ __forceinline__ void tc_wait_ld16x2(uint32_t (&a)[16], uint32_t (&b)[
                  :: "memory");
 }
 
+// ||v||^2 (and, with L1, ||v||_1) of row `tok` of a [128 tokens][128 bf16] tile stored as two
+// swizzle-128B halves.  Any order of the row's 16-byte pieces gives the same sums; this one is free
+// of bank conflicts when consecutive threads take consecutive rows.
+template <bool L1>
+__device__ __forceinline__ void value_norms(const uint8_t* vt, int tok, float& l2, float& l1) {
+    float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0, ab0 = acc0, ab1 = acc0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+            const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
+            const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
+            const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
+            acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
+            acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
+            if (L1) {
+                ab0 = __fadd2_rn(ab0, __fadd2_rn(make_float2(fabsf(f0.x), fabsf(f0.y)), make_float2(fabsf(f1.x), fabsf(f1.y))));
+                ab1 = __fadd2_rn(ab1, __fadd2_rn(make_float2(fabsf(f2.x), fabsf(f2.y)), make_float2(fabsf(f3.x), fabsf(f3.y))));
+            }
+        }
+    const float2 sum = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
+    l2 = sum.x + sum.y;
+    const float2 sab = __fadd2_rn(ab0, ab1);
+    l1 = sab.x + sab.y;
+}
+
 // Running sums of one token over the window rows, two rows per packed fp32x2 lane.  With
 // a = A_rp, u = a z (z the unscaled logit), b = a + scale u = a (1 + Z):
 //   Eq. 6   sum_r a^2 ||(1+Z) v - Z o_r||^2 = |v|^2 S1 + scale S2 + scale^2 S3
@@ -266,7 +298,7 @@ __device__ __forceinline__ void score_rows16(const uint32_t (&zr)[16], const uin
             if (VARS & OBC_VAR_K) { S.s4 = __ffma2_rn(uu, t2, S.s4); S.s5 = __fadd2_rn(uu, S.s5); }
         }
         if (VARS & OBC_VAR_V) S.s6 = __ffma2_rn(a, a, S.s6);
-        if (VARS & OBC_VAR_ATTN) S.s7 = __fadd2_rn(a, S.s7);
+        if (VARS & (OBC_VAR_ATTN | OBC_VAR_VATP)) S.s7 = __fadd2_rn(a, S.s7);
     }
 }
 
@@ -290,8 +322,9 @@ __device__ __forceinline__ void score_chunk(uint32_t zt, uint32_t tt, int chunk_
     }
 }
 
-// VARS: variants this instantiation computes (a superset of p.variants)
-template <unsigned VARS>
+// VARS: variants this instantiation computes (a superset of p.variants).  OWN_NV: no pass 1 ran (the
+// caller supplied the attention outputs), so warps 2-3 compute the value norms from the V tiles here.
+template <unsigned VARS, bool OWN_NV>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
                 const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -303,6 +336,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_TMEM);
     float4* sConst = reinterpret_cast<float4*>(smem + OFF_CONST);   // [8 epilogue warps][64 row pairs]
+    float2* sNv = reinterpret_cast<float2*>(smem + OFF_NV);         // [NSLOT][128] (||v||^2, ||v||_1)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     span_begin(p.span);
@@ -310,7 +344,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_k); prefetch_tmap(&map_v); prefetch_tmap(&map_q); prefetch_tmap(&map_o);
-        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
+        // a K/V stage is released by the MMA commit and, when the norms are computed here, by warps 2-3
+        for (int i = 0; i < NSTAGE; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), OWN_NV ? 3 : 1); }
+        if (OWN_NV) for (int i = 0; i < 2 * NSLOT; ++i) mbar_init(bar(BAR_NV + i), 2);
         mbar_init(bar(BAR_QO_FULL), 1); mbar_init(bar(BAR_QO_EMPTY), 1);
         for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_TM_FULL + i), 1);
         for (int i = 0; i < 2; ++i) mbar_init(bar(BAR_TM_EMPTY + i), 4);
@@ -332,8 +368,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // Every role walks the same tiles (TileWalk); all window rows of a unit (at most 128) are one chunk.
     // Tiles go to the two epilogue groups alternately.  What an epilogue group waits for (accumulators
     // ready) is signalled on barriers of its own, so that each waiter sees every phase of the barriers
-    // it uses; a parity wait must never fall two phases behind.  ||v_p||^2 comes from pass 1 and the
-    // per-row constants from the combine kernel, so no warp here reads the K/V tiles.
+    // it uses; a parity wait must never fall two phases behind.  ||v_p||^2 comes from pass 1 (or, with
+    // OWN_NV, from warps 2-3 through a ring of NSLOT slots) and the per-row constants from the combine kernel.
     // `item` counts the (tile, chunk) pairs processed so far and indexes the smem stage, TMEM
     // buffer and constant-slot rings.
     TileWalk tw;
@@ -412,7 +448,29 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 ++item;
             }
         }
-    } else if (warp >= 4) {
+    } else if (warp < 4) {
+        // ================= value norms of every tile (only when no pass 1 supplied them) ===========
+        if (OWN_NV) {
+            const int t64 = threadIdx.x - 64;                      // 0..63
+            uint32_t item = 0;
+            for (; !tw.done() && !failed; tw.next(), ++item) {
+                const uint32_t st = item % NSTAGE, slot = item % NSLOT, owner = item & 1;
+                if (!mbar_wait(bar(BAR_FULL + st), (item / NSTAGE) & 1)) { failed = true; fail_site = __LINE__; break; }
+                const uint8_t* vt = smem + OFF_V + st * kOperandBytes;
+                // slot `slot` was last read for the tile four back, whose owner took it into registers before
+                // releasing the accumulators that the MMA of the tile two back (whose commit freed this stage) needed
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int tok = t64 + 64 * j;
+                    float l2, l1;
+                    value_norms<(VARS & OBC_VAR_VATP) != 0>(vt, tok, l2, l1);
+                    sNv[slot * TILE + tok] = make_float2(l2, l1);
+                }
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(bar(BAR_NV + owner * NSLOT + slot)); mbar_arrive(bar(BAR_EMPTY + st)); }
+            }
+        }
+    } else {
         // ======================================= epilogue =======================================
         const int wg = (warp - 4) >> 2;                            // 0: even tiles, 1: odd tiles
         const int lane_grp = warp & 3;                             // TMEM lanes 32*lane_grp .. +31
@@ -420,7 +478,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const float2 sl2 = make_float2(p.scale * kLog2e, p.scale * kLog2e), sc = make_float2(p.scale, p.scale);
         const size_t plane = (size_t)units * p.Nmax;
         uint32_t item = 0, tile_seq = 0;
-        uint32_t full_par = 0;                                     // phase parity of this group's barriers, one bit each
+        uint32_t full_par = 0, nv_par = 0;                         // phase parity of this group's barriers, one bit each
         float4* my_const = sConst + (warp - 4) * 64;               // this warp's copy of the unit's row constants
         int const_unit = -1;
         for (; !tw.done() && !failed; tw.next()) {
@@ -436,7 +494,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
             const uint32_t buf = item & 1;
-            const float nv = ptok < N ? p.nv[(size_t)unit * p.Nmax + ptok] : 0.f;      // used after the row loop
+            float nv = 0.f, nv1 = 0.f;                             // used after the row loop
+            if (!OWN_NV && ptok < N) nv = p.nv[(size_t)unit * p.Nmax + ptok];
             if (unit != const_unit) {                              // at most once per unit: (-lse2, |o|^2) of every row pair
                 __syncwarp();
                 for (int i = lane; i < 64; i += 32) {
@@ -450,6 +509,13 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (!mbar_wait(bar(BAR_TM_FULL + wg * 2 + buf), (full_par >> buf) & 1)) { failed = true; fail_site = __LINE__; break; }
             full_par ^= 1u << buf;
             tc_fence_after();
+            if (OWN_NV) {                                          // the norms of this tile (ready long before the accumulators)
+                const uint32_t slot = item % NSLOT;
+                if (!mbar_wait(bar(BAR_NV + wg * NSLOT + slot), (nv_par >> slot) & 1)) { failed = true; fail_site = __LINE__; break; }
+                nv_par ^= 1u << slot;
+                const float2 n21 = sNv[slot * TILE + tok];
+                nv = n21.x; nv1 = n21.y;
+            }
             const float4* cst = my_const;
             const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u, tt = zt + 128u;
             if (masked_tile)
@@ -470,6 +536,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] =
                     live ? fmaf(nv, S.s1.x + S.s1.y, fmaf(p.scale, S.s2.x + S.s2.y, s2 * (S.s3.x + S.s3.y))) : 0.f;
                 if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? S.s7.x + S.s7.y : 0.f;
+                if (p.variants & OBC_VAR_VATP) out[(size_t)(pl++) * plane + ptok] = live ? nv1 * (S.s7.x + S.s7.y) : 0.f;
             }
         }
         // padding beyond the last tile of a shorter sequence: zeros
@@ -508,8 +575,8 @@ constexpr uint32_t kQoBuf = 4 * kHalfB64;                         // Q chunk (2 
 constexpr uint32_t MC_OFF_QO = 0;                                 // 2 buffers x 32 KB
 constexpr uint32_t MC_OFF_K = MC_OFF_QO + 2 * kQoBuf;             // 2 tiles x 32 KB
 constexpr uint32_t MC_OFF_V = MC_OFF_K + 2 * kOperandBytes;
-constexpr uint32_t MC_OFF_NV = MC_OFF_V + 2 * kOperandBytes;      // [pair parity][tile of the pair][128] floats
-constexpr uint32_t MC_OFF_CONST = MC_OFF_NV + 4 * TILE * 4;       // 4 slots x 32 float4 (per chunk)
+constexpr uint32_t MC_OFF_NV = MC_OFF_V + 2 * kOperandBytes;      // [pair parity][tile of the pair][128] x (||v||^2, ||v||_1)
+constexpr uint32_t MC_OFF_CONST = MC_OFF_NV + 4 * TILE * 8;       // 4 slots x 32 float4 (per chunk)
 constexpr uint32_t MC_OFF_BAR = MC_OFF_CONST + 4 * 32 * 16;
 enum { MC_FULL = 0, MC_EMPTY = 2, MC_QO_FULL = 4, MC_QO_EMPTY = 6, MC_TM_FULL = 8, MC_TM_EMPTY = 12,
        MC_NV = 16, MC_CONST = 18, MC_NBARS = 22 };
@@ -527,7 +594,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     const uint32_t bars = sbase + MC_OFF_BAR;
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + MC_OFF_TMEM);
-    float* sNv = reinterpret_cast<float*>(smem + MC_OFF_NV);
+    float2* sNv = reinterpret_cast<float2*>(smem + MC_OFF_NV);
     float* sConst = reinterpret_cast<float*>(smem + MC_OFF_CONST);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -645,23 +712,13 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             for (int j = 0; j < 2 && !failed; ++j) {
                 if (!mbar_wait(bar(MC_FULL + j), pitem & 1)) { failed = true; fail_site = __LINE__; break; }
                 const uint8_t* vt = smem + MC_OFF_V + j * kOperandBytes;
-                float* nvdst = sNv + ((pitem & 1) * 2 + j) * TILE;
+                float2* nvdst = sNv + ((pitem & 1) * 2 + j) * TILE;
 #pragma unroll
                 for (int jj = 0; jj < 2; ++jj) {
                     const int tok = t64 + 64 * jj;
-                    float2 acc0 = make_float2(0.f, 0.f), acc1 = acc0, acc2 = acc0, acc3 = acc0;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int ch = 0; ch < 8; ++ch) {
-                            const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
-                            const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
-                            const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
-                            acc0 = __ffma2_rn(f0, f0, acc0); acc1 = __ffma2_rn(f1, f1, acc1);
-                            acc2 = __ffma2_rn(f2, f2, acc2); acc3 = __ffma2_rn(f3, f3, acc3);
-                        }
-                    const float2 sum = __fadd2_rn(__fadd2_rn(acc0, acc1), __fadd2_rn(acc2, acc3));
-                    nvdst[tok] = sum.x + sum.y;
+                    float l2, l1;
+                    value_norms<(VARS & OBC_VAR_VATP) != 0>(vt, tok, l2, l1);
+                    nvdst[tok] = make_float2(l2, l1);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(MC_EMPTY + j));
@@ -715,7 +772,8 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             }
             if (failed) break;
             if (!mbar_wait(bar(MC_NV + (pitem & 1)), (pitem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
-            const float nv = sNv[((pitem & 1) * 2 + wg) * TILE + tok];
+            const float2 nv21 = sNv[((pitem & 1) * 2 + wg) * TILE + tok];
+            const float nv = nv21.x, nv1 = nv21.y;
             if (ptok < p.Nmax) {
                 float* out = p.scores + (size_t)unit * p.Nmax;
                 const bool live = ptok < N;
@@ -727,6 +785,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] =
                     live ? fmaf(nv, S.s1.x + S.s1.y, fmaf(p.scale, S.s2.x + S.s2.y, s2 * (S.s3.x + S.s3.y))) : 0.f;
                 if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? S.s7.x + S.s7.y : 0.f;
+                if (p.variants & OBC_VAR_VATP) out[(size_t)(pl++) * plane + ptok] = live ? nv1 * (S.s7.x + S.s7.y) : 0.f;
             }
         }
         // padding beyond the last tile of a shorter sequence: zeros
@@ -975,7 +1034,6 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int ch = 0; ch < 8; ++ch) {
-                            // any order of the row's 16-byte chunks gives the same sum; this one is bank-conflict free
                             const uint4 u = *reinterpret_cast<const uint4*>(vt + h * kHalfBytes + tok * 128 + ((ch ^ (tok & 7)) << 4));
                             const float2 f0 = bf16x2_to_f32x2(u.x), f1 = bf16x2_to_f32x2(u.y);
                             const float2 f2 = bf16x2_to_f32x2(u.z), f3 = bf16x2_to_f32x2(u.w);
@@ -1267,7 +1325,7 @@ static SimtPlan make_tc_plan(const ScoreShape& s) {
 size_t tc_workspace_bytes(const ScoreShape& s) { return make_tc_plan(s).bytes; }
 
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
-                           float* scores, void* ws, cudaStream_t stream) {
+                           float* scores, void* ws, cudaStream_t stream, const GivenAttention* given) {
     const TcChunks ch = tc_chunks(s.R);
     const SimtPlan plan = make_tc_plan(s);
     char* wsb = (char*)ws;
@@ -1290,7 +1348,10 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
             return OBC_ERR_CUDA;
         }
     }
-    {   // pass 1 + combine
+    if (given) {   // the caller's O and LSE take the place of pass 1 + combine; pass 2 computes the value norms itself
+        obc_status st = launch_given_prep(s, plan, *given, ws, stream);
+        if (st != OBC_OK) return st;
+    } else {       // pass 1 + combine
         P1Params p1{};
         p1.B = s.B; p1.Hq = s.Hq; p1.Hkv = s.Hkv; p1.G = s.G; p1.W = s.W; p1.R = s.R; p1.Nmax = s.Nmax;
         p1.seq_lens = s.seq_lens; p1.scale = s.scale; p1.causal = s.causal;
@@ -1339,7 +1400,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         };
         if (s.variants == OBC_VAR_VK) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_VK>);
         if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_K | OBC_VAR_VK>);
-        return launch_multi(tc_pass2_multi_kernel<OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN>);
+        return launch_multi(tc_pass2_multi_kernel<kAllVariants>);
     }
 
     auto launch = [&](auto kernel) -> obc_status {
@@ -1347,9 +1408,16 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         { ProfScope ps("tc_pass2", stream); OBC_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mq, mo, mk, mv, p)); }
         return OBC_OK;
     };
-    if (s.variants == OBC_VAR_VK) return launch(tc_pass2_kernel<OBC_VAR_VK>);
-    if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch(tc_pass2_kernel<OBC_VAR_K | OBC_VAR_VK>);
-    return launch(tc_pass2_kernel<OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN>);
+    if (given) {
+        if (s.variants == OBC_VAR_VK) return launch(tc_pass2_kernel<OBC_VAR_VK, true>);
+        if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch(tc_pass2_kernel<OBC_VAR_K | OBC_VAR_VK, true>);
+        return launch(tc_pass2_kernel<kAllVariants, true>);
+    }
+    if (s.variants == OBC_VAR_VK) return launch(tc_pass2_kernel<OBC_VAR_VK, false>);
+    if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch(tc_pass2_kernel<OBC_VAR_K | OBC_VAR_VK, false>);
+    // pass 1 leaves only ||v||^2; the l1 variant takes both norms from the V tiles in pass 2
+    if (s.variants & OBC_VAR_VATP) return launch(tc_pass2_kernel<kAllVariants, true>);
+    return launch(tc_pass2_kernel<kAllVariants & ~OBC_VAR_VATP, false>);
 }
 
 }  // namespace obc
