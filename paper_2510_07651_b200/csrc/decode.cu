@@ -78,6 +78,42 @@ __device__ __forceinline__ void store_rows(uint4* dst, const uint4 (&v)[16]) {
 }
 __device__ __forceinline__ uint4 staged_chunk(const uint4* src, int r, int c) { return src[r * 16 + (c ^ (r & 15))]; }
 
+// ---- warp-level tensor-core pieces ------------------------------------------------------------------
+// The contractions of a chunk are tiny (256 slots x at most 8 heads x 128 channels) and the kernels are
+// bound by memory traffic, but on CUDA cores their instruction count (about 3000 per thread and chunk)
+// was what limited the blocks in flight.  One m16n8k16 MMA per 16 slots and 16 channels replaces 128
+// multiply-adds per lane; the operands come out of the staged rows with ldmatrix (the 16-byte pieces of
+// the swizzled rows are exactly its 8x8 tiles).
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void* p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], const void* p) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+// d += a (16x16, row-major) * b (16x8, column-major), bf16 operands, fp32 accumulators
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// address of the 8x8 tile that lane `lane` names for an x4 load covering 16 staged rows from `row0` and the two
+// 16-byte pieces `piece0`, `piece0 + 1`.  rows_major: tiles ordered (rows 0-7, p0), (rows 8-15, p0), (rows 0-7, p1),
+// (rows 8-15, p1), the A operand of slots x channels; otherwise (rows 0-7, p0), (rows 0-7, p1), (rows 8-15, p0), ...
+__device__ __forceinline__ const uint4* tile_addr(const uint4* sRows, int row0, int piece0, int lane, bool rows_major) {
+    const int mi = lane >> 3, rr = lane & 7;
+    const int row = row0 + (rows_major ? (mi & 1) : (mi >> 1)) * 8 + rr;
+    const int piece = piece0 + (rows_major ? (mi >> 1) : (mi & 1));
+    return sRows + row * 16 + (piece ^ (row & 15));
+}
+// x = hi + lo with both halves bf16: two MMAs then carry an fp32 operand to about 16 bits
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
 template <int G>
 __global__ void __launch_bounds__(CH)
 decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt, TensorView vt,
@@ -85,7 +121,6 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
                     int step_pos, char* ws) {
     pdl_wait();
     extern __shared__ __align__(16) uint4 sRows[];                      // [CH][16]: the chunk's K rows
-    __shared__ __align__(16) float sQ[G][kD];
     __shared__ float sP[G][CH];
     __shared__ __align__(16) float sO[8][G][kD];
     __shared__ float sRed[8][G];
@@ -104,9 +139,16 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         if (tid < G) { part_m[tid] = -INFINITY; part_l[tid] = 0.f; }
         return;
     }
-    for (int i = tid; i < G * kD; i += CH) {
-        const int r = i / kD, c = i % kD;
-        sQ[r][c] = __bfloat162float(bf_row(q, b, g * G + r, 0)[c]);
+    // B operand of the logits: lane (n = lane / 4, t = lane % 4) holds q_n[16 ks + 2t .. +1] and [.. + 8 .. +9]
+    uint32_t qf[8][2];
+    {
+        const int n = lane >> 2, t = lane & 3;
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(bf_row(q, b, g * G + (n < G ? n : 0), 0));
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qf[ks][0] = n < G ? qrow[ks * 8 + t] : 0u;
+            qf[ks][1] = n < G ? qrow[ks * 8 + 4 + t] : 0u;
+        }
     }
     if (valid && next >= c0 && next < c0 + CH) {       // this chunk owns the slot of the new token
         __nv_bfloat16* kdst = const_cast<__nv_bfloat16*>(bf_row(kc, b, g, next));
@@ -125,28 +167,26 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
     const int slot = c0 + tid;
     const bool live = slot < hi && ((valid && slot == next) || pos[(size_t)unit * s.cap + slot] >= 0);
     const float sl2 = s.scale * kLog2e;
+    // logits of the warp's 32 slots: two 16-slot tiles, eight 16-channel steps each
+#pragma unroll
+    for (int tile = 0; tile < 2; ++tile) {
+        const int row0 = warp * 32 + tile * 16;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a[4];
+            ldsm_x4(a, tile_addr(sRows, row0, 2 * ks, lane, true));
+            mma_bf16(acc, a, qf[ks][0], qf[ks][1]);
+        }
+        // acc[0], acc[1]: slot row0 + lane / 4, heads 2 (lane % 4), + 1; acc[2], acc[3]: slot + 8
+        const int sl = row0 + (lane >> 2), h0 = 2 * (lane & 3);
+        if (h0 < G) { sP[h0][sl] = acc[0]; sP[h0][sl + 8] = acc[2]; }
+        if (h0 + 1 < G) { sP[h0 + 1][sl] = acc[1]; sP[h0 + 1][sl + 8] = acc[3]; }
+    }
+    __syncthreads();
     float z2[G];
 #pragma unroll
-    for (int r = 0; r < G; ++r) z2[r] = 0.f;
-    if (live) {
-        float2 zz[G];                                      // two partial dot products per row (packed fp32x2)
-#pragma unroll
-        for (int r = 0; r < G; ++r) zz[r] = make_float2(0.f, 0.f);
-#pragma unroll 4
-        for (int c = 0; c < 16; ++c) {
-            float2 kf[4];
-            unpack8x2(staged_chunk(sRows, tid, c), kf);
-#pragma unroll
-            for (int r = 0; r < G; ++r) {
-                const float4 qa = *reinterpret_cast<const float4*>(&sQ[r][c * 8]);
-                const float4 qb = *reinterpret_cast<const float4*>(&sQ[r][c * 8 + 4]);
-                zz[r] = __ffma2_rn(make_float2(qa.x, qa.y), kf[0], zz[r]); zz[r] = __ffma2_rn(make_float2(qa.z, qa.w), kf[1], zz[r]);
-                zz[r] = __ffma2_rn(make_float2(qb.x, qb.y), kf[2], zz[r]); zz[r] = __ffma2_rn(make_float2(qb.z, qb.w), kf[3], zz[r]);
-            }
-        }
-#pragma unroll
-        for (int r = 0; r < G; ++r) z2[r] = zz[r].x + zz[r].y;
-    }
+    for (int r = 0; r < G; ++r) z2[r] = sP[r][tid];        // this thread's slot; sP[.][tid] is rewritten below by this thread only
     float* zbuf = (float*)(ws + plan.off_z) + (size_t)unit * G * s.cap;
 #pragma unroll
     for (int r = 0; r < G; ++r) {
@@ -174,30 +214,36 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
 #pragma unroll
     for (int r = 0; r < G; ++r) if (lane == 0) sRed[warp][r] = lsum[r];
 
-    // partial outputs: warp w covers slots c0+32w .. +31, lane owns channels 4*lane .. +3
-    const unsigned live_mask = __ballot_sync(0xffffffffu, live);
-    float o[G][4];
-#pragma unroll
-    for (int r = 0; r < G; ++r) { o[r][0] = o[r][1] = o[r][2] = o[r][3] = 0.f; }
+    // partial outputs of the warp's 32 slots, transposed: (16 channels) x (8 heads) tiles of V^T P^T.  The
+    // probabilities enter as bf16 high and low halves; slots without a live token carry p = 0.
     __syncthreads();                                       // V rows staged
-    for (int t = 0; t < 32; ++t) {
-        if (!((live_mask >> t) & 1u)) continue;
-        // channels 4*lane .. +3 of slot row: half (lane & 1) of the 16-byte chunk lane / 2
-        const int row = warp * 32 + t;
-        const uint2 raw = reinterpret_cast<const uint2*>(&sRows[row * 16 + ((lane >> 1) ^ (row & 15))])[lane & 1];
-        float4 vv;
-        vv.x = __uint_as_float(raw.x << 16); vv.y = __uint_as_float(raw.x & 0xffff0000u);
-        vv.z = __uint_as_float(raw.y << 16); vv.w = __uint_as_float(raw.y & 0xffff0000u);
+    {
+        uint32_t ph[2][2], pl[2][2];                       // [16-slot step][k half]: p of head lane / 4, slots 2 (lane % 4), + 1 (+ 8)
+        const int n = lane >> 2, t = lane & 3;
 #pragma unroll
-        for (int r = 0; r < G; ++r) {
-            const float p = sP[r][warp * 32 + t];
-            o[r][0] = fmaf(p, vv.x, o[r][0]); o[r][1] = fmaf(p, vv.y, o[r][1]);
-            o[r][2] = fmaf(p, vv.z, o[r][2]); o[r][3] = fmaf(p, vv.w, o[r][3]);
+        for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const int sl = warp * 32 + kk * 16 + hf * 8 + 2 * t;
+                const float p0 = n < G ? sP[n][sl] : 0.f, p1 = n < G ? sP[n][sl + 1] : 0.f;
+                split_bf16x2(p0, p1, ph[kk][hf], pl[kk][hf]);
+            }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {                      // channels 16 j .. 16 j + 15
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+                uint32_t a[4];
+                ldsm_x4_trans(a, tile_addr(sRows, warp * 32 + kk * 16, 2 * j, lane, false));
+                mma_bf16(acc, a, ph[kk][0], ph[kk][1]);
+                mma_bf16(acc, a, pl[kk][0], pl[kk][1]);
+            }
+            // acc[0], acc[1]: channel 16 j + lane / 4, heads 2 (lane % 4), + 1; acc[2], acc[3]: channel + 8
+            const int ch = 16 * j + (lane >> 2), h0 = 2 * t;
+            if (h0 < G) { sO[warp][h0][ch] = acc[0]; sO[warp][h0][ch + 8] = acc[2]; }
+            if (h0 + 1 < G) { sO[warp][h0 + 1][ch] = acc[1]; sO[warp][h0 + 1][ch + 8] = acc[3]; }
         }
     }
-#pragma unroll
-    for (int r = 0; r < G; ++r)
-        *reinterpret_cast<float4*>(&sO[warp][r][lane * 4]) = make_float4(o[r][0], o[r][1], o[r][2], o[r][3]);
     __syncthreads();
     float* part_o = (float*)(ws + plan.off_po) + ((size_t)unit * plan.chunks + chunk) * G * kD;
     for (int i = tid; i < G * kD; i += CH) {
