@@ -316,13 +316,13 @@ decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
 }
 
 template <int G>
-__global__ void __launch_bounds__(CH)
+__global__ void __launch_bounds__(CH, 3)
 decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc, const int32_t* pos,
                     const int32_t* state, int step_pos, char* ws) {
     pdl_wait();
     extern __shared__ __align__(16) uint4 sRows[];                      // [CH][16]: the chunk's V rows
-    __shared__ __align__(16) float sO[G][kD];
     __shared__ float sLse[G], sNo[G];
+    __shared__ float sT[G + 1][CH];                                     // v_slot . o_r (r < G) and ||v_slot||^2
     __shared__ MinCand sMin[8];
 
     const int unit = blockIdx.y, chunk = blockIdx.x, c0 = chunk * CH;
@@ -336,7 +336,6 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
         if (tid == 0) *part_min = MinCand{INFINITY, -1, -1, 0};
         return;
     }
-    for (int i = tid; i < G * kD; i += CH) sO[i / kD][i % kD] = ((const float*)(ws + plan.off_o))[(size_t)unit * G * kD + i];
     if (tid < G) {
         sLse[tid] = ((const float*)(ws + plan.off_lse))[(size_t)unit * G + tid];
         sNo[tid] = ((const float*)(ws + plan.off_no))[(size_t)unit * G + tid];
@@ -346,34 +345,56 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
         load_rows(stage, vc, b, g, c0, hi);
         store_rows(sRows, stage);
     }
+    // B operand of v . o: lane (n = lane / 4, t = lane % 4) holds o_n[16 ks + 2t .. +1] and [.. + 8 .. +9],
+    // each fp32 value as a bf16 high and low half
+    uint32_t oh[8][2], ol[8][2];
+    {
+        const int n = lane >> 2, t = lane & 3;
+        const float2* orow = reinterpret_cast<const float2*>((const float*)(ws + plan.off_o) + ((size_t)unit * G + (n < G ? n : 0)) * kD);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const float2 o2 = n < G ? orow[ks * 8 + hf * 4 + t] : make_float2(0.f, 0.f);
+                split_bf16x2(o2.x, o2.y, oh[ks][hf], ol[ks][hf]);
+            }
+    }
     __syncthreads();
 
     const int slot = c0 + tid;
     const int my_pos = slot < hi ? pos[(size_t)unit * s.cap + slot] : -1;
     const bool live = my_pos >= 0;
     MinCand cand{INFINITY, -1, -1, 0};
-    if (live) {
-        float nv, t[G];
-        float2 nn = make_float2(0.f, 0.f), tt[G];          // packed fp32x2 partial sums
+    // v . o_r and ||v||^2 of the warp's 32 slots: two 16-slot tiles, eight 16-channel steps each.  The norms are
+    // the diagonal of (tile) x (tile)^T, whose B operand is the tile's own A fragment.
 #pragma unroll
-        for (int r = 0; r < G; ++r) tt[r] = make_float2(0.f, 0.f);
-#pragma unroll 4
-        for (int c = 0; c < 16; ++c) {
-            float2 vf[4];
-            unpack8x2(staged_chunk(sRows, tid, c), vf);
+    for (int tile = 0; tile < 2; ++tile) {
+        const int row0 = warp * 32 + tile * 16;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f}, n_lo[4] = {0.f, 0.f, 0.f, 0.f}, n_hi[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) nn = __ffma2_rn(vf[j], vf[j], nn);
-#pragma unroll
-            for (int r = 0; r < G; ++r) {
-                const float4 oa = *reinterpret_cast<const float4*>(&sO[r][c * 8]);
-                const float4 ob = *reinterpret_cast<const float4*>(&sO[r][c * 8 + 4]);
-                tt[r] = __ffma2_rn(make_float2(oa.x, oa.y), vf[0], tt[r]); tt[r] = __ffma2_rn(make_float2(oa.z, oa.w), vf[1], tt[r]);
-                tt[r] = __ffma2_rn(make_float2(ob.x, ob.y), vf[2], tt[r]); tt[r] = __ffma2_rn(make_float2(ob.z, ob.w), vf[3], tt[r]);
-            }
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a[4];
+            ldsm_x4(a, tile_addr(sRows, row0, 2 * ks, lane, true));
+            mma_bf16(acc, a, oh[ks][0], oh[ks][1]);
+            mma_bf16(acc, a, ol[ks][0], ol[ks][1]);
+            mma_bf16(n_lo, a, a[0], a[2]);                 // columns = slots row0 .. + 7
+            mma_bf16(n_hi, a, a[1], a[3]);                 // columns = slots row0 + 8 .. + 15
         }
-        nv = nn.x + nn.y;
+        // acc[0], acc[1]: slot row0 + lane / 4, heads 2 (lane % 4), + 1; acc[2], acc[3]: slot + 8
+        const int gq = lane >> 2, tq = lane & 3, sl = row0 + gq, h0 = 2 * tq;
+        if (h0 < G) { sT[h0][sl] = acc[0]; sT[h0][sl + 8] = acc[2]; }
+        if (h0 + 1 < G) { sT[h0 + 1][sl] = acc[1]; sT[h0 + 1][sl + 8] = acc[3]; }
+        // the lane whose column pair 2 tq, 2 tq + 1 contains its own row holds the diagonal entries
+        if (tq == (gq >> 1)) {
+            sT[G][sl] = (gq & 1) ? n_lo[1] : n_lo[0];
+            sT[G][sl + 8] = (gq & 1) ? n_hi[3] : n_hi[2];
+        }
+    }
+    __syncthreads();
+    if (live) {
+        float nv = sT[G][tid], t[G];
 #pragma unroll
-        for (int r = 0; r < G; ++r) t[r] = tt[r].x + tt[r].y;
+        for (int r = 0; r < G; ++r) t[r] = sT[r][tid];
         const float* zbuf = (const float*)(ws + plan.off_z) + (size_t)unit * G * s.cap;
         float sc = 0.f;
 #pragma unroll
