@@ -2,9 +2,11 @@
 // cache).  Sec. 3 "Decoding" / "Cache Eviction"; Sec. 4.2 (scores accumulated over steps);
 // App. C.2.2 (sinks + recent window protected, one eviction per step once over budget).
 //
-// CUDA cores only: with G <= 8 score rows per KV head the contractions are matrix-vector
-// products bound by HBM traffic, so one thread owns one cache slot (a 256-byte K or V row read
-// as 16-byte vectors) and reductions over slots use warp shuffles.
+// With G <= 8 score rows per KV head the contractions are thin (slots x heads x 128 channels) and
+// the step is bound by HBM traffic.  A CTA takes one chunk of 256 slots of one KV head: the 256-byte
+// K or V rows are staged in shared memory (16-byte pieces XOR-swizzled by row) and the contractions
+// run as warp-level m16n8k16 MMAs fed by ldmatrix; one thread per slot does the softmax and score
+// arithmetic, and reductions over slots use warp shuffles.
 //
 //   decode_pass1   append (k_t, v_t); logits of every live slot (kept in the workspace so K is
 //                  read once); per-chunk softmax statistics and partial outputs
@@ -44,14 +46,6 @@ DecodePlan make_plan(const DecodeShape& s) {
 
 struct MinCand { float val; int pos; int slot; int pad; };
 
-// four packed pairs (lo, hi) of the eight bf16 of a 16-byte chunk
-__device__ __forceinline__ void unpack8x2(uint4 u, float2 (&f)[4]) {
-    f[0] = make_float2(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
-    f[1] = make_float2(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
-    f[2] = make_float2(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
-    f[3] = make_float2(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
-}
-
 __device__ __forceinline__ const __nv_bfloat16* bf_row(const TensorView& t, int b, int h, long long tok) {
     return reinterpret_cast<const __nv_bfloat16*>(t.ptr) + b * t.sb + h * t.sh + tok * t.st;
 }
@@ -59,8 +53,8 @@ __device__ __forceinline__ const __nv_bfloat16* bf_row(const TensorView& t, int 
 // Cooperative copy of the 256-byte rows [c0, c0 + CH) of one cache into shared memory, in two steps so
 // that the caller can put work between them: load_rows issues all 16 loads of a thread before any
 // use (a warp reads two whole rows per instruction, coalesced; rows at or beyond `hi` are not
-// read), store_rows puts the 16-byte chunk c of row r at chunk c ^ (r & 15), so that the thread
-// that owns row r later reads its row without bank conflicts.
+// read), store_rows puts the 16-byte chunk c of row r at chunk c ^ (r & 15), so that the eight
+// rows of an 8x8 tile fall into distinct banks when ldmatrix reads them.
 __device__ __forceinline__ void load_rows(uint4 (&v)[16], const TensorView& t, int b, int g, int c0, int hi) {
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
@@ -76,7 +70,6 @@ __device__ __forceinline__ void store_rows(uint4* dst, const uint4 (&v)[16]) {
         dst[r * 16 + (c ^ (r & 15))] = v[k];
     }
 }
-__device__ __forceinline__ uint4 staged_chunk(const uint4* src, int r, int c) { return src[r * 16 + (c ^ (r & 15))]; }
 
 // ---- warp-level tensor-core pieces ------------------------------------------------------------------
 // The contractions of a chunk are tiny (256 slots x at most 8 heads x 128 channels) and the kernels are
