@@ -81,3 +81,9 @@ def test_decode_multi_chunk_steady_state():
 @pytest.mark.parametrize("variant", ["V", "K", "ATTN"])
 def test_decode_other_variants(variant):
     _run(B=1, Hq=7, Hkv=1, n0=300, budget=310, cap=330, n_sink=2, n_recent=16, steps=20, variant=variant)
+
+
+@pytest.mark.parametrize("G", [1, 2, 3, 5, 6, 8])
+def test_decode_every_group_size(G):
+    # the MMA tiles pad the query heads of a group to 8 columns: every group size, two chunks, an odd extent
+    _run(B=1, Hq=2 * G, Hkv=2, n0=290, budget=300, cap=301, n_sink=3, n_recent=20, steps=24)
