@@ -20,6 +20,8 @@
  *   scores from a given O/LSE  Eq. 4-6 with A = exp(Z - lse) and o_i as supplied by the caller
  *                              (the attention kernel's own outputs instead of a recompute)
  *   GQA reduction              App. A.5 (sum over the query heads of a KV head's group)
+ *   head-adaptive select       the AdaKV budget allocation the paper pairs its scores with (Sec. 5.1,
+ *                              App. C.2.1): global ranking across heads with a per-head safeguard
  *   pool / select / compact    Algorithm 2 (top-k below the cutoff, indices sorted ascending,
  *                              gather, recent tail appended) with SnapKV-style 1-D pooling
  *   decode step pieces         Sec. 3 "Decoding"/"Cache Eviction", Sec. 4.2 last paragraph
@@ -331,6 +333,70 @@ int obc_oracle_select(const float* pooled, int N, int budget, int n_sink, int n_
     for (; w < idx_len; ++w) idx[w] = -1;
     free(c);
     return 0;
+}
+
+/* ------------------------------------------------------------------ head-adaptive select */
+typedef struct { float s; int32_t h; int32_t i; } hcand_t;
+static int hcand_cmp(const void* a, const void* b) {
+    const hcand_t* x = (const hcand_t*)a; const hcand_t* y = (const hcand_t*)b;
+    if (x->s > y->s) return -1;
+    if (x->s < y->s) return 1;
+    if (x->h != y->h) return (x->h > y->h) - (x->h < y->h);  /* equal scores: lowest head, then lowest index */
+    return (x->i > y->i) - (x->i < y->i);
+}
+
+/*
+ * Head-adaptive budgets (the AdaKV allocation of App. C.2.1 and Sec. 5.1: the top-k eviction scores are
+ * ranked globally across the heads of a layer, with a safeguard fraction of the budget guaranteed to
+ * every head), for one batch item.
+ *   pooled [H, N]   the heads' pooled scores (row stride N)
+ *   budget          kept tokens per head on average; n_hh = budget - n_sink - n_recent slots per head
+ *                   are for scored tokens, H * n_hh in total
+ *   safeguard       fraction of n_hh every head keeps by its own ranking: s = floor(safeguard * n_hh)
+ * Every head first takes its s best candidates of [n_sink, N - n_recent) (ties: lowest index); the
+ * other H * (n_hh - s) slots go to the best remaining candidates of all heads ranked together (ties:
+ * lowest head, then lowest index).  idx [H, idx_len]: per head the sinks, the selected tokens in
+ * ascending order and the recent tail, padded with -1; counts [H] = kept tokens of the head.
+ * Returns 0, or -1 on bad arguments or when a head would keep more than idx_len tokens.
+ */
+int obc_oracle_select_adaptive(const float* pooled, int H, int N, int budget, int n_sink, int n_recent,
+                               float safeguard, int32_t* idx, int32_t* counts, int idx_len) {
+    if (!pooled || !idx || !counts || H < 1 || N < 1 || budget > N) return -1;
+    if (n_sink < 0 || n_recent < 0 || budget < n_sink + n_recent) return -1;
+    if (!(safeguard >= 0.0f && safeguard <= 1.0f)) return -1;
+    const int lo = n_sink, hi = N - n_recent, n_hh = budget - n_sink - n_recent, n = hi - lo;
+    if (n < n_hh) return -1;
+    int s = (int)floor((double)safeguard * (double)n_hh);
+    if (s > n_hh) s = n_hh;
+    const long extra = (long)H * (n_hh - s);
+    char* taken = (char*)calloc((size_t)H * (size_t)(n > 0 ? n : 1), 1);
+    cand_t* c = (cand_t*)malloc(sizeof(cand_t) * (size_t)(n > 0 ? n : 1));
+    hcand_t* rest = (hcand_t*)malloc(sizeof(hcand_t) * (size_t)H * (size_t)(n > 0 ? n : 1));
+    if (!taken || !c || !rest) { free(taken); free(c); free(rest); return -1; }
+    long n_rest = 0;
+    for (int h = 0; h < H; ++h) {                          /* the safeguarded share of every head */
+        for (int p = lo; p < hi; ++p) { c[p - lo].s = pooled[(long)h * N + p]; c[p - lo].i = p; }
+        qsort(c, (size_t)n, sizeof(cand_t), cand_cmp);
+        for (int j = 0; j < s; ++j) taken[(long)h * n + (c[j].i - lo)] = 1;
+        for (int j = s; j < n; ++j) { rest[n_rest].s = c[j].s; rest[n_rest].h = h; rest[n_rest].i = c[j].i; ++n_rest; }
+    }
+    qsort(rest, (size_t)n_rest, sizeof(hcand_t), hcand_cmp);   /* all heads ranked together */
+    for (long j = 0; j < extra; ++j) taken[(long)rest[j].h * n + (rest[j].i - lo)] = 1;
+    int rc = 0;
+    for (int h = 0; h < H && rc == 0; ++h) {
+        int w = 0;
+        int32_t* out = idx + (long)h * idx_len;
+        int kept = n_sink + n_recent;
+        for (int p = 0; p < n; ++p) kept += taken[(long)h * n + p];
+        if (kept > idx_len) { rc = -1; break; }
+        for (int p = 0; p < n_sink; ++p) out[w++] = p;
+        for (int p = lo; p < hi; ++p) if (taken[(long)h * n + (p - lo)]) out[w++] = p;
+        for (int p = hi; p < N; ++p) out[w++] = p;
+        counts[h] = w;
+        for (; w < idx_len; ++w) out[w] = -1;
+    }
+    free(taken); free(c); free(rest);
+    return rc;
 }
 
 /* ------------------------------------------------------------------ compact */

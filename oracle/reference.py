@@ -45,6 +45,7 @@ def lib():
                                              C.c_double, C.c_int, C.c_int, dp, dp, dp, dp, dp, C.c_int]
         L.obc_oracle_pool.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, fp]
         L.obc_oracle_select.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, ip, C.c_int]
+        L.obc_oracle_select_adaptive.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, ip, ip, C.c_int]
         L.obc_oracle_compact.argtypes = [C.c_void_p, C.c_int, C.c_int, ip, C.c_int, C.c_void_p]
         L.obc_oracle_decode_scores.argtypes = [fp, fp, fp, ip, C.c_int, C.c_int, C.c_int, C.c_int,
                                                C.c_double, C.c_int, dp]
@@ -158,6 +159,33 @@ def select_pipeline(scores, seq_lens, budgets, n_sink, n_recent, pool_mode, pool
             pooled = pool(s, n_sink, n - n_recent, pool_mode, pool_kernel)
             idx[b, h] = select(pooled, int(budgets[b]), n_sink, n_recent, idx_len)
     return idx
+
+
+def select_adaptive(pooled, budget, n_sink, n_recent, safeguard, idx_len):
+    """Head-adaptive selection for one batch item: pooled [H,N] -> (idx [H,idx_len], counts [H])."""
+    s, sp = _f(pooled)
+    H, N = s.shape
+    idx = np.empty((H, idx_len), dtype=np.int32)
+    counts = np.empty(H, dtype=np.int32)
+    rc = lib().obc_oracle_select_adaptive(sp, H, N, budget, n_sink, n_recent, float(safeguard),
+                                          idx.ctypes.data_as(C.POINTER(C.c_int32)),
+                                          counts.ctypes.data_as(C.POINTER(C.c_int32)), idx_len)
+    if rc != 0:
+        raise ValueError("obc_oracle_select_adaptive rejected its arguments")
+    return idx, counts
+
+
+def select_adaptive_pipeline(scores, seq_lens, budgets, n_sink, n_recent, pool_mode, pool_kernel, safeguard, idx_len):
+    """pool + head-adaptive select for scores [B,Hkv,Nmax] -> (idx [B,Hkv,idx_len], counts [B,Hkv])."""
+    B, H, _ = scores.shape
+    idx = np.full((B, H, idx_len), -1, dtype=np.int32)
+    counts = np.zeros((B, H), dtype=np.int32)
+    for b in range(B):
+        n = int(seq_lens[b])
+        pooled = np.stack([pool(np.ascontiguousarray(scores[b, h, :n], dtype=np.float32), n_sink, n - n_recent,
+                                pool_mode, pool_kernel) for h in range(H)])
+        idx[b], counts[b] = select_adaptive(pooled, int(budgets[b]), n_sink, n_recent, safeguard, idx_len)
+    return idx, counts
 
 
 def decode_scores(qg, kc, vc, pos, hi, variant="VK", scale=0.0):

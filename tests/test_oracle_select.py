@@ -136,3 +136,84 @@ def test_decode_state_keeps_sinks_and_recents_and_respects_budget():
         assert len(set(livepos.tolist())) == budget
         assert set(range(n_sink)) <= set(livepos.tolist())
         assert set(range(step_pos - n_recent + 1, step_pos + 1)) <= set(livepos.tolist())
+
+
+# ---- head-adaptive budgets (global ranking across heads with a per-head safeguard) ----------------
+def brute_adaptive(pooled, budget, n_sink, n_recent, safeguard):
+    """Plain-Python statement: every head's s best candidates, then the best of the rest of all heads."""
+    H, N = pooled.shape
+    lo, hi, n_hh = n_sink, N - n_recent, budget - n_sink - n_recent
+    s = int(np.floor(float(np.float32(safeguard)) * n_hh))
+    kept = [set() for _ in range(H)]
+    rest = []
+    for h in range(H):
+        order = sorted(range(lo, hi), key=lambda p: (-float(pooled[h, p]), p))
+        kept[h].update(order[:s])
+        rest += [(-float(pooled[h, p]), h, p) for p in order[s:]]
+    for _, h, p in sorted(rest)[:H * (n_hh - s)]:
+        kept[h].add(p)
+    return [np.array(list(range(n_sink)) + sorted(k) + list(range(hi, N)), np.int32) for k in kept]
+
+
+@pytest.mark.parametrize("seed", range(3))
+@pytest.mark.parametrize("safeguard", [0.0, 0.2, 0.5, 1.0])
+def test_adaptive_select_matches_brute_force_with_ties(seed, safeguard):
+    rng = np.random.default_rng(100 + seed)
+    H, N = 3, 120
+    pooled = rng.integers(0, 9, (H, N)).astype(np.float32) / 4          # many ties, within and across heads
+    pooled[1] *= 2.0                                                     # one head scores higher overall
+    for budget, n_sink, n_recent in [(30, 0, 8), (40, 4, 16), (N, 0, 0), (25, 4, 20)]:
+        idx_len = n_sink + n_recent + H * (budget - n_sink - n_recent)
+        idx_len = min(idx_len, N)
+        idx, counts = ref.select_adaptive(pooled, budget, n_sink, n_recent, safeguard, idx_len)
+        want = brute_adaptive(pooled, budget, n_sink, n_recent, safeguard)
+        assert counts.sum() == H * budget
+        for h in range(H):
+            assert counts[h] == len(want[h])
+            assert (idx[h, :counts[h]] == want[h]).all() and (idx[h, counts[h]:] == -1).all()
+
+
+def test_adaptive_select_limits():
+    rng = np.random.default_rng(7)
+    H, N, budget, n_sink, n_recent = 4, 200, 50, 2, 10
+    pooled = rng.random((H, N), dtype=np.float32)
+    # safeguard 1: every head keeps exactly its own top budget, i.e. the per-head selection
+    idx, counts = ref.select_adaptive(pooled, budget, n_sink, n_recent, 1.0, budget)
+    for h in range(H):
+        assert counts[h] == budget and (idx[h] == ref.select(pooled[h], budget, n_sink, n_recent)).all()
+    # safeguard 0 with distinct scores: the library's top-k over all heads' candidates at once
+    idx, counts = ref.select_adaptive(pooled, budget, n_sink, n_recent, 0.0, N)
+    n_hh = budget - n_sink - n_recent
+    flat = torch.from_numpy(pooled[:, n_sink:N - n_recent].copy()).reshape(-1)
+    top = torch.topk(flat, H * n_hh).indices.numpy()
+    n = N - n_sink - n_recent
+    for h in range(H):
+        want = np.sort(top[top // n == h] % n + n_sink)
+        got = idx[h, n_sink:counts[h] - n_recent]
+        assert (got == want).all()
+        assert (idx[h, :n_sink] == np.arange(n_sink)).all() and (idx[h, counts[h] - n_recent:counts[h]] == np.arange(N - n_recent, N)).all()
+
+
+def test_adaptive_select_moves_budget_to_the_head_that_scores_higher():
+    # head 0 scores 10 everywhere, head 1 scores 1: with a quarter safeguarded (1 of 4 slots), head 1 keeps
+    # its one guaranteed token and head 0 takes the other seven
+    pooled = np.stack([np.full(12, 10.0, np.float32), np.full(12, 1.0, np.float32)])
+    idx, counts = ref.select_adaptive(pooled, 4, 0, 0, 0.25, 8)
+    assert counts.tolist() == [7, 1]
+    assert idx[0, :7].tolist() == list(range(7)) and idx[1, 0] == 0 and (idx[1, 1:] == -1).all()
+    # a head may not outgrow the index buffer
+    with pytest.raises(ValueError):
+        ref.select_adaptive(pooled, 4, 0, 0, 0.25, 6)
+
+
+def test_adaptive_pipeline_pools_each_head_before_ranking():
+    rng = np.random.default_rng(11)
+    scores = rng.random((2, 3, 90), dtype=np.float32)
+    lens = np.array([90, 61], np.int32)
+    idx, counts = ref.select_adaptive_pipeline(scores, lens, [20, 15], 1, 6, "max", 5, 0.2, 60)
+    for b in range(2):
+        n = int(lens[b])
+        pooled = np.stack([ref.pool(scores[b, h, :n], 1, n - 6, "max", 5) for h in range(3)])
+        want = brute_adaptive(pooled, [20, 15][b], 1, 6, 0.2)
+        for h in range(3):
+            assert (idx[b, h, :counts[b, h]] == want[h]).all() and (idx[b, h, counts[b, h]:] == -1).all()
