@@ -177,6 +177,27 @@ obc_status obc_select_workspace(const obc_select_params* p, size_t* bytes /* hos
 obc_status obc_select(const obc_select_params* p, const float* scores, int32_t* idx,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * obc_select_adaptive: head-adaptive budgets, the AdaKV allocation that the paper pairs its scores
+ * with for its strongest results (Sec. 5.1 "Baselines"; App. C.2.1 "AdaKV": the top-k eviction scores
+ * are ranked globally across all heads of the layer; safeguard 0.2).  Per batch item, with
+ * n_hh = budget - n_sink - n_recent and H = n_kv_heads: every head first keeps its own
+ * floor(safeguard * n_hh) best candidates (pooled scores, ties: lowest index); the remaining
+ * H * n_hh - H * floor(..) slots go to the best remaining candidates of all heads ranked together
+ * (ties: lowest head, then lowest index).  A head keeps its sinks, its chosen tokens in ascending
+ * order and its recent tail.
+ *   p          as for obc_select; p->budgets must be NULL (one budget per call); p->idx_stride is
+ *              the most one head may keep (a head that would keep more gets a row of -1 and
+ *              counts = -1, as does a budget that does not fit its sequence)
+ *   idx        device int32 [B,Hkv,idx_stride], rows padded with -1 (obc_compact skips those)
+ *   counts     device int32 [B,Hkv]: tokens kept per head; they add up to Hkv * budget per batch item
+ *   workspace  device, 256-byte aligned, obc_select_adaptive_workspace() bytes
+ * ------------------------------------------------------------------------------------------ */
+obc_status obc_select_adaptive_workspace(const obc_select_params* p, float safeguard, size_t* bytes /* host out */);
+obc_status obc_select_adaptive(const obc_select_params* p, float safeguard, const float* scores,
+                               int32_t* idx, int32_t* counts, void* workspace, size_t workspace_bytes,
+                               void* stream);
+
 /*
  * obc_select_noalloc: obc_select for callers that have no device memory to give as workspace and
  * may not allocate any.  (The paper has no counterpart: this is a packaging variant of obc_select.)

@@ -24,7 +24,7 @@ POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
 EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_given", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
-           "obc_select_noalloc", "obc_compact",
+           "obc_select_noalloc", "obc_select_adaptive_workspace", "obc_select_adaptive", "obc_compact",
            "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
            "obc_status_string", "obc_last_cuda_error", "obc_version"]
 
@@ -88,6 +88,8 @@ def lib():
         L.obc_select_workspace.argtypes = [C.POINTER(obc_select_params), sz]
         L.obc_select.argtypes = [C.POINTER(obc_select_params), vp, vp, vp, C.c_size_t, vp]
         L.obc_select_noalloc.argtypes = [C.POINTER(obc_select_params), vp, vp, vp]
+        L.obc_select_adaptive_workspace.argtypes = [C.POINTER(obc_select_params), C.c_float, sz]
+        L.obc_select_adaptive.argtypes = [C.POINTER(obc_select_params), C.c_float, vp, vp, vp, vp, C.c_size_t, vp]
         L.obc_compact.argtypes = [C.c_int32] * 5 + [obc_tensor, obc_tensor, vp, obc_tensor, obc_tensor, vp, vp, vp]
         L.obc_decode_workspace.argtypes = [C.POINTER(obc_decode_params), sz]
         L.obc_decode_step.argtypes = [C.POINTER(obc_decode_params)] + [obc_tensor] * 5 + [vp, vp, vp, C.c_int32, vp, C.c_size_t, vp]
@@ -232,6 +234,25 @@ def obc_select(scores, *, budget=0, budgets=None, idx_stride=None, seq_lens=None
     _check(lib().obc_select(C.byref(p), scores.data_ptr(), idx.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
            "obc_select")
     return idx
+
+
+def obc_select_adaptive(scores, *, budget, safeguard=0.2, idx_stride=None, seq_lens=None, n_sink=0, n_recent=0,
+                        pool="none", pool_kernel=1, idx=None, counts=None, workspace=None):
+    """Head-adaptive budgets: scores fp32 [B,Hkv,Nmax] -> (idx int32 [B,Hkv,idx_stride] padded with -1,
+    counts int32 [B,Hkv]).  Every head keeps floor(safeguard * n_hh) tokens by its own ranking; the rest of the
+    layer's Hkv * n_hh slots go to the best remaining tokens of all heads together."""
+    p = select_params(scores, budget=budget, idx_stride=idx_stride, seq_lens=seq_lens, n_sink=n_sink,
+                      n_recent=n_recent, pool=pool, pool_kernel=pool_kernel)
+    if idx is None:
+        idx = torch.empty((p.batch, p.n_kv_heads, p.idx_stride), dtype=torch.int32, device=scores.device)
+    if counts is None:
+        counts = torch.empty((p.batch, p.n_kv_heads), dtype=torch.int32, device=scores.device)
+    n = C.c_size_t(0)
+    _check(lib().obc_select_adaptive_workspace(C.byref(p), float(safeguard), C.byref(n)), "obc_select_adaptive_workspace")
+    ws = _workspace(n.value, scores, workspace)
+    _check(lib().obc_select_adaptive(C.byref(p), float(safeguard), scores.data_ptr(), idx.data_ptr(), counts.data_ptr(),
+                                     ws.data_ptr(), ws.numel(), _stream()), "obc_select_adaptive")
+    return idx, counts
 
 
 SELECT_NOALLOC_MAX_KEYS = 1 << 20

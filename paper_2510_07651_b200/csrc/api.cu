@@ -2,6 +2,7 @@
 // Every function here runs on the host and only enqueues work; see include/obcache.h.
 #include "obc_common.cuh"
 #include <atomic>
+#include <cmath>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -201,6 +202,40 @@ obc_status obc_select(const obc_select_params* p, const float* scores, int32_t* 
     if (!workspace || workspace_bytes < select_workspace_bytes(s.B, s.Hkv, s.Nmax)) return OBC_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
     return launch_select(s, scores, idx, workspace, (cudaStream_t)stream);
+}
+
+// scored tokens every head keeps by its own ranking: floor(safeguard * n_hh), in double like the size query
+static obc_status resolve_adaptive(const obc_select_params* p, float safeguard, SelectShape* s, int* n_safe) {
+    obc_status st = resolve_select(p, s);
+    if (st != OBC_OK) return st;
+    if (p->budgets) return OBC_ERR_UNSUPPORTED;            // one budget for the whole batch
+    if (!(safeguard >= 0.f && safeguard <= 1.f)) return OBC_ERR_SHAPE;
+    if ((long long)s->Hkv * s->Nmax > 0x7fffffffLL || (long long)s->Hkv * s->budget > 0x7fffffffLL) return OBC_ERR_SHAPE;
+    const int n_hh = s->budget - s->n_sink - s->n_recent;
+    int ns = (int)floor((double)safeguard * (double)n_hh);
+    if (ns > n_hh) ns = n_hh;
+    *n_safe = ns;
+    return OBC_OK;
+}
+
+obc_status obc_select_adaptive_workspace(const obc_select_params* p, float safeguard, size_t* bytes) {
+    if (!bytes) return OBC_ERR_NULL;
+    SelectShape s; int n_safe = 0;
+    obc_status st = resolve_adaptive(p, safeguard, &s, &n_safe);
+    if (st != OBC_OK) return st;
+    *bytes = select_adaptive_workspace_bytes(s, n_safe);
+    return OBC_OK;
+}
+
+obc_status obc_select_adaptive(const obc_select_params* p, float safeguard, const float* scores,
+                               int32_t* idx, int32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
+    SelectShape s; int n_safe = 0;
+    obc_status st = resolve_adaptive(p, safeguard, &s, &n_safe);
+    if (st != OBC_OK) return st;
+    if (!scores || !idx || !counts) return OBC_ERR_NULL;
+    if (!workspace || workspace_bytes < select_adaptive_workspace_bytes(s, n_safe)) return OBC_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
+    return launch_select_adaptive(s, n_safe, scores, idx, counts, workspace, (cudaStream_t)stream);
 }
 
 obc_status obc_select_noalloc(const obc_select_params* p, const float* scores, int32_t* idx, void* stream) {

@@ -91,6 +91,9 @@ struct SelectShape {
 };
 size_t select_workspace_bytes(int B, int Hkv, int Nmax);
 obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx, void* ws, cudaStream_t stream);
+size_t select_adaptive_workspace_bytes(const SelectShape& s, int n_safe);
+obc_status launch_select_adaptive(const SelectShape& s, int n_safe, const float* scores, int32_t* idx, int32_t* counts,
+                                  void* ws, cudaStream_t stream);
 obc_status launch_select_static(const SelectShape& s, const float* scores, int32_t* idx, cudaStream_t stream);
 obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_bytes,
                          TensorView k, TensorView v, TensorView ko, TensorView vo, const int32_t* idx,

@@ -429,6 +429,53 @@ gather_kernel(int units, int Hkv, int idx_stride, int vecs, int elem_bytes,
         }
 }
 
+
+// ---- head-adaptive budgets: pieces around the two selection kernels ------------------------------------
+// keys of the tokens every head keeps by its own ranking are raised to the largest key, so that the
+// ranking across heads takes them first
+__global__ void __launch_bounds__(256)
+adaptive_boost_kernel(int units, int Nmax, int n_sink, int n_safe, int safe_stride,
+                      const int32_t* __restrict__ idx_safe, uint32_t* __restrict__ keys) {
+    pdl_wait();
+    const int unit = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (unit >= units || j >= n_safe) return;
+    const int p = idx_safe[(size_t)unit * safe_stride + n_sink + j];
+    if (p >= 0 && p < Nmax) keys[(size_t)unit * Nmax + p] = 0xffffffffu;
+}
+
+// vidx [B][total]: the tokens chosen across the heads of a batch item, ascending in h * Nmax + p.  One block
+// per (b, h) finds its head's stretch by binary search and writes the head's row of idx: sinks, chosen
+// tokens, recent tail, -1 padding; counts[b, h] = tokens kept (or -1, with a row of -1, when the row does
+// not fit idx_stride or the budget does not fit the sequence).
+__global__ void __launch_bounds__(256)
+adaptive_split_kernel(SelectShape s, int total, const int32_t* __restrict__ vidx_all,
+                      int32_t* __restrict__ idx_all, int32_t* __restrict__ counts) {
+    pdl_wait();
+    const int unit = blockIdx.x, b = unit / s.Hkv, h = unit % s.Hkv;
+    const int N = seq_len(s, b), lo = s.n_sink, hi = N - s.n_recent;
+    const int n_hh = s.budget - s.n_sink - s.n_recent;
+    const int32_t* vidx = vidx_all + (size_t)b * total;
+    int32_t* idx = idx_all + (size_t)unit * s.idx_stride;
+    auto lower_bound = [&](int v) {                       // first position whose virtual index is >= v
+        int a = 0, z = total;
+        while (a < z) { const int m = (a + z) >> 1; if (vidx[m] < v) a = m + 1; else z = m; }
+        return a;
+    };
+    const int seg0 = lower_bound(h * s.Nmax), seg1 = lower_bound((h + 1) * s.Nmax), c = seg1 - seg0;
+    const int kept = s.n_sink + c + s.n_recent;
+    const bool bad = N > s.Nmax || hi < lo || n_hh < 0 || n_hh > hi - lo || kept > s.idx_stride;
+    if (bad) {
+        for (int j = threadIdx.x; j < s.idx_stride; j += blockDim.x) idx[j] = -1;
+        if (threadIdx.x == 0) counts[unit] = -1;
+        return;
+    }
+    for (int j = threadIdx.x; j < s.n_sink; j += blockDim.x) idx[j] = j;
+    for (int j = threadIdx.x; j < c; j += blockDim.x) idx[s.n_sink + j] = vidx[seg0 + j] - h * s.Nmax;
+    for (int j = threadIdx.x; j < s.n_recent; j += blockDim.x) idx[s.n_sink + c + j] = hi + j;
+    for (int j = kept + threadIdx.x; j < s.idx_stride; j += blockDim.x) idx[j] = -1;
+    if (threadIdx.x == 0) counts[unit] = kept;
+}
+
 }  // namespace
 
 size_t select_workspace_bytes(int B, int Hkv, int Nmax) { return align_up((size_t)B * Hkv * Nmax * 4, 256); }
@@ -517,6 +564,51 @@ obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_byte
         OBC_CUDA_TRY(launch_pdl(gather_kernel, dim3((unsigned)((total + 255) / 256), B * Hkv), dim3(256), 0, stream, 1,
                                 B * Hkv, Hkv, idx_stride, vecs, elem_bytes, k, v, ko, vo, idx, s_in, s_out, Nmax));
     }
+    return OBC_OK;
+}
+
+// ---- head-adaptive budgets -------------------------------------------------------------------------------
+// workspace: pooled keys [units][Nmax] | every head's own selection [units][n_sink + n_safe + n_recent] |
+// the selection across heads [B][Hkv * n_hh]
+struct AdaptivePlan { size_t off_keys, off_safe, off_vidx, bytes; int safe_stride, total; };
+static AdaptivePlan make_adaptive_plan(const SelectShape& s, int n_safe) {
+    AdaptivePlan p{};
+    const size_t units = (size_t)s.B * s.Hkv;
+    const int n_hh = s.budget - s.n_sink - s.n_recent;
+    p.safe_stride = s.n_sink + n_safe + s.n_recent;
+    p.total = s.Hkv * (n_hh > 0 ? n_hh : 0);
+    size_t off = 0;
+    p.off_keys = off; off = align_up(off + units * s.Nmax * 4, 256);
+    p.off_safe = off; off = align_up(off + units * (size_t)(p.safe_stride > 0 ? p.safe_stride : 1) * 4, 256);
+    p.off_vidx = off; off = align_up(off + (size_t)s.B * (size_t)(p.total > 0 ? p.total : 1) * 4, 256);
+    p.bytes = off;
+    return p;
+}
+size_t select_adaptive_workspace_bytes(const SelectShape& s, int n_safe) { return make_adaptive_plan(s, n_safe).bytes; }
+
+obc_status launch_select_adaptive(const SelectShape& s, int n_safe, const float* scores, int32_t* idx, int32_t* counts,
+                                  void* ws, cudaStream_t stream) {
+    const AdaptivePlan plan = make_adaptive_plan(s, n_safe);
+    const int units = s.B * s.Hkv;
+    uint32_t* keys = (uint32_t*)((char*)ws + plan.off_keys);
+    int32_t* idx_safe = (int32_t*)((char*)ws + plan.off_safe);
+    int32_t* vidx = (int32_t*)((char*)ws + plan.off_vidx);
+    { ProfScope ps("pool_key", stream); OBC_CUDA_TRY(launch_pdl(pool_key_kernel, dim3((s.Nmax + 255) / 256, units), dim3(256), 0, stream, 1, s, scores, keys)); }
+    if (n_safe > 0) {
+        SelectShape own = s;                              // every head's own ranking, n_safe scored tokens each
+        own.budget = s.n_sink + n_safe + s.n_recent; own.budgets = nullptr; own.idx_stride = plan.safe_stride;
+        { ProfScope ps("select", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(units), dim3(SEL_NT), 0, stream, 1, own, (const uint32_t*)keys, idx_safe)); }
+        { ProfScope ps("adaptive_boost", stream);
+          OBC_CUDA_TRY(launch_pdl(adaptive_boost_kernel, dim3((n_safe + 255) / 256, units), dim3(256), 0, stream, 1, units, s.Nmax, s.n_sink, n_safe, plan.safe_stride, (const int32_t*)idx_safe, keys)); }
+    }
+    if (plan.total > 0) {
+        // all heads of a batch item as one sequence of Hkv * Nmax keys (the keys of protected and padding
+        // positions are 0 and rank below every candidate); equal keys keep the lowest head, then the lowest index
+        SelectShape all{s.B, 1, s.Hkv * s.Nmax, nullptr, plan.total, nullptr, plan.total, 0, 0, OBC_POOL_NONE, 1};
+        { ProfScope ps("select_layer", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(s.B), dim3(SEL_NT), 0, stream, 1, all, (const uint32_t*)keys, vidx)); }
+    }
+    { ProfScope ps("adaptive_split", stream);
+      OBC_CUDA_TRY(launch_pdl(adaptive_split_kernel, dim3(units), dim3(256), 0, stream, 1, s, plan.total, (const int32_t*)vidx, idx, counts)); }
     return OBC_OK;
 }
 
