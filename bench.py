@@ -450,7 +450,8 @@ def run_other(args):
         return
 
     given = args.workload.endswith("-given")     # the caller's attention outputs instead of a recompute
-    idx_cfg = {"llama32k": 2, "qwen128k": 3, "ragged": 4}[args.workload.replace("-given", "")]
+    adaptive = args.workload.endswith("-adaptive")    # head-adaptive budgets (safeguard 0.2) instead of one budget per head
+    idx_cfg = {"llama32k": 2, "qwen128k": 3, "ragged": 4}[args.workload.replace("-given", "").replace("-adaptive", "")]
     case, run = synth.config(idx_cfg)
     q, k, v = bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)
     lens = None if (case.seq_lens == case.Nmax).all() else torch.from_numpy(case.seq_lens).cuda()
@@ -458,13 +459,18 @@ def run_other(args):
     budgets = np.asarray(run["budget"] if isinstance(run["budget"], list) else [run["budget"]] * case.B, np.int32)
     uniform = bool((budgets == budgets[0]).all())
     bud_d = None if uniform else torch.from_numpy(budgets).cuda()
-    stride = int(budgets.max())
+    stride = int(budgets.max()) * (4 if adaptive else 1)      # adaptive: a head may keep up to four average budgets
     sp = api.score_params(q, k, seq_lens=lens, variants=order)
     ws_score = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
     scores = torch.empty((len(order), case.B, case.Hkv, case.Nmax), dtype=torch.float32, device="cuda")
     selp = api.select_params(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
                              seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"])
     ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
+    if adaptive:
+        n_ws = api.C.c_size_t(0)
+        api._check(api.lib().obc_select_adaptive_workspace(api.C.byref(selp), 0.2, api.C.byref(n_ws)), "obc_select_adaptive_workspace")
+        ws_sel = torch.empty(n_ws.value, dtype=torch.uint8, device="cuda")
+    counts = torch.empty((case.B, case.Hkv), dtype=torch.int32, device="cuda")
     idx = torch.empty((case.B, case.Hkv, stride), dtype=torch.int32, device="cuda")
     k_out = torch.empty((case.B, case.Hkv, stride, 128), dtype=torch.bfloat16, device="cuda")
     v_out = torch.empty_like(k_out)
@@ -493,9 +499,14 @@ def run_other(args):
             api.obc_score_given(q, k, v, o_win, lse_win, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
         else:
             api.obc_score(q, k, v, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
-        api.obc_select(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
-                       seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
-                       idx=idx, workspace=ws_sel)
+        if adaptive:
+            api.obc_select_adaptive(scores[-1], budget=int(budgets[0]), safeguard=0.2, idx_stride=stride, seq_lens=lens,
+                                    n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
+                                    idx=idx, counts=counts, workspace=ws_sel)
+        else:
+            api.obc_select(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
+                           seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
+                           idx=idx, workspace=ws_sel)
         api.obc_compact(k, v, idx, k_out=k_out, v_out=v_out)
     for _ in range(3):
         step()
@@ -526,7 +537,8 @@ def run_other(args):
             "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{case.name}: B{case.B} Hq{case.Hq} Hkv{case.Hkv} d128 Nmax{case.Nmax} W{case.W} bf16, "
                                    f"variants {order}, pool {run['pool_mode']} {run['pool_kernel']}, tokens/step {tokens}"
-                                   + (", window O and LSE supplied by the caller (no recompute)" if given else ""),
+                                   + (", window O and LSE supplied by the caller (no recompute)" if given else "")
+                                   + (", head-adaptive budgets (safeguard 0.2)" if adaptive else ""),
                        "launch": launch_mode, "ms_per_step_by_launch": {k_: v_ / steps for k_, v_ in ms_by_mode.items()},
                        "l2": "inputs (K+V) larger than L2" if tokens * case.Hkv * 512 > 126e6 else "single input copy"},
             "kernels": {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}}
@@ -542,7 +554,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--eager", action="store_true", help="time plain library calls instead of replaying CUDA graphs")
-    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given"],
+    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive"],
                     help="llama32k is the headline benchmark; the others print a shorter line (1 GPU)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"

@@ -186,7 +186,8 @@ struct ClusterShared {                        // fixed part of the CTA's shared 
 };
 
 __global__ void __launch_bounds__(CL_NT)
-select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* __restrict__ idx_all, int seg_cap) {
+select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* __restrict__ idx_all, int seg_cap,
+                      const uint32_t* __restrict__ keys_in) {
     extern __shared__ __align__(16) uint8_t sel_smem[];
     ClusterShared& sh = *reinterpret_cast<ClusterShared*>(sel_smem);
     uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(ClusterShared));
@@ -219,51 +220,56 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;   // sum[3][] and local[]
     if (tid == 0) sh.n_list = 0;
 
-    // pooled keys: stage the scores with their halo, then pool out of shared memory
-    const float* sc = scores + (size_t)unit * s.Nmax;
-    const int half = (s.pool_mode == OBC_POOL_NONE) ? 0 : s.pool_kernel / 2;
-    const float pad = s.pool_mode == OBC_POOL_MAX ? -INFINITY : 0.f;
-    for (int base = 0; base < m + 2 * half; base += 8 * CL_NT) {      // eight loads in flight per thread
-        float val[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = base + u * CL_NT + tid, p = lo + c0 + i - half;
-            val[u] = (i < m + 2 * half && p >= lo && p < hi) ? sc[p] : pad;
+    if (keys_in) {                                 // the caller has the (pooled) keys already: [units][Nmax]
+        const uint32_t* kin = keys_in + (size_t)unit * s.Nmax + lo + c0;
+        for (int i = tid; i < m; i += CL_NT) keys[i] = kin[i];
+    } else {
+        // pooled keys: stage the scores with their halo, then pool out of shared memory
+        const float* sc = scores + (size_t)unit * s.Nmax;
+        const int half = (s.pool_mode == OBC_POOL_NONE) ? 0 : s.pool_kernel / 2;
+        const float pad = s.pool_mode == OBC_POOL_MAX ? -INFINITY : 0.f;
+        for (int base = 0; base < m + 2 * half; base += 8 * CL_NT) {      // eight loads in flight per thread
+            float val[8];
+    #pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = base + u * CL_NT + tid, p = lo + c0 + i - half;
+                val[u] = (i < m + 2 * half && p >= lo && p < hi) ? sc[p] : pad;
+            }
+    #pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = base + u * CL_NT + tid;
+                if (i < m + 2 * half) stage[i] = val[u];
+            }
         }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = base + u * CL_NT + tid;
-            if (i < m + 2 * half) stage[i] = val[u];
-        }
-    }
-    __syncthreads();
-    for (int i = tid; i < m; i += CL_NT) {
-        float val;
-        if (half == 0) {
-            val = stage[i];
-        } else if (half <= 3) {                    // kernels up to 7: all taps read before they are combined
-            float tap[7];
-#pragma unroll
-            for (int t = 0; t < 7; ++t) tap[t] = t <= 2 * half ? stage[i + t] : pad;
-            if (s.pool_mode == OBC_POOL_MAX) {
+        __syncthreads();
+        for (int i = tid; i < m; i += CL_NT) {
+            float val;
+            if (half == 0) {
+                val = stage[i];
+            } else if (half <= 3) {                    // kernels up to 7: all taps read before they are combined
+                float tap[7];
+    #pragma unroll
+                for (int t = 0; t < 7; ++t) tap[t] = t <= 2 * half ? stage[i + t] : pad;
+                if (s.pool_mode == OBC_POOL_MAX) {
+                    val = -INFINITY;
+    #pragma unroll
+                    for (int t = 0; t < 7; ++t) val = fmaxf(val, tap[t]);      // padding taps are -inf
+                } else {                               // taps in ascending index order; padding adds +0
+                    val = 0.f;
+    #pragma unroll
+                    for (int t = 0; t < 7; ++t) if (t <= 2 * half) val = __fadd_rn(val, tap[t]);
+                    val = __fdiv_rn(val, (float)s.pool_kernel);
+                }
+            } else if (s.pool_mode == OBC_POOL_MAX) {
                 val = -INFINITY;
-#pragma unroll
-                for (int t = 0; t < 7; ++t) val = fmaxf(val, tap[t]);      // padding taps are -inf
-            } else {                               // taps in ascending index order; padding adds +0
+                for (int t = 0; t <= 2 * half; ++t) val = fmaxf(val, stage[i + t]);
+            } else {
                 val = 0.f;
-#pragma unroll
-                for (int t = 0; t < 7; ++t) if (t <= 2 * half) val = __fadd_rn(val, tap[t]);
+                for (int t = 0; t <= 2 * half; ++t) val = __fadd_rn(val, stage[i + t]);
                 val = __fdiv_rn(val, (float)s.pool_kernel);
             }
-        } else if (s.pool_mode == OBC_POOL_MAX) {
-            val = -INFINITY;
-            for (int t = 0; t <= 2 * half; ++t) val = fmaxf(val, stage[i + t]);
-        } else {
-            val = 0.f;
-            for (int t = 0; t <= 2 * half; ++t) val = __fadd_rn(val, stage[i + t]);
-            val = __fdiv_rn(val, (float)s.pool_kernel);
+            keys[i] = float_key(val);
         }
-        keys[i] = float_key(val);
     }
     cluster.sync();                                // histograms zeroed and keys written everywhere
 
@@ -490,7 +496,15 @@ static int select_cluster_size(int Nmax, int* seg_cap) {
     return C;
 }
 
+// keys_in: when given, [units][Nmax] keys that take the place of pooling `scores` (which may then be null);
+// `ws` is then not written
+static obc_status launch_select_impl(const SelectShape& s, const float* scores, const uint32_t* keys_in, int32_t* idx,
+                                     void* ws, cudaStream_t stream);
 obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx, void* ws, cudaStream_t stream) {
+    return launch_select_impl(s, scores, nullptr, idx, ws, stream);
+}
+static obc_status launch_select_impl(const SelectShape& s, const float* scores, const uint32_t* keys_in, int32_t* idx,
+                                     void* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
     int seg_cap = 0;
     const int C = select_cluster_size(s.Nmax, &seg_cap);
@@ -507,10 +521,14 @@ obc_status launch_select(const SelectShape& s, const float* scores, int32_t* idx
         int max_clusters = 0;
         if (cudaOccupancyMaxActiveClusters(&max_clusters, select_cluster_kernel, &cfg) == cudaSuccess && max_clusters > 0) {
             { ProfScope ps("select_cluster", stream);
-              OBC_CUDA_TRY(launch_pdl(select_cluster_kernel, dim3((unsigned)(units * C)), dim3(CL_NT), smem, stream, C, s, scores, idx, seg_cap)); }
+              OBC_CUDA_TRY(launch_pdl(select_cluster_kernel, dim3((unsigned)(units * C)), dim3(CL_NT), smem, stream, C, s, scores, idx, seg_cap, keys_in)); }
             return OBC_OK;
         }
         (void)cudaGetLastError();                  // the device cannot host such a cluster: one CTA per head
+    }
+    if (keys_in) {
+        { ProfScope ps("select", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(units), dim3(SEL_NT), 0, stream, 1, s, keys_in, idx)); }
+        return OBC_OK;
     }
     uint32_t* keys = (uint32_t*)ws;
     { ProfScope ps("pool_key", stream); OBC_CUDA_TRY(launch_pdl(pool_key_kernel, dim3((s.Nmax + 255) / 256, units), dim3(256), 0, stream, 1, s, scores, keys)); }
@@ -597,7 +615,8 @@ obc_status launch_select_adaptive(const SelectShape& s, int n_safe, const float*
     if (n_safe > 0) {
         SelectShape own = s;                              // every head's own ranking, n_safe scored tokens each
         own.budget = s.n_sink + n_safe + s.n_recent; own.budgets = nullptr; own.idx_stride = plan.safe_stride;
-        { ProfScope ps("select", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(units), dim3(SEL_NT), 0, stream, 1, own, (const uint32_t*)keys, idx_safe)); }
+        obc_status st = launch_select_impl(own, nullptr, keys, idx_safe, nullptr, stream);
+        if (st != OBC_OK) return st;
         { ProfScope ps("adaptive_boost", stream);
           OBC_CUDA_TRY(launch_pdl(adaptive_boost_kernel, dim3((n_safe + 255) / 256, units), dim3(256), 0, stream, 1, units, s.Nmax, s.n_sink, n_safe, plan.safe_stride, (const int32_t*)idx_safe, keys)); }
     }
@@ -605,7 +624,8 @@ obc_status launch_select_adaptive(const SelectShape& s, int n_safe, const float*
         // all heads of a batch item as one sequence of Hkv * Nmax keys (the keys of protected and padding
         // positions are 0 and rank below every candidate); equal keys keep the lowest head, then the lowest index
         SelectShape all{s.B, 1, s.Hkv * s.Nmax, nullptr, plan.total, nullptr, plan.total, 0, 0, OBC_POOL_NONE, 1};
-        { ProfScope ps("select_layer", stream); OBC_CUDA_TRY(launch_pdl(select_kernel, dim3(s.B), dim3(SEL_NT), 0, stream, 1, all, (const uint32_t*)keys, vidx)); }
+        obc_status st = launch_select_impl(all, nullptr, keys, vidx, nullptr, stream);
+        if (st != OBC_OK) return st;
     }
     { ProfScope ps("adaptive_split", stream);
       OBC_CUDA_TRY(launch_pdl(adaptive_split_kernel, dim3(units), dim3(256), 0, stream, 1, s, plan.total, (const int32_t*)vidx, idx, counts)); }
