@@ -88,6 +88,25 @@ def test_select_validation(L):
     assert L.obc_select(C.byref(_selp()), 4096, 4096, 4096, 16, None) == -5
 
 
+def test_given_and_adaptive_validation(L):
+    t = lambda ptr, dt=1: api.obc_tensor(ptr, dt, 0, 256 * 128, 128)
+    p = _sp()
+    # the attention outputs and their log-sum-exp are both required; o may be fp32 next to a bf16 cache
+    assert L.obc_score_given(C.byref(p), t(4096), t(4096), t(4096), t(4096), None, 4096, 4096, 1 << 30, None) == -1
+    assert L.obc_score_given(C.byref(p), t(4096), t(4096), t(4096), t(None), 4096, 4096, 4096, 1 << 30, None) == -1
+    assert L.obc_score_given(C.byref(p), t(4096), t(4096), t(4096), t(4096, 0), 4096, 4096, 4096, 16, None) == -5
+    assert L.obc_score_given(C.byref(_sp(variants=16)), t(4096), t(4096), t(4096), t(4104), 4096, 4096, 4096, 1 << 30, None) == -4
+    n = C.c_size_t(0)
+    assert L.obc_select_adaptive_workspace(C.byref(_selp()), 0.2, C.byref(n)) == 0 and n.value >= 2 * 256 * 4
+    assert L.obc_select_adaptive_workspace(C.byref(_selp()), 1.5, C.byref(n)) == -2
+    assert L.obc_select_adaptive_workspace(C.byref(_selp()), -0.1, C.byref(n)) == -2
+    assert L.obc_select_adaptive_workspace(C.byref(_selp(budgets=4096)), 0.2, C.byref(n)) == -3
+    assert L.obc_select_adaptive(C.byref(_selp()), 0.2, 4096, 4096, None, 4096, 1 << 20, None) == -1
+    assert L.obc_select_adaptive(C.byref(_selp()), 0.2, 4096, 4096, 4096, 4096, 16, None) == -5
+    d1, d2 = C.c_double(0), C.c_double(0)
+    assert L.obc_score_kernel_spans(None, None, C.byref(d1), C.byref(d2)) == -1
+
+
 def test_compact_and_decode_validation(L):
     t = lambda ptr: api.obc_tensor(ptr, 1, 0, 256 * 128, 128)
     assert L.obc_compact(1, 2, 64, 16, 256, t(4096), t(4096), 4096, t(4096), t(4096), None, None, None) == -3
