@@ -3,10 +3,10 @@
 // App. C.2.2 (sinks + recent window protected, one eviction per step once over budget).
 //
 // With G <= 8 score rows per KV head the contractions are thin (slots x heads x 128 channels) and
-// the step is bound by HBM traffic.  A CTA takes one chunk of 256 slots of one KV head: the 256-byte
-// K or V rows are staged in shared memory (16-byte pieces XOR-swizzled by row) and the contractions
-// run as warp-level m16n8k16 MMAs fed by ldmatrix; one thread per slot does the softmax and score
-// arithmetic, and reductions over slots use warp shuffles.
+// the step is bound by HBM traffic.  A CTA takes one chunk of 128 slots of one KV head: the 256-byte
+// K and V rows travel into shared memory by asynchronous copies (16-byte pieces XOR-swizzled by row)
+// and the contractions run as warp-level m16n8k16 MMAs fed by ldmatrix; one thread per slot does the
+// softmax and score arithmetic, and reductions over slots use warp shuffles.
 //
 //   decode_pass1   append (k_t, v_t); logits of every live slot (kept in the workspace so K is
 //                  read once); per-chunk softmax statistics and partial outputs
@@ -19,7 +19,8 @@
 namespace obc {
 namespace {
 
-constexpr int CH = 256;                  // slots per chunk = threads per block
+constexpr int CH = 128;                  // slots per chunk = threads per block
+constexpr int NWARP = CH / 32;
 constexpr size_t kStageBytes = (size_t)CH * 256;   // one chunk of 256-byte rows in shared memory
 
 struct DecodePlan {
@@ -50,26 +51,26 @@ __device__ __forceinline__ const __nv_bfloat16* bf_row(const TensorView& t, int 
     return reinterpret_cast<const __nv_bfloat16*>(t.ptr) + b * t.sb + h * t.sh + tok * t.st;
 }
 
-// Cooperative copy of the 256-byte rows [c0, c0 + CH) of one cache into shared memory, in two steps so
-// that the caller can put work between them: load_rows issues all 16 loads of a thread before any
-// use (a warp reads two whole rows per instruction, coalesced; rows at or beyond `hi` are not
-// read), store_rows puts the 16-byte chunk c of row r at chunk c ^ (r & 15), so that the eight
-// rows of an 8x8 tile fall into distinct banks when ldmatrix reads them.
-__device__ __forceinline__ void load_rows(uint4 (&v)[16], const TensorView& t, int b, int g, int c0, int hi) {
+// The 256-byte rows [c0, c0 + CH) of one cache travel into shared memory by asynchronous 16-byte copies
+// (cp.async: no registers hold them on the way, and a CTA has its K and its V rows under way together).
+// A warp copies two whole rows per instruction, coalesced; rows at or beyond `hi` are not read and are
+// zeroed.  The 16-byte piece c of row r lands at piece c ^ (r & 15), so that the eight rows of an 8x8
+// tile fall into distinct banks when ldmatrix reads them.
+__device__ __forceinline__ void copy_rows_async(uint4* dst, const TensorView& t, int b, int g, int c0, int hi) {
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
         const int i = threadIdx.x + k * CH, r = i >> 4, c = i & 15;
-        // plain loads: the new token's row was stored by this CTA just before
-        v[k] = c0 + r < hi ? reinterpret_cast<const uint4*>(bf_row(t, b, g, c0 + r))[c] : make_uint4(0, 0, 0, 0);
+        uint4* d = dst + r * 16 + (c ^ (r & 15));
+        if (c0 + r < hi) {
+            const uint4* src = reinterpret_cast<const uint4*>(bf_row(t, b, g, c0 + r)) + c;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(d)), "l"(src) : "memory");
+        } else {
+            *d = make_uint4(0, 0, 0, 0);
+        }
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
 }
-__device__ __forceinline__ void store_rows(uint4* dst, const uint4 (&v)[16]) {
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
-        const int i = threadIdx.x + k * CH, r = i >> 4, c = i & 15;
-        dst[r * 16 + (c ^ (r & 15))] = v[k];
-    }
-}
+template <int N> __device__ __forceinline__ void copy_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // ---- warp-level tensor-core pieces ------------------------------------------------------------------
 // The contractions of a chunk are tiny (256 slots x at most 8 heads x 128 channels) and the kernels are
@@ -113,10 +114,10 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, const int32_t* state,
                     int step_pos, char* ws) {
     pdl_wait();
-    extern __shared__ __align__(16) uint4 sRows[];                      // [CH][16]: the chunk's K rows
+    extern __shared__ __align__(16) uint4 sStage[];                     // [2][CH][16]: the chunk's K rows, then its V rows
     __shared__ float sP[G][CH];
-    __shared__ __align__(16) float sO[8][G][kD];
-    __shared__ float sRed[8][G];
+    __shared__ __align__(16) float sO[NWARP][G][kD];
+    __shared__ float sRed[NWARP][G];
     __shared__ float sM[G];
 
     const int unit = blockIdx.y, chunk = blockIdx.x, c0 = chunk * CH;
@@ -151,14 +152,14 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         else if (tid == 32) { pos[(size_t)unit * s.cap + next] = step_pos; s_acc[(size_t)unit * s.cap + next] = 0.f; }
     }
     __syncthreads();                                       // the new token's row is in place
-    uint4 stage[16];
-    load_rows(stage, kc, b, g, c0, hi);
-    store_rows(sRows, stage);
-    __syncthreads();
-    load_rows(stage, vc, b, g, c0, hi);                    // V rows travel while the logits are computed
-
+    const uint4* sRows = sStage;                           // K rows
+    const uint4* sVrows = sStage + CH * 16;                // V rows, under way while the logits are computed
+    copy_rows_async(sStage, kc, b, g, c0, hi);
+    copy_rows_async(sStage + CH * 16, vc, b, g, c0, hi);
     const int slot = c0 + tid;
     const bool live = slot < hi && ((valid && slot == next) || pos[(size_t)unit * s.cap + slot] >= 0);
+    copy_wait<1>();                                        // this thread's K pieces have landed
+    __syncthreads();
     const float sl2 = s.scale * kLog2e;
     // logits of the warp's 32 slots: two 16-slot tiles, eight 16-channel steps each
 #pragma unroll
@@ -191,7 +192,7 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
     __syncthreads();
     if (tid < G) {
         float m = -INFINITY;
-        for (int w = 0; w < 8; ++w) m = fmaxf(m, sRed[w][tid]);
+        for (int w = 0; w < NWARP; ++w) m = fmaxf(m, sRed[w][tid]);
         sM[tid] = m;
     }
     __syncthreads();
@@ -202,14 +203,13 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         sP[r][tid] = p;
         lsum[r] = warp_sum(p);
     }
-    __syncthreads();                                       // sRed reads done, sP complete, K rows no longer read
-    store_rows(sRows, stage);
+    copy_wait<0>();                                        // this thread's V pieces have landed
+    __syncthreads();                                       // sRed reads done, sP complete, V rows staged
 #pragma unroll
     for (int r = 0; r < G; ++r) if (lane == 0) sRed[warp][r] = lsum[r];
 
     // partial outputs of the warp's 32 slots, transposed: (16 channels) x (8 heads) tiles of V^T P^T.  The
     // probabilities enter as bf16 high and low halves; slots without a live token carry p = 0.
-    __syncthreads();                                       // V rows staged
     {
         uint32_t ph[2][2], pl[2][2];                       // [16-slot step][k half]: p of head lane / 4, slots 2 (lane % 4), + 1 (+ 8)
         const int n = lane >> 2, t = lane & 3;
@@ -227,7 +227,7 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk) {
                 uint32_t a[4];
-                ldsm_x4_trans(a, tile_addr(sRows, warp * 32 + kk * 16, 2 * j, lane, false));
+                ldsm_x4_trans(a, tile_addr(sVrows, warp * 32 + kk * 16, 2 * j, lane, false));
                 mma_bf16(acc, a, ph[kk][0], ph[kk][1]);
                 mma_bf16(acc, a, pl[kk][0], pl[kk][1]);
             }
@@ -243,12 +243,12 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         const int r = i / kD, c = i % kD;
         float acc = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) acc += sO[w][r][c];
+        for (int w = 0; w < NWARP; ++w) acc += sO[w][r][c];
         part_o[i] = acc;
     }
     if (tid < G) {
         float l = 0.f;
-        for (int w = 0; w < 8; ++w) l += sRed[w][tid];
+        for (int w = 0; w < NWARP; ++w) l += sRed[w][tid];
         part_m[tid] = sM[tid]; part_l[tid] = l;
     }
 }
@@ -309,34 +309,33 @@ decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
 }
 
 template <int G>
-__global__ void __launch_bounds__(CH, 3)
+__global__ void __launch_bounds__(CH)
 decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc, const int32_t* pos,
                     const int32_t* state, int step_pos, char* ws) {
-    pdl_wait();
     extern __shared__ __align__(16) uint4 sRows[];                      // [CH][16]: the chunk's V rows
     __shared__ float sLse[G], sNo[G];
     __shared__ float sT[G + 1][CH];                                     // v_slot . o_r (r < G) and ||v_slot||^2
-    __shared__ MinCand sMin[8];
+    __shared__ MinCand sMin[NWARP];
 
     const int unit = blockIdx.y, chunk = blockIdx.x, c0 = chunk * CH;
     const int b = unit / s.Hkv, g = unit % s.Hkv;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // The V rows are requested before anything else, and before the wait on the preceding kernel: the cache
+    // was last written two kernels back (the new token's row), and which rows are live is sorted out below.
+    copy_rows_async(sRows, vc, b, g, c0, s.cap);
+    pdl_wait();
     const int next = state[unit * 4 + 1], hi_old = state[unit * 4 + 2];
     const bool valid = next >= 0 && next < s.cap;
     const int hi = valid ? max(hi_old, next + 1) : hi_old;
     MinCand* part_min = (MinCand*)(ws + plan.off_min) + (size_t)unit * plan.chunks + chunk;
     if (c0 >= hi) {
         if (tid == 0) *part_min = MinCand{INFINITY, -1, -1, 0};
+        copy_wait<0>();                                                 // no copy may be under way when the CTA leaves
         return;
     }
     if (tid < G) {
         sLse[tid] = ((const float*)(ws + plan.off_lse))[(size_t)unit * G + tid];
         sNo[tid] = ((const float*)(ws + plan.off_no))[(size_t)unit * G + tid];
-    }
-    {
-        uint4 stage[16];
-        load_rows(stage, vc, b, g, c0, hi);
-        store_rows(sRows, stage);
     }
     // B operand of v . o: lane (n = lane / 4, t = lane % 4) holds o_n[16 ks + 2t .. +1] and [.. + 8 .. +9],
     // each fp32 value as a bf16 high and low half
@@ -352,10 +351,14 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
                 split_bf16x2(o2.x, o2.y, oh[ks][hf], ol[ks][hf]);
             }
     }
-    __syncthreads();
-
     const int slot = c0 + tid;
     const int my_pos = slot < hi ? pos[(size_t)unit * s.cap + slot] : -1;
+    copy_wait<0>();
+    __syncthreads();
+    if (c0 + CH > hi) {                                    // rows beyond the live extent may hold anything: zero them
+        for (int i = tid; i < CH * 16; i += CH) if (c0 + (i >> 4) >= hi) sRows[i] = make_uint4(0, 0, 0, 0);
+        __syncthreads();
+    }
     const bool live = my_pos >= 0;
     MinCand cand{INFINITY, -1, -1, 0};
     // v . o_r and ||v||^2 of the warp's 32 slots: two 16-slot tiles, eight 16-channel steps each.  The norms are
@@ -420,7 +423,7 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
     __syncthreads();
     if (tid == 0) {
         MinCand best = sMin[0];
-        for (int w = 1; w < 8; ++w) {
+        for (int w = 1; w < NWARP; ++w) {
             const MinCand o2 = sMin[w];
             if (o2.slot >= 0 && (best.slot < 0 || o2.val < best.val || (o2.val == best.val && o2.pos > best.pos))) best = o2;
         }
@@ -463,8 +466,8 @@ obc_status launch_g(const DecodeShape& s, const DecodePlan& plan, TensorView q, 
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
                     int step_pos, char* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
-    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_pass1_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageBytes));
-      OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), kStageBytes, stream, 1, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
+    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_pass1_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * kStageBytes)));
+      OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), 2 * kStageBytes, stream, 1, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
     { ProfScope ps("decode_combine", stream); OBC_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(units * s.G), dim3(kD), 0, stream, 1, s, plan, ws)); }
     { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_score_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageBytes));
       OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G>, dim3(plan.chunks, units), dim3(CH), kStageBytes, stream, 1, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
