@@ -273,8 +273,15 @@ decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
     const float* pm = (const float*)(ws + plan.off_pm) + (size_t)unit * plan.chunks * G + r;
     const float* pl = (const float*)(ws + plan.off_pl) + (size_t)unit * plan.chunks * G + r;
     const float* po = (const float*)(ws + plan.off_po) + ((size_t)unit * plan.chunks * G + r) * kD + c;
+    // the statistics of chunk c (and c + 128, ...) are read once; the partial outputs are requested CMB at a
+    // time before their weights are known (a chunk without a live slot wrote none: its value is dropped, not
+    // multiplied), so the block costs a couple of round trips to L2 however many chunks there are
+    constexpr int CMB = 20;
     float M = -INFINITY;
     for (int ch = c; ch < plan.chunks; ch += kD) M = fmaxf(M, pm[(size_t)ch * G]);
+    float first[CMB];
+#pragma unroll
+    for (int u = 0; u < CMB; ++u) first[u] = u < plan.chunks ? po[(size_t)u * G * kD] : 0.f;
     M = decode_block_reduce(M, true, red);
     float L = 0.f, oc = 0.f;
     for (int base = 0; base < plan.chunks; base += kD) {
@@ -287,15 +294,20 @@ decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
         __syncthreads();
         sW[c] = w;
         __syncthreads();
-        for (int j0 = 0; j0 < cnt; j0 += 8) {
-            float o8[8], w8[8];
+        for (int j0 = 0; j0 < cnt; j0 += CMB) {
+            float o[CMB];
+            if (base == 0 && j0 == 0) {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {                  // chunks without a live slot hold no partial output
-                w8[u] = j0 + u < cnt ? sW[j0 + u] : 0.f;
-                o8[u] = w8[u] != 0.f ? po[(size_t)(base + j0 + u) * G * kD] : 0.f;
+                for (int u = 0; u < CMB; ++u) o[u] = first[u];
+            } else {
+#pragma unroll
+                for (int u = 0; u < CMB; ++u) o[u] = j0 + u < cnt ? po[(size_t)(base + j0 + u) * G * kD] : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) oc = fmaf(o8[u], w8[u], oc);
+            for (int u = 0; u < CMB; ++u) {
+                const float wu = j0 + u < cnt ? sW[j0 + u] : 0.f;
+                oc = wu != 0.f ? fmaf(o[u], wu, oc) : oc;
+            }
         }
     }
     L = decode_block_reduce(L, false, red);
@@ -431,34 +443,46 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
     }
 }
 
+// one warp per (b, g): the lanes read the chunks' candidates side by side and reduce them with shuffles
 __global__ void __launch_bounds__(128)
 decode_final_kernel(DecodeShape s, DecodePlan plan, int32_t* pos, int32_t* state, const char* ws) {
     pdl_wait();
-    const int unit = blockIdx.x * blockDim.x + threadIdx.x;
+    const int unit = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (unit >= s.B * s.Hkv) return;
     int live = state[unit * 4 + 0];
     const int next = state[unit * 4 + 1], hi_old = state[unit * 4 + 2];
     const bool valid = next >= 0 && next < s.cap;
-    if (!valid) { state[unit * 4 + 3] = 1; return; }       // no room: the step was not applied
+    if (!valid) { if (lane == 0) state[unit * 4 + 3] = 1; return; }       // no room: the step was not applied
     const int hi = max(hi_old, next + 1);
     live += 1;
     int new_next = hi;
-    if (live > s.budget) {
+    if (live > s.budget) {                                   // uniform over the warp
         const MinCand* pm = (const MinCand*)(ws + plan.off_min) + (size_t)unit * plan.chunks;
         MinCand best{INFINITY, -1, -1, 0};
-        for (int ch = 0; ch < plan.chunks; ++ch) {
+        for (int ch = lane; ch < plan.chunks; ch += 32) {
             const MinCand o2 = pm[ch];
             if (o2.slot >= 0 && (best.slot < 0 || o2.val < best.val || (o2.val == best.val && o2.pos > best.pos))) best = o2;
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            MinCand other;
+            other.val = __shfl_xor_sync(0xffffffffu, best.val, o);
+            other.pos = __shfl_xor_sync(0xffffffffu, best.pos, o);
+            other.slot = __shfl_xor_sync(0xffffffffu, best.slot, o);
+            if (other.slot >= 0 && (best.slot < 0 || other.val < best.val || (other.val == best.val && other.pos > best.pos)))
+                { best.val = other.val; best.pos = other.pos; best.slot = other.slot; }
+        }
         if (best.slot >= 0) {
-            pos[(size_t)unit * s.cap + best.slot] = -1;
+            if (lane == 0) pos[(size_t)unit * s.cap + best.slot] = -1;
             live -= 1;
             new_next = best.slot;
         }
     }
-    state[unit * 4 + 0] = live;
-    state[unit * 4 + 1] = new_next;
-    state[unit * 4 + 2] = hi;
+    if (lane == 0) {
+        state[unit * 4 + 0] = live;
+        state[unit * 4 + 1] = new_next;
+        state[unit * 4 + 2] = hi;
+    }
 }
 
 template <int G>
@@ -471,7 +495,7 @@ obc_status launch_g(const DecodeShape& s, const DecodePlan& plan, TensorView q, 
     { ProfScope ps("decode_combine", stream); OBC_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(units * s.G), dim3(kD), 0, stream, 1, s, plan, ws)); }
     { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_score_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageBytes));
       OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G>, dim3(plan.chunks, units), dim3(CH), kStageBytes, stream, 1, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
-    { ProfScope ps("decode_final", stream); OBC_CUDA_TRY(launch_pdl(decode_final_kernel, dim3((units + 127) / 128), dim3(128), 0, stream, 1, s, plan, pos, state, ws)); }
+    { ProfScope ps("decode_final", stream); OBC_CUDA_TRY(launch_pdl(decode_final_kernel, dim3((units + 3) / 4), dim3(128), 0, stream, 1, s, plan, pos, state, ws)); }
     return OBC_OK;
 }
 
