@@ -25,7 +25,7 @@ constexpr size_t kStageBytes = (size_t)CH * 256;   // one chunk of 256-byte rows
 
 struct DecodePlan {
     int chunks;
-    size_t off_z, off_pm, off_pl, off_po, off_lse, off_no, off_o, off_min, bytes;
+    size_t off_z, off_pm, off_pl, off_po, off_lse, off_no, off_o, off_ohi, off_olo, off_min, bytes;
 };
 
 DecodePlan make_plan(const DecodeShape& s) {
@@ -40,6 +40,8 @@ DecodePlan make_plan(const DecodeShape& s) {
     p.off_lse = off; off = align_up(off + units * s.G * 4, 256);
     p.off_no = off;  off = align_up(off + units * s.G * 4, 256);
     p.off_o = off;   off = align_up(off + units * s.G * kD * 4, 256);
+    p.off_ohi = off; off = align_up(off + units * s.G * kD * 2, 256);     // o as bf16 high and low halves (o = hi + lo)
+    p.off_olo = off; off = align_up(off + units * s.G * kD * 2, 256);
     p.off_min = off; off = align_up(off + units * p.chunks * 16, 256);
     p.bytes = off;
     return p;
@@ -57,16 +59,18 @@ __device__ __forceinline__ const __nv_bfloat16* bf_row(const TensorView& t, int 
 // zeroed.  The 16-byte piece c of row r lands at piece c ^ (r & 15), so that the eight rows of an 8x8
 // tile fall into distinct banks when ldmatrix reads them.
 __device__ __forceinline__ void copy_rows_async(uint4* dst, const TensorView& t, int b, int g, int c0, int hi) {
+    // thread t copies piece c = t % 16 of rows t / 16, t / 16 + 8, ...: one source pointer that advances by eight
+    // rows, and a destination whose swizzle (r & 15) alternates between two values
+    const int c = threadIdx.x & 15, r0 = threadIdx.x >> 4;
+    const char* src = reinterpret_cast<const char*>(bf_row(t, b, g, c0 + r0)) + c * 16;
+    const size_t step = (size_t)t.st * 2 * (CH / 16);                  // bytes between rows CH / 16 apart
+    const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(dst);
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
-        const int i = threadIdx.x + k * CH, r = i >> 4, c = i & 15;
-        uint4* d = dst + r * 16 + (c ^ (r & 15));
-        if (c0 + r < hi) {
-            const uint4* src = reinterpret_cast<const uint4*>(bf_row(t, b, g, c0 + r)) + c;
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(d)), "l"(src) : "memory");
-        } else {
-            *d = make_uint4(0, 0, 0, 0);
-        }
+        const int r = r0 + k * (CH / 16);
+        const uint32_t d = d0 + (uint32_t)(r * 16 + (c ^ (r & 15))) * 16u;
+        if (c0 + r < hi) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + k * step) : "memory");
+        else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
@@ -314,6 +318,11 @@ decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
     oc = L > 0.f ? oc / L : 0.f;
     const float sq = decode_block_reduce(oc * oc, false, red);
     ((float*)(ws + plan.off_o))[((size_t)unit * G + r) * kD + c] = oc;
+    {   // the score kernel's MMA operand: o to about 16 bits as two bf16 halves
+        const __nv_bfloat16 hi = __float2bfloat16_rn(oc);
+        ((__nv_bfloat16*)(ws + plan.off_ohi))[((size_t)unit * G + r) * kD + c] = hi;
+        ((__nv_bfloat16*)(ws + plan.off_olo))[((size_t)unit * G + r) * kD + c] = __float2bfloat16_rn(oc - __bfloat162float(hi));
+    }
     if (c == 0) {
         ((float*)(ws + plan.off_lse))[(size_t)unit * G + r] = M + log2f(L);
         ((float*)(ws + plan.off_no))[(size_t)unit * G + r] = sq;
@@ -350,17 +359,19 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
         sNo[tid] = ((const float*)(ws + plan.off_no))[(size_t)unit * G + tid];
     }
     // B operand of v . o: lane (n = lane / 4, t = lane % 4) holds o_n[16 ks + 2t .. +1] and [.. + 8 .. +9],
-    // each fp32 value as a bf16 high and low half
+    // each fp32 value as a bf16 high and low half (split once per step by the combine kernel)
     uint32_t oh[8][2], ol[8][2];
     {
         const int n = lane >> 2, t = lane & 3;
-        const float2* orow = reinterpret_cast<const float2*>((const float*)(ws + plan.off_o) + ((size_t)unit * G + (n < G ? n : 0)) * kD);
+        const size_t row = ((size_t)unit * G + (n < G ? n : 0)) * (kD / 2);
+        const uint32_t* hrow = reinterpret_cast<const uint32_t*>(ws + plan.off_ohi) + row;
+        const uint32_t* lrow = reinterpret_cast<const uint32_t*>(ws + plan.off_olo) + row;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-                const float2 o2 = n < G ? orow[ks * 8 + hf * 4 + t] : make_float2(0.f, 0.f);
-                split_bf16x2(o2.x, o2.y, oh[ks][hf], ol[ks][hf]);
+                oh[ks][hf] = n < G ? hrow[ks * 8 + hf * 4 + t] : 0u;
+                ol[ks][hf] = n < G ? lrow[ks * 8 + hf * 4 + t] : 0u;
             }
     }
     const int slot = c0 + tid;
