@@ -118,7 +118,7 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, const int32_t* state,
                     int step_pos, char* ws) {
     pdl_wait();
-    extern __shared__ __align__(16) uint4 sStage[];                     // [2][CH][16]: the chunk's K rows, then its V rows
+    extern __shared__ __align__(16) uint4 sStage[];                     // [CH][16]: the chunk's K rows, later its V rows
     __shared__ float sP[G][CH];
     __shared__ __align__(16) float sO[NWARP][G][kD];
     __shared__ float sRed[NWARP][G];
@@ -156,13 +156,14 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         else if (tid == 32) { pos[(size_t)unit * s.cap + next] = step_pos; s_acc[(size_t)unit * s.cap + next] = 0.f; }
     }
     __syncthreads();                                       // the new token's row is in place
-    const uint4* sRows = sStage;                           // K rows
-    const uint4* sVrows = sStage + CH * 16;                // V rows, under way while the logits are computed
+    // One buffer: the K rows first; the V rows take their place as soon as the logits are out and travel during
+    // the softmax arithmetic.  (Half the shared memory per CTA lets more CTAs of the SM overlap their round trips.)
+    const uint4* sRows = sStage;
+    const uint4* sVrows = sStage;
     copy_rows_async(sStage, kc, b, g, c0, hi);
-    copy_rows_async(sStage + CH * 16, vc, b, g, c0, hi);
     const int slot = c0 + tid;
     const bool live = slot < hi && ((valid && slot == next) || pos[(size_t)unit * s.cap + slot] >= 0);
-    copy_wait<1>();                                        // this thread's K pieces have landed
+    copy_wait<0>();                                        // this thread's K pieces have landed
     __syncthreads();
     const float sl2 = s.scale * kLog2e;
     // logits of the warp's 32 slots: two 16-slot tiles, eight 16-channel steps each
@@ -181,7 +182,8 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         if (h0 < G) { sP[h0][sl] = acc[0]; sP[h0][sl + 8] = acc[2]; }
         if (h0 + 1 < G) { sP[h0 + 1][sl] = acc[1]; sP[h0 + 1][sl + 8] = acc[3]; }
     }
-    __syncthreads();
+    __syncthreads();                                       // the K rows are no longer read
+    copy_rows_async(sStage, vc, b, g, c0, hi);
     float z2[G];
 #pragma unroll
     for (int r = 0; r < G; ++r) z2[r] = sP[r][tid];        // this thread's slot; sP[.][tid] is rewritten below by this thread only
@@ -501,8 +503,8 @@ obc_status launch_g(const DecodeShape& s, const DecodePlan& plan, TensorView q, 
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
                     int step_pos, char* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
-    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_pass1_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * kStageBytes)));
-      OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), 2 * kStageBytes, stream, 1, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
+    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_pass1_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageBytes));
+      OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), kStageBytes, stream, 1, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
     { ProfScope ps("decode_combine", stream); OBC_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(units * s.G), dim3(kD), 0, stream, 1, s, plan, ws)); }
     { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_score_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageBytes));
       OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G>, dim3(plan.chunks, units), dim3(CH), kStageBytes, stream, 1, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
