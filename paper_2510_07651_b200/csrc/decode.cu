@@ -346,6 +346,16 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
     // The V rows are requested before anything else, and before the wait on the preceding kernel: the cache
     // was last written two kernels back (the new token's row), and which rows are live is sorted out below.
     copy_rows_async(sRows, vc, b, g, c0, s.cap);
+    // Likewise this slot's position, logits and accumulator, all written two kernels back or earlier: asked for
+    // whether or not the slot turns out to be live, so that no later load has to wait for an earlier one.
+    const int slot = c0 + tid;
+    const bool in_cache = slot < s.cap;
+    const int pos_in = in_cache ? pos[(size_t)unit * s.cap + slot] : -1;
+    const float* zbuf = (const float*)(ws + plan.off_z) + (size_t)unit * G * s.cap;
+    float zin[G];
+#pragma unroll
+    for (int r = 0; r < G; ++r) zin[r] = in_cache ? zbuf[(size_t)r * s.cap + slot] : 0.f;
+    const float acc_in = in_cache ? s_acc[(size_t)unit * s.cap + slot] : 0.f;
     pdl_wait();
     const int next = state[unit * 4 + 1], hi_old = state[unit * 4 + 2];
     const bool valid = next >= 0 && next < s.cap;
@@ -376,8 +386,7 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
                 ol[ks][hf] = n < G ? lrow[ks * 8 + hf * 4 + t] : 0u;
             }
     }
-    const int slot = c0 + tid;
-    const int my_pos = slot < hi ? pos[(size_t)unit * s.cap + slot] : -1;
+    const int my_pos = slot < hi ? pos_in : -1;
     copy_wait<0>();
     __syncthreads();
     if (c0 + CH > hi) {                                    // rows beyond the live extent may hold anything: zero them
@@ -416,11 +425,10 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
         float nv = sT[G][tid], t[G];
 #pragma unroll
         for (int r = 0; r < G; ++r) t[r] = sT[r][tid];
-        const float* zbuf = (const float*)(ws + plan.off_z) + (size_t)unit * G * s.cap;
         float sc = 0.f;
 #pragma unroll
         for (int r = 0; r < G; ++r) {
-            const float z2 = zbuf[(size_t)r * s.cap + slot];
+            const float z2 = zin[r];
             const float a = exp2f(z2 - sLse[r]);
             const float Z = z2 * 0.6931471805599453f;          // back from log2 units: scale * q.k
             const float a2 = a * a;
@@ -430,7 +438,7 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
                 sc += a2 * nv + a2 * Z * Z * (sNo[r] + nv - 2.f * t[r]) + 2.f * a2 * Z * (nv - t[r]);
             else sc += a;
         }
-        const float acc = s_acc[(size_t)unit * s.cap + slot] + sc;
+        const float acc = acc_in + sc;
         s_acc[(size_t)unit * s.cap + slot] = acc;
         if (my_pos >= s.n_sink && my_pos <= step_pos - s.n_recent) cand = MinCand{acc, my_pos, slot, 0};
     }
