@@ -122,6 +122,8 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
 // become resident while the preceding kernel of the stream is still draining.  A kernel executes
 // pdl_wait() before its first access to memory that an earlier kernel may have written (or may
 // still read, for its own writes); what precedes the wait is set-up that touches no such memory.
+// (Releasing the next kernel earlier, with griddepcontrol.launch_dependents after the wait, was measured
+// and is not done: CTAs of the next kernel that sit waiting on an SM slowed the kernel at work.)
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>

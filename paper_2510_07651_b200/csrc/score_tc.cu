@@ -102,6 +102,17 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
     asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
                  ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// the same copy with an L2 eviction-priority hint (a policy made by l2_policy_*)
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                 int c0, int c1, int c2, int c3, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
@@ -168,6 +179,7 @@ struct TcParams {
     float* scores;                            // [planes][units][Nmax]
     unsigned int* status;                     // device status word (workspace header)
     unsigned long long* span;                 // [2]: ~(earliest CTA start), latest CTA end, in globaltimer ns
+    int l2_stream;                            // K/V copies carry the "evict first" L2 hint (their last use)
 };
 
 __device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
@@ -380,16 +392,24 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (lane == 0) {
             uint32_t item = 0, qo_loads = 0;
             int qo_unit = -1;
+            const uint64_t pol_stream = l2_policy_evict_first();
             for (; !tw.done() && !failed; tw.next()) {
                 const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv, t0 = tw.tile * TILE;
                 const uint32_t st = item % NSTAGE, use = item / NSTAGE;
                 if (!mbar_wait(bar(BAR_EMPTY + st), (use & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                 mbar_expect_tx(bar(BAR_FULL + st), 2 * kOperandBytes);
                 const uint32_t dk = sbase + OFF_K + st * kOperandBytes, dv = sbase + OFF_V + st * kOperandBytes;
-                tma_load_4d(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b);
-                tma_load_4d(dk + kHalfBytes, &map_k, bar(BAR_FULL + st), 64, t0, g, b);
-                tma_load_4d(dv, &map_v, bar(BAR_FULL + st), 0, t0, g, b);
-                tma_load_4d(dv + kHalfBytes, &map_v, bar(BAR_FULL + st), 64, t0, g, b);
+                if (p.l2_stream) {                             // last use of the tile: it may leave the cache first
+                    tma_load_4d_hint(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b, pol_stream);
+                    tma_load_4d_hint(dk + kHalfBytes, &map_k, bar(BAR_FULL + st), 64, t0, g, b, pol_stream);
+                    tma_load_4d_hint(dv, &map_v, bar(BAR_FULL + st), 0, t0, g, b, pol_stream);
+                    tma_load_4d_hint(dv + kHalfBytes, &map_v, bar(BAR_FULL + st), 64, t0, g, b, pol_stream);
+                } else {
+                    tma_load_4d(dk, &map_k, bar(BAR_FULL + st), 0, t0, g, b);
+                    tma_load_4d(dk + kHalfBytes, &map_k, bar(BAR_FULL + st), 64, t0, g, b);
+                    tma_load_4d(dv, &map_v, bar(BAR_FULL + st), 0, t0, g, b);
+                    tma_load_4d(dv + kHalfBytes, &map_v, bar(BAR_FULL + st), 64, t0, g, b);
+                }
                 // K, V and the sequence lengths were read by pass 1 of this call, so the first tile
                 // may be fetched while the preceding kernel drains; -2 O is that kernel's output
                 if (item == 0) pdl_wait();
@@ -851,6 +871,7 @@ struct P1Params {
     int causal;
     int n_chunks, chunk_rows;
     int n_splits, tiles_per_split;                         // CTAs per (unit, chunk); each writes one partial
+    int l2_stream;                                         // K/V copies carry the "evict first" L2 hint
     float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
     float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the chunk-0 CTAs
     unsigned int* status;
@@ -962,16 +983,24 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tma_load_2d(sbase + P1_OFF_Q, &map_q, bar(P1_QFULL), 0, qrow);
             tma_load_2d(sbase + P1_OFF_Q + kHalfBytes, &map_q, bar(P1_QFULL), 64, qrow);
             int issued = 0;
+            const uint64_t pol_stream = l2_policy_evict_first();
             for (int i = 0; i < n_tiles; ++i) {
                 const uint32_t st = i % P1_NSTAGE;
                 if (!mbar_wait(bar(P1_EMPTY + st), ((i / P1_NSTAGE) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                 mbar_expect_tx(bar(P1_FULL + st), 2 * kOperandBytes);
                 const uint32_t dk = sbase + P1_OFF_K + st * kOperandBytes, dv = sbase + P1_OFF_V + st * kOperandBytes;
                 const int t0 = (tile_lo + i) * TILE;
-                tma_load_4d(dk, &map_k, bar(P1_FULL + st), 0, t0, g, b);
-                tma_load_4d(dk + kHalfBytes, &map_k, bar(P1_FULL + st), 64, t0, g, b);
-                tma_load_4d(dv, &map_v, bar(P1_FULL + st), 0, t0, g, b);
-                tma_load_4d(dv + kHalfBytes, &map_v, bar(P1_FULL + st), 64, t0, g, b);
+                if (p.l2_stream) {                             // the cache cannot hold K and V until pass 2 anyway
+                    tma_load_4d_hint(dk, &map_k, bar(P1_FULL + st), 0, t0, g, b, pol_stream);
+                    tma_load_4d_hint(dk + kHalfBytes, &map_k, bar(P1_FULL + st), 64, t0, g, b, pol_stream);
+                    tma_load_4d_hint(dv, &map_v, bar(P1_FULL + st), 0, t0, g, b, pol_stream);
+                    tma_load_4d_hint(dv + kHalfBytes, &map_v, bar(P1_FULL + st), 64, t0, g, b, pol_stream);
+                } else {
+                    tma_load_4d(dk, &map_k, bar(P1_FULL + st), 0, t0, g, b);
+                    tma_load_4d(dk + kHalfBytes, &map_k, bar(P1_FULL + st), 64, t0, g, b);
+                    tma_load_4d(dv, &map_v, bar(P1_FULL + st), 0, t0, g, b);
+                    tma_load_4d(dv + kHalfBytes, &map_v, bar(P1_FULL + st), 64, t0, g, b);
+                }
                 ++issued;
             }
             for (int back = 0; back < P1_NSTAGE && back < issued; ++back) {   // drain own copies
@@ -1273,6 +1302,16 @@ TcChunks tc_chunks(int R) {
     return c;
 }
 
+size_t l2_bytes() {
+    static size_t n = 0;
+    if (!n) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, dev) != cudaSuccess || v <= 0) v = 126 << 20;
+        n = (size_t)v;
+    }
+    return n;
+}
+
 int sm_count() {
     static int n = 0;
     if (!n) {
@@ -1348,6 +1387,11 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
             return OBC_ERR_CUDA;
         }
     }
+    // A cache that cannot hold K and V from pass 1 to pass 2 is better streamed through: with the "evict
+    // first" hint on the K/V copies pass 1 ran 2 us faster on the 32k Llama layer (134 MB against 126 MB of L2).
+    // Smaller caches keep the default policy, so that pass 2 finds in L2 what pass 1 read.
+    const bool l2_stream = ch.n_chunks == 1 && !given &&
+        (double)units * s.Nmax * kD * 2 * 2 > 0.75 * (double)l2_bytes();
     if (given) {   // the caller's O and LSE take the place of pass 1 + combine; pass 2 computes the value norms itself
         obc_status st = launch_given_prep(s, plan, *given, ws, stream);
         if (st != OBC_OK) return st;
@@ -1357,6 +1401,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.seq_lens = s.seq_lens; p1.scale = s.scale; p1.causal = s.causal;
         p1.n_chunks = ch.n_chunks; p1.chunk_rows = ch.chunk_rows;
         p1.n_splits = plan.n_splits; p1.tiles_per_split = plan.tiles_per_split;
+        p1.l2_stream = l2_stream ? 1 : 0;
         p1.part_m = (float*)(wsb + plan.off_part_m); p1.part_l = (float*)(wsb + plan.off_part_l);
         p1.part_o = (float*)(wsb + plan.off_part_o);
         p1.nv = (float*)(wsb + plan.off_nv);
@@ -1379,6 +1424,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     p.span = (unsigned long long*)(wsb + plan.off_flag + kSpanOffset) + 2;
     p.cpair = (const float4*)(wsb + plan.off_cpair);
     p.nv = (const float*)(wsb + plan.off_nv);
+    p.l2_stream = l2_stream ? 1 : 0;
     const long long n_tiles = (long long)units * ((s.Nmax + TILE - 1) / TILE);
     const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
 

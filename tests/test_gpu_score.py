@@ -79,6 +79,20 @@ def test_tensor_core_row_counts(N, W, Hq, Hkv):
     _check(case, ["V", "K", "VK", "ATTN", "VATP"], path="tc", tight=2e-2)
 
 
+@pytest.mark.parametrize("N,Hq,Hkv,dtype,path", [
+    (96, 2, 1, "f32", "auto"),            # R = 192 on CUDA cores
+    (384, 2, 2, "bf16", "simt"),
+    (384, 4, 2, "bf16", "auto"),          # R = 768: twelve row chunks of 64 on tensor cores
+    (640, 1, 1, "bf16", "tc"),            # R = 640, five token tiles, every tile needs the mask
+])
+def test_full_history_window(N, Hq, Hkv, dtype, path):
+    """The perturbation window is the whole sequence (w = 1 in Sec. 4.3, the accumulation H2O uses): every
+    query position is a window row and row i sees the tokens p <= i."""
+    case = synth.make_prefill("history", B=1, Hq=Hq, Hkv=Hkv, d=128, W=N, N=N, dtype=dtype, seed=311 + N,
+                              hh_frac=0.02)
+    _check(case, ["V", "K", "VK", "ATTN", "VATP"], path=path, tight=2e-2 if dtype == "bf16" else None)
+
+
 def test_peaky_attention_cancellation_case():
     # some attention weights approach 1, so ||v_p - o_i||^2 cancels heavily
     case = synth.make_prefill("peaky", B=1, Hq=8, Hkv=2, d=128, W=16, N=2048, dtype="bf16", seed=5,
