@@ -464,8 +464,11 @@ def run_other(args):
 
     given = args.workload.endswith("-given")     # the caller's attention outputs instead of a recompute
     adaptive = args.workload.endswith("-adaptive")    # head-adaptive budgets (safeguard 0.2) instead of one budget per head
-    idx_cfg = {"llama32k": 2, "qwen128k": 3, "ragged": 4}[args.workload.replace("-given", "").replace("-adaptive", "")]
-    case, run = synth.config(idx_cfg)
+    if args.workload == "history4k":             # the whole sequence as perturbation window (W = N = 4096)
+        case, run = synth.full_history(4096)
+    else:
+        idx_cfg = {"llama32k": 2, "qwen128k": 3, "ragged": 4}[args.workload.replace("-given", "").replace("-adaptive", "")]
+        case, run = synth.config(idx_cfg)
     q, k, v = bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)
     lens = None if (case.seq_lens == case.Nmax).all() else torch.from_numpy(case.seq_lens).cuda()
     order = [n for n in ("V", "K", "VK") if n in run["variants"]]
@@ -567,7 +570,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--eager", action="store_true", help="time plain library calls instead of replaying CUDA graphs")
-    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive"],
+    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive", "history4k"],
                     help="llama32k is the headline benchmark; the others print a shorter line (1 GPU)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"

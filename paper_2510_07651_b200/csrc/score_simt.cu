@@ -261,6 +261,63 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     }
 }
 
+// The same merge with one warp per (unit, output row), for few splits and many rows (a window of thousands of
+// queries): no block-wide barrier, lane t holds head-dim elements 4t..4t+3, the splits are added in order.
+constexpr int CMBW_MAX_SPLITS = 8;
+__global__ void __launch_bounds__(CMB_NT)
+simt_combine_rows_kernel(ScoreShape s, SimtPlan plan, float* ws) {
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long rows_total = (long long)s.B * s.Hkv * plan.rows_out;
+    const long long orow = (long long)blockIdx.x * (CMB_NT / 32) + (threadIdx.x >> 5);
+    if (orow >= rows_total) return;
+    const int r = (int)(orow % plan.rows_out), unit = (int)(orow / plan.rows_out);
+    __nv_bfloat16* obf = plan.want_obf ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + plan.off_obf) : nullptr;
+    float* cpair = plan.want_obf ? ws + plan.off_cpair / 4 + (orow >> 1) * 4 + (orow & 1) : nullptr;
+    float4 oc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lse2 = INFINITY, onorm = 0.f;                    // padding rows weigh 0
+    if (r < s.R) {
+        const float* part_m = ws + plan.off_part_m / 4;
+        const float* part_l = ws + plan.off_part_l / 4;
+        const float* part_o = ws + plan.off_part_o / 4;
+        const size_t row0 = (size_t)unit * plan.n_splits * s.R + r;          // split sp: row0 + sp * R
+        float m[CMBW_MAX_SPLITS], l[CMBW_MAX_SPLITS];
+        float4 o4[CMBW_MAX_SPLITS];
+#pragma unroll
+        for (int sp = 0; sp < CMBW_MAX_SPLITS; ++sp) {                       // every load before the first use
+            const bool on = sp < plan.n_splits;
+            m[sp] = on ? part_m[row0 + (size_t)sp * s.R] : -INFINITY;
+            l[sp] = on ? part_l[row0 + (size_t)sp * s.R] : 0.f;
+            o4[sp] = on ? *reinterpret_cast<const float4*>(part_o + (row0 + (size_t)sp * s.R) * kD + lane * 4)
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float M = -INFINITY, L = 0.f;
+#pragma unroll
+        for (int sp = 0; sp < CMBW_MAX_SPLITS; ++sp) M = fmaxf(M, m[sp]);
+#pragma unroll
+        for (int sp = 0; sp < CMBW_MAX_SPLITS; ++sp) {
+            const float w = m[sp] == -INFINITY ? 0.f : exp2f(m[sp] - M);
+            L = fmaf(l[sp], w, L);
+            oc.x = fmaf(o4[sp].x, w, oc.x); oc.y = fmaf(o4[sp].y, w, oc.y);
+            oc.z = fmaf(o4[sp].z, w, oc.z); oc.w = fmaf(o4[sp].w, w, oc.w);
+        }
+        oc.x /= L; oc.y /= L; oc.z /= L; oc.w /= L;
+        onorm = warp_sum((oc.x * oc.x + oc.y * oc.y) + (oc.z * oc.z + oc.w * oc.w));
+        lse2 = M + log2f(L);
+    }
+    *reinterpret_cast<float4*>(ws + plan.off_o / 4 + orow * kD + lane * 4) = oc;
+    if (obf) {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(-2.f * oc.x, -2.f * oc.y), hi = __floats2bfloat162_rn(-2.f * oc.z, -2.f * oc.w);
+        *reinterpret_cast<uint2*>(obf + orow * kD + lane * 4) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+    if (lane == 0) {
+        (ws + plan.off_lse2 / 4)[orow] = lse2;
+        (ws + plan.off_onorm / 4)[orow] = onorm;
+        if (cpair) { cpair[0] = -lse2; cpair[2] = onorm; }
+    }
+}
+
 // One block of 128 threads per (unit, output row), like the combine kernel, but the row comes from the
 // caller: o [B,Hq,W,d] and the natural-log LSE [B,Hq,W] of an attention kernel that already ran.
 // Row r of KV head g is (query head g*G + r / W, window query r % W).
@@ -466,6 +523,13 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
 }
 
 obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream) {
+    const long long rows = (long long)s.B * s.Hkv * plan.rows_out;
+    if (plan.n_splits <= CMBW_MAX_SPLITS && rows >= 1024) {           // many rows, few splits: a warp per row
+        ProfScope ps("combine", stream);
+        OBC_CUDA_TRY(launch_pdl(simt_combine_rows_kernel, dim3((unsigned)((rows + CMB_NT / 32 - 1) / (CMB_NT / 32))), dim3(CMB_NT), 0,
+                                stream, 1, s, plan, (float*)ws));
+        return OBC_OK;
+    }
     { ProfScope ps("combine", stream); OBC_CUDA_TRY(launch_pdl(simt_combine_kernel, dim3(s.B * s.Hkv * plan.rows_out), dim3(CMB_NT), 0, stream, 1, s, plan, (float*)ws)); }
     return OBC_OK;
 }

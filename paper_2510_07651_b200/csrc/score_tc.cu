@@ -185,6 +185,14 @@ struct TcParams {
 __device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
 __device__ __forceinline__ int tc_seq_len(const TcParams& p, int b) { return tc_seq_len_raw(p.seq_lens, b, p.Nmax); }
 
+// Last token that any of the window rows [r0, r1] of a unit sees (row r is query position N - W + r mod W
+// of its head): tiles that begin after it contribute nothing to these rows and are not visited.  With a
+// short window every chunk of rows reaches the end of the cache; with the whole sequence as the window
+// (W = N) about half of the (row chunk, token tile) pairs drop out.
+__device__ __forceinline__ int rows_last_token(int r0, int r1, int W, int N, int causal) {
+    return (causal && r0 / W == r1 / W) ? N - W + (r1 % W) : N - 1;
+}
+
 // Walks the CTA's share of the token tiles.  All non-empty 128-token tiles of all (batch item,
 // KV head) units, in (unit, tile) order, are cut into gridDim.x contiguous, equally long runs, so
 // that a CTA stays inside one unit for as long as possible (its Q / O operands stay in shared
@@ -669,7 +677,9 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     tma_load_4d(dv + kHalfBytes, &map_v, bar(MC_FULL + j), 64, t0, g, b);
                 }
                 if (pitem == 0) pdl_wait();                        // K and V were read by pass 1; -2 O is the preceding kernel's output
-                for (int c = 0; c < nc && !failed; ++c, ++citem) {
+                const int pair_first = tw.tile * 2 * TILE, Nu = tc_seq_len(p, b);
+                for (int c = 0; c < nc && !failed; ++c) {
+                    if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, p.causal) < pair_first) continue;
                     const uint32_t qb = citem & 1;
                     if (!mbar_wait(bar(MC_QO_EMPTY + qb), ((citem >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                     mbar_expect_tx(bar(MC_QO_FULL + qb), qo_bytes);
@@ -680,6 +690,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     tma_load_2d(dq + kHalfB64, &map_q, bar(MC_QO_FULL + qb), 64, qrow);
                     tma_load_2d(dob, &map_o, bar(MC_QO_FULL + qb), 0, orow);
                     tma_load_2d(dob + kHalfB64, &map_o, bar(MC_QO_FULL + qb), 64, orow);
+                    ++citem;
                 }
             }
             // drain: every copy this thread issued must have landed before the CTA may exit
@@ -699,7 +710,9 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             uint32_t pitem = 0, citem = 0;
             for (; !tw.done() && !failed; tw.next(), ++pitem) {
                 if (!mbar_wait(bar(MC_FULL + 0), pitem & 1) || !mbar_wait(bar(MC_FULL + 1), pitem & 1)) { failed = true; fail_site = __LINE__; break; }
-                for (int c = 0; c < nc && !failed; ++c, ++citem) {
+                const int pair_first = tw.tile * 2 * TILE, Nu = tc_seq_len(p, tw.unit / p.Hkv);
+                for (int c = 0; c < nc && !failed; ++c) {
+                    if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, p.causal) < pair_first) continue;
                     const uint32_t qb = citem & 1;
                     if (!mbar_wait(bar(MC_QO_FULL + qb), (citem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
                     const uint32_t bq = desc_lo_k(sbase + MC_OFF_QO + qb * kQoBuf), bo = bq + ((2 * kHalfB64) >> 4);
@@ -719,6 +732,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     }
                     if (failed) break;
                     tc_commit(bar(MC_QO_EMPTY + qb));              // this Q / O buffer may be refilled
+                    ++citem;
                 }
                 if (!failed) { tc_commit(bar(MC_EMPTY + 0)); tc_commit(bar(MC_EMPTY + 1)); }   // both tiles no longer read
             }
@@ -745,7 +759,9 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             }
             if (failed) break;
             if (lane == 0) mbar_arrive(bar(MC_NV + (pitem & 1)));
-            for (int c = 0; c < nc; ++c, ++citem) {
+            const int pair_first = tw.tile * 2 * TILE, Nu = tc_seq_len(p, unit / p.Hkv);
+            for (int c = 0; c < nc; ++c) {
+                if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, p.causal) < pair_first) continue;
                 const uint32_t cs = citem & 3;
                 const size_t crow = (size_t)unit * p.rows_out + (size_t)c * MC_ROWS + t64;
                 const float2 cst = make_float2(-p.lse2[crow], p.onorm[crow] * (VARS == OBC_VAR_VK ? p.scale : 1.f));
@@ -758,6 +774,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 cdst[0] = cst.x; cdst[2] = cst.y;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(MC_CONST + cs));
+                ++citem;
             }
         }
     } else {
@@ -775,7 +792,9 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
-            for (int c = 0; c < nc; ++c, ++citem) {
+            const int pair_first = tw.tile * 2 * TILE;
+            for (int c = 0; c < nc; ++c) {
+                if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, N, p.causal) < pair_first) continue;
                 const uint32_t item = 2 * citem + wg, buf = item & 3, cs = citem & 3;
                 if (!mbar_wait(bar(MC_CONST + cs), (citem >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
                 if (!mbar_wait(bar(MC_TM_FULL + buf), (item >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
@@ -789,6 +808,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(MC_TM_EMPTY + buf));
+                ++citem;
             }
             if (failed) break;
             if (!mbar_wait(bar(MC_NV + (pitem & 1)), (pitem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
@@ -873,7 +893,7 @@ struct P1Params {
     int n_splits, tiles_per_split;                         // CTAs per (unit, chunk); each writes one partial
     int l2_stream;                                         // K/V copies carry the "evict first" L2 hint
     float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
-    float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the chunk-0 CTAs
+    float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the CTAs of the last row chunk
     unsigned int* status;
     unsigned long long* span;                              // [2]: ~(earliest CTA start), latest CTA end, in globaltimer ns
 };
@@ -951,8 +971,8 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
-        // a K/V stage is released by the MMA commit and, in chunk-0 CTAs, by the two ||v||^2 warps
-        for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), c == 0 ? 3 : 1); }
+        // a K/V stage is released by the MMA commit and, in the CTAs of the last row chunk, by the two ||v||^2 warps
+        for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), c == p.n_chunks - 1 ? 3 : 1); }
         mbar_init(bar(P1_QFULL), 1); mbar_init(bar(P1_ODONE), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(bar(P1_SFULL + i), 1); mbar_init(bar(P1_PFULL + i), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -972,7 +992,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.status = 0u;
     const int N = tc_seq_len_raw(p.seq_lens, b, p.Nmax);
     const int tile_lo = split * p.tiles_per_split;
-    const int tile_hi = min(tile_lo + p.tiles_per_split, (N + TILE - 1) / TILE);
+    // tiles past the last token that any row of this chunk sees are not visited
+    const int chunk_last = rows_last_token(c * p.chunk_rows, min((c + 1) * p.chunk_rows, p.R) - 1, p.W, N, p.causal);
+    const int tile_hi = min(min(tile_lo + p.tiles_per_split, (N + TILE - 1) / TILE), chunk_last / TILE + 1);
     const int n_tiles = max(tile_hi - tile_lo, 0);
 
     if (warp == 0) {
@@ -1045,10 +1067,11 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (!failed) tc_commit(bar(P1_ODONE));
         }
     } else if (warp < 4) {
-        // ====================== ||v_p||^2 of every cached token (chunk-0 CTAs) ===================
+        // ============ ||v_p||^2 of every cached token (CTAs of the last row chunk) ===============
         // Pass 2 needs it per token; the V tile is in shared memory here anyway, and these two warps
         // have nothing else to do, whereas in pass 2 every issue slot next to the epilogue counts.
-        if (c == 0) {
+        // (The last chunk holds the last window row, which sees every token, so its CTAs visit every tile.)
+        if (c == p.n_chunks - 1) {
             const int t64 = threadIdx.x - 64;                                // 0..63
             for (int i = 0; i < n_tiles && !failed; ++i) {
                 const uint32_t st = i % P1_NSTAGE;

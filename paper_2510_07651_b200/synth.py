@@ -156,6 +156,14 @@ def config(idx: int, *, shrink: int = 1, seed: int | None = None) -> tuple[Prefi
     return c, run
 
 
+def full_history(n: int = 4096, *, seed: int = 1240) -> tuple[PrefillCase, dict]:
+    """Llama-3-8B-shaped layer scored with the whole sequence as the perturbation window (W = N): every
+    query position is a window row, as in the w = 1 accumulation the paper attributes to H2O (Sec. 4.3)."""
+    c = make_prefill("history", B=1, Hq=32, Hkv=8, d=128, W=n, N=n, dtype="bf16", seed=seed)
+    run = dict(variants=["VK"], budget=n // 8, pool_mode="max", pool_kernel=7, n_sink=0, n_recent=32)
+    return c, run
+
+
 @dataclasses.dataclass
 class DecodeCase:
     """Decode-time rescoring problem: an initial cache plus per-step (q, k, v)."""
