@@ -413,7 +413,7 @@ def run_other(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     steps, warmup = args.steps, max(args.warmup, 3)
 
-    if args.workload == "decode":
+    if args.workload in ("decode", "decode-window"):
         # Llama-3-8B shapes, batch 32: a 16384-token context already reduced to the 4096-token budget;
         # every step appends one token, rescores all 4097 live slots (W = 1) and evicts one.
         B, Hq, Hkv, n0, budget, n_sink, n_recent = 32, 32, 8, 4096, 4096, 4, 256
@@ -434,10 +434,13 @@ def run_other(args):
         v_t = [vd[t].unsqueeze(2) for t in range(ns)]
         p = api.decode_params(q_t[0], kc, budget=budget, n_sink=n_sink, n_recent=n_recent)
         ws = torch.empty(api.obc_decode_workspace(p), dtype=torch.uint8, device="cuda")
+        window = 16 if args.workload == "decode-window" else 0       # scores accumulated over the last 16 steps only
+        hist = torch.zeros((B, Hkv, window, cap), dtype=torch.float32, device="cuda") if window else None
 
         def step(t):
             api.obc_decode_step(q_t[t % ns], k_t[t % ns], v_t[t % ns], kc, vc, s_acc, pos, state, n0 + t,
-                                budget=budget, n_sink=n_sink, n_recent=n_recent, variant="VK", workspace=ws)
+                                budget=budget, n_sink=n_sink, n_recent=n_recent, variant="VK", workspace=ws,
+                                acc_window=window, s_hist=hist)
         for t in range(warmup):
             step(t)
         torch.cuda.synchronize()
@@ -456,7 +459,8 @@ def run_other(args):
         line = {"metric": "decode rescoring steps/sec", "value": steps / (ms * 1e-3), "unit": "steps/s",
                 "ms_per_step": ms / steps, "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": "decode: B32 Hq32 Hkv8 d128, live 4096 -> 4097 -> 4096 per step, W1, OBCache-V&K, "
-                                       "4 sinks, 256 recent, one eviction per head per step"},
+                                       "4 sinks, 256 recent, one eviction per head per step"
+                                       + (f", accumulator = the last {window} steps' scores" if window else "")},
                 "hbm_gbs_algorithmic": live_bytes / (ms / steps * 1e-3) / 1e9,
                 "kernels": {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}}
         print(json.dumps(line))
@@ -570,7 +574,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--eager", action="store_true", help="time plain library calls instead of replaying CUDA graphs")
-    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive", "history4k"],
+    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive", "history4k", "decode-window"],
                     help="llama32k is the headline benchmark; the others print a shorter line (1 GPU)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"

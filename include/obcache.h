@@ -251,6 +251,16 @@ obc_status obc_compact(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int3
  *   4. if live > budget: frees the live slot with the smallest s_acc among tokens with
  *      n_sink <= pos <= step_pos - n_recent (equal values: the highest pos), which becomes
  *      next_slot; otherwise next_slot = hi.
+ *
+ * Accumulation window (Sec. 6, "Choice of Perturbation Window in Decoding": scores accumulated
+ * only within a recent window instead of over the whole history).  With acc_window = w > 0 step 3
+ * becomes  s_acc[slot] = sum of the slot's scores of the last w steps (this one included, fewer
+ * while the token is younger than w steps).  The per-step scores are kept in the ring s_hist, fp32
+ * [B,Hkv,w,capacity], which the caller zero-fills before the first step and then leaves alone; the
+ * step with position step_pos uses ring row step_pos mod w, so consecutive steps must advance
+ * step_pos by one.  The sum is formed afresh every step, rows 0..w-1 in order; what s_acc held
+ * before is not used (a token's column of the ring is cleared when the token enters the cache).
+ * acc_window = 0 (s_hist ignored) accumulates over all steps.  acc_window > 4096: OBC_ERR_SHAPE.
  * ------------------------------------------------------------------------------------------ */
 typedef struct {
     size_t struct_size;
@@ -259,6 +269,8 @@ typedef struct {
     int32_t budget, n_sink, n_recent;
     uint32_t variant;         /* exactly one OBC_VAR_* bit */
     float scale;              /* <= 0 selects 1/sqrt(head_dim) */
+    int32_t acc_window;       /* 0: accumulate over all steps; w > 0: over the last w steps */
+    float* s_hist;            /* device, [B,Hkv,acc_window,capacity]; NULL when acc_window == 0 */
 } obc_decode_params;
 
 obc_status obc_decode_workspace(const obc_decode_params* p, size_t* bytes /* host out */);

@@ -211,8 +211,12 @@ class DecodeState:
     queries -> s_acc += score -> if live > budget, evict one slot (it becomes next_slot).
     """
 
-    def __init__(self, k0, v0, cap, s_acc0=None):
+    def __init__(self, k0, v0, cap, s_acc0=None, window=0):
+        """`window` = w > 0: the accumulator is the sum of a token's scores over the last w steps only
+        (Sec. 6, accumulation within a recent window); 0: over every step since the token entered."""
         n0, d = k0.shape
+        self.window = int(window)
+        self.hist = np.zeros((self.window, cap), np.float64)      # ring of per-step scores, row = step_pos mod w
         self.k = np.zeros((cap, d), np.float32); self.v = np.zeros((cap, d), np.float32)
         self.k[:n0] = k0; self.v[:n0] = v0
         self.pos = np.full(cap, -1, np.int32); self.pos[:n0] = np.arange(n0)
@@ -224,11 +228,21 @@ class DecodeState:
     def append(self, k_t, v_t, step_pos):
         s = self.next_slot
         self.k[s] = k_t; self.v[s] = v_t; self.pos[s] = step_pos; self.s_acc[s] = 0.0
+        if self.window:
+            self.hist[:, s] = 0.0
         self.live += 1
         self.hi = max(self.hi, s + 1)
 
     def scores(self, qg, variant="VK"):
         return decode_scores(qg, self.k, self.v, self.pos, self.hi, variant)
+
+    def accumulate(self, sc, step_pos):
+        """The accumulator after this step's scores `sc` [cap] (float64; the state's own s_acc is left to the
+        caller, who may store a rounded or a teacher-forced value)."""
+        if not self.window:
+            return self.s_acc.astype(np.float64) + sc
+        self.hist[step_pos % self.window] = np.where(self.pos >= 0, sc, 0.0)
+        return self.hist.sum(axis=0)
 
     def evict(self, step_pos, budget, n_sink, n_recent):
         """Evict per the fp32 accumulator if over budget; returns the evicted slot or -1."""

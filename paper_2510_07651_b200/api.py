@@ -61,7 +61,7 @@ class obc_decode_params(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("batch", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("capacity", C.c_int32),
                 ("budget", C.c_int32), ("n_sink", C.c_int32), ("n_recent", C.c_int32),
-                ("variant", C.c_uint32), ("scale", C.c_float)]
+                ("variant", C.c_uint32), ("scale", C.c_float), ("acc_window", C.c_int32), ("s_hist", C.c_void_p)]
 
 
 class obc_kernel_time(C.Structure):
@@ -287,11 +287,15 @@ def obc_compact(k, v, idx, *, k_out=None, v_out=None, scores_in=None, scores_out
     return (k_out, v_out) if scores_in is None else (k_out, v_out, scores_out)
 
 
-def decode_params(q_t, k_cache, *, budget, n_sink, n_recent, variant="VK", scale=0.0) -> obc_decode_params:
+def decode_params(q_t, k_cache, *, budget, n_sink, n_recent, variant="VK", scale=0.0, acc_window=0,
+                  s_hist=None) -> obc_decode_params:
     B, Hq, _, d = q_t.shape
     _, Hkv, cap, _ = k_cache.shape
+    if acc_window > 0 and s_hist is not None:
+        assert s_hist.dtype == torch.float32 and s_hist.is_contiguous() and tuple(s_hist.shape) == (B, Hkv, acc_window, cap)
     return obc_decode_params(C.sizeof(obc_decode_params), B, Hq, Hkv, d, cap, budget, n_sink, n_recent,
-                             VARIANTS[variant] if isinstance(variant, str) else variant, float(scale))
+                             VARIANTS[variant] if isinstance(variant, str) else variant, float(scale),
+                             int(acc_window), _ptr(s_hist))
 
 
 def obc_decode_workspace(p: obc_decode_params) -> int:
@@ -301,9 +305,12 @@ def obc_decode_workspace(p: obc_decode_params) -> int:
 
 
 def obc_decode_step(q_t, k_t, v_t, k_cache, v_cache, s_acc, pos, state, step_pos, *, budget, n_sink, n_recent,
-                    variant="VK", scale=0.0, workspace=None):
-    """One in-place decode rescoring + eviction step (see include/obcache.h)."""
-    p = decode_params(q_t, k_cache, budget=budget, n_sink=n_sink, n_recent=n_recent, variant=variant, scale=scale)
+                    variant="VK", scale=0.0, workspace=None, acc_window=0, s_hist=None):
+    """One in-place decode rescoring + eviction step (see include/obcache.h).  With acc_window = w > 0 the
+    accumulator is the sum of the last w steps' scores and s_hist is the zero-initialised fp32 ring
+    [B,Hkv,w,capacity] that holds them."""
+    p = decode_params(q_t, k_cache, budget=budget, n_sink=n_sink, n_recent=n_recent, variant=variant, scale=scale,
+                      acc_window=acc_window, s_hist=s_hist)
     ws = _workspace(obc_decode_workspace(p), k_cache, workspace)
     _check(lib().obc_decode_step(C.byref(p), as_tensor4(q_t), as_tensor4(k_t), as_tensor4(v_t), as_tensor4(k_cache),
                                  as_tensor4(v_cache), s_acc.data_ptr(), pos.data_ptr(), state.data_ptr(),

@@ -275,9 +275,11 @@ static obc_status resolve_decode(const obc_decode_params* p, DecodeShape* s) {
     if (p->variant != OBC_VAR_V && p->variant != OBC_VAR_K && p->variant != OBC_VAR_VK && p->variant != OBC_VAR_ATTN)
         return OBC_ERR_UNSUPPORTED;
     if ((long long)p->batch * p->n_kv_heads > 65535) return OBC_ERR_SHAPE;
+    if (p->acc_window < 0 || p->acc_window > 4096) return OBC_ERR_SHAPE;
     *s = DecodeShape{p->batch, p->n_q_heads, p->n_kv_heads, p->n_q_heads / p->n_kv_heads, p->capacity,
                      p->budget, p->n_sink, p->n_recent, p->variant,
-                     p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)kD)};
+                     p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)kD),
+                     p->acc_window, p->acc_window > 0 ? p->s_hist : nullptr};
     return OBC_OK;
 }
 
@@ -298,6 +300,8 @@ obc_status obc_decode_step(const obc_decode_params* p, obc_tensor q_t, obc_tenso
     obc_status st = resolve_decode(p, &s);
     if (st != OBC_OK) return st;
     if (!s_acc || !pos || !state) return OBC_ERR_NULL;
+    if (s.acc_window > 0 && !s.s_hist) return OBC_ERR_NULL;
+    if (s.acc_window > 0 && ((uintptr_t)s.s_hist & 3) != 0) return OBC_ERR_ALIGN;
     const obc_tensor* ts[5] = {&q_t, &k_t, &v_t, &k_cache, &v_cache};
     for (int i = 0; i < 5; ++i) {
         if ((st = check_tensor(*ts[i], true)) != OBC_OK) return st;

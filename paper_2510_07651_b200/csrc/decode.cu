@@ -154,6 +154,8 @@ decode_pass1_kernel(DecodeShape s, DecodePlan plan, TensorView q, TensorView kt,
         if (tid < 16) reinterpret_cast<uint4*>(kdst)[tid] = reinterpret_cast<const uint4*>(bf_row(kt, b, g, 0))[tid];
         else if (tid < 32) reinterpret_cast<uint4*>(vdst)[tid - 16] = reinterpret_cast<const uint4*>(bf_row(vt, b, g, 0))[tid - 16];
         else if (tid == 32) { pos[(size_t)unit * s.cap + next] = step_pos; s_acc[(size_t)unit * s.cap + next] = 0.f; }
+        // a token that enters the cache starts with an empty score history (the slot's former tenant left its own)
+        for (int r = tid; r < s.acc_window; r += CH) s.s_hist[((size_t)unit * s.acc_window + r) * s.cap + next] = 0.f;
     }
     __syncthreads();                                       // the new token's row is in place
     // One buffer: the K rows first; the V rows take their place as soon as the logits are out and travel during
@@ -438,7 +440,20 @@ decode_score_kernel(DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
                 sc += a2 * nv + a2 * Z * Z * (sNo[r] + nv - 2.f * t[r]) + 2.f * a2 * Z * (nv - t[r]);
             else sc += a;
         }
-        const float acc = acc_in + sc;
+        float acc = acc_in + sc;
+        if (s.acc_window > 0) {                                // the last acc_window steps only, summed afresh in ring order
+            float* hcol = s.s_hist + (size_t)unit * s.acc_window * s.cap + slot;
+            const int now = step_pos % s.acc_window;
+            acc = 0.f;
+            for (int r0 = 0; r0 < s.acc_window; r0 += 8) {      // eight loads in flight
+                float hv[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) hv[u] = (r0 + u < s.acc_window && r0 + u != now) ? hcol[(size_t)(r0 + u) * s.cap] : 0.f;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) acc += (r0 + u == now) ? sc : hv[u];
+            }
+            hcol[(size_t)now * s.cap] = sc;
+        }
         s_acc[(size_t)unit * s.cap + slot] = acc;
         if (my_pos >= s.n_sink && my_pos <= step_pos - s.n_recent) cand = MinCand{acc, my_pos, slot, 0};
     }

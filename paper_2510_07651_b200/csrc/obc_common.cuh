@@ -104,6 +104,8 @@ struct DecodeShape {
     int B, Hq, Hkv, G, cap, budget, n_sink, n_recent;
     unsigned variant;
     float scale;
+    int acc_window;                      // 0, or the number of steps whose scores make up the accumulator
+    float* s_hist;                       // [B,Hkv,acc_window,cap] ring of per-step scores
 };
 size_t decode_workspace_bytes(const DecodeShape& s);
 obc_status launch_decode(const DecodeShape& s, TensorView q, TensorView kt, TensorView vt,

@@ -119,6 +119,14 @@ def test_compact_and_decode_validation(L):
     assert L.obc_decode_workspace(C.byref(dp), C.byref(n)) == -2
     dp.capacity, dp.variant = 65, 3
     assert L.obc_decode_workspace(C.byref(dp), C.byref(n)) == -3
+    dp.variant, dp.acc_window = 4, -1                          # accumulation window: 0..4096 steps
+    assert L.obc_decode_workspace(C.byref(dp), C.byref(n)) == -2
+    dp.acc_window = 4097
+    assert L.obc_decode_workspace(C.byref(dp), C.byref(n)) == -2
+    dp.acc_window = 8                                          # a window needs its ring of per-step scores
+    assert L.obc_decode_workspace(C.byref(dp), C.byref(n)) == 0
+    assert L.obc_decode_step(C.byref(dp), t(4096), t(4096), t(4096), t(4096), t(4096), 4096, 4096, 4096, 70,
+                             4096, n.value, None) == -1
 
 
 def test_missing_library_fails_loudly(monkeypatch):

@@ -13,7 +13,7 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", seed=55, s_acc0=False):
+def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", seed=55, s_acc0=False, window=0):
     G = Hq // Hkv
     dc = synth.make_decode(B=B, Hq=Hq, Hkv=Hkv, d=128, n0=n0, steps=steps, seed=seed)
     dev = "cuda"
@@ -30,8 +30,9 @@ def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", see
         s_acc[:, :, :n0] = torch.from_numpy(init).cuda()
     state = torch.zeros((B, Hkv, 4), dtype=torch.int32, device=dev)
     state[..., 0] = n0; state[..., 1] = n0; state[..., 2] = n0
-    sts = [[ref.DecodeState(dc.k0[b, h], dc.v0[b, h], cap, None if init is None else init[b, h])
+    sts = [[ref.DecodeState(dc.k0[b, h], dc.v0[b, h], cap, None if init is None else init[b, h], window=window)
             for h in range(Hkv)] for b in range(B)]
+    hist = torch.zeros((B, Hkv, window, cap), dtype=torch.float32, device=dev) if window else None
     qd, kd, vd = H.dev_bf16(dc.q_t_bits), H.dev_bf16(dc.k_t_bits), H.dev_bf16(dc.v_t_bits)
     ws = None
     n_evicted = 0
@@ -39,7 +40,7 @@ def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", see
         step_pos = n0 + t
         ws = api.obc_decode_step(qd[t].unsqueeze(2), kd[t].unsqueeze(2), vd[t].unsqueeze(2), kc, vc, s_acc, pos,
                                  state, step_pos, budget=budget, n_sink=n_sink, n_recent=n_recent, variant=variant,
-                                 workspace=ws)
+                                 workspace=ws, acc_window=window, s_hist=hist)
         torch.cuda.synchronize()
         g_acc, g_pos, g_state = s_acc.cpu().numpy(), pos.cpu().numpy(), state.cpu().numpy()
         for b in range(B):
@@ -47,7 +48,7 @@ def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", see
                 st = sts[b][h]
                 st.append(dc.k_t[t, b, h], dc.v_t[t, b, h], step_pos)
                 sc = st.scores(dc.q_t[t, b, h * G:(h + 1) * G], variant)
-                want_acc = st.s_acc.astype(np.float64) + sc
+                want_acc = st.accumulate(sc, step_pos)
                 livemask = st.pos >= 0
                 H.assert_scores_close(g_acc[b, h][livemask], want_acc[livemask], "bf16", tight=2e-2,
                                       what=f"step {t} unit {b},{h}")
@@ -87,3 +88,11 @@ def test_decode_other_variants(variant):
 def test_decode_every_group_size(G):
     # the MMA tiles pad the query heads of a group to 8 columns: every group size, two chunks, an odd extent
     _run(B=1, Hq=2 * G, Hkv=2, n0=290, budget=300, cap=301, n_sink=3, n_recent=20, steps=24)
+
+
+@pytest.mark.parametrize("window", [1, 5, 16])
+def test_decode_accumulation_window(window):
+    """Scores accumulated over the last `window` steps only: steady-state eviction with slot reuse, several
+    chunks, a window shorter and longer than a token's usual stay beyond the protected recents."""
+    ev = _run(B=2, Hq=8, Hkv=2, n0=280, budget=290, cap=291, n_sink=4, n_recent=12, steps=40, window=window)
+    assert ev == 2 * 2 * 30

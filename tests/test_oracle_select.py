@@ -138,6 +138,43 @@ def test_decode_state_keeps_sinks_and_recents_and_respects_budget():
         assert set(range(step_pos - n_recent + 1, step_pos + 1)) <= set(livepos.tolist())
 
 
+@pytest.mark.parametrize("window", [1, 3, 7, 64])
+def test_decode_window_accumulator_matches_a_log_kept_per_token(window):
+    """Accumulation within a recent window (Sec. 6): the state's ring, indexed by slot and step mod w, must
+    give every live token the sum of the scores it received in the last w steps, as read off a plain log
+    keyed by (token position, step) that knows nothing of slots or rings."""
+    rng = np.random.default_rng(40 + window)
+    G, d, n0, budget, n_sink, n_recent, steps = 2, 8, 10, 12, 2, 3, 40
+    k0 = rng.standard_normal((n0, d)).astype(np.float32)
+    v0 = rng.standard_normal((n0, d)).astype(np.float32)
+    st = ref.DecodeState(k0, v0, cap=budget + 1, window=window)
+    full = ref.DecodeState(k0, v0, cap=budget + 1)                       # accumulates over every step
+    log = {}                                                             # (position, step) -> score
+    for t in range(steps):
+        step_pos = n0 + t
+        k_t, v_t = rng.standard_normal(d).astype(np.float32), rng.standard_normal(d).astype(np.float32)
+        q_t = rng.standard_normal((G, d)).astype(np.float32)
+        st.append(k_t, v_t, step_pos)
+        sc = st.scores(q_t)
+        for slot in np.flatnonzero(st.pos >= 0):
+            log[(int(st.pos[slot]), t)] = float(sc[slot])
+        acc = st.accumulate(sc, step_pos)
+        for slot in np.flatnonzero(st.pos >= 0):
+            want = sum(log.get((int(st.pos[slot]), u), 0.0) for u in range(max(0, t - window + 1), t + 1))
+            assert abs(acc[slot] - want) <= 1e-12 * max(1.0, abs(want))
+        if window == 1:                                                  # only this step's scores
+            np.testing.assert_array_equal(acc[st.pos >= 0], sc[st.pos >= 0])
+        st.s_acc[:] = acc.astype(np.float32)
+        st.evict(step_pos, budget, n_sink, n_recent)
+        if window >= steps:                                              # never slides: the plain accumulation
+            full.append(k_t, v_t, step_pos)
+            facc = full.accumulate(full.scores(q_t), step_pos)
+            full.s_acc[:] = facc.astype(np.float32)
+            full.evict(step_pos, budget, n_sink, n_recent)
+            assert np.array_equal(full.pos, st.pos)
+            np.testing.assert_allclose(acc[st.pos >= 0], facc[st.pos >= 0], rtol=1e-6, atol=1e-12)
+
+
 # ---- head-adaptive budgets (global ranking across heads with a per-head safeguard) ----------------
 def brute_adaptive(pooled, budget, n_sink, n_recent, safeguard):
     """Plain-Python statement: every head's s best candidates, then the best of the rest of all heads."""
