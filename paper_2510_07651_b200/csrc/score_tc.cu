@@ -180,6 +180,8 @@ struct TcParams {
     unsigned int* status;                     // device status word (workspace header)
     unsigned long long* span;                 // [2]: ~(earliest CTA start), latest CTA end, in globaltimer ns
     int l2_stream;                            // K/V copies carry the "evict first" L2 hint (their last use)
+    int csplit;                               // multi-chunk kernel: CTAs that share the row chunks of one tile pair
+    float* partial;                           // csplit > 1: [csplit][planes][units][Nmax] partial scores
 };
 
 __device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
@@ -193,6 +195,17 @@ __device__ __forceinline__ int rows_last_token(int r0, int r1, int W, int N, int
     return (causal && r0 / W == r1 / W) ? N - W + (r1 % W) : N - 1;
 }
 
+// Multi-chunk pass 2 with the row chunks of a tile pair shared by `csplit` CTAs: position t of a unit with
+// P pairs stands for pair zigzag(t mod P) and the chunks c = t / P, t / P + csplit, ...  The zigzag (first,
+// last, second, second to last, ...) puts a pair that many rows see next to one that few rows see, so that
+// the contiguous runs of positions that the CTAs take weigh about the same under a causal window.
+__device__ __forceinline__ void split_position(int t, int positions_in_unit, int csplit, int& pair, int& cs) {
+    if (csplit == 1) { pair = t; cs = 0; return; }
+    const int P = positions_in_unit / csplit, q = t % P;
+    cs = t / P;
+    pair = (q & 1) ? P - 1 - (q >> 1) : (q >> 1);
+}
+
 // Walks the CTA's share of the token tiles.  All non-empty 128-token tiles of all (batch item,
 // KV head) units, in (unit, tile) order, are cut into gridDim.x contiguous, equally long runs, so
 // that a CTA stays inside one unit for as long as possible (its Q / O operands stay in shared
@@ -202,11 +215,12 @@ struct TileWalk {
     long long left;                           // positions still to visit, including the current one
     const TcParams* p;
     int span;                                 // consecutive tiles of a unit that one position stands for
+    int reps;                                 // positions per such group of tiles (CTAs that share its row chunks)
     __device__ __forceinline__ int tiles_of(int b) const {
-        return ((tc_seq_len(*p, b) + TILE - 1) / TILE + span - 1) / span;
+        return ((tc_seq_len(*p, b) + TILE - 1) / TILE + span - 1) / span * reps;
     }
-    __device__ void init(const TcParams& prm, int tiles_per_position = 1) {
-        p = &prm; span = tiles_per_position;
+    __device__ void init(const TcParams& prm, int tiles_per_position = 1, int positions_per_group = 1) {
+        p = &prm; span = tiles_per_position; reps = positions_per_group;
         long long total = 0;
         if (p->seq_lens) { for (int b = 0; b < p->B; ++b) total += (long long)p->Hkv * tiles_of(b); }
         else total = (long long)p->B * p->Hkv * tiles_of(0);
@@ -611,7 +625,9 @@ enum { MC_FULL = 0, MC_EMPTY = 2, MC_QO_FULL = 4, MC_QO_EMPTY = 6, MC_TM_FULL = 
 constexpr uint32_t MC_OFF_TMEM = MC_OFF_BAR + MC_NBARS * 8;
 constexpr uint32_t kSmemMulti = MC_OFF_TMEM + 16 + 1024;
 
-template <unsigned VARS>
+// SPLIT: the general walk (row chunks of a pair shared by several CTAs, hidden tile pairs skipped); without
+// it every CTA takes whole pairs and every chunk, which is all a short window over a long cache needs.
+template <unsigned VARS, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
                       const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -658,7 +674,11 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
     // items 2 * citem + j.  Rings: K/V stage j; Q/O buffer citem & 1; constant slot citem & 3; TMEM
     // buffer item & 3, so that epilogue group j always sees buffers j and j + 2.
     TileWalk tw;
-    tw.init(p, 2);
+    tw.init(p, 2, SPLIT ? p.csplit : 1);
+    const int cstep = SPLIT ? p.csplit : 1;
+    // a chunk of 64 rows can lose sight of a tile pair only if the window is longer than the chunk (with up to
+    // 64 window rows per head every chunk holds some head's last query, which sees the whole cache)
+    const bool may_skip = SPLIT && p.causal && p.W > MC_ROWS;
     if (!(warp == 0 && lane == 0)) pdl_wait();       // the producer thread waits after its first K/V copies
     if (warp == 0) {
         // ===================================== TMA producer =====================================
@@ -666,9 +686,11 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             uint32_t pitem = 0, citem = 0;
             for (; !tw.done() && !failed; tw.next(), ++pitem) {
                 const int unit = tw.unit, b = unit / p.Hkv, g = unit % p.Hkv;
+                int pair, cs;
+                if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
                 for (int j = 0; j < 2 && !failed; ++j) {
                     if (!mbar_wait(bar(MC_EMPTY + j), (pitem & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
-                    const int t0 = (tw.tile * 2 + j) * TILE;
+                    const int t0 = (pair * 2 + j) * TILE;
                     mbar_expect_tx(bar(MC_FULL + j), 2 * kOperandBytes);
                     const uint32_t dk = sbase + MC_OFF_K + j * kOperandBytes, dv = sbase + MC_OFF_V + j * kOperandBytes;
                     tma_load_4d(dk, &map_k, bar(MC_FULL + j), 0, t0, g, b);
@@ -677,9 +699,9 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     tma_load_4d(dv + kHalfBytes, &map_v, bar(MC_FULL + j), 64, t0, g, b);
                 }
                 if (pitem == 0) pdl_wait();                        // K and V were read by pass 1; -2 O is the preceding kernel's output
-                const int pair_first = tw.tile * 2 * TILE, Nu = tc_seq_len(p, b);
-                for (int c = 0; c < nc && !failed; ++c) {
-                    if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, p.causal) < pair_first) continue;
+                const int pair_first = pair * 2 * TILE, Nu = tc_seq_len(p, b);
+                for (int c = cs; c < nc && !failed; c += cstep) {
+                    if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, 1) < pair_first) continue;
                     const uint32_t qb = citem & 1;
                     if (!mbar_wait(bar(MC_QO_EMPTY + qb), ((citem >> 1) & 1) ^ 1)) { failed = true; fail_site = __LINE__; break; }
                     mbar_expect_tx(bar(MC_QO_FULL + qb), qo_bytes);
@@ -710,9 +732,11 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             uint32_t pitem = 0, citem = 0;
             for (; !tw.done() && !failed; tw.next(), ++pitem) {
                 if (!mbar_wait(bar(MC_FULL + 0), pitem & 1) || !mbar_wait(bar(MC_FULL + 1), pitem & 1)) { failed = true; fail_site = __LINE__; break; }
-                const int pair_first = tw.tile * 2 * TILE, Nu = tc_seq_len(p, tw.unit / p.Hkv);
-                for (int c = 0; c < nc && !failed; ++c) {
-                    if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, p.causal) < pair_first) continue;
+                int pair, cs;
+                if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
+                const int pair_first = pair * 2 * TILE, Nu = tc_seq_len(p, tw.unit / p.Hkv);
+                for (int c = cs; c < nc && !failed; c += cstep) {
+                    if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, 1) < pair_first) continue;
                     const uint32_t qb = citem & 1;
                     if (!mbar_wait(bar(MC_QO_FULL + qb), (citem >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
                     const uint32_t bq = desc_lo_k(sbase + MC_OFF_QO + qb * kQoBuf), bo = bq + ((2 * kHalfB64) >> 4);
@@ -759,9 +783,11 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             }
             if (failed) break;
             if (lane == 0) mbar_arrive(bar(MC_NV + (pitem & 1)));
-            const int pair_first = tw.tile * 2 * TILE, Nu = tc_seq_len(p, unit / p.Hkv);
-            for (int c = 0; c < nc; ++c) {
-                if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, p.causal) < pair_first) continue;
+            int pair, cs;
+            if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
+            const int pair_first = pair * 2 * TILE, Nu = tc_seq_len(p, unit / p.Hkv);
+            for (int c = cs; c < nc; c += cstep) {
+                if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, 1) < pair_first) continue;
                 const uint32_t cs = citem & 3;
                 const size_t crow = (size_t)unit * p.rows_out + (size_t)c * MC_ROWS + t64;
                 const float2 cst = make_float2(-p.lse2[crow], p.onorm[crow] * (VARS == OBC_VAR_VK ? p.scale : 1.f));
@@ -787,14 +813,16 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         uint32_t pitem = 0, citem = 0;
         for (; !tw.done() && !failed; tw.next(), ++pitem) {
             const int unit = tw.unit, b = unit / p.Hkv;
-            const int N = tc_seq_len(p, b), t0 = (tw.tile * 2 + wg) * TILE;
+            int pair, cs;
+            if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
+            const int N = tc_seq_len(p, b), t0 = (pair * 2 + wg) * TILE;
             const int ptok = t0 + tok;
             const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
-            const int pair_first = tw.tile * 2 * TILE;
-            for (int c = 0; c < nc; ++c) {
-                if (rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, N, p.causal) < pair_first) continue;
+            const int pair_first = pair * 2 * TILE;
+            for (int c = cs; c < nc; c += cstep) {
+                if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, N, 1) < pair_first) continue;
                 const uint32_t item = 2 * citem + wg, buf = item & 3, cs = citem & 3;
                 if (!mbar_wait(bar(MC_CONST + cs), (citem >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
                 if (!mbar_wait(bar(MC_TM_FULL + buf), (item >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
@@ -815,7 +843,9 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             const float2 nv21 = sNv[((pitem & 1) * 2 + wg) * TILE + tok];
             const float nv = nv21.x, nv1 = nv21.y;
             if (ptok < p.Nmax) {
-                float* out = p.scores + (size_t)unit * p.Nmax;
+                // with the chunks of the pair shared by several CTAs each writes its part of the sums (the scores are
+                // linear in them) into its own copy of the planes; tc_partial_sum_kernel adds the copies in order
+                float* out = (cstep > 1 ? p.partial + (size_t)cs * __popc(p.variants) * plane : p.scores) + (size_t)unit * p.Nmax;
                 const bool live = ptok < N;
                 const float s2 = p.scale * p.scale;
                 int pl = 0;
@@ -848,6 +878,24 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
+}
+
+// scores = sum over the csplit partial copies, in order, for the tokens that pass 2 visited (whole tile
+// pairs up to the unit's length; the zero padding beyond is written by pass 2 itself)
+__global__ void __launch_bounds__(256)
+tc_partial_sum_kernel(TcParams p, int n_planes) {
+    pdl_wait();
+    const int unit = blockIdx.y, b = unit / p.Hkv;
+    const int N = tc_seq_len(p, b);
+    const int end = min((N + 2 * TILE - 1) / (2 * TILE) * (2 * TILE), p.Nmax);
+    const size_t plane = (size_t)p.B * p.Hkv * p.Nmax;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < end; i += gridDim.x * blockDim.x)
+        for (int pl = 0; pl < n_planes; ++pl) {
+            const size_t at = (size_t)pl * plane + (size_t)unit * p.Nmax + i;
+            float sum = 0.f;
+            for (int cs = 0; cs < p.csplit; ++cs) sum += p.partial[(size_t)cs * n_planes * plane + at];
+            p.scores[at] = sum;
+        }
 }
 
 // =================================================================================================
@@ -1354,6 +1402,19 @@ bool tc_supported(const ScoreShape& s, int dtype, const TensorView& q) {
     return q.sh == (long long)s.W * q.st && q.sb == (long long)s.Hq * q.sh;
 }
 
+// Multi-chunk pass 2: with fewer tile pairs than about two per SM (a short cache scored over a long window)
+// the row chunks of every pair are shared by several CTAs.
+static int tc_chunk_split(const ScoreShape& s, const TcChunks& ch) {
+    if (ch.n_chunks <= 1) return 1;
+    const long long pairs = (long long)s.B * s.Hkv * (((s.Nmax + TILE - 1) / TILE + 1) / 2);
+    const int nc = ch.rows_out / MC_ROWS, sms = sm_count();
+    if (pairs >= 2LL * sms) return 1;
+    int c = (int)((3LL * sms + pairs - 1) / pairs);
+    if (c > 8) c = 8;
+    if (c > nc) c = nc;
+    return c < 1 ? 1 : c;
+}
+
 // Workspace plan of the tensor-core path: the SIMT plan's layout with splits counted in 128-token tiles.
 static SimtPlan make_tc_plan(const ScoreShape& s) {
     const TcChunks ch = tc_chunks(s.R);
@@ -1384,7 +1445,13 @@ static SimtPlan make_tc_plan(const ScoreShape& s) {
     return p;
 }
 
-size_t tc_workspace_bytes(const ScoreShape& s) { return make_tc_plan(s).bytes; }
+// the partial score planes of a shared multi-chunk pass 2 follow the plan's arrays
+static size_t tc_partial_bytes(const ScoreShape& s) {
+    const int cs = tc_chunk_split(s, tc_chunks(s.R));
+    return cs > 1 ? (size_t)cs * s.n_planes * s.B * s.Hkv * s.Nmax * 4 : 0;
+}
+
+size_t tc_workspace_bytes(const ScoreShape& s) { return make_tc_plan(s).bytes + tc_partial_bytes(s); }
 
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
                            float* scores, void* ws, cudaStream_t stream, const GivenAttention* given) {
@@ -1448,6 +1515,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     p.cpair = (const float4*)(wsb + plan.off_cpair);
     p.nv = (const float*)(wsb + plan.off_nv);
     p.l2_stream = l2_stream ? 1 : 0;
+    p.csplit = 1; p.partial = nullptr;
     const long long n_tiles = (long long)units * ((s.Nmax + TILE - 1) / TILE);
     const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
 
@@ -1462,14 +1530,27 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
             return OBC_ERR_CUDA;
         }
         p.n_chunks = ch.rows_out / MC_ROWS; p.chunk_rows = MC_ROWS;
+        p.csplit = tc_chunk_split(s, ch);
+        p.partial = (float*)(wsb + plan.bytes);
+        const long long positions = (long long)units * (((s.Nmax + TILE - 1) / TILE + 1) / 2) * p.csplit;
+        const int mgrid = (int)(positions < sm_count() ? positions : sm_count());
         auto launch_multi = [&](auto kernel) -> obc_status {
             OBC_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMulti));
-            { ProfScope ps("tc_pass2", stream); OBC_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmemMulti, stream, 1, mq64, mo64, mk, mv, p)); }
+            { ProfScope ps("tc_pass2", stream); OBC_CUDA_TRY(launch_pdl(kernel, dim3(mgrid), dim3(kThreads), kSmemMulti, stream, 1, mq64, mo64, mk, mv, p)); }
+            if (p.csplit > 1) {
+                ProfScope ps("partial_sum", stream);
+                OBC_CUDA_TRY(launch_pdl(tc_partial_sum_kernel, dim3((s.Nmax + 255) / 256, units), dim3(256), 0, stream, 1, p, s.n_planes));
+            }
             return OBC_OK;
         };
-        if (s.variants == OBC_VAR_VK) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_VK>);
-        if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_K | OBC_VAR_VK>);
-        return launch_multi(tc_pass2_multi_kernel<kAllVariants>);
+        if (p.csplit > 1 || (s.causal && s.W > MC_ROWS)) {
+            if (s.variants == OBC_VAR_VK) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_VK, true>);
+            if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_K | OBC_VAR_VK, true>);
+            return launch_multi(tc_pass2_multi_kernel<kAllVariants, true>);
+        }
+        if (s.variants == OBC_VAR_VK) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_VK, false>);
+        if (s.variants == (OBC_VAR_K | OBC_VAR_VK)) return launch_multi(tc_pass2_multi_kernel<OBC_VAR_K | OBC_VAR_VK, false>);
+        return launch_multi(tc_pass2_multi_kernel<kAllVariants, false>);
     }
 
     auto launch = [&](auto kernel) -> obc_status {
