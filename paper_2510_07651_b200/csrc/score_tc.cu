@@ -1014,7 +1014,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     span_begin(p.span);
 
     const int split = blockIdx.x, vu = blockIdx.y;
-    const int unit = vu / p.n_chunks, c = vu % p.n_chunks;
+    // row chunks are taken last to first: under a causal window the later chunks see more of the cache, and
+    // with more CTAs than SMs the long ones should start first
+    const int unit = vu / p.n_chunks, c = p.n_chunks - 1 - vu % p.n_chunks;
     const int b = unit / p.Hkv, g = unit % p.Hkv;
 
     if (threadIdx.x == 0) {
