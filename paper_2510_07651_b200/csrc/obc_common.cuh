@@ -49,6 +49,7 @@ constexpr size_t kSpanOffset = 64;   // byte offset, in the workspace header, of
 struct SimtPlan {
     int n_splits;                        // KV splits of pass 1
     int tiles_per_split;
+    int tile_tokens;                     // tokens per tile of the pass-1 kernel the plan is for
     int rows_out;                        // rows per unit in the combined arrays (R, or R padded)
     int want_obf;                        // also write the bf16 copy of -2*O (tensor-core pass 2)
     size_t off_flag;                             // 256-byte header: device status word, kernel spans at kSpanOffset

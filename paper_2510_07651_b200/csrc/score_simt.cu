@@ -106,6 +106,7 @@ simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
 
     const int tile_lo = split * plan.tiles_per_split;
     const int tile_hi = min(tile_lo + plan.tiles_per_split, (N + TN - 1) / TN);
+    if (tile_lo >= (N + TN - 1) / TN) return;      // a split past the end of a shorter sequence: the merge does not read it
     for (int tile = tile_lo; tile < tile_hi; ++tile) {
         const int t0 = tile * TN;
         __syncthreads();
@@ -176,6 +177,11 @@ simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
 // split t, warp w the float4 partial outputs of splits w, w+4, ... (pass 1 writes every partial,
 // zeros where a split saw no token), so a block costs one round trip to L2 instead of one per split.
 constexpr int CMB_NT = 128;
+// splits that hold tokens of a sequence of N tokens: the others ran no tile and wrote nothing
+__device__ __forceinline__ int active_splits(const SimtPlan& plan, int N) {
+    const int tiles = (N + plan.tile_tokens - 1) / plan.tile_tokens;
+    return min(plan.n_splits, (tiles + plan.tiles_per_split - 1) / plan.tiles_per_split);
+}
 constexpr int CMB_INFLIGHT = 10;                       // float4 loads in flight per thread
 
 __device__ __forceinline__ float block128_reduce(float x, bool take_max, float* red) {
@@ -213,10 +219,11 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     const size_t sstride = (size_t)s.R * kD;                             // floats between the outputs of two splits
     float M = -INFINITY, L = 0.f, Mrun = -INFINITY;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int base = 0; base < plan.n_splits; base += CMB_NT) {
-        const int sp = base + tid, cnt = min(CMB_NT, plan.n_splits - base);
-        const float m = sp < plan.n_splits ? part_m[row0 + (size_t)sp * s.R] : -INFINITY;
-        const float l = sp < plan.n_splits ? part_l[row0 + (size_t)sp * s.R] : 0.f;
+    const int n_act = active_splits(plan, seq_len(s, unit / s.Hkv));
+    for (int base = 0; base < n_act; base += CMB_NT) {
+        const int sp = base + tid, cnt = min(CMB_NT, n_act - base);
+        const float m = sp < n_act ? part_m[row0 + (size_t)sp * s.R] : -INFINITY;
+        const float l = sp < n_act ? part_l[row0 + (size_t)sp * s.R] : 0.f;
         const float* po = part_o + (row0 + (size_t)base * s.R) * kD + lane * 4;
         for (int j0 = warp; j0 < cnt || j0 == warp; j0 += 4 * CMB_INFLIGHT) {
             float4 o4[CMB_INFLIGHT];
@@ -283,9 +290,10 @@ simt_combine_rows_kernel(ScoreShape s, SimtPlan plan, float* ws) {
         const size_t row0 = (size_t)unit * plan.n_splits * s.R + r;          // split sp: row0 + sp * R
         float m[CMBW_MAX_SPLITS], l[CMBW_MAX_SPLITS];
         float4 o4[CMBW_MAX_SPLITS];
+        const int n_act = active_splits(plan, seq_len(s, unit / s.Hkv));
 #pragma unroll
         for (int sp = 0; sp < CMBW_MAX_SPLITS; ++sp) {                       // every load before the first use
-            const bool on = sp < plan.n_splits;
+            const bool on = sp < n_act;
             m[sp] = on ? part_m[row0 + (size_t)sp * s.R] : -INFINITY;
             l[sp] = on ? part_l[row0 + (size_t)sp * s.R] : 0.f;
             o4[sp] = on ? *reinterpret_cast<const float4*>(part_o + (row0 + (size_t)sp * s.R) * kD + lane * 4)
@@ -506,6 +514,7 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
     if (n < 1) n = 1;
     p.tiles_per_split = (tiles + n - 1) / n;
     p.n_splits = (tiles + p.tiles_per_split - 1) / p.tiles_per_split;
+    p.tile_tokens = TN;
     p.rows_out = rows_out;
     p.want_obf = want_obf ? 1 : 0;
     size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, orow = (size_t)units * rows_out, off = 0;

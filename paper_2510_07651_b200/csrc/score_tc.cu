@@ -1018,6 +1018,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // with more CTAs than SMs the long ones should start first
     const int unit = vu / p.n_chunks, c = p.n_chunks - 1 - vu % p.n_chunks;
     const int b = unit / p.Hkv, g = unit % p.Hkv;
+    // a split past the end of a shorter sequence has nothing to do and the merge does not read its partial result
+    // (the sequence lengths are the caller's input, so they may be read before the wait on the preceding kernel)
+    if (split > 0 && split * p.tiles_per_split * TILE >= tc_seq_len_raw(p.seq_lens, b, p.Nmax)) return;
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
@@ -1429,6 +1432,7 @@ static SimtPlan make_tc_plan(const ScoreShape& s) {
     SimtPlan p{};
     p.tiles_per_split = (tiles + n - 1) / n;                                   // per pass-1 CTA
     p.n_splits = (tiles + p.tiles_per_split - 1) / p.tiles_per_split;          // CTAs, and partial results, per unit
+    p.tile_tokens = TILE;
     p.rows_out = ch.rows_out;
     p.want_obf = 1;
     const size_t rows = (size_t)units * s.R, prow = rows * p.n_splits, orow = (size_t)units * ch.rows_out;

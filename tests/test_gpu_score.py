@@ -125,6 +125,21 @@ def test_workspace_poison_does_not_leak():
     H.assert_scores_close(s[0].cpu().numpy(), want, "f32", tight=2e-5)
 
 
+@pytest.mark.parametrize("path", ["simt", "tc"])
+def test_ragged_batch_with_poisoned_workspace(path):
+    """Splits past the end of a shorter sequence run nothing and write nothing: whatever the workspace held
+    there (here a NaN pattern) must not reach the scores."""
+    case = synth.make_prefill("ragpoison", B=3, Hq=8, Hkv=2, d=128, W=16, N=[9000, 700, 2500], dtype="bf16", seed=21)
+    q, k, v = H.upload(case)
+    lens = H.lens_dev(case)
+    p = api.score_params(q, k, seq_lens=lens, variants=["VK"], path=path)
+    ws = torch.full((api.obc_score_workspace(p),), 0xFF, dtype=torch.uint8, device="cuda")
+    s = api.obc_score(q, k, v, seq_lens=lens, variants=["VK"], path=path, workspace=ws)
+    api.obc_score_status(ws)
+    want = H.oracle_scores(case, ["VK"])["VK"]
+    H.assert_scores_close(s[0].cpu().numpy(), want, "bf16", tight=2e-2, what=f"ragged poison {path}")
+
+
 def test_kernel_spans_are_recorded_and_cleared():
     """Both tensor-core kernels leave a plausible device-side extent in the workspace header; reading
     it zeroes it; the CUDA-core path leaves nothing."""
