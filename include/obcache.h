@@ -92,6 +92,11 @@ typedef struct {
     int32_t causal;           /* nonzero: window row i sees keys p <= N_b - W + i */
     uint32_t variants;        /* OBC_VAR_* bitmask, at least one bit */
     int32_t path;             /* OBC_PATH_* */
+    const int32_t* mask_lens; /* device [batch] or NULL.  For a cache whose tokens are one shard of a longer
+                                 sequence (see obc_window_attention): M_b = the sequence's length minus the
+                                 position of the shard's first token.  Window row i then sees the shard's tokens
+                                 p <= M_b - W + i, and the preconditions become W <= M_b, 1 <= seq_lens[b].
+                                 NULL: M_b = N_b (the cache is the whole sequence). */
 } obc_score_params;
 
 /* Bytes of device workspace obc_score needs for these parameters (host computation only). */
@@ -120,6 +125,28 @@ obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_
 obc_status obc_score_given(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
                            obc_tensor o, const float* lse,
                            float* scores, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Token-sharded caches (a sequence whose K/V is split by token range over several caches, e.g. one per GPU
+ * under context parallelism).  The window attention of Sec. 3 is a softmax over ALL cached tokens, so the
+ * shards must agree on it before any of them can score; the scores themselves (Eq. 4-6) are then local to
+ * a shard's tokens.  Three steps, with one exchange of R x (d + 1) numbers per head between them:
+ *   1. obc_window_attention on every shard (params.mask_lens set): the shard's own softmax over its tokens,
+ *      o_out fp32 [B,Hq,W,d] contiguous and lse_out fp32 [B,Hq,W] (natural log of the row's sum of
+ *      exp(scaled logit) over the shard's visible tokens; -inf and a zero row of o_out where it sees none);
+ *   2. the shards' (o, lse) are gathered (by the caller: NCCL all-gather, peer copies, ...) and
+ *      obc_merge_attention combines n_parts of them, stored [n_parts][B,Hq,W,(d)] contiguous, into the
+ *      attention over the whole sequence:  lse = log sum_s exp(lse_s),  o = sum_s exp(lse_s - lse) o_s;
+ *   3. obc_score_given on every shard with the merged (o, lse) and the same mask_lens.
+ * obc_window_attention takes the workspace of obc_score_workspace for the same parameters (variants are
+ * ignored but must be valid).  obc_merge_attention needs no workspace; rows = B * Hq * W.
+ * ------------------------------------------------------------------------------------------ */
+obc_status obc_window_attention(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                                float* o_out, float* lse_out,
+                                void* workspace, size_t workspace_bytes, void* stream);
+obc_status obc_merge_attention(int32_t n_parts, int64_t rows, int32_t head_dim,
+                               const float* o_parts, const float* lse_parts,
+                               float* o_out, float* lse_out, void* stream);
 
 /*
  * Reads the device status word that obc_score keeps in the first bytes of its workspace.  The

@@ -23,7 +23,7 @@ VARIANTS = {"V": OBC_VAR_V, "K": OBC_VAR_K, "VK": OBC_VAR_VK, "ATTN": OBC_VAR_AT
 POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
-EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_given", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
+EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_given", "obc_window_attention", "obc_merge_attention", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
            "obc_select_noalloc", "obc_select_adaptive_workspace", "obc_select_adaptive", "obc_compact",
            "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
            "obc_status_string", "obc_last_cuda_error", "obc_version"]
@@ -47,7 +47,7 @@ class obc_score_params(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("batch", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("window", C.c_int32),
                 ("max_len", C.c_int32), ("seq_lens", C.c_void_p), ("scale", C.c_float),
-                ("causal", C.c_int32), ("variants", C.c_uint32), ("path", C.c_int32)]
+                ("causal", C.c_int32), ("variants", C.c_uint32), ("path", C.c_int32), ("mask_lens", C.c_void_p)]
 
 
 class obc_select_params(C.Structure):
@@ -83,6 +83,8 @@ def lib():
         L.obc_score_workspace.argtypes = [C.POINTER(obc_score_params), sz]
         L.obc_score.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, vp, vp, C.c_size_t, vp]
         L.obc_score_given.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, obc_tensor, vp, vp, vp, C.c_size_t, vp]
+        L.obc_window_attention.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, vp, vp, vp, C.c_size_t, vp]
+        L.obc_merge_attention.argtypes = [C.c_int32, C.c_int64, C.c_int32, vp, vp, vp, vp, vp]
         L.obc_score_status.argtypes = [vp, vp]
         L.obc_score_kernel_spans.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.obc_select_workspace.argtypes = [C.POINTER(obc_select_params), sz]
@@ -145,11 +147,13 @@ def variants_mask(variants) -> int:
     return m
 
 
-def score_params(q, k, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",), path="auto") -> obc_score_params:
+def score_params(q, k, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",), path="auto",
+                 mask_lens=None) -> obc_score_params:
     B, Hq, W, d = q.shape
     _, Hkv, Nmax, _ = k.shape
     return obc_score_params(C.sizeof(obc_score_params), B, Hq, Hkv, d, W, Nmax, _ptr(seq_lens), float(scale),
-                            int(bool(causal)), variants_mask(variants), PATHS[path] if isinstance(path, str) else path)
+                            int(bool(causal)), variants_mask(variants), PATHS[path] if isinstance(path, str) else path,
+                            _ptr(mask_lens))
 
 
 def obc_score_workspace(p: obc_score_params) -> int:
@@ -173,11 +177,44 @@ def obc_score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",
     return scores
 
 
+def obc_window_attention(q, k, v, *, seq_lens=None, mask_lens=None, scale=0.0, causal=True, path="auto",
+                         o_out=None, lse_out=None, workspace=None):
+    """Window attention of one token shard: (o fp32 [B,Hq,W,d], lse fp32 [B,Hq,W]) over the shard's own
+    tokens; mask_lens int32 [B] = sequence length minus the position of the shard's first token."""
+    p = score_params(q, k, seq_lens=seq_lens, scale=scale, causal=causal, variants=("VK",), path=path, mask_lens=mask_lens)
+    B, Hq, W, d = q.shape
+    if o_out is None:
+        o_out = torch.empty((B, Hq, W, d), dtype=torch.float32, device=k.device)
+    if lse_out is None:
+        lse_out = torch.empty((B, Hq, W), dtype=torch.float32, device=k.device)
+    ws = _workspace(obc_score_workspace(p), k, workspace)
+    _check(lib().obc_window_attention(C.byref(p), as_tensor4(q), as_tensor4(k), as_tensor4(v), o_out.data_ptr(),
+                                      lse_out.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "obc_window_attention")
+    return o_out, lse_out
+
+
+def obc_merge_attention(o_parts, lse_parts, *, o_out=None, lse_out=None):
+    """Attention over the whole sequence from its shards': o_parts fp32 [P,B,Hq,W,d], lse_parts fp32 [P,B,Hq,W]."""
+    if o_parts.dtype != torch.float32 or lse_parts.dtype != torch.float32 or not (o_parts.is_contiguous() and lse_parts.is_contiguous()):
+        raise ValueError("o_parts and lse_parts must be contiguous float32 tensors")
+    if tuple(o_parts.shape[:-1]) != tuple(lse_parts.shape):
+        raise ValueError("lse_parts must be shaped like o_parts without its last axis")
+    P, d = o_parts.shape[0], o_parts.shape[-1]
+    rows = lse_parts[0].numel()
+    if o_out is None:
+        o_out = torch.empty(o_parts.shape[1:], dtype=torch.float32, device=o_parts.device)
+    if lse_out is None:
+        lse_out = torch.empty(lse_parts.shape[1:], dtype=torch.float32, device=o_parts.device)
+    _check(lib().obc_merge_attention(P, rows, d, o_parts.data_ptr(), lse_parts.data_ptr(), o_out.data_ptr(),
+                                     lse_out.data_ptr(), _stream()), "obc_merge_attention")
+    return o_out, lse_out
+
+
 def obc_score_given(q, k, v, o, lse, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",), path="auto",
-                    scores=None, workspace=None):
+                    scores=None, workspace=None, mask_lens=None):
     """obc_score from attention outputs the caller already has: o [B,Hq,W,d] (f32 or bf16) and lse
     fp32 [B,Hq,W] (natural log, contiguous) of the window rows; no window attention is recomputed."""
-    p = score_params(q, k, seq_lens=seq_lens, scale=scale, causal=causal, variants=variants, path=path)
+    p = score_params(q, k, seq_lens=seq_lens, scale=scale, causal=causal, variants=variants, path=path, mask_lens=mask_lens)
     B, Hkv, Nmax = k.shape[0], k.shape[1], k.shape[2]
     if tuple(o.shape) != tuple(q.shape) or tuple(lse.shape) != tuple(q.shape[:3]):
         raise ValueError("o must be shaped like q and lse like q without its last axis")

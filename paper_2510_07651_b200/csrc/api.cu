@@ -57,13 +57,13 @@ obc_status resolve_score(const obc_score_params* p, ScoreShape* s) {
     if (p->struct_size != sizeof(obc_score_params)) return OBC_ERR_UNSUPPORTED;
     if (p->head_dim != kD) return OBC_ERR_UNSUPPORTED;
     if (p->batch < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->n_q_heads % p->n_kv_heads) return OBC_ERR_SHAPE;
-    if (p->window < 1 || p->max_len < 1 || p->window > p->max_len) return OBC_ERR_SHAPE;
+    if (p->window < 1 || p->max_len < 1 || (!p->mask_lens && p->window > p->max_len)) return OBC_ERR_SHAPE;
     if ((long long)p->batch * p->n_kv_heads > 65535) return OBC_ERR_SHAPE;
     const unsigned known = OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_ATTN | OBC_VAR_VATP;
     if (p->variants == 0 || (p->variants & ~known)) return OBC_ERR_UNSUPPORTED;
     if (p->path < OBC_PATH_AUTO || p->path > OBC_PATH_TC) return OBC_ERR_UNSUPPORTED;
     s->B = p->batch; s->Hq = p->n_q_heads; s->Hkv = p->n_kv_heads; s->G = s->Hq / s->Hkv;
-    s->W = p->window; s->R = s->G * s->W; s->Nmax = p->max_len; s->seq_lens = p->seq_lens;
+    s->W = p->window; s->R = s->G * s->W; s->Nmax = p->max_len; s->seq_lens = p->seq_lens; s->mask_lens = p->mask_lens;
     s->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)kD);
     s->causal = p->causal != 0; s->variants = p->variants;
     s->n_planes = __builtin_popcount(p->variants);
@@ -129,6 +129,45 @@ static obc_status score_impl(const obc_score_params* p, obc_tensor q, obc_tensor
            : launch_simt_pass1_combine(s, plan, q.dtype, view(q), view(k), view(v), workspace, (cudaStream_t)stream);
     if (st != OBC_OK) return st;
     return launch_simt_pass2(s, plan, q.dtype, view(q), view(k), view(v), scores, workspace, (cudaStream_t)stream);
+}
+
+obc_status obc_window_attention(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
+                                float* o_out, float* lse_out,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    ScoreShape s;
+    obc_status st = resolve_score(p, &s);
+    if (st != OBC_OK) return st;
+    if (!o_out || !lse_out) return OBC_ERR_NULL;
+    if ((st = check_tensor(q, true)) != OBC_OK) return st;
+    if ((st = check_tensor(k, true)) != OBC_OK) return st;
+    if ((st = check_tensor(v, true)) != OBC_OK) return st;
+    if (q.dtype != k.dtype || k.dtype != v.dtype) return OBC_ERR_UNSUPPORTED;
+    if (((uintptr_t)o_out & 15) != 0 || ((uintptr_t)lse_out & 3) != 0) return OBC_ERR_ALIGN;
+    size_t need = 0;
+    if ((st = obc_score_workspace(p, &need)) != OBC_OK) return st;
+    if (!workspace || workspace_bytes < need) return OBC_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255) != 0) return OBC_ERR_ALIGN;
+    const bool tc = want_tc(p, s, q.dtype, view(q));
+    if (p->path == OBC_PATH_TC && !tc) return OBC_ERR_UNSUPPORTED;
+    SimtPlan plan;
+    if (tc) {
+        st = launch_attention_tc(s, view(q), view(k), view(v), workspace, (cudaStream_t)stream, &plan);
+    } else {
+        plan = make_simt_plan(s, s.R, false);
+        st = launch_simt_pass1_combine(s, plan, q.dtype, view(q), view(k), view(v), workspace, (cudaStream_t)stream);
+    }
+    if (st != OBC_OK) return st;
+    return launch_export_attention(s, plan, workspace, o_out, lse_out, (cudaStream_t)stream);
+}
+
+obc_status obc_merge_attention(int32_t n_parts, int64_t rows, int32_t head_dim,
+                               const float* o_parts, const float* lse_parts,
+                               float* o_out, float* lse_out, void* stream) {
+    if (head_dim != kD) return OBC_ERR_UNSUPPORTED;
+    if (n_parts < 1 || n_parts > 4096 || rows < 1 || rows > 0x7fffffffLL) return OBC_ERR_SHAPE;
+    if (!o_parts || !lse_parts || !o_out || !lse_out) return OBC_ERR_NULL;
+    if ((((uintptr_t)o_parts | (uintptr_t)o_out) & 15) != 0 || (((uintptr_t)lse_parts | (uintptr_t)lse_out) & 3) != 0) return OBC_ERR_ALIGN;
+    return launch_merge_attention(n_parts, rows, o_parts, lse_parts, o_out, lse_out, (cudaStream_t)stream);
 }
 
 obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,

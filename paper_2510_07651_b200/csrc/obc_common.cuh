@@ -37,6 +37,7 @@ struct TensorView {                      // element strides; d contiguous
 struct ScoreShape {
     int B, Hq, Hkv, G, W, R, Nmax;
     const int32_t* seq_lens;             // device or nullptr
+    const int32_t* mask_lens;            // device or nullptr: length the causal mask counts from (token-sharded caches)
     float scale;                         // 1/sqrt(d) resolved
     int causal;
     unsigned variants;
@@ -78,6 +79,14 @@ obc_status launch_given_prep(const ScoreShape& s, const SimtPlan& plan, const Gi
 obc_status launch_simt_pass1_combine(const ScoreShape& s, const SimtPlan& plan, int dtype,
                                      TensorView q, TensorView k, TensorView v, void* ws, cudaStream_t stream);
 obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream);
+// the combined window attention of the workspace as o [B,Hq,W,d] and natural-log lse [B,Hq,W]
+obc_status launch_export_attention(const ScoreShape& s, const SimtPlan& plan, const void* ws, float* o_out, float* lse_out,
+                                   cudaStream_t stream);
+obc_status launch_merge_attention(int n_parts, long long rows, const float* o_parts, const float* lse_parts,
+                                  float* o_out, float* lse_out, cudaStream_t stream);
+// pass 1 + combine of the tensor-core path alone (the workspace then holds the shard's window attention)
+obc_status launch_attention_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v, void* ws, cudaStream_t stream,
+                               SimtPlan* plan_out);
 obc_status launch_simt_pass2(const ScoreShape& s, const SimtPlan& plan, int dtype,
                              TensorView q, TensorView k, TensorView v,
                              float* scores, void* ws, cudaStream_t stream);
@@ -118,7 +127,8 @@ bool tc_shape_supported(const ScoreShape& s);                       // R large e
 bool tc_supported(const ScoreShape& s, int dtype, const TensorView& q);   // + bf16, uniformly strided Q rows
 size_t tc_workspace_bytes(const ScoreShape& s);
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
-                           float* scores, void* ws, cudaStream_t stream, const GivenAttention* given = nullptr);
+                           float* scores, void* ws, cudaStream_t stream, const GivenAttention* given = nullptr,
+                           SimtPlan* attention_only = nullptr);   // non-null: stop after pass 1 + combine, return the plan
 
 // ---- programmatic dependent launch ------------------------------------------------------------
 // Every kernel of the library is launched with programmatic stream serialization: its CTAs may

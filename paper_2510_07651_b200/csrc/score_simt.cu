@@ -22,6 +22,9 @@ constexpr int NT = 256;
 __device__ __forceinline__ int seq_len(const ScoreShape& s, int b) {
     return s.seq_lens ? s.seq_lens[b] : s.Nmax;
 }
+// length the causal mask counts from: the sequence's own length, or (token-sharded caches) the distance from the
+// shard's first token to the end of the whole sequence
+__device__ __forceinline__ int mask_len(const ScoreShape& s, int b) { return s.mask_lens ? s.mask_lens[b] : seq_len(s, b); }
 
 template <typename T>
 __device__ __forceinline__ const T* row_ptr(const TensorView& t, int b, int h, long long tok) {
@@ -101,7 +104,7 @@ simt_pass1_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         int r = r0 + warp * 4 + i;
-        last[i] = (r < s.R) ? (s.causal ? (long long)N - s.W + (r % s.W) : (long long)N - 1) : -1;
+        last[i] = (r < s.R) ? (s.causal ? min((long long)mask_len(s, b) - s.W + (r % s.W), (long long)N - 1) : (long long)N - 1) : -1;
     }
 
     const int tile_lo = split * plan.tiles_per_split;
@@ -256,7 +259,8 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     }
     *reinterpret_cast<float4*>(&sAcc[warp][lane * 4]) = acc;
     L = block128_reduce(L, false, red);                // its barriers also publish sAcc
-    const float oc = ((sAcc[0][tid] + sAcc[1][tid]) + (sAcc[2][tid] + sAcc[3][tid])) / L;
+    // (L = 0: the row saw no token, which only a shard of a longer sequence can show; it then weighs nothing in the merge)
+    const float oc = L > 0.f ? ((sAcc[0][tid] + sAcc[1][tid]) + (sAcc[2][tid] + sAcc[3][tid])) / L : 0.f;
     const float onorm = block128_reduce(oc * oc, false, red);
     (ws + plan.off_o / 4)[orow * kD + tid] = oc;
     if (obf) obf[orow * kD + tid] = __float2bfloat16(-2.f * oc);
@@ -309,7 +313,7 @@ simt_combine_rows_kernel(ScoreShape s, SimtPlan plan, float* ws) {
             oc.x = fmaf(o4[sp].x, w, oc.x); oc.y = fmaf(o4[sp].y, w, oc.y);
             oc.z = fmaf(o4[sp].z, w, oc.z); oc.w = fmaf(o4[sp].w, w, oc.w);
         }
-        oc.x /= L; oc.y /= L; oc.z /= L; oc.w /= L;
+        if (L > 0.f) { oc.x /= L; oc.y /= L; oc.z /= L; oc.w /= L; }       // L = 0: a shard in which the row sees no token
         onorm = warp_sum((oc.x * oc.x + oc.y * oc.y) + (oc.z * oc.z + oc.w * oc.w));
         lse2 = M + log2f(L);
     }
@@ -429,7 +433,7 @@ simt_pass2_kernel(ScoreShape s, SimtPlan plan, TensorView q, TensorView k, Tenso
         for (int i = 0; i < 4; ++i) {
             const int r = r0 + warp * 4 + i;
             if (r >= s.R) continue;
-            const long long last = s.causal ? (long long)N - s.W + (r % s.W) : (long long)N - 1;
+            const long long last = s.causal ? min((long long)mask_len(s, b) - s.W + (r % s.W), (long long)N - 1) : (long long)N - 1;
             const float lse = sLse[warp * 4 + i], no = sNo[warp * 4 + i];
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
@@ -529,6 +533,63 @@ SimtPlan make_simt_plan(const ScoreShape& s, int rows_out, bool want_obf) {
     p.off_cpair = off; p.off_nv = off;             // tensor-core plan only
     p.bytes = off;
     return p;
+}
+
+// ---- token-sharded caches: a shard's window attention out of the workspace, and the merge of the shards' ----------
+// one warp per window row: o [B,Hq,W,d] fp32 and the natural-log lse [B,Hq,W] from the combined arrays
+__global__ void __launch_bounds__(CMB_NT)
+export_attention_kernel(ScoreShape s, SimtPlan plan, const float* ws, float* o_out, float* lse_out) {
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * (CMB_NT / 32) + (threadIdx.x >> 5);   // (unit, r) = ((b, g), (head of the group, query))
+    if (row >= (long long)s.B * s.Hkv * s.R) return;
+    const long long unit = row / s.R, r = row % s.R;
+    const size_t src = (size_t)unit * plan.rows_out + r;
+    // rows of a unit are its G heads' W queries in order, and the units follow (b, g): the same order as [B,Hq,W]
+    *reinterpret_cast<float4*>(o_out + (size_t)row * kD + lane * 4) =
+        *reinterpret_cast<const float4*>(ws + plan.off_o / 4 + src * kD + lane * 4);
+    if (lane == 0) lse_out[row] = (ws + plan.off_lse2 / 4)[src] * 0.6931471805599453f;
+}
+
+// one warp per row: lse = log sum_s exp(lse_s), o = sum_s exp(lse_s - lse) o_s over the n_parts shards
+__global__ void __launch_bounds__(CMB_NT)
+merge_attention_kernel(int n_parts, long long rows, const float* __restrict__ o_parts, const float* __restrict__ lse_parts,
+                       float* __restrict__ o_out, float* __restrict__ lse_out) {
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * (CMB_NT / 32) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    float M = -INFINITY;
+    for (int sp = 0; sp < n_parts; ++sp) M = fmaxf(M, lse_parts[(size_t)sp * rows + row]);
+    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sp = 0; sp < n_parts; ++sp) {
+        const float ls = lse_parts[(size_t)sp * rows + row];
+        const float w = ls == -INFINITY ? 0.f : expf(ls - M);
+        const float4 o4 = *reinterpret_cast<const float4*>(o_parts + ((size_t)sp * rows + row) * kD + lane * 4);
+        L += w;
+        acc.x = fmaf(o4.x, w, acc.x); acc.y = fmaf(o4.y, w, acc.y); acc.z = fmaf(o4.z, w, acc.z); acc.w = fmaf(o4.w, w, acc.w);
+    }
+    if (L > 0.f) { acc.x /= L; acc.y /= L; acc.z /= L; acc.w /= L; }
+    *reinterpret_cast<float4*>(o_out + (size_t)row * kD + lane * 4) = acc;
+    if (lane == 0) lse_out[row] = M + logf(L);
+}
+
+obc_status launch_export_attention(const ScoreShape& s, const SimtPlan& plan, const void* ws, float* o_out, float* lse_out,
+                                   cudaStream_t stream) {
+    const long long rows = (long long)s.B * s.Hkv * s.R;
+    ProfScope ps("export_attention", stream);
+    OBC_CUDA_TRY(launch_pdl(export_attention_kernel, dim3((unsigned)((rows + CMB_NT / 32 - 1) / (CMB_NT / 32))), dim3(CMB_NT), 0, stream, 1,
+                            s, plan, (const float*)ws, o_out, lse_out));
+    return OBC_OK;
+}
+
+obc_status launch_merge_attention(int n_parts, long long rows, const float* o_parts, const float* lse_parts,
+                                  float* o_out, float* lse_out, cudaStream_t stream) {
+    ProfScope ps("merge_attention", stream);
+    OBC_CUDA_TRY(launch_pdl(merge_attention_kernel, dim3((unsigned)((rows + CMB_NT / 32 - 1) / (CMB_NT / 32))), dim3(CMB_NT), 0, stream, 1,
+                            n_parts, rows, o_parts, lse_parts, o_out, lse_out));
+    return OBC_OK;
 }
 
 obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, cudaStream_t stream) {

@@ -168,6 +168,7 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int n) {
 struct TcParams {
     int B, Hkv, G, W, R, Nmax;
     const int32_t* seq_lens;
+    const int32_t* mask_lens;                 // or nullptr: length the causal mask counts from (token-sharded caches)
     float scale;
     int causal;
     unsigned variants;
@@ -186,6 +187,7 @@ struct TcParams {
 
 __device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
 __device__ __forceinline__ int tc_seq_len(const TcParams& p, int b) { return tc_seq_len_raw(p.seq_lens, b, p.Nmax); }
+__device__ __forceinline__ int tc_mask_len(const TcParams& p, int b) { return p.mask_lens ? p.mask_lens[b] : tc_seq_len(p, b); }
 
 // Last token that any of the window rows [r0, r1] of a unit sees (row r is query position N - W + r mod W
 // of its head): tiles that begin after it contribute nothing to these rows and are not visited.  With a
@@ -532,7 +534,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             float* out = p.scores + (size_t)unit * p.Nmax;
             const int ptok = t0 + tok;
             // rows of the window that do not see this tile's last token need the causal mask
-            const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
+            const int Nm = tc_mask_len(p, b);
+            const bool masked_tile = p.causal && (t0 + TILE - 1 > Nm - p.W);
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
             const uint32_t buf = item & 1;
@@ -561,7 +564,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const float4* cst = my_const;
             const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u, tt = zt + 128u;
             if (masked_tile)
-                score_chunk<VARS, true>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, N - p.W, p.W, 0);
+                score_chunk<VARS, true>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, Nm - p.W, p.W, 0);
             else
                 score_chunk<VARS, false>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, 0, 0, 0);
             tc_fence_before();
@@ -699,7 +702,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                     tma_load_4d(dv + kHalfBytes, &map_v, bar(MC_FULL + j), 64, t0, g, b);
                 }
                 if (pitem == 0) pdl_wait();                        // K and V were read by pass 1; -2 O is the preceding kernel's output
-                const int pair_first = pair * 2 * TILE, Nu = tc_seq_len(p, b);
+                const int pair_first = pair * 2 * TILE, Nu = tc_mask_len(p, b);
                 for (int c = cs; c < nc && !failed; c += cstep) {
                     if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, 1) < pair_first) continue;
                     const uint32_t qb = citem & 1;
@@ -734,7 +737,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 if (!mbar_wait(bar(MC_FULL + 0), pitem & 1) || !mbar_wait(bar(MC_FULL + 1), pitem & 1)) { failed = true; fail_site = __LINE__; break; }
                 int pair, cs;
                 if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
-                const int pair_first = pair * 2 * TILE, Nu = tc_seq_len(p, tw.unit / p.Hkv);
+                const int pair_first = pair * 2 * TILE, Nu = tc_mask_len(p, tw.unit / p.Hkv);
                 for (int c = cs; c < nc && !failed; c += cstep) {
                     if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, 1) < pair_first) continue;
                     const uint32_t qb = citem & 1;
@@ -785,7 +788,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             if (lane == 0) mbar_arrive(bar(MC_NV + (pitem & 1)));
             int pair, cs;
             if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
-            const int pair_first = pair * 2 * TILE, Nu = tc_seq_len(p, unit / p.Hkv);
+            const int pair_first = pair * 2 * TILE, Nu = tc_mask_len(p, unit / p.Hkv);
             for (int c = cs; c < nc; c += cstep) {
                 if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, 1) < pair_first) continue;
                 const uint32_t cs = citem & 3;
@@ -815,14 +818,14 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
             const int unit = tw.unit, b = unit / p.Hkv;
             int pair, cs;
             if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
-            const int N = tc_seq_len(p, b), t0 = (pair * 2 + wg) * TILE;
+            const int N = tc_seq_len(p, b), Nm = tc_mask_len(p, b), t0 = (pair * 2 + wg) * TILE;
             const int ptok = t0 + tok;
-            const bool masked_tile = p.causal && (t0 + TILE - 1 > N - p.W);
+            const bool masked_tile = p.causal && (t0 + TILE - 1 > Nm - p.W);
             RowSums S;
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
             const int pair_first = pair * 2 * TILE;
             for (int c = cs; c < nc; c += cstep) {
-                if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, N, 1) < pair_first) continue;
+                if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nm, 1) < pair_first) continue;
                 const uint32_t item = 2 * citem + wg, buf = item & 3, cs = citem & 3;
                 if (!mbar_wait(bar(MC_CONST + cs), (citem >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
                 if (!mbar_wait(bar(MC_TM_FULL + buf), (item >> 2) & 1)) { failed = true; fail_site = __LINE__; break; }
@@ -830,7 +833,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 const float4* cst = reinterpret_cast<const float4*>(sConst + cs * 128);
                 const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 128u, tt = zt + 64u;
                 if (masked_tile)
-                    score_chunk<VARS, true>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, N - p.W, p.W, (c * MC_ROWS) % p.W);
+                    score_chunk<VARS, true>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, Nm - p.W, p.W, (c * MC_ROWS) % p.W);
                 else
                     score_chunk<VARS, false>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, 0, 0, 0);
                 tc_fence_before();
@@ -935,6 +938,7 @@ constexpr float kRescaleThreshold = 8.f;                   // log2 units
 struct P1Params {
     int B, Hq, Hkv, G, W, R, Nmax;
     const int32_t* seq_lens;
+    const int32_t* mask_lens;                              // or nullptr: length the causal mask counts from
     float scale;
     int causal;
     int n_chunks, chunk_rows;
@@ -1046,7 +1050,8 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int N = tc_seq_len_raw(p.seq_lens, b, p.Nmax);
     const int tile_lo = split * p.tiles_per_split;
     // tiles past the last token that any row of this chunk sees are not visited
-    const int chunk_last = rows_last_token(c * p.chunk_rows, min((c + 1) * p.chunk_rows, p.R) - 1, p.W, N, p.causal);
+    const int Nm = p.mask_lens ? p.mask_lens[b] : N;       // a shard of a longer sequence: its distance to that sequence's end
+    const int chunk_last = rows_last_token(c * p.chunk_rows, min((c + 1) * p.chunk_rows, p.R) - 1, p.W, Nm, p.causal);
     const int tile_hi = min(min(tile_lo + p.tiles_per_split, (N + TILE - 1) / TILE), chunk_last / TILE + 1);
     const int n_tiles = max(tile_hi - tile_lo, 0);
 
@@ -1160,8 +1165,8 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int rows_valid = min(p.chunk_rows, p.R - c * p.chunk_rows);
         const int r = c * p.chunk_rows + row;
         const bool valid = row < rows_valid;
-        const int last = valid ? (p.causal ? N - p.W + (r % p.W) : N - 1) : -1;   // last visible token
-        const int first_masked = min(p.causal ? N - p.W + 1 : N, N);         // tiles reaching it need the mask
+        const int last = valid ? (p.causal ? min(Nm - p.W + (r % p.W), N - 1) : N - 1) : -1;   // last visible token
+        const int first_masked = min(p.causal ? Nm - p.W + 1 : N, N);        // tiles reaching it need the mask
         const float sl2 = p.scale * kLog2e;
         const uint32_t lane_addr = (uint32_t)(lane_grp * 32) << 16;
         const uint32_t tS = tmem_base + lane_addr + w * 128u, tO = tmem_base + lane_addr + 256u + w * 128u;
@@ -1459,8 +1464,14 @@ static size_t tc_partial_bytes(const ScoreShape& s) {
 
 size_t tc_workspace_bytes(const ScoreShape& s) { return make_tc_plan(s).bytes + tc_partial_bytes(s); }
 
+obc_status launch_attention_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v, void* ws, cudaStream_t stream,
+                               SimtPlan* plan_out) {
+    return launch_score_tc(s, q, k, v, nullptr, ws, stream, nullptr, plan_out);
+}
+
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
-                           float* scores, void* ws, cudaStream_t stream, const GivenAttention* given) {
+                           float* scores, void* ws, cudaStream_t stream, const GivenAttention* given,
+                           SimtPlan* attention_only) {
     const TcChunks ch = tc_chunks(s.R);
     const SimtPlan plan = make_tc_plan(s);
     char* wsb = (char*)ws;
@@ -1494,7 +1505,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
     } else {       // pass 1 + combine
         P1Params p1{};
         p1.B = s.B; p1.Hq = s.Hq; p1.Hkv = s.Hkv; p1.G = s.G; p1.W = s.W; p1.R = s.R; p1.Nmax = s.Nmax;
-        p1.seq_lens = s.seq_lens; p1.scale = s.scale; p1.causal = s.causal;
+        p1.seq_lens = s.seq_lens; p1.mask_lens = s.mask_lens; p1.scale = s.scale; p1.causal = s.causal;
         p1.n_chunks = ch.n_chunks; p1.chunk_rows = ch.chunk_rows;
         p1.n_splits = plan.n_splits; p1.tiles_per_split = plan.tiles_per_split;
         p1.l2_stream = l2_stream ? 1 : 0;
@@ -1509,8 +1520,9 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         obc_status st = launch_combine(s, plan, ws, stream);
         if (st != OBC_OK) return st;
     }
+    if (attention_only) { *attention_only = plan; return OBC_OK; }      // the workspace holds the window attention
     TcParams p{};
-    p.B = s.B; p.Hkv = s.Hkv; p.G = s.G; p.W = s.W; p.R = s.R; p.Nmax = s.Nmax; p.seq_lens = s.seq_lens;
+    p.B = s.B; p.Hkv = s.Hkv; p.G = s.G; p.W = s.W; p.R = s.R; p.Nmax = s.Nmax; p.seq_lens = s.seq_lens; p.mask_lens = s.mask_lens;
     p.scale = s.scale; p.causal = s.causal; p.variants = s.variants;
     p.n_chunks = ch.n_chunks; p.chunk_rows = ch.chunk_rows; p.rows_out = ch.rows_out;
     p.lse2 = (const float*)(wsb + plan.off_lse2);

@@ -4,6 +4,11 @@ Every (batch item, KV head) unit is independent through score, select and compac
 group's query heads with their KV head), so the units are partitioned across ranks and no collective
 touches the data path.  `torch.distributed` is only used to agree on a step time (max over ranks) and,
 if the caller wants the whole index tensor on every rank, to gather the per-unit results.
+
+A cache sharded by TOKEN range instead (context parallelism: a sequence too long for one GPU) has one
+real exchange: the window attention of Sec. 3 is a softmax over all cached tokens, so the ranks
+all-gather their shards' (o, lse) of the R window rows, merge them, and then score their own tokens
+(`context_parallel_scores`); the scores are gathered before the selection (`gather_token_shards`).
 """
 from __future__ import annotations
 
@@ -52,3 +57,49 @@ def gather_head_shards(local: torch.Tensor, n_kv_heads: int) -> torch.Tensor:
     bufs = [torch.empty_like(pad) for _ in range(world)]
     dist.all_gather(bufs, pad)
     return torch.cat([bufs[r][:, :parts[r][1] - parts[r][0]] for r in range(world)], dim=1).view(dtype)
+
+
+def token_shards(n_tokens: int, world: int) -> list[tuple[int, int]]:
+    """Contiguous, balanced [begin, end) token ranges of a sequence, one per rank."""
+    return partition_units(n_tokens, world)
+
+
+def context_parallel_scores(q, k_local, v_local, *, offset: int, total_len: int, variants=("VK",), causal=True,
+                            scale=0.0, path="auto", group=None, ops=None):
+    """This rank's scores [n_variants,B,Hkv,n_local] of a cache sharded by token range.
+
+    q [B,Hq,W,d] are the window queries (the last W positions of the whole sequence, the same on every
+    rank); k_local, v_local [B,Hkv,n_local,d] hold tokens offset .. offset + n_local - 1 of a sequence of
+    total_len tokens.  Steps: the shard's own window attention; all-gather of (o, lse) over `group`
+    (B*Hq*W*(d+1) floats per rank); merge; scores of the local tokens from the merged attention.
+    `ops` supplies obc_window_attention / obc_merge_attention / obc_score_given (default: the library)."""
+    if ops is None:
+        from . import api as ops
+    B = q.shape[0]
+    mask = torch.full((B,), int(total_len) - int(offset), dtype=torch.int32, device=q.device)
+    o, lse = ops.obc_window_attention(q, k_local, v_local, mask_lens=mask, scale=scale, causal=causal, path=path)
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    if world > 1:
+        o_parts = [torch.empty_like(o) for _ in range(world)]
+        lse_parts = [torch.empty_like(lse) for _ in range(world)]
+        dist.all_gather(o_parts, o.contiguous(), group=group)
+        dist.all_gather(lse_parts, lse.contiguous(), group=group)
+        o_parts, lse_parts = torch.stack(o_parts), torch.stack(lse_parts)
+    else:
+        o_parts, lse_parts = o.unsqueeze(0).contiguous(), lse.unsqueeze(0).contiguous()
+    o_all, lse_all = ops.obc_merge_attention(o_parts, lse_parts)
+    return ops.obc_score_given(q, k_local, v_local, o_all, lse_all, mask_lens=mask, variants=variants, causal=causal,
+                               scale=scale, path=path)
+
+
+def gather_token_shards(local: torch.Tensor, total_len: int, group=None) -> torch.Tensor:
+    """All-gather of per-token results `[..., n_local]` (this rank's token range of `token_shards`) into
+    `[..., total_len]` on every rank, e.g. the scores before a selection that every rank repeats."""
+    world = dist.get_world_size(group)
+    parts = token_shards(total_len, world)
+    most = max(hi - lo for lo, hi in parts)
+    pad = torch.zeros(tuple(local.shape[:-1]) + (most,), dtype=local.dtype, device=local.device)
+    pad[..., :local.shape[-1]] = local
+    bufs = [torch.empty_like(pad) for _ in range(world)]
+    dist.all_gather(bufs, pad, group=group)
+    return torch.cat([bufs[r][..., :parts[r][1] - parts[r][0]] for r in range(world)], dim=-1)

@@ -1,0 +1,76 @@
+"""A cache sharded by token range (context parallelism), on one GPU: the shards are scored one after another
+through obc_window_attention -> obc_merge_attention -> obc_score_given, exactly the calls each rank of a
+multi-GPU job makes (the all-gather between them is a stack here), and the concatenated scores are compared
+with the CPU checker's scores of the whole, unsharded cache."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_07651_b200 import api, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _sharded_scores(case, cuts, variants, path):
+    q, k, v = H.upload(case)
+    N, B = case.Nmax, case.B
+    bounds = [0] + list(cuts) + [N]
+    shards = [(lo, hi) for lo, hi in zip(bounds[:-1], bounds[1:])]
+    masks = [torch.full((B,), N - lo, dtype=torch.int32, device="cuda") for lo, _ in shards]
+    parts = [api.obc_window_attention(q, k[:, :, lo:hi], v[:, :, lo:hi], mask_lens=m, path=path)
+             for (lo, hi), m in zip(shards, masks)]
+    o_all, lse_all = api.obc_merge_attention(torch.stack([p[0] for p in parts]), torch.stack([p[1] for p in parts]))
+    order = [n for n in H.VARIANT_ORDER if n in variants]
+    out = []
+    for (lo, hi), m in zip(shards, masks):
+        ks, vs = k[:, :, lo:hi], v[:, :, lo:hi]
+        p = api.score_params(q, ks, variants=order, path=path, mask_lens=m)
+        ws = torch.empty(api.obc_score_workspace(p), dtype=torch.uint8, device="cuda")
+        s = api.obc_score_given(q, ks, vs, o_all, lse_all, variants=order, path=path, mask_lens=m, workspace=ws)
+        api.obc_score_status(ws)
+        out.append(s)
+    torch.cuda.synchronize()
+    s = torch.cat(out, dim=-1).cpu().numpy()
+    return {n: s[i] for i, n in enumerate(order)}, o_all, lse_all
+
+
+@pytest.mark.parametrize("N,W,Hq,Hkv,dtype,path,cuts", [
+    (3000, 64, 8, 2, "bf16", "tc", (1100, 2950)),        # R = 256 (row chunks of 64); the last shard (50 tokens) is shorter than the window
+    (2500, 32, 8, 2, "bf16", "auto", (777, 1500, 2490)), # R = 128: the single-chunk kernels; uneven shards, one of 10 tokens
+    (900, 16, 4, 2, "f32", "auto", (300, 640)),          # CUDA-core kernels, fp32
+    (1500, 24, 6, 2, "bf16", "simt", (1490,)),           # CUDA-core kernels, bf16; the second shard lies inside the window
+])
+def test_token_sharded_cache_scores_like_the_whole(N, W, Hq, Hkv, dtype, path, cuts):
+    case = synth.make_prefill("sharded", B=2, Hq=Hq, Hkv=Hkv, d=128, W=W, N=N, dtype=dtype, seed=500 + N, hh_frac=0.02)
+    variants = ["V", "K", "VK", "ATTN"]
+    got, o_all, lse_all = _sharded_scores(case, cuts, variants, path)
+    want = H.oracle_scores(case, variants)
+    mx = max(np.abs(want[n]).max() for n in ("V", "K", "VK"))
+    for n in variants:
+        H.assert_scores_close(got[n], want[n], dtype, tight=2e-2 if dtype == "bf16" else None,
+                              what=f"sharded {n} {path}", mx=None if n == "ATTN" else mx)
+    # the merged attention is the attention over the whole cache
+    from oracle import reference as ref
+    att = ref.score(case.q, case.k, case.v, want=("ATTN",), return_attention=True)
+    o_ref = att["O"].reshape(case.B, Hq, W, 128)
+    lse_ref = (att["m"] + np.log(att["l"])).reshape(case.B, Hq, W)
+    tol = 2e-2 if dtype == "bf16" else 1e-4
+    assert np.abs(lse_all.cpu().numpy() - lse_ref).max() <= tol
+    assert np.abs(o_all.cpu().numpy() - o_ref).max() <= tol * max(1.0, np.abs(o_ref).max())
+
+
+def test_merge_attention_weights_and_empty_shards():
+    """lse = log sum exp(lse_s), o = sum exp(lse_s - lse) o_s; a shard that saw nothing (lse = -inf) weighs 0."""
+    g = torch.Generator(device="cpu").manual_seed(3)
+    P, rows = 4, 37
+    o = torch.randn((P, rows, 128), generator=g)
+    lse = torch.randn((P, rows), generator=g) * 3
+    lse[2, :10] = float("-inf")
+    lse[:, 5] = float("-inf"); lse[1, 5] = 0.25                  # only one shard saw row 5
+    want_lse = torch.logsumexp(lse.double(), dim=0)
+    want_o = (torch.exp(lse.double() - want_lse).unsqueeze(-1) * o.double()).sum(0)
+    got_o, got_lse = api.obc_merge_attention(o.cuda(), lse.cuda())
+    assert torch.allclose(got_lse.cpu().double(), want_lse, rtol=1e-5, atol=1e-5)
+    assert torch.allclose(got_o.cpu().double(), want_o, rtol=1e-4, atol=1e-5)
+    assert torch.equal(got_o[5].cpu(), o[1, 5])

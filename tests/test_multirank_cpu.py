@@ -73,3 +73,81 @@ def test_two_ranks_sharded_by_kv_head_match_the_unsharded_job():
         assert p.exitcode == 0
     assert same_idx and same_kept
     assert slow == pytest.approx(11.0)
+
+
+# ---- cache sharded by token range: the exchange of the window attention -------------------------------
+class _CpuOps:
+    """Stand-ins for the three library calls, in plain double-precision tensor code, with the library's
+    conventions: natural-log lse, -inf and a zero row where a shard shows a window row no token, and
+    `mask_lens` = sequence length minus the position of the shard's first token."""
+
+    @staticmethod
+    def _logits(q, k, mask_lens, causal, scale):
+        B, Hq, W, d = q.shape
+        Hkv, n = k.shape[1], k.shape[2]
+        G = Hq // Hkv
+        z = torch.einsum("bhwd,bhnd->bhwn", q.double(), k.double().repeat_interleave(G, dim=1)) * (scale or d ** -0.5)
+        if causal:
+            last = mask_lens.view(B, 1, 1, 1).double() - W + torch.arange(W).view(1, 1, W, 1)
+            z = z.masked_fill(torch.arange(n).view(1, 1, 1, n) > last, float("-inf"))
+        return z, G
+
+    @classmethod
+    def obc_window_attention(cls, q, k, v, *, mask_lens, scale=0.0, causal=True, path="auto"):
+        z, G = cls._logits(q, k, mask_lens, causal, scale)
+        lse = torch.logsumexp(z, dim=-1)
+        a = torch.exp(z - torch.where(torch.isinf(lse), torch.zeros_like(lse), lse).unsqueeze(-1))
+        o = torch.einsum("bhwn,bhnd->bhwd", a, v.double().repeat_interleave(G, dim=1))
+        return o.float(), lse.float()
+
+    @staticmethod
+    def obc_merge_attention(o_parts, lse_parts):
+        lse = torch.logsumexp(lse_parts.double(), dim=0)
+        w = torch.exp(lse_parts.double() - lse)
+        return (w.unsqueeze(-1) * o_parts.double()).sum(0).float(), lse.float()
+
+    @classmethod
+    def obc_score_given(cls, q, k, v, o, lse, *, mask_lens, variants=("ATTN",), causal=True, scale=0.0, path="auto"):
+        # the attention-only plane sum_r A_rp (Sec. 4.3) is enough to show which lse and which mask were used
+        z, G = cls._logits(q, k, mask_lens, causal, scale)
+        a = torch.exp(z - lse.double().unsqueeze(-1))
+        B, Hq, W, n = a.shape
+        return a.view(B, Hq // G, G * W, n).sum(2).unsqueeze(0).float()
+
+
+def _cp_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        case = synth.make_prefill("cp", B=2, Hq=4, Hkv=2, d=128, W=40, N=107, dtype="f32", seed=77)
+        q, k, v = (torch.from_numpy(x) for x in (case.q, case.k, case.v))
+        N = case.Nmax
+        lo, hi = multirank.token_shards(N, world)[rank]          # world 3: the last shard is shorter than the window
+        s_loc = multirank.context_parallel_scores(q, k[:, :, lo:hi], v[:, :, lo:hi], offset=lo, total_len=N,
+                                                  variants=("ATTN",), ops=_CpuOps)
+        s_all = multirank.gather_token_shards(s_loc, N)
+        if rank == 0:
+            full = _CpuOps.obc_window_attention(q, k, v, mask_lens=torch.full((2,), N, dtype=torch.int32))
+            want = _CpuOps.obc_score_given(q, k, v, *full, mask_lens=torch.full((2,), N, dtype=torch.int32))
+            out.put((tuple(s_all.shape), float((s_all - want).abs().max()), float(s_all.sum())))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_token_shards_exchange_the_window_attention():
+    """Three gloo ranks, each with a third of the tokens: after the all-gather and merge of the shards' (o, lse)
+    every rank's attention weights are those of the whole sequence, so the gathered attention-only scores
+    equal the unsharded ones and sum to the number of window rows."""
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_cp_worker, args=(r, 3, port, out)) for r in range(3)]
+    for p in procs:
+        p.start()
+    shape, err, total = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert shape == (1, 2, 2, 107)
+    assert err < 1e-5
+    assert total == pytest.approx(2 * 4 * 40, rel=1e-5)       # every softmax row sums to 1
