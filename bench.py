@@ -466,6 +466,67 @@ def run_other(args):
         print(json.dumps(line))
         return
 
+    if args.workload == "llama32k-sharded":
+        # One rank's share of the 32k Llama layer sharded by token range over two ranks (context parallelism):
+        # this rank holds the second half of the tokens (the window's own tokens are among them).  Per step:
+        # the shard's window attention, the merge with the other rank's (o, lse) (computed once during set-up;
+        # in a real job it arrives by all-gather: B*Hq*W*(d+1) floats = 0.5 MB), the scores of the local tokens,
+        # and the selection over the whole sequence's scores (the other half filled in once during set-up).
+        case, run = synth.config(2)
+        q, k, v = bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)
+        N, half = case.Nmax, case.Nmax // 2
+        m0 = torch.full((case.B,), N, dtype=torch.int32, device="cuda")
+        m1 = torch.full((case.B,), N - half, dtype=torch.int32, device="cuda")
+        k0, v0, k1, v1 = k[:, :, :half], v[:, :, :half], k[:, :, half:], v[:, :, half:]
+        o_parts = torch.empty((2, case.B, case.Hq, case.W, 128), dtype=torch.float32, device="cuda")
+        lse_parts = torch.empty((2, case.B, case.Hq, case.W), dtype=torch.float32, device="cuda")
+        api.obc_window_attention(q, k0, v0, mask_lens=m0, o_out=o_parts[0], lse_out=lse_parts[0])
+        o_all, lse_all = torch.empty_like(o_parts[0]), torch.empty_like(lse_parts[0])
+        sp = api.score_params(q, k1, variants=["VK"], mask_lens=m1)
+        ws = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
+        scores = torch.zeros((1, case.B, case.Hkv, N), dtype=torch.float32, device="cuda")
+        loc = torch.empty((1, case.B, case.Hkv, N - half), dtype=torch.float32, device="cuda")
+        api.obc_window_attention(q, k1, v1, mask_lens=m1, o_out=o_parts[1], lse_out=lse_parts[1], workspace=ws)
+        api.obc_merge_attention(o_parts, lse_parts, o_out=o_all, lse_out=lse_all)
+        sp0 = api.score_params(q, k0, variants=["VK"], mask_lens=m0)
+        ws0 = torch.empty(api.obc_score_workspace(sp0), dtype=torch.uint8, device="cuda")
+        scores[..., :half] = api.obc_score_given(q, k0, v0, o_all, lse_all, variants=["VK"], mask_lens=m0, workspace=ws0)
+        selp = api.select_params(scores[0], budget=run["budget"], n_recent=run["n_recent"], pool=run["pool_mode"],
+                                 pool_kernel=run["pool_kernel"])
+        ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
+        idx = torch.empty((case.B, case.Hkv, run["budget"]), dtype=torch.int32, device="cuda")
+
+        def step():
+            api.obc_window_attention(q, k1, v1, mask_lens=m1, o_out=o_parts[1], lse_out=lse_parts[1], workspace=ws)
+            api.obc_merge_attention(o_parts, lse_parts, o_out=o_all, lse_out=lse_all)
+            api.obc_score_given(q, k1, v1, o_all, lse_all, variants=["VK"], mask_lens=m1, scores=loc, workspace=ws)
+            scores[..., half:].copy_(loc)                       # stands for the all-gather of the scores
+            api.obc_select(scores[0], budget=run["budget"], n_recent=run["n_recent"], pool=run["pool_mode"],
+                           pool_kernel=run["pool_kernel"], idx=idx, workspace=ws_sel)
+        for _ in range(warmup):
+            step()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        api.obc_profile_begin()
+        for _ in range(min(steps, 50)):
+            step()
+        torch.cuda.synchronize()
+        prof = api.obc_profile_end()
+        line = {"metric": METRIC, "value": N * steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps,
+                "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "one of two ranks of the 32k Llama layer sharded by token range (this rank: tokens "
+                                       f"{half}..{N - 1}), emulated on one GPU: window attention of the shard, merge with the "
+                                       "peer's (o, lse), local scores, selection over the gathered scores; no compaction",
+                           "l2": "single input copy (K+V of the shard = 67 MB)"},
+                "kernels": {k_: {"launches": v_[0], "avg_us": 1e3 * v_[1] / v_[0]} for k_, v_ in sorted(prof.items())}}
+        print(json.dumps(line))
+        return
+
     given = args.workload.endswith("-given")     # the caller's attention outputs instead of a recompute
     adaptive = args.workload.endswith("-adaptive")    # head-adaptive budgets (safeguard 0.2) instead of one budget per head
     if args.workload == "history4k":             # the whole sequence as perturbation window (W = N = 4096)
@@ -574,7 +635,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--eager", action="store_true", help="time plain library calls instead of replaying CUDA graphs")
-    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive", "history4k", "decode-window"],
+    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive", "history4k", "decode-window", "llama32k-sharded"],
                     help="llama32k is the headline benchmark; the others print a shorter line (1 GPU)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"
