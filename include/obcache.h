@@ -147,6 +147,16 @@ obc_status obc_window_attention(const obc_score_params* p, obc_tensor q, obc_ten
 obc_status obc_merge_attention(int32_t n_parts, int64_t rows, int32_t head_dim,
                                const float* o_parts, const float* lse_parts,
                                float* o_out, float* lse_out, void* stream);
+/*
+ * After the selection over the gathered scores (Algorithm 2; identical on every rank) a shard keeps the rows it
+ * owns: obc_shard_indices writes, for every (b, g), the entries of idx [B,Hkv,idx_stride] (ascending, -1 padded,
+ * positions in the whole sequence) that lie in [token_offset, token_offset + n_local), relative to the shard, in
+ * ascending order into idx_local [B,Hkv,idx_stride] (-1 padded) and their number into counts [B,Hkv].
+ * obc_compact with the shard's k, v and idx_local then fills the first counts[b,g] rows of the shard's compacted
+ * cache.  idx and idx_local must not be the same buffer.
+ */
+obc_status obc_shard_indices(int32_t batch, int32_t n_kv_heads, int32_t idx_stride, const int32_t* idx,
+                             int32_t token_offset, int32_t n_local, int32_t* idx_local, int32_t* counts, void* stream);
 
 /*
  * Reads the device status word that obc_score keeps in the first bytes of its workspace.  The

@@ -23,7 +23,7 @@ VARIANTS = {"V": OBC_VAR_V, "K": OBC_VAR_K, "VK": OBC_VAR_VK, "ATTN": OBC_VAR_AT
 POOLS = {"none": OBC_POOL_NONE, "avg": OBC_POOL_AVG, "max": OBC_POOL_MAX}
 PATHS = {"auto": OBC_PATH_AUTO, "simt": OBC_PATH_SIMT, "tc": OBC_PATH_TC}
 
-EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_given", "obc_window_attention", "obc_merge_attention", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
+EXPORTS = ["obc_score_workspace", "obc_score", "obc_score_given", "obc_window_attention", "obc_merge_attention", "obc_shard_indices", "obc_score_status", "obc_score_kernel_spans", "obc_select_workspace", "obc_select",
            "obc_select_noalloc", "obc_select_adaptive_workspace", "obc_select_adaptive", "obc_compact",
            "obc_decode_workspace", "obc_decode_step", "obc_profile_begin", "obc_profile_end",
            "obc_status_string", "obc_last_cuda_error", "obc_version"]
@@ -85,6 +85,7 @@ def lib():
         L.obc_score_given.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, obc_tensor, vp, vp, vp, C.c_size_t, vp]
         L.obc_window_attention.argtypes = [C.POINTER(obc_score_params), obc_tensor, obc_tensor, obc_tensor, vp, vp, vp, C.c_size_t, vp]
         L.obc_merge_attention.argtypes = [C.c_int32, C.c_int64, C.c_int32, vp, vp, vp, vp, vp]
+        L.obc_shard_indices.argtypes = [C.c_int32, C.c_int32, C.c_int32, vp, C.c_int32, C.c_int32, vp, vp, vp]
         L.obc_score_status.argtypes = [vp, vp]
         L.obc_score_kernel_spans.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.obc_select_workspace.argtypes = [C.POINTER(obc_select_params), sz]
@@ -208,6 +209,20 @@ def obc_merge_attention(o_parts, lse_parts, *, o_out=None, lse_out=None):
     _check(lib().obc_merge_attention(P, rows, d, o_parts.data_ptr(), lse_parts.data_ptr(), o_out.data_ptr(),
                                      lse_out.data_ptr(), _stream()), "obc_merge_attention")
     return o_out, lse_out
+
+
+def obc_shard_indices(idx, token_offset: int, n_local: int, *, idx_local=None, counts=None):
+    """A token shard's share of the kept indices idx int32 [B,Hkv,stride]: (idx_local, counts), see include/obcache.h."""
+    if idx.dtype != torch.int32 or not idx.is_contiguous():
+        raise ValueError("idx must be a contiguous int32 tensor")
+    B, Hkv, stride = idx.shape
+    if idx_local is None:
+        idx_local = torch.empty_like(idx)
+    if counts is None:
+        counts = torch.empty((B, Hkv), dtype=torch.int32, device=idx.device)
+    _check(lib().obc_shard_indices(B, Hkv, stride, idx.data_ptr(), int(token_offset), int(n_local), idx_local.data_ptr(),
+                                   counts.data_ptr(), _stream()), "obc_shard_indices")
+    return idx_local, counts
 
 
 def obc_score_given(q, k, v, o, lse, *, seq_lens=None, scale=0.0, causal=True, variants=("VK",), path="auto",

@@ -170,6 +170,15 @@ obc_status obc_merge_attention(int32_t n_parts, int64_t rows, int32_t head_dim,
     return launch_merge_attention(n_parts, rows, o_parts, lse_parts, o_out, lse_out, (cudaStream_t)stream);
 }
 
+obc_status obc_shard_indices(int32_t batch, int32_t n_kv_heads, int32_t idx_stride, const int32_t* idx,
+                             int32_t token_offset, int32_t n_local, int32_t* idx_local, int32_t* counts, void* stream) {
+    if (batch < 1 || n_kv_heads < 1 || idx_stride < 1 || token_offset < 0 || n_local < 1) return OBC_ERR_SHAPE;
+    if ((long long)batch * n_kv_heads > 0x7fffffffLL || (long long)token_offset + n_local > 0x7fffffffLL) return OBC_ERR_SHAPE;
+    if (!idx || !idx_local || !counts) return OBC_ERR_NULL;
+    if (idx == idx_local) return OBC_ERR_SHAPE;
+    return launch_shard_indices(batch * n_kv_heads, idx_stride, token_offset, n_local, idx, idx_local, counts, (cudaStream_t)stream);
+}
+
 obc_status obc_score(const obc_score_params* p, obc_tensor q, obc_tensor k, obc_tensor v,
                      float* scores, void* workspace, size_t workspace_bytes, void* stream) {
     return score_impl(p, q, k, v, nullptr, nullptr, scores, workspace, workspace_bytes, stream);

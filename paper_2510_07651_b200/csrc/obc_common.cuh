@@ -105,6 +105,8 @@ size_t select_adaptive_workspace_bytes(const SelectShape& s, int n_safe);
 obc_status launch_select_adaptive(const SelectShape& s, int n_safe, const float* scores, int32_t* idx, int32_t* counts,
                                   void* ws, cudaStream_t stream);
 obc_status launch_select_static(const SelectShape& s, const float* scores, int32_t* idx, cudaStream_t stream);
+obc_status launch_shard_indices(int units, int idx_stride, int t0, int n, const int32_t* idx, int32_t* local, int32_t* counts,
+                                cudaStream_t stream);
 obc_status launch_gather(int B, int Hkv, int idx_stride, int Nmax, int elem_bytes,
                          TensorView k, TensorView v, TensorView ko, TensorView vo, const int32_t* idx,
                          const float* s_in, float* s_out, cudaStream_t stream);

@@ -482,7 +482,33 @@ adaptive_split_kernel(SelectShape s, int total, const int32_t* __restrict__ vidx
     if (threadIdx.x == 0) counts[unit] = kept;
 }
 
+// A token shard's share of the kept indices: row (b, h) of idx is ascending (padding -1 at the end), so the entries
+// in [t0, t0 + n) are one stretch, found by binary search; written relative to the shard, padded with -1.
+__global__ void __launch_bounds__(256)
+shard_indices_kernel(int idx_stride, int t0, int n, const int32_t* __restrict__ idx_all,
+                     int32_t* __restrict__ local_all, int32_t* __restrict__ counts) {
+    pdl_wait();
+    const int unit = blockIdx.x;
+    const int32_t* idx = idx_all + (size_t)unit * idx_stride;
+    int32_t* local = local_all + (size_t)unit * idx_stride;
+    auto lower_bound = [&](int v) {                       // first entry >= v; the -1 padding counts as past every token
+        int a = 0, z = idx_stride;
+        while (a < z) { const int m = (a + z) >> 1; const int x = idx[m]; if (x >= 0 && x < v) a = m + 1; else z = m; }
+        return a;
+    };
+    const int seg0 = lower_bound(t0), seg1 = lower_bound(t0 + n), c = seg1 - seg0;
+    for (int j = threadIdx.x; j < idx_stride; j += blockDim.x) local[j] = j < c ? idx[seg0 + j] - t0 : -1;
+    if (threadIdx.x == 0) counts[unit] = c;
+}
+
 }  // namespace
+
+obc_status launch_shard_indices(int units, int idx_stride, int t0, int n, const int32_t* idx, int32_t* local, int32_t* counts,
+                                cudaStream_t stream) {
+    ProfScope ps("shard_indices", stream);
+    OBC_CUDA_TRY(launch_pdl(shard_indices_kernel, dim3((unsigned)units), dim3(256), 0, stream, 1, idx_stride, t0, n, idx, local, counts));
+    return OBC_OK;
+}
 
 size_t select_workspace_bytes(int B, int Hkv, int Nmax) { return align_up((size_t)B * Hkv * Nmax * 4, 256); }
 

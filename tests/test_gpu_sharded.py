@@ -74,3 +74,36 @@ def test_merge_attention_weights_and_empty_shards():
     assert torch.allclose(got_lse.cpu().double(), want_lse, rtol=1e-5, atol=1e-5)
     assert torch.allclose(got_o.cpu().double(), want_o, rtol=1e-4, atol=1e-5)
     assert torch.equal(got_o[5].cpu(), o[1, 5])
+
+
+def test_shard_indices_and_local_compaction():
+    """Every shard gathers the kept rows it owns; put side by side the shards' compacted rows are the compacted cache."""
+    case = synth.make_prefill("shardidx", B=2, Hq=4, Hkv=2, d=128, W=8, N=[1000, 640], dtype="bf16", seed=9)
+    q, k, v = H.upload(case)
+    lens = H.lens_dev(case)
+    s = api.obc_score(q, k, v, seq_lens=lens, variants=["VK"])
+    budgets = torch.tensor([100, 64], dtype=torch.int32, device="cuda")
+    idx = api.obc_select(s[0], budget=0, budgets=budgets, idx_stride=100, seq_lens=lens, n_recent=8, pool="max", pool_kernel=7)
+    k_all, v_all = api.obc_compact(k, v, idx)
+    torch.cuda.synchronize()
+    idx_h = idx.cpu().numpy()
+    cuts = [0, 300, 310, 900, 1000]                           # a shard of ten tokens; the last one holds the recent tail
+    filled = np.zeros((2, 2), np.int64)
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        loc, cnt = api.obc_shard_indices(idx, lo, hi - lo)
+        ko = torch.zeros((2, 2, 100, 128), dtype=torch.bfloat16, device="cuda")
+        vo = torch.zeros_like(ko)
+        api.obc_compact(k[:, :, lo:hi], v[:, :, lo:hi], loc, k_out=ko, v_out=vo)
+        torch.cuda.synchronize()
+        loc_h, cnt_h = loc.cpu().numpy(), cnt.cpu().numpy()
+        for b in range(2):
+            for h in range(2):
+                row = idx_h[b, h]
+                want = row[(row >= lo) & (row < hi)] - lo
+                assert cnt_h[b, h] == len(want)
+                assert np.array_equal(loc_h[b, h, :len(want)], want) and (loc_h[b, h, len(want):] == -1).all()
+                f = int(filled[b, h])
+                assert torch.equal(ko[b, h, :len(want)], k_all[b, h, f:f + len(want)])
+                assert torch.equal(vo[b, h, :len(want)], v_all[b, h, f:f + len(want)])
+                filled[b, h] += len(want)
+    assert (filled == np.array([[100, 100], [64, 64]])).all()
