@@ -5,7 +5,7 @@ import torch
 from oracle import reference as ref
 from paper_2510_07651_b200 import api, synth
 
-# spec tolerances: |gpu - ref| <= atol + rtol * |ref|
+# tolerances of the parity tests: |gpu - ref| <= atol + rtol * |ref|
 BF16_RTOL, BF16_ATOL = 2e-2, 1e-4
 F32_RTOL = 1e-5            # fp32 caches: atol = 1e-5 * max|ref|
 VARIANT_ORDER = ("V", "K", "VK", "ATTN", "VATP")     # plane order of the scores buffer
@@ -29,7 +29,7 @@ def lens_dev(case):
 
 def assert_scores_close(got: np.ndarray, want: np.ndarray, dtype: str, *, tight: float | None = None, what="",
                         mx: float | None = None):
-    """Spec tolerance, plus (tight) a relative bound normalised by the largest reference
+    """The stated tolerance, plus (tight) a relative bound normalised by the largest reference
     score, which stays meaningful when scores are far below the absolute tolerance.  `mx` is the
     magnitude the fp32 absolute tolerance scales with (default: the largest reference value of
     this plane; callers pass the largest OBCache score of the case so that a plane that is
