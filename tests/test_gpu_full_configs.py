@@ -70,6 +70,17 @@ def test_config4_ragged_batch_full():
     _prefill_full(4)
 
 
+def test_whole_sequence_window_llama_shapes_1k():
+    # Llama shapes with every one of 1024 query positions as a window row (R = 4096 rows per KV head): shared row
+    # chunks, skipped tile pairs and the warp-per-row merge, every element against the checker
+    case, run = synth.full_history(1024)
+    got = H.gpu_scores(case, ["K", "VK"])
+    want = H.oracle_scores(case, ["K", "VK"])
+    mx = max(np.abs(want[n]).max() for n in ("K", "VK"))
+    for n in ("K", "VK"):
+        H.assert_scores_close(got[n], want[n], "bf16", tight=2e-2, what=f"history1k/{n}", mx=mx)
+
+
 def test_config5_decode_full_shapes_sampled_units():
     # Llama shapes, batch 32, 256 steps in steady state (live 4096 -> 4097 -> 4096 per step); the
     # checker replays 6 sampled units teacher-forced on the GPU's own accumulators.

@@ -107,3 +107,38 @@ def test_shard_indices_and_local_compaction():
                 assert torch.equal(vo[b, h, :len(want)], v_all[b, h, f:f + len(want)])
                 filled[b, h] += len(want)
     assert (filled == np.array([[100, 100], [64, 64]])).all()
+
+
+def test_llama_32k_layer_sharded_over_two_ranks_full():
+    """The 32k Llama layer at full size, its tokens split evenly over two shards: scores against the checker's
+    scores of the whole cache, then the selection on the gathered scores and every shard's own compaction against
+    the checker's selection and gather."""
+    from oracle import reference as ref
+    case, run = synth.config(2)
+    got, _, _ = _sharded_scores(case, (case.Nmax // 2,), ["VK"], "auto")
+    want = H.oracle_scores(case, ["VK"])["VK"]
+    H.assert_scores_close(got["VK"], want, "bf16", tight=2e-2, what="sharded config 2")
+    scores = torch.from_numpy(got["VK"]).cuda()
+    budget = run["budget"]
+    idx = api.obc_select(scores, budget=budget, n_sink=run["n_sink"], n_recent=run["n_recent"], pool=run["pool_mode"],
+                         pool_kernel=run["pool_kernel"])
+    torch.cuda.synchronize()
+    want_idx = ref.select_pipeline(got["VK"], case.seq_lens, [budget], run["n_sink"], run["n_recent"], run["pool_mode"],
+                                   run["pool_kernel"], budget)
+    assert np.array_equal(idx.cpu().numpy(), want_idx)
+    q, k, v = H.upload(case)
+    half = case.Nmax // 2
+    filled = np.zeros((case.B, case.Hkv), np.int64)
+    for lo, hi in ((0, half), (half, case.Nmax)):
+        loc, cnt = api.obc_shard_indices(idx, lo, hi - lo)
+        ko, vo = api.obc_compact(k[:, :, lo:hi], v[:, :, lo:hi], loc)
+        torch.cuda.synchronize()
+        kb, vb, c = ko.view(torch.int16).cpu().numpy(), vo.view(torch.int16).cpu().numpy(), cnt.cpu().numpy()
+        for h in range(case.Hkv):
+            f, n = int(filled[0, h]), int(c[0, h])
+            rows = want_idx[0, h, f:f + n]
+            assert ((rows >= lo) & (rows < hi)).all()
+            assert np.array_equal(kb[0, h, :n], case.k_bits[0, h].view(np.int16)[rows])
+            assert np.array_equal(vb[0, h, :n], case.v_bits[0, h].view(np.int16)[rows])
+            filled[0, h] += n
+    assert (filled == budget).all()
