@@ -107,6 +107,31 @@ def test_given_and_adaptive_validation(L):
     assert L.obc_score_kernel_spans(None, None, C.byref(d1), C.byref(d2)) == -1
 
 
+def test_token_shard_calls_validation(L):
+    t = lambda ptr, dt=1: api.obc_tensor(ptr, dt, 0, 256 * 128, 128)
+    n = C.c_size_t(0)
+    # a window longer than the cache is only meaningful for a shard of a longer sequence (mask_lens given)
+    long_w = _sp(window=300)
+    assert L.obc_score_workspace(C.byref(long_w), C.byref(n)) == -2
+    long_w.mask_lens = 4096
+    assert L.obc_score_workspace(C.byref(long_w), C.byref(n)) == 0
+    p = _sp()
+    assert L.obc_window_attention(C.byref(p), t(4096), t(4096), t(4096), None, 4096, 4096, 1 << 30, None) == -1
+    assert L.obc_window_attention(C.byref(p), t(4096), t(4096), t(4096), 4096, None, 4096, 1 << 30, None) == -1
+    assert L.obc_window_attention(C.byref(p), t(4096), t(4096), t(4096), 4100, 4096, 4096, 1 << 30, None) == -4
+    assert L.obc_window_attention(C.byref(p), t(4096), t(4096), t(4096), 4096, 4096, 4096, 16, None) == -5
+    assert L.obc_window_attention(C.byref(p), t(4096), t(4096, 0), t(4096), 4096, 4096, 4096, 1 << 30, None) == -3
+    assert L.obc_merge_attention(0, 64, 128, 4096, 4096, 4096, 4096, None) == -2
+    assert L.obc_merge_attention(2, 0, 128, 4096, 4096, 4096, 4096, None) == -2
+    assert L.obc_merge_attention(2, 64, 64, 4096, 4096, 4096, 4096, None) == -3
+    assert L.obc_merge_attention(2, 64, 128, None, 4096, 4096, 4096, None) == -1
+    assert L.obc_merge_attention(2, 64, 128, 4100, 4096, 4096, 4096, None) == -4
+    assert L.obc_shard_indices(1, 2, 64, 4096, 0, 0, 8192, 4096, None) == -2        # an empty shard
+    assert L.obc_shard_indices(1, 2, 64, 4096, -1, 10, 8192, 4096, None) == -2
+    assert L.obc_shard_indices(1, 2, 64, None, 0, 10, 8192, 4096, None) == -1
+    assert L.obc_shard_indices(1, 2, 64, 4096, 0, 10, 4096, 4096, None) == -2       # in place
+
+
 def test_compact_and_decode_validation(L):
     t = lambda ptr: api.obc_tensor(ptr, 1, 0, 256 * 128, 128)
     assert L.obc_compact(1, 2, 64, 16, 256, t(4096), t(4096), 4096, t(4096), t(4096), None, None, None) == -3
