@@ -275,6 +275,8 @@ simt_combine_kernel(ScoreShape s, SimtPlan plan, float* ws) {
 // The same merge with one warp per (unit, output row), for many rows (a window of thousands of queries, a large
 // batch): no block-wide barrier, lane t holds head-dim elements 4t..4t+3, the splits are added in order, eight at a time.
 constexpr int CMBW_MAX_SPLITS = 8;
+// FEW: at most CMBW_MAX_SPLITS splits, one batch of loads and the maximum taken from it (one round trip to L2 in all)
+template <bool FEW>
 __global__ void __launch_bounds__(CMB_NT)
 simt_combine_rows_kernel(ScoreShape s, SimtPlan plan, float* ws) {
     pdl_wait();
@@ -294,13 +296,11 @@ simt_combine_rows_kernel(ScoreShape s, SimtPlan plan, float* ws) {
         const size_t row0 = (size_t)unit * plan.n_splits * s.R + r;          // split sp: row0 + sp * R
         const int n_act = active_splits(plan, seq_len(s, unit / s.Hkv));
         float M = -INFINITY, L = 0.f;
-        for (int sp = lane; sp < n_act; sp += 32) M = fmaxf(M, part_m[row0 + (size_t)sp * s.R]);   // the row's maximum over the splits
-        M = warp_max(M);
-        for (int base = 0; base < n_act; base += CMBW_MAX_SPLITS) {
-            float m[CMBW_MAX_SPLITS], l[CMBW_MAX_SPLITS];
-            float4 o4[CMBW_MAX_SPLITS];
+        float m[CMBW_MAX_SPLITS], l[CMBW_MAX_SPLITS];
+        float4 o4[CMBW_MAX_SPLITS];
+        auto load_batch = [&](int base) {                                    // every load of the batch before the first use
 #pragma unroll
-            for (int u = 0; u < CMBW_MAX_SPLITS; ++u) {                      // every load of the batch before the first use
+            for (int u = 0; u < CMBW_MAX_SPLITS; ++u) {
                 const int sp = base + u;
                 const bool on = sp < n_act;
                 m[u] = on ? part_m[row0 + (size_t)sp * s.R] : -INFINITY;
@@ -308,6 +308,18 @@ simt_combine_rows_kernel(ScoreShape s, SimtPlan plan, float* ws) {
                 o4[u] = on ? *reinterpret_cast<const float4*>(part_o + (row0 + (size_t)sp * s.R) * kD + lane * 4)
                            : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+        };
+        load_batch(0);
+        // the row's maximum over the splits: from the first batch when that is all of them (one round trip in all),
+        // otherwise the lanes read the splits' maxima side by side
+        float mrest = -INFINITY;
+        if (!FEW)
+            for (int sp = CMBW_MAX_SPLITS + lane; sp < n_act; sp += 32) mrest = fmaxf(mrest, part_m[row0 + (size_t)sp * s.R]);
+#pragma unroll
+        for (int u = 0; u < CMBW_MAX_SPLITS; ++u) M = fmaxf(M, m[u]);
+        if (!FEW && n_act > CMBW_MAX_SPLITS) M = fmaxf(M, warp_max(mrest));
+        for (int base = 0; base < (FEW ? 1 : n_act); base += CMBW_MAX_SPLITS) {
+            if (base > 0) load_batch(base);
 #pragma unroll
             for (int u = 0; u < CMBW_MAX_SPLITS; ++u) {
                 const float w = m[u] == -INFINITY ? 0.f : exp2f(m[u] - M);
@@ -601,8 +613,9 @@ obc_status launch_combine(const ScoreShape& s, const SimtPlan& plan, void* ws, c
     // block per row; with 1024 rows of 18 splits (one 32k layer) the block per row wins, 8.5 us against 14.5 us
     if ((plan.n_splits <= CMBW_MAX_SPLITS && rows >= 1024) || rows >= 4096) {
         ProfScope ps("combine", stream);
-        OBC_CUDA_TRY(launch_pdl(simt_combine_rows_kernel, dim3((unsigned)((rows + CMB_NT / 32 - 1) / (CMB_NT / 32))), dim3(CMB_NT), 0,
-                                stream, 1, s, plan, (float*)ws));
+        const dim3 grid((unsigned)((rows + CMB_NT / 32 - 1) / (CMB_NT / 32)));
+        if (plan.n_splits <= CMBW_MAX_SPLITS) OBC_CUDA_TRY(launch_pdl(simt_combine_rows_kernel<true>, grid, dim3(CMB_NT), 0, stream, 1, s, plan, (float*)ws));
+        else OBC_CUDA_TRY(launch_pdl(simt_combine_rows_kernel<false>, grid, dim3(CMB_NT), 0, stream, 1, s, plan, (float*)ws));
         return OBC_OK;
     }
     { ProfScope ps("combine", stream); OBC_CUDA_TRY(launch_pdl(simt_combine_kernel, dim3(s.B * s.Hkv * plan.rows_out), dim3(CMB_NT), 0, stream, 1, s, plan, (float*)ws)); }
