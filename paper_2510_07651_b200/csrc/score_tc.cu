@@ -626,12 +626,13 @@ constexpr uint32_t MC_OFF_BAR = MC_OFF_CONST + 4 * 32 * 16;
 enum { MC_FULL = 0, MC_EMPTY = 2, MC_QO_FULL = 4, MC_QO_EMPTY = 6, MC_TM_FULL = 8, MC_TM_EMPTY = 12,
        MC_NV = 16, MC_CONST = 18, MC_NBARS = 22 };
 constexpr uint32_t MC_OFF_TMEM = MC_OFF_BAR + MC_NBARS * 8;
+constexpr int kThreadsMulti = kThreads + 32;                      // + warp 12: the second MMA-issuing thread
 constexpr uint32_t kSmemMulti = MC_OFF_TMEM + 16 + 1024;
 
 // SPLIT: the general walk (row chunks of a pair shared by several CTAs, hidden tile pairs skipped); without
 // it every CTA takes whole pairs and every chunk, which is all a short window over a long cache needs.
 template <unsigned VARS, bool SPLIT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsMulti, 1)
 tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_o,
                       const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                       const __grid_constant__ TcParams p) {
@@ -651,9 +652,10 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_k); prefetch_tmap(&map_v); prefetch_tmap(&map_q); prefetch_tmap(&map_o);
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(MC_FULL + i), 1); mbar_init(bar(MC_EMPTY + i), 3); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(MC_QO_FULL + i), 1); mbar_init(bar(MC_QO_EMPTY + i), 1); }
-        for (int i = 0; i < 4; ++i) { mbar_init(bar(MC_TM_FULL + i), 1); mbar_init(bar(MC_TM_EMPTY + i), 4); }
+        // two threads issue the MMAs (see below), so what an MMA commit signals takes two arrivals
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(MC_FULL + i), 1); mbar_init(bar(MC_EMPTY + i), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(MC_QO_FULL + i), 1); mbar_init(bar(MC_QO_EMPTY + i), 2); }
+        for (int i = 0; i < 4; ++i) { mbar_init(bar(MC_TM_FULL + i), 2); mbar_init(bar(MC_TM_EMPTY + i), 4); }
         for (int i = 0; i < 2; ++i) mbar_init(bar(MC_NV + i), 2);
         for (int i = 0; i < 4; ++i) mbar_init(bar(MC_CONST + i), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -728,8 +730,13 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 (void)mbar_wait(bar(MC_QO_FULL + (it & 1)), (it >> 1) & 1);
             }
         }
-    } else if (warp == 1) {
-        // ===================================== MMA issuer =======================================
+    } else if (warp == 1 || warp == 12) {
+        // ===================================== MMA issuers ======================================
+        // One thread gets a tcgen05.mma out about every 88 cycles here (it shares its scheduler with two epilogue
+        // warps), and a 128x64x16 MMA keeps the tensor pipe busy for 32: so two threads issue, warp 1 the logits
+        // Z = K Q^T and warp 12 the cross terms T' = V (-2 O)^T.  Each commits what it issued; the barriers that
+        // an MMA commit signals count two arrivals.
+        const bool z_side = warp == 1;
         if (lane == 0) {
             const uint32_t idesc = idesc_bf16(MC_ROWS);
             uint32_t pitem = 0, citem = 0;
@@ -749,13 +756,16 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                         tc_fence_after();
                         const uint32_t zt = tmem_base + buf * 128u, tt = zt + 64u;
                         const uint32_t ak = desc_lo_k(sbase + MC_OFF_K + j * kOperandBytes), av = desc_lo_k(sbase + MC_OFF_V + j * kOperandBytes);
+                        if (z_side) {
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)             // d = 128 = 8 steps of K = 16
-                            tc_mma(zt, desc_make(ak + desc_kstep(ks, kHalfBytes)), desc_make(bq + desc_kstep(ks, kHalfB64)), idesc, ks > 0);
+                            for (int ks = 0; ks < 8; ++ks)         // d = 128 = 8 steps of K = 16
+                                tc_mma(zt, desc_make(ak + desc_kstep(ks, kHalfBytes)), desc_make(bq + desc_kstep(ks, kHalfB64)), idesc, ks > 0);
+                        } else {
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            tc_mma(tt, desc_make(av + desc_kstep(ks, kHalfBytes)), desc_make(bo + desc_kstep(ks, kHalfB64)), idesc, ks > 0);
-                        tc_commit(bar(MC_TM_FULL + buf));          // accumulators ready for epilogue group j
+                            for (int ks = 0; ks < 8; ++ks)
+                                tc_mma(tt, desc_make(av + desc_kstep(ks, kHalfBytes)), desc_make(bo + desc_kstep(ks, kHalfB64)), idesc, ks > 0);
+                        }
+                        tc_commit(bar(MC_TM_FULL + buf));          // this thread's accumulator of the item is ready
                     }
                     if (failed) break;
                     tc_commit(bar(MC_QO_EMPTY + qb));              // this Q / O buffer may be refilled
@@ -806,7 +816,7 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 ++citem;
             }
         }
-    } else {
+    } else if (warp < 12) {
         // ======================================= epilogue =======================================
         const int wg = (warp - 4) >> 2;                            // owns tile wg of every pair
         const int lane_grp = warp & 3;                             // TMEM lanes 32*lane_grp .. +31
@@ -1554,7 +1564,7 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         const int mgrid = (int)(positions < sm_count() ? positions : sm_count());
         auto launch_multi = [&](auto kernel) -> obc_status {
             OBC_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMulti));
-            { ProfScope ps("tc_pass2", stream); OBC_CUDA_TRY(launch_pdl(kernel, dim3(mgrid), dim3(kThreads), kSmemMulti, stream, 1, mq64, mo64, mk, mv, p)); }
+            { ProfScope ps("tc_pass2", stream); OBC_CUDA_TRY(launch_pdl(kernel, dim3(mgrid), dim3(kThreadsMulti), kSmemMulti, stream, 1, mq64, mo64, mk, mv, p)); }
             if (p.csplit > 1) {
                 ProfScope ps("partial_sum", stream);
                 OBC_CUDA_TRY(launch_pdl(tc_partial_sum_kernel, dim3((s.Nmax + 255) / 256, units), dim3(256), 0, stream, 1, p, s.n_planes));
