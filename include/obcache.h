@@ -289,7 +289,7 @@ obc_status obc_compact(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int3
  *      n_sink <= pos <= step_pos - n_recent (equal values: the highest pos), which becomes
  *      next_slot; otherwise next_slot = hi.
  *
- * Accumulation window (Sec. 6, "Choice of Perturbation Window in Decoding": scores accumulated
+ * Accumulation window (App. B, "Choice of Perturbation Window in Decoding": scores accumulated
  * only within a recent window instead of over the whole history).  With acc_window = w > 0 step 3
  * becomes  s_acc[slot] = sum of the slot's scores of the last w steps (this one included, fewer
  * while the token is younger than w steps).  The per-step scores are kept in the ring s_hist, fp32

@@ -213,7 +213,7 @@ class DecodeState:
 
     def __init__(self, k0, v0, cap, s_acc0=None, window=0):
         """`window` = w > 0: the accumulator is the sum of a token's scores over the last w steps only
-        (Sec. 6, accumulation within a recent window); 0: over every step since the token entered."""
+        (App. B, accumulation within a recent window); 0: over every step since the token entered."""
         n0, d = k0.shape
         self.window = int(window)
         self.hist = np.zeros((self.window, cap), np.float64)      # ring of per-step scores, row = step_pos mod w

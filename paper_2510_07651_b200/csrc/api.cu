@@ -219,6 +219,7 @@ static obc_status resolve_select(const obc_select_params* p, SelectShape* s) {
     if (!p) return OBC_ERR_NULL;
     if (p->struct_size != sizeof(obc_select_params)) return OBC_ERR_UNSUPPORTED;
     if (p->batch < 1 || p->n_kv_heads < 1 || p->max_len < 1) return OBC_ERR_SHAPE;
+    if ((long long)p->batch * p->n_kv_heads > 65535) return OBC_ERR_SHAPE;      // units index gridDim.y
     if (p->n_sink < 0 || p->n_recent < 0 || p->idx_stride < 1) return OBC_ERR_SHAPE;
     if (p->pool_mode < OBC_POOL_NONE || p->pool_mode > OBC_POOL_MAX) return OBC_ERR_UNSUPPORTED;
     if (p->pool_kernel < 1 || p->pool_kernel % 2 == 0) return OBC_ERR_SHAPE;
@@ -300,6 +301,7 @@ obc_status obc_compact(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int3
                        const float* scores_in, float* scores_out, void* stream) {
     if (head_dim != kD) return OBC_ERR_UNSUPPORTED;
     if (batch < 1 || n_kv_heads < 1 || idx_stride < 1 || max_len < 1) return OBC_ERR_SHAPE;
+    if ((long long)batch * n_kv_heads > 65535) return OBC_ERR_SHAPE;            // units index gridDim.y
     if (!idx) return OBC_ERR_NULL;
     if ((scores_in == nullptr) != (scores_out == nullptr)) return OBC_ERR_NULL;
     obc_status st;
@@ -384,7 +386,7 @@ obc_status obc_profile_end(obc_kernel_time* out, int32_t max_out, int32_t* n_out
         int j = 0;
         for (; j < n; ++j) if (std::strcmp(out[j].name, r.name) == 0) break;
         if (j == n) {
-            if (n == max_out) continue;
+            if (n == max_out) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); continue; }
             std::memset(&out[n], 0, sizeof(out[n]));
             std::strncpy(out[n].name, r.name, sizeof(out[n].name) - 1);
             ++n;

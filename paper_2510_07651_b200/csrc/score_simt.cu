@@ -19,8 +19,10 @@ constexpr int RC = 32;        // window rows per chunk (8 warps x 4 rows)
 constexpr int KS = kD + 4;    // padded row stride (floats) of the token-major smem tiles
 constexpr int NT = 256;
 
+// A length read on the device cannot be checked by the host: it is clamped to [0, max_len] so that no row
+// beyond the caller's buffers is ever addressed.
 __device__ __forceinline__ int seq_len(const ScoreShape& s, int b) {
-    return s.seq_lens ? s.seq_lens[b] : s.Nmax;
+    return s.seq_lens ? min(max(s.seq_lens[b], 0), s.Nmax) : s.Nmax;
 }
 // length the causal mask counts from: the sequence's own length, or (token-sharded caches) the distance from the
 // shard's first token to the end of the whole sequence

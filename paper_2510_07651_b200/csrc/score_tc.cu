@@ -9,12 +9,17 @@
 // the sum over window queries and the GQA group (App. A.5) needs no cross-thread reduction and no
 // W x N matrix ever leaves the SM.
 //
-// Warp roles of the 384-thread CTA (persistent, one CTA per SM):
+// Warp roles of the 640-thread CTA (persistent, one CTA per SM):
 //   warp 0      TMA producer: K/V tiles into a 2-stage ring, Q / -2O when the unit changes
 //   warp 1      MMA issuer (one elected lane), double-buffered TMEM accumulators (2 x 256 columns)
 //   warps 2-3   idle when pass 1 ran (its two spare warps computed ||v_p||^2 with the V tile at hand);
 //               otherwise (attention outputs supplied by the caller, or the l1 variant) the value norms of every tile
-//   warps 4-7   epilogue group 0 (even tiles), warps 8-11 epilogue group 1 (odd tiles)
+//   warps 4-11  epilogue of the even tiles, warps 12-19 epilogue of the odd tiles.  Each tile has two
+//               warpgroups: both hold one token per thread (a warp reads the TMEM lanes 32 (warp mod 4) ..),
+//               the first sums the first half of the window rows, the second the other half and hands
+//               its sums over through shared memory; the first adds them and stores the token's scores.
+//               (One warpgroup per tile spent most of its time waiting on its own dependent instructions:
+//               an SM sub-partition then runs two epilogue warps; with four it hides them.)
 //
 // Every mbarrier wait is bounded: on a timeout the kernel raises the status word in the workspace
 // header, stops issuing work, waits (bounded) for its own copies in flight, frees TMEM and returns.
@@ -31,7 +36,8 @@ constexpr unsigned kAllVariants = OBC_VAR_V | OBC_VAR_K | OBC_VAR_VK | OBC_VAR_A
 constexpr int NSTAGE = 2;
 constexpr uint32_t kHalfBytes = 128 * 128;      // [128 rows][64 bf16] = 16 KB, one swizzle-128B block
 constexpr uint32_t kOperandBytes = 2 * kHalfBytes;
-constexpr int kThreads = 384;
+constexpr int kThreads = 640;                   // single-chunk pass 2: 4 service warps + 4 epilogue warpgroups
+constexpr int kThreadsBase = 384;               // the multi-chunk pass 2 keeps two epilogue warpgroups
 constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s per wait
 
 // ---- shared memory map (offsets from a 1024-byte aligned base) ------------------------------
@@ -39,18 +45,21 @@ constexpr uint32_t OFF_Q = 0;
 constexpr uint32_t OFF_O = OFF_Q + kOperandBytes;
 constexpr uint32_t OFF_K = OFF_O + kOperandBytes;                 // NSTAGE x 32 KB
 constexpr uint32_t OFF_V = OFF_K + NSTAGE * kOperandBytes;        // NSTAGE x 32 KB
-constexpr uint32_t OFF_CONST = OFF_V + NSTAGE * kOperandBytes;    // 8 epilogue warps x 64 float4 (row-pair constants)
+constexpr uint32_t OFF_CONST = OFF_V + NSTAGE * kOperandBytes;    // 16 epilogue warps x 32 float4 (row-pair constants of the warp's half)
 constexpr int NSLOT = 4;                                          // ring depth of the per-tile value norms
-constexpr uint32_t OFF_NV = OFF_CONST + 8 * 64 * 16;              // NSLOT x 128 x (||v||^2, ||v||_1), own-norm kernels only
-constexpr uint32_t OFF_BAR = OFF_NV + NSLOT * TILE * 8;
-constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + 2 + 2 * NSLOT;
+constexpr uint32_t OFF_NV = OFF_CONST + 16 * 32 * 16;             // NSLOT x 128 x (||v||^2, ||v||_1), own-norm kernels only
+constexpr int kNumSums = 7;                                       // running sums a token carries (RowSums)
+constexpr uint32_t OFF_XCH = OFF_NV + NSLOT * TILE * 8;           // [tile parity][2][kNumSums][128] floats: the second half's sums
+constexpr uint32_t OFF_BAR = OFF_XCH + 2 * 2 * kNumSums * TILE * 4;
+constexpr uint32_t kNumBars = 2 * NSTAGE + 2 + 4 + 2 + 2 * NSLOT + 4;
 constexpr uint32_t OFF_TMEM = OFF_BAR + kNumBars * 8;
 constexpr uint32_t kSmemBytes = OFF_TMEM + 16 + 1024;             // + alignment slack
 
 enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_QO_FULL = 2 * NSTAGE, BAR_QO_EMPTY = 2 * NSTAGE + 1,
        BAR_TM_FULL = 2 * NSTAGE + 2,      // [epilogue group][TMEM buffer]
        BAR_TM_EMPTY = 2 * NSTAGE + 6,     // [TMEM buffer]
-       BAR_NV = 2 * NSTAGE + 8 };         // [epilogue group][slot], own-norm kernels only
+       BAR_NV = 2 * NSTAGE + 8,           // [epilogue group][slot], own-norm kernels only
+       BAR_XCH = 2 * NSTAGE + 8 + 2 * NSLOT };   // [tile parity][2]: the second row half's sums are in shared memory
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -185,7 +194,8 @@ struct TcParams {
     float* partial;                           // csplit > 1: [csplit][planes][units][Nmax] partial scores
 };
 
-__device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? lens[b] : nmax; }
+// (a device-side length is clamped to [0, max_len]: the host cannot check it)
+__device__ __forceinline__ int tc_seq_len_raw(const int32_t* lens, int b, int nmax) { return lens ? min(max(lens[b], 0), nmax) : nmax; }
 __device__ __forceinline__ int tc_seq_len(const TcParams& p, int b) { return tc_seq_len_raw(p.seq_lens, b, p.Nmax); }
 __device__ __forceinline__ int tc_mask_len(const TcParams& p, int b) { return p.mask_lens ? p.mask_lens[b] : tc_seq_len(p, b); }
 
@@ -358,6 +368,21 @@ __device__ __forceinline__ void score_chunk(uint32_t zt, uint32_t tt, int chunk_
     }
 }
 
+// The same item with one batch of 16 rows in registers at a time (half the registers): for kernels whose SM
+// sub-partitions run four epilogue warps, where the other warps cover the wait for the next batch.
+template <unsigned VARS, bool MASKED>
+__device__ __forceinline__ void score_chunk_lean(uint32_t zt, uint32_t tt, int chunk_rows, const float4* cst,
+                                                 float2 sl2, float2 sc, RowSums& S, int ptok, int mask_base, int W, int wi) {
+    uint32_t z0[16], t0[16];
+#pragma unroll 1
+    for (int c0 = 0; c0 < chunk_rows; c0 += 16) {
+        tc_ld16(zt + c0, z0);
+        tc_ld16(tt + c0, t0);
+        tc_wait_ld16x2(z0, t0);
+        score_rows16<VARS, MASKED>(z0, t0, cst + (c0 >> 1), sl2, sc, S, ptok, mask_base, W, wi);
+    }
+}
+
 // VARS: variants this instantiation computes (a superset of p.variants).  OWN_NV: no pass 1 ran (the
 // caller supplied the attention outputs), so warps 2-3 compute the value norms from the V tiles here.
 template <unsigned VARS, bool OWN_NV>
@@ -371,8 +396,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const uint32_t bars = sbase + OFF_BAR;
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_TMEM);
-    float4* sConst = reinterpret_cast<float4*>(smem + OFF_CONST);   // [8 epilogue warps][64 row pairs]
+    float4* sConst = reinterpret_cast<float4*>(smem + OFF_CONST);   // [16 epilogue warps][32 row pairs]
     float2* sNv = reinterpret_cast<float2*>(smem + OFF_NV);         // [NSLOT][128] (||v||^2, ||v||_1)
+    float* sXch = reinterpret_cast<float*>(smem + OFF_XCH);         // [tile parity][2][kNumSums][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     span_begin(p.span);
@@ -385,7 +411,8 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (OWN_NV) for (int i = 0; i < 2 * NSLOT; ++i) mbar_init(bar(BAR_NV + i), 2);
         mbar_init(bar(BAR_QO_FULL), 1); mbar_init(bar(BAR_QO_EMPTY), 1);
         for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_TM_FULL + i), 1);
-        for (int i = 0; i < 2; ++i) mbar_init(bar(BAR_TM_EMPTY + i), 4);
+        for (int i = 0; i < 2; ++i) mbar_init(bar(BAR_TM_EMPTY + i), 8);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_XCH + i), 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -516,14 +543,18 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
     } else {
         // ======================================= epilogue =======================================
-        const int wg = (warp - 4) >> 2;                            // 0: even tiles, 1: odd tiles
+        const int wg = (warp - 4) >> 3;                            // 0: even tiles, 1: odd tiles
+        const int half = ((warp - 4) >> 2) & 1;                    // 0: first half of the window rows (and the stores), 1: the rest
         const int lane_grp = warp & 3;                             // TMEM lanes 32*lane_grp .. +31
         const int tok = lane_grp * 32 + lane;                      // token within the tile
+        // the chunk's rows in two runs of whole 16-row batches
+        const int rows0 = min(p.chunk_rows, (p.chunk_rows / 2 + 15) / 16 * 16);
+        const int r_begin = half ? rows0 : 0, r_count = half ? p.chunk_rows - rows0 : rows0;
         const float2 sl2 = make_float2(p.scale * kLog2e, p.scale * kLog2e), sc = make_float2(p.scale, p.scale);
         const size_t plane = (size_t)units * p.Nmax;
-        uint32_t item = 0, tile_seq = 0;
+        uint32_t item = 0, tile_seq = 0, mine_seq = 0;
         uint32_t full_par = 0, nv_par = 0;                         // phase parity of this group's barriers, one bit each
-        float4* my_const = sConst + (warp - 4) * 64;               // this warp's copy of the unit's row constants
+        float4* my_const = sConst + (warp - 4) * 32;               // this warp's copy of its rows' constants
         int const_unit = -1;
         for (; !tw.done() && !failed; tw.next()) {
             const bool mine = (tile_seq & 1) == (uint32_t)wg;
@@ -540,13 +571,14 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             S.s1 = S.s2 = S.s3 = S.s4 = S.s5 = S.s6 = S.s7 = make_float2(0.f, 0.f);
             const uint32_t buf = item & 1;
             float nv = 0.f, nv1 = 0.f;                             // used after the row loop
-            if (!OWN_NV && ptok < N) nv = p.nv[(size_t)unit * p.Nmax + ptok];
-            if (unit != const_unit) {                              // at most once per unit: (-lse2, |o|^2) of every row pair
+            if (!OWN_NV && half == 0 && ptok < N) nv = p.nv[(size_t)unit * p.Nmax + ptok];
+            if (unit != const_unit) {                              // at most once per unit: (-lse2, |o|^2) of the warp's row pairs
                 __syncwarp();
-                for (int i = lane; i < 64; i += 32) {
-                    float4 c4 = i * 2 < p.chunk_rows ? p.cpair[(((size_t)unit * p.rows_out) >> 1) + i] : make_float4(-INFINITY, -INFINITY, 0.f, 0.f);
+                {
+                    const int rp = (r_begin >> 1) + lane;          // row pair of the chunk
+                    float4 c4 = lane * 2 < r_count ? p.cpair[(((size_t)unit * p.rows_out) >> 1) + rp] : make_float4(-INFINITY, -INFINITY, 0.f, 0.f);
                     if (VARS == OBC_VAR_VK) { c4.z *= p.scale; c4.w *= p.scale; }
-                    my_const[i] = c4;
+                    my_const[lane] = c4;
                 }
                 __syncwarp();
                 const_unit = unit;
@@ -554,7 +586,7 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (!mbar_wait(bar(BAR_TM_FULL + wg * 2 + buf), (full_par >> buf) & 1)) { failed = true; fail_site = __LINE__; break; }
             full_par ^= 1u << buf;
             tc_fence_after();
-            if (OWN_NV) {                                          // the norms of this tile (ready long before the accumulators)
+            if (OWN_NV && half == 0) {                             // the norms of this tile (ready long before the accumulators)
                 const uint32_t slot = item % NSLOT;
                 if (!mbar_wait(bar(BAR_NV + wg * NSLOT + slot), (nv_par >> slot) & 1)) { failed = true; fail_site = __LINE__; break; }
                 nv_par ^= 1u << slot;
@@ -562,36 +594,63 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 nv = n21.x; nv1 = n21.y;
             }
             const float4* cst = my_const;
-            const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u, tt = zt + 128u;
-            if (masked_tile)
-                score_chunk<VARS, true>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, Nm - p.W, p.W, 0);
-            else
-                score_chunk<VARS, false>(zt, tt, p.chunk_rows, cst, sl2, sc, S, ptok, 0, 0, 0);
+            const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u + (uint32_t)r_begin, tt = zt + 128u;
+            if (r_count > 0) {
+                if (masked_tile)
+                    score_chunk_lean<VARS, true>(zt, tt, r_count, cst, sl2, sc, S, ptok, Nm - p.W, p.W, r_begin % p.W);
+                else
+                    score_chunk_lean<VARS, false>(zt, tt, r_count, cst, sl2, sc, S, ptok, 0, 0, 0);
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_TM_EMPTY + buf));
             ++item;
-            if (!failed && ptok < p.Nmax) {
+            // the two row halves of the token meet: sums 1..7 of RowSums, packed lanes folded
+            float sum[kNumSums] = {S.s1.x + S.s1.y, S.s2.x + S.s2.y, S.s3.x + S.s3.y, S.s4.x + S.s4.y,
+                                   S.s5.x + S.s5.y, S.s6.x + S.s6.y, S.s7.x + S.s7.y};
+            // slot xs was last used two of this group's tiles ago; the first half read it before it released the
+            // accumulators of the tile after that one, without which the tile at hand could not have been computed
+            const uint32_t xs = mine_seq & 1;
+            float* xch = sXch + ((wg * 2 + xs) * kNumSums) * TILE + tok;
+            if (half == 1) {
+#pragma unroll
+                for (int j = 0; j < kNumSums; ++j) {
+                    const bool used = VARS == OBC_VAR_VK ? j < 2 : true;
+                    if (used) xch[j * TILE] = sum[j];
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_XCH + wg * 2 + xs));
+                ++mine_seq;
+                continue;
+            }
+            if (!mbar_wait(bar(BAR_XCH + wg * 2 + xs), (mine_seq >> 1) & 1)) { failed = true; fail_site = __LINE__; break; }
+            ++mine_seq;
+#pragma unroll
+            for (int j = 0; j < kNumSums; ++j) {
+                const bool used = VARS == OBC_VAR_VK ? j < 2 : true;
+                if (used) sum[j] += xch[j * TILE];
+            }
+            if (ptok < p.Nmax) {
                 const bool live = ptok < N;
                 const float s2 = p.scale * p.scale;
                 int pl = 0;
-                if (p.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + ptok] = live ? nv * (S.s6.x + S.s6.y) : 0.f;
+                if (p.variants & OBC_VAR_V)    out[(size_t)(pl++) * plane + ptok] = live ? nv * sum[5] : 0.f;
                 if (p.variants & OBC_VAR_K)    out[(size_t)(pl++) * plane + ptok] =
-                    live ? s2 * (fmaf(nv, S.s5.x + S.s5.y, S.s3.x + S.s3.y) + (S.s4.x + S.s4.y)) : 0.f;
+                    live ? s2 * (fmaf(nv, sum[4], sum[2]) + sum[3]) : 0.f;
                 if (p.variants & OBC_VAR_VK)   out[(size_t)(pl++) * plane + ptok] =
-                    live ? fmaf(nv, S.s1.x + S.s1.y, fmaf(p.scale, S.s2.x + S.s2.y, s2 * (S.s3.x + S.s3.y))) : 0.f;
-                if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? S.s7.x + S.s7.y : 0.f;
-                if (p.variants & OBC_VAR_VATP) out[(size_t)(pl++) * plane + ptok] = live ? nv1 * (S.s7.x + S.s7.y) : 0.f;
+                    live ? fmaf(nv, sum[0], fmaf(p.scale, sum[1], s2 * sum[2])) : 0.f;
+                if (p.variants & OBC_VAR_ATTN) out[(size_t)(pl++) * plane + ptok] = live ? sum[6] : 0.f;
+                if (p.variants & OBC_VAR_VATP) out[(size_t)(pl++) * plane + ptok] = live ? nv1 * sum[6] : 0.f;
             }
         }
         // padding beyond the last tile of a shorter sequence: zeros
         if (p.seq_lens) {
-            const int et = threadIdx.x - 128;                      // 0..255
+            const int et = threadIdx.x - 128;                      // 0..511
             const int n_planes = __popc(p.variants);
             for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
                 const int first = (tc_seq_len(p, unit / p.Hkv) + TILE - 1) / TILE * TILE;
                 for (int pl = 0; pl < n_planes; ++pl)
-                    for (int i = first + et; i < p.Nmax; i += 256) p.scores[(size_t)pl * plane + (size_t)unit * p.Nmax + i] = 0.f;
+                    for (int i = first + et; i < p.Nmax; i += 512) p.scores[(size_t)pl * plane + (size_t)unit * p.Nmax + i] = 0.f;
             }
         }
     }
@@ -626,7 +685,7 @@ constexpr uint32_t MC_OFF_BAR = MC_OFF_CONST + 4 * 32 * 16;
 enum { MC_FULL = 0, MC_EMPTY = 2, MC_QO_FULL = 4, MC_QO_EMPTY = 6, MC_TM_FULL = 8, MC_TM_EMPTY = 12,
        MC_NV = 16, MC_CONST = 18, MC_NBARS = 22 };
 constexpr uint32_t MC_OFF_TMEM = MC_OFF_BAR + MC_NBARS * 8;
-constexpr int kThreadsMulti = kThreads + 32;                      // + warp 12: the second MMA-issuing thread
+constexpr int kThreadsMulti = kThreadsBase + 32;                      // + warp 12: the second MMA-issuing thread
 constexpr uint32_t kSmemMulti = MC_OFF_TMEM + 16 + 1024;
 
 // SPLIT: the general walk (row chunks of a pair shared by several CTAs, hidden tile pairs skipped); without
@@ -1032,10 +1091,6 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // with more CTAs than SMs the long ones should start first
     const int unit = vu / p.n_chunks, c = p.n_chunks - 1 - vu % p.n_chunks;
     const int b = unit / p.Hkv, g = unit % p.Hkv;
-    // a split past the end of a shorter sequence has nothing to do and the merge does not read its partial result
-    // (the sequence lengths are the caller's input, so they may be read before the wait on the preceding kernel)
-    if (split > 0 && split * p.tiles_per_split * TILE >= tc_seq_len_raw(p.seq_lens, b, p.Nmax)) return;
-
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
         // a K/V stage is released by the MMA commit and, in the CTAs of the last row chunk, by the two ||v||^2 warps
@@ -1054,10 +1109,13 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
     int fail_site = 0;                             // source line of the wait that gave up (status word)
-    pdl_wait();                                    // nothing above reads or writes global memory
+    pdl_wait();                                    // above, only the span words of the workspace header were touched (atomically)
     // the status word starts at 0: no wait of this call can have given up yet (each lasts seconds)
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.status = 0u;
     const int N = tc_seq_len_raw(p.seq_lens, b, p.Nmax);
+    // a split past the end of a shorter sequence has nothing to do and the merge does not read its partial result
+    // (the lengths may be the preceding kernel's output, so they are read after the wait)
+    const bool idle_split = split > 0 && split * p.tiles_per_split * TILE >= N;
     const int tile_lo = split * p.tiles_per_split;
     // tiles past the last token that any row of this chunk sees are not visited
     const int Nm = p.mask_lens ? p.mask_lens[b] : N;       // a shard of a longer sequence: its distance to that sequence's end
@@ -1065,7 +1123,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int tile_hi = min(min(tile_lo + p.tiles_per_split, (N + TILE - 1) / TILE), chunk_last / TILE + 1);
     const int n_tiles = max(tile_hi - tile_lo, 0);
 
-    if (warp == 0) {
+    if (idle_split) {
+        // nothing to compute and nothing to store
+    } else if (warp == 0) {
         // ===================================== TMA producer =====================================
         if (lane == 0 && n_tiles > 0) {
             mbar_expect_tx(bar(P1_QFULL), (uint32_t)p.chunk_rows * 256u);

@@ -1,5 +1,5 @@
-// Pooling + per-head top-budget selection + ordered index emission (Algorithm 2's
-// "topk(S[..., :cutoff], num_hh) -> sort"), and the row gather that builds the compacted cache.
+// Pooling + per-head top-budget selection + ordered index emission (Algorithm 2: the num_hh best
+// candidates below the cutoff, their indices ascending), and the row gather that builds the compacted cache.
 //
 //   select_cluster_kernel  one thread-block cluster per (batch item, KV head).  Every CTA pools
 //                     its contiguous share of the candidates into order-preserving uint32 keys

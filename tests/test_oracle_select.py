@@ -140,7 +140,7 @@ def test_decode_state_keeps_sinks_and_recents_and_respects_budget():
 
 @pytest.mark.parametrize("window", [1, 3, 7, 64])
 def test_decode_window_accumulator_matches_a_log_kept_per_token(window):
-    """Accumulation within a recent window (Sec. 6): the state's ring, indexed by slot and step mod w, must
+    """Accumulation within a recent window (App. B): the state's ring, indexed by slot and step mod w, must
     give every live token the sum of the scores it received in the last w steps, as read off a plain log
     keyed by (token position, step) that knows nothing of slots or rings."""
     rng = np.random.default_rng(40 + window)
