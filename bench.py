@@ -5,11 +5,18 @@ A "step" is one pass of the whole path over one Llama-3-8B-shaped layer cache (3
 8 KV heads, head_dim 128, N = 32768 cached tokens, window W = 32, bf16, OBCache-V&K, max-pool 7,
 budget 2048 per head).  The metric is cached tokens scored+compacted per second per layer.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 With N > 1 it is launched by torch.distributed.run, one rank per GPU; every rank processes its
 own cache (the (batch, KV head) units are independent, so there is no data-path collective) and
 the reported value is the sum over ranks divided by the slowest rank's time (weak scaling).
+
+Timing: W warm-up steps, then rounds of exactly K steps, each round bracketed by a barrier and a
+device synchronisation and timed with CUDA events; rounds are repeated until at least half a
+second has been timed and the median round is reported (with few steps a single round lasts a
+millisecond or two, less than one clock sample).  Every workload prints one JSON line with the
+clocks sampled during the rounds, the roofline of its dominant kernel and of the whole step, the
+plain-ALU and special-function bounds, and the CPU checker timed on a bounded sample.
 
 `--impl reference` times the CPU checker (oracle/) as it stands on the host cores.
 """
@@ -31,7 +38,12 @@ METRIC = "cached tokens scored+compacted/sec per layer"
 UNIT = "tokens/s"
 WORKLOAD = ("llama3-8b-layer-32k: B1 Hq32 Hkv8 d128 N32768 W32 bf16, OBCache-V&K, max-pool 7, "
             "budget 2048/head, n_recent 32")
-N_COPIES = 4            # distinct input copies rotated between steps (4 x 135 MB > 126 MB L2)
+NOMINAL_HBM_GBS, NOMINAL_BF16_TFLOPS = 8000.0, 2250.0
+N_SM, FP32_LANES, SFU_LANES = 148, 128, 16        # per SM: fp32 lanes, special-function lanes
+MIN_TIMED_S = 0.5
+PREFILL = {"llama32k": 2, "qwen128k": 3, "ragged": 4}
+WORKLOADS = ["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive",
+             "history4k", "decode-window", "llama32k-sharded"]
 
 
 def load_peaks():
@@ -56,7 +68,7 @@ class ClockSampler:
         self.t0 = time.time()
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu=timestamp,{self.FIELDS}", "--format=csv,noheader,nounits",
-                                       "-lms", "50", "-i", str(device_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-lms", "20", "-i", str(device_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
         self.marks = {}
@@ -67,7 +79,7 @@ class ClockSampler:
     def stop(self):
         if self.p is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        time.sleep(0.06)
+        time.sleep(0.05)
         self.p.terminate()
         self.p.wait()
         self.f.flush()
@@ -83,7 +95,7 @@ class ClockSampler:
                 continue
         a, b = self.marks.get("timed_begin", self.t0), self.marks.get("timed_end", time.time())
         inside = [x for x in parsed if a <= x[0] <= b]
-        where = "timed region"
+        where = "timed rounds"
         if not inside:                       # region shorter than the sampling period
             inside, where = parsed, "whole run"
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -109,67 +121,291 @@ def ncu_traffic(kernel):
     return float(rec[kernel]) if kernel in rec else None
 
 
-def make_case(seed):
-    from paper_2510_07651_b200 import synth
-    return synth.config(2, seed=seed)
+# ---------------------------------------------------------------------------------------------------
+# what each workload is: name, how the inputs relate to the L2, how it shards
+# ---------------------------------------------------------------------------------------------------
+def workload_config(name, world=1):
+    """The `config` object of the JSON line: the same for the library arm and the reference arm."""
+    text = {
+        "llama32k": WORKLOAD,
+        "qwen128k": "qwen2.5-7b-layer-128k: B1 Hq28 Hkv4 d128 N131072 W64 bf16, OBCache-K and V&K (one launch), max-pool 7, "
+                    "budget 4096/head, n_recent 64",
+        "ragged": "llama3-8b-layer, batch 8, ragged lengths uniform in [8192, 65536] (seeded): Hq32 Hkv8 d128 W32 bf16, "
+                  "OBCache-V&K, no pooling, budget 10% of each length, n_recent 32",
+        "decode": "decode rescoring: B32 Hq32 Hkv8 d128 bf16, live 4096 -> 4097 -> 4096 slots per head and step (a 16384-token "
+                  "context already reduced to the 4096 budget), W1, OBCache-V&K accumulated, 4 sinks, 256 recent, one eviction "
+                  "per head per step",
+        "decode-window": "decode rescoring as `decode`, the accumulator limited to the scores of the last 16 steps",
+        "llama32k-given": WORKLOAD + "; window O and LSE supplied by the caller (no attention recompute)",
+        "qwen128k-given": "qwen2.5-7b-layer-128k as `qwen128k`; window O and LSE supplied by the caller (no attention recompute)",
+        "llama32k-adaptive": WORKLOAD + "; head-adaptive budgets (safeguard 0.2) instead of one budget per head",
+        "history4k": "llama3-8b-layer, whole sequence as perturbation window: B1 Hq32 Hkv8 d128 N4096 W4096 bf16 (16384 window "
+                     "rows per KV head, causal), OBCache-V&K, max-pool 7, budget 512/head",
+        "llama32k-sharded": "one of two ranks of the 32k Llama layer sharded by token range (this rank: tokens 16384..32767), "
+                            "emulated on one GPU: window attention of the shard, merge with the peer's (o, lse), local scores, "
+                            "selection over the gathered scores; no compaction",
+    }[name]
+    l2 = {
+        "llama32k": "4 distinct input copies rotated between steps (4 x 135 MB > 126 MB L2)",
+        "llama32k-given": "4 distinct input copies rotated between steps (4 x 135 MB > 126 MB L2)",
+        "llama32k-adaptive": "4 distinct input copies rotated between steps (4 x 135 MB > 126 MB L2)",
+        "qwen128k": "inputs larger than L2 (K+V = 268 MB)", "qwen128k-given": "inputs larger than L2 (K+V = 268 MB)",
+        "ragged": "inputs larger than L2 (K+V = 1.2 GB)",
+        "decode": "inputs larger than L2 (live K+V = 537 MB per step)",
+        "decode-window": "inputs larger than L2 (live K+V = 537 MB per step)",
+        "history4k": "16 distinct input copies rotated between steps (16 x 17 MB > 2 x 126 MB L2)",
+        "llama32k-sharded": "4 distinct input copies rotated between steps (4 x 67 MB > 2 x 126 MB L2)",
+    }[name]
+    return {"workload": text, "l2": l2,
+            "parallelism": f"{world} independent layer caches, one per GPU, no collective"}
 
 
-def run_reference(args):
-    """The CPU checker as it stands, timed on the host cores (rank 0 only).  Each step scores,
-    selects and compacts a bounded sample of the workload: the first `heads` of the 8 KV heads
-    (all 32768 tokens, all their query heads), sized so that the whole run ends within minutes."""
-    if int(os.environ.get("RANK", "0")) != 0:
-        return
-    import numpy as np
-    from oracle import reference as ref
-    ref.build()
-    case, run = make_case(1236)
-    cores = ref.host_threads()
-    G = case.G
+def time_rounds(run_step, steps, warmup, barrier, min_total_s=MIN_TIMED_S, max_rounds=2000):
+    """Median over rounds of exactly `steps` steps; each round has a barrier + synchronise on both sides.
+    Returns (median ms per round, number of rounds)."""
+    import torch
+    from paper_2510_07651_b200 import multirank
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(warmup):
+        run_step(i)
+    rounds, total, it = [], 0.0, warmup
+    while True:
+        barrier()
+        e0.record()
+        for _ in range(steps):
+            run_step(it); it += 1
+        e1.record()
+        torch.cuda.synchronize()
+        barrier()
+        ms = multirank.max_over_ranks(e0.elapsed_time(e1), "cuda")      # every rank sees the same figure
+        rounds.append(ms); total += ms * 1e-3
+        if total >= min_total_s or len(rounds) >= max_rounds:
+            break
+    return statistics.median(rounds), len(rounds)
 
-    def step(heads, n_tok):
-        q, k, v = case.q[:, :heads * G], case.k[:, :heads, :n_tok], case.v[:, :heads, :n_tok]
-        s = ref.score(q, k, v, want=("VK",))["VK"].astype(np.float32)
-        budget = min(run["budget"], n_tok)
-        idx = ref.select_pipeline(s, np.array([n_tok], np.int32), [budget], 0, run["n_recent"], run["pool_mode"],
-                                  run["pool_kernel"], budget)
-        for h in range(heads):
-            ref.compact(case.k_bits[0, h, :n_tok], idx[0, h], budget)
-            ref.compact(case.v_bits[0, h, :n_tok], idx[0, h], budget)
 
-    # size the per-step sample so that warm-up + timed steps take about two minutes in all
-    t0 = time.time()
-    step(1, 4096)
-    t_unit = (time.time() - t0) / 4096                      # seconds per token of one KV head
-    per_step = 120.0 / (args.steps + args.warmup)
-    heads = int(max(1, min(case.Hkv, per_step / (t_unit * case.Nmax))))
-    n_tok = case.Nmax
-    if heads == 1 and t_unit * case.Nmax > per_step:
-        n_tok = int(max(1024, min(case.Nmax, per_step / t_unit)) // 1024 * 1024)
-    for _ in range(args.warmup):
-        step(heads, n_tok)
-    t0 = time.time()
-    for _ in range(args.steps):
-        step(heads, n_tok)
-    dt = time.time() - t0
-    value = n_tok * (heads / case.Hkv) * args.steps / dt           # layer-equivalent tokens per second
-    sample = (f"{heads} of {case.Hkv} KV heads x the first {n_tok} of {case.Nmax} cached tokens per step, "
-              "scaled to one layer (all 8 KV heads)")
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "sample": sample},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
-            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+def bounds_of(alg, seconds, peaks, clock_mhz):
+    """Roofline record of one kernel (or of the whole step) from its algorithmic work.
+    alg: dict(bytes, flops, pairs, fp32_per_pair, ex2_per_pair)."""
+    t_hbm = alg["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_mma = alg.get("flops", 0) / (peaks["bf16_tflops_sustained"] * 1e12)
+    rec = {"algorithmic_bytes": alg["bytes"], "algorithmic_flops": alg.get("flops", 0),
+           "t_hbm_us": t_hbm * 1e6, "t_mma_us": t_mma * 1e6}
+    if t_hbm >= t_mma:
+        ach = alg["bytes"] / seconds / 1e9
+        rec.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
+                   frac_of_nominal=ach / NOMINAL_HBM_GBS, nominal_peak=NOMINAL_HBM_GBS,
+                   peak_source=f"{peaks['source']} STREAM-style copy")
+    else:
+        ach = alg["flops"] / seconds / 1e12
+        rec.update(bound="tensor", achieved=ach, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                   frac=ach / peaks["bf16_tflops_sustained"], frac_of_nominal=ach / NOMINAL_BF16_TFLOPS,
+                   nominal_peak=NOMINAL_BF16_TFLOPS, peak_source=f"{peaks['source']} cuBLAS bf16 sustained")
+    if alg.get("pairs"):
+        hz = (clock_mhz or peaks["sm_max_mhz"]) * 1e6
+        rec["t_fp32_us"] = alg["pairs"] * alg["fp32_per_pair"] / (N_SM * FP32_LANES * hz) * 1e6
+        rec["t_sfu_us"] = alg["pairs"] * alg["ex2_per_pair"] / (N_SM * SFU_LANES * hz) * 1e6
+        rec["alu_note"] = (f"{alg['pairs']:.3g} (row, token) pairs x {alg['fp32_per_pair']} fp32 instructions on {N_SM} x {FP32_LANES} "
+                           f"lanes and x {alg['ex2_per_pair']} ex2 on {N_SM} x {SFU_LANES} lanes at {hz / 1e6:.0f} MHz")
+    return rec
+
+
+def prefill_model(case, run, given=False):
+    """Algorithmic work of the prefill path on `case`: per kernel kind and for the whole step."""
+    d, es = case.d, 2 if case.dtype == "bf16" else 4
+    tok_heads = int(case.seq_lens.sum()) * case.Hkv                  # cached tokens x KV heads
+    planes = len(run["variants"])
+    # (row, token) pairs a pass visits: every window row sees the tokens up to its own position
+    pairs = 0
+    for n in case.seq_lens:
+        n = int(n)
+        vis = sum(n - case.W + i + 1 for i in range(case.W)) if case.W < 4096 else case.W * (2 * n - case.W + 1) // 2
+        pairs += vis * case.G * case.Hkv
+    kv = tok_heads * d * es * 2
+    contraction = 2 * d * pairs                                      # flops of one contraction over the visible pairs
+    fp32 = 7 if run["variants"] == ["VK"] else 10 if set(run["variants"]) == {"K", "VK"} else 12
+    budgets = run["budget"] if isinstance(run["budget"], list) else [run["budget"]] * case.B
+    kept = sum(min(int(b), int(n)) for b, n in zip(budgets, case.seq_lens)) * case.Hkv
+    gather = kept * d * es * 2 * 2                                   # K and V rows read and written
+    score_rw = tok_heads * 4 * (planes + 1)                          # planes written, the selected plane read
+    model = {
+        "pass1": dict(bytes=kv, flops=2 * contraction, pairs=pairs, fp32_per_pair=5, ex2_per_pair=1),
+        "pass2": dict(bytes=kv + tok_heads * 4 * planes, flops=2 * contraction, pairs=pairs, fp32_per_pair=fp32, ex2_per_pair=1),
+        "gather": dict(bytes=gather), "select": dict(bytes=tok_heads * 4 + kept * 4),
+        "step": dict(bytes=kv + score_rw + gather + kept * 4, flops=(2 if given else 4) * contraction,
+                     pairs=pairs * (1 if given else 2), fp32_per_pair=(fp32 if given else (fp32 + 5) / 2), ex2_per_pair=1),
+    }
+    return model
+
+
+def kernel_kind(name):
+    for k in ("pass1", "pass2", "gather", "select"):
+        if k in name:
+            return k
+    return None
+
+
+def finish_line(*, name, world, args, metric, unit, value, ms_round, rounds, prof, prof_steps, model, peaks, clocks,
+                cpu, e2e=None, headline_kernel=None, spans=None, extra=None, launch=None):
+    ms_step = ms_round / args.steps
+    clock = clocks.get("sm_mhz") if clocks else None
+    kernels = {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}
+    by_kernel = {}
+    for k, rec in kernels.items():
+        kind = kernel_kind(k)
+        if kind and kind in model:
+            by_kernel[k] = dict(avg_us=rec["avg_us"], **bounds_of(model[kind], rec["avg_us"] * 1e-6, peaks, clock))
+    if spans:
+        for k, span in spans.items():
+            if k in kernels and span > 0:
+                kernels[k]["device_span_us"] = span
+                if k in by_kernel:
+                    by_kernel[k]["device_span_us"] = span
+                    by_kernel[k]["frac_device_span"] = by_kernel[k]["frac"] * by_kernel[k]["avg_us"] / span
+    dom = headline_kernel if headline_kernel in by_kernel else None
+    if dom is None and by_kernel:
+        dom = max((k for k in by_kernel if kernel_kind(k) in ("pass1", "pass2")), key=lambda k: kernels[k]["avg_us"], default=None)
+    roof = {"kernel": dom, "launches": kernels[dom]["launches"] if dom else None, "traffic": None}
+    if dom:
+        roof.update(by_kernel[dom])
+        roof["traffic"] = ncu_traffic(dom)
+    roof["kernels"] = by_kernel
+    roof["step"] = dict(us=ms_step * 1e3, **bounds_of(model["step"], ms_step * 1e-3, peaks, clock))
+    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": workload_config(name, world),
+            "timing": {"rounds": rounds, "steps_per_round": args.steps, "reported": "median round",
+                       "min_timed_s": MIN_TIMED_S, "launch": launch},
+            "clocks": clocks, "e2e": e2e,
+            "gpu_launches": (sum(v[0] for v in prof.values()) // max(prof_steps, 1)) * args.steps,
+            "roofline": roof, "kernels": kernels, "cpu_baseline": cpu}
+    if extra:
+        line.update(extra)
     print(json.dumps(line))
 
 
-def run_ours(args):
+# ---------------------------------------------------------------------------------------------------
+# CPU checker legs (bounded samples of each workload)
+# ---------------------------------------------------------------------------------------------------
+def cpu_prefill_sample(case, run, *, heads=None, batch=None, given=False, adaptive=False, budget_s=10.0, max_reps=8):
+    """The checker on a sample of `case`: KV heads [0, heads) of batch items [0, batch); score, pool + select,
+    compact.  Returns (layer-equivalent tokens per second, description, seconds)."""
     import numpy as np
+    from oracle import reference as ref
+    ref.build()
+    B = case.B if batch is None else batch
+    H = case.Hkv if heads is None else heads
+    G = case.G
+    q, k, v = case.q[:B, :H * G], case.k[:B, :H], case.v[:B, :H]
+    lens = case.seq_lens[:B]
+    want = tuple(run["variants"])
+    budgets = run["budget"] if isinstance(run["budget"], list) else [run["budget"]] * case.B
+    stride = int(max(budgets)) * (4 if adaptive else 1)
+    giv = None
+    if given:                                  # the window attention a caller would hand over (untimed)
+        out = ref.score(q, k, v, seq_lens=lens, want=("ATTN",), return_attention=True)
+        giv = (out["O"].reshape(B, H * G, case.W, case.d).astype(np.float32),
+               (out["m"] + np.log(out["l"])).reshape(B, H * G, case.W).astype(np.float32))
+    reps, t0 = 0, time.time()
+    while reps < 1 or (time.time() - t0 < budget_s and reps < max_reps):
+        s = ref.score(q, k, v, seq_lens=lens, want=want, given=giv)[want[-1]].astype(np.float32)
+        if adaptive:
+            ridx, _ = ref.select_adaptive_pipeline(s, lens, budgets[:B], run["n_sink"], run["n_recent"], run["pool_mode"],
+                                                   run["pool_kernel"], 0.2, stride)
+        else:
+            ridx = ref.select_pipeline(s, lens, budgets[:B], run["n_sink"], run["n_recent"], run["pool_mode"],
+                                       run["pool_kernel"], stride)
+        for b in range(B):
+            for h in range(H):
+                n, cnt = int(lens[b]), int((ridx[b, h] >= 0).sum())     # rows are padded with -1 beyond the kept tokens
+                ref.compact(case.k_bits[b, h, :n], ridx[b, h, :cnt], cnt)
+                ref.compact(case.v_bits[b, h, :n], ridx[b, h, :cnt], cnt)
+        reps += 1
+    dt = time.time() - t0
+    tokens = int(lens.sum()) * (H / case.Hkv)            # layer-equivalent tokens (all KV heads of a layer)
+    desc = (f"KV heads 0..{H - 1} of {case.Hkv}, batch items 0..{B - 1} of {case.B} ({int(lens.sum())} tokens per head), "
+            f"{reps} repetition(s), {dt:.1f} s; scaled to one layer by the head count")
+    return tokens * reps / dt, desc, dt
+
+
+def cpu_decode_sample(dc, *, n0, budget, n_sink, n_recent, steps=8, window=0):
+    """`steps` decode steps of the checker over every (batch item, KV head): append, W = 1 scores, accumulate, evict."""
+    import numpy as np
+    from oracle import reference as ref
+    ref.build()
+    B, Hkv, G, cap = dc.k0.shape[0], dc.k0.shape[1], dc.q_t.shape[2] // dc.k0.shape[1], budget + 1
+    sts = [[ref.DecodeState(dc.k0[b, h], dc.v0[b, h], cap, window=window) for h in range(Hkv)] for b in range(B)]
+    t0 = time.time()
+    for t in range(steps):
+        for b in range(B):
+            for h in range(Hkv):
+                st = sts[b][h]
+                st.append(dc.k_t[t, b, h], dc.v_t[t, b, h], n0 + t)
+                acc = st.accumulate(st.scores(dc.q_t[t, b, h * G:(h + 1) * G], "VK"), n0 + t)
+                live = st.pos >= 0
+                st.s_acc[live] = acc[live].astype(np.float32)
+                st.evict(n0 + t, budget, n_sink, n_recent)
+    dt = time.time() - t0
+    return steps / dt, f"{steps} steps over all {B} x {Hkv} heads ({n0 + 1} live slots each), {dt:.1f} s", dt
+
+
+# ---------------------------------------------------------------------------------------------------
+# reference arm: the CPU checker
+# ---------------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The CPU checker as it stands, timed on the host cores (rank 0 only).  Each step is a bounded sample of
+    the workload, sized so that the whole run ends within a few minutes; the value is scaled to the metric's unit."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import reference as ref
+    from paper_2510_07651_b200 import synth
+    ref.build()
+    cores = ref.host_threads()
+    name = args.workload
+    per_step = 120.0 / (args.steps + args.warmup)
+    if name.startswith("decode"):
+        n0, budget = 4096, 4096
+        dc = synth.make_decode(B=32, Hq=32, Hkv=8, d=128, n0=n0, steps=args.steps + args.warmup, seed=1239)
+        window = 16 if name == "decode-window" else 0
+        val, desc, dt = cpu_decode_sample(dc, n0=n0, budget=budget, n_sink=4, n_recent=256,
+                                          steps=min(max(1, args.steps), dc.q_t.shape[0]), window=window)
+        value, metric, unit, ms_step, sample = val, "decode rescoring steps/sec", "steps/s", 1e3 / val, desc
+    else:
+        base = name.replace("-given", "").replace("-adaptive", "").replace("-sharded", "")
+        case, run = synth.full_history(4096) if base == "history4k" else synth.config(PREFILL[base], seed=1236 if base == "llama32k" else None)
+        given, adaptive = name.endswith("-given"), name.endswith("-adaptive")
+        # size the sample: time one KV head of one batch item, then take as many heads (and batch items) as fit a step
+        heads, batch = 1, 1
+        v0, _, dt0 = cpu_prefill_sample(case, run, heads=1, batch=1, given=given, adaptive=adaptive, budget_s=0.0, max_reps=1)
+        per_head_s = dt0
+        heads = int(max(1, min(case.Hkv, per_step / max(per_head_s, 1e-3))))
+        if heads == case.Hkv and case.B > 1:
+            batch = int(max(1, min(case.B, per_step / max(per_head_s * case.Hkv, 1e-3))))
+        for _ in range(args.warmup):
+            cpu_prefill_sample(case, run, heads=heads, batch=batch, given=given, adaptive=adaptive, budget_s=0.0, max_reps=1)
+        t0, tok = time.time(), 0.0
+        for _ in range(args.steps):
+            v, sample, dt = cpu_prefill_sample(case, run, heads=heads, batch=batch, given=given, adaptive=adaptive, budget_s=0.0, max_reps=1)
+            tok += v * dt
+        total = time.time() - t0
+        value, metric, unit, ms_step = tok / total, METRIC, UNIT, 1e3 * total / args.steps
+        sample = sample.split(", 1 repetition")[0] + " per step; scaled to one layer by the head count"
+    line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(name, args.gpus),
+            "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------
+# the library arm
+# ---------------------------------------------------------------------------------------------------
+def setup_gpu():
     import torch
     import torch.distributed as dist
-    from paper_2510_07651_b200 import api, build, multirank, synth
-
+    from paper_2510_07651_b200 import api, build
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -178,114 +414,194 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     build.build()
     api.lib()
-    peaks = load_peaks()
-
-    # ---- inputs: N_COPIES distinct seeded caches, resident in HBM ------------------------------
-    bf = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
-    cases, dev = [], []
-    for c in range(N_COPIES):
-        case, run = make_case(1236 + 100 * rank + c)
-        cases.append(case)
-        dev.append((bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)))
-    case = cases[0]
-    B, Hkv, N, d, budget = case.B, case.Hkv, case.Nmax, case.d, run["budget"]
-    tokens_per_step = int(case.seq_lens.sum())
-
-    # ---- preallocated outputs and workspaces (nothing is allocated inside the timed region) -----
-    sp = api.score_params(dev[0][0], dev[0][1], variants=run["variants"], path=args.path)
-    ws_score = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
-    scores = torch.empty((1, B, Hkv, N), dtype=torch.float32, device="cuda")
-    selp = api.select_params(scores[0], budget=budget, n_recent=run["n_recent"], pool=run["pool_mode"],
-                             pool_kernel=run["pool_kernel"])
-    ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
-    idx = torch.empty((B, Hkv, budget), dtype=torch.int32, device="cuda")
-    k_out = torch.empty((B, Hkv, budget, d), dtype=torch.bfloat16, device="cuda")
-    v_out = torch.empty_like(k_out)
-
-    def step(q, k, v):
-        api.obc_score(q, k, v, variants=run["variants"], path=args.path, scores=scores, workspace=ws_score)
-        api.obc_select(scores[0], budget=budget, n_recent=run["n_recent"], pool=run["pool_mode"],
-                       pool_kernel=run["pool_kernel"], idx=idx, workspace=ws_sel)
-        api.obc_compact(k, v, idx, k_out=k_out, v_out=v_out)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+    return world, rank, local, barrier
+
+
+def run_prefill(args):
+    """llama32k (the headline), qwen128k, ragged, their -given / -adaptive variants and history4k."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2510_07651_b200 import api, synth
+
+    name = args.workload
+    world, rank, local, barrier = setup_gpu()
+    if world > 1 and name != "llama32k":
+        raise SystemExit("only the headline workload runs on several GPUs")
+    peaks = load_peaks()
+    given, adaptive = name.endswith("-given"), name.endswith("-adaptive")
+    base = name.replace("-given", "").replace("-adaptive", "")
+    headline = name == "llama32k"
+    n_copies = {"llama32k": 4, "history4k": 16}.get(base, 1)
+
+    bf = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    cases, dev = [], []
+    for c in range(n_copies):
+        if base == "history4k":
+            case, run = synth.full_history(4096, seed=1240 + c)
+        elif base == "llama32k":
+            case, run = synth.config(2, seed=1236 + 100 * rank + c)
+        else:
+            case, run = synth.config(PREFILL[base])
+        cases.append(case)
+        dev.append((bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)))
+    case = cases[0]
+    B, Hkv, N, d = case.B, case.Hkv, case.Nmax, case.d
+    tokens_per_step = int(case.seq_lens.sum())
+    lens = None if (case.seq_lens == case.Nmax).all() else torch.from_numpy(case.seq_lens).cuda()
+    order = [n for n in ("V", "K", "VK") if n in run["variants"]]
+    budgets = np.asarray(run["budget"] if isinstance(run["budget"], list) else [run["budget"]] * B, np.int32)
+    uniform = bool((budgets == budgets[0]).all())
+    bud_d = None if uniform else torch.from_numpy(budgets).cuda()
+    stride = int(budgets.max()) * (4 if adaptive else 1)      # adaptive: a head may keep up to four average budgets
+
+    # ---- preallocated outputs and workspaces (nothing is allocated inside the timed region) -----
+    sp = api.score_params(dev[0][0], dev[0][1], seq_lens=lens, variants=order, path=args.path)
+    ws_score = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
+    scores = torch.empty((len(order), B, Hkv, N), dtype=torch.float32, device="cuda")
+    selp = api.select_params(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
+                             seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"])
+    ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
+    if adaptive:
+        n_ws = api.C.c_size_t(0)
+        api._check(api.lib().obc_select_adaptive_workspace(api.C.byref(selp), 0.2, api.C.byref(n_ws)), "obc_select_adaptive_workspace")
+        ws_sel = torch.empty(n_ws.value, dtype=torch.uint8, device="cuda")
+    counts = torch.empty((B, Hkv), dtype=torch.int32, device="cuda")
+    idx = torch.empty((B, Hkv, stride), dtype=torch.int32, device="cuda")
+    k_out = torch.empty((B, Hkv, stride, d), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+
+    given_dev = []
+    if given:
+        # what the model's attention kernel would hand over for the window rows, made here (untimed set-up)
+        # with plain tensor ops: O = softmax(scale * Q K^T) V and the natural-log LSE, causal over the window
+        G, W, scale = case.G, case.W, 1.0 / np.sqrt(128.0)
+        for (q, k, v) in dev:
+            o_win = torch.empty((B, case.Hq, W, 128), dtype=torch.bfloat16, device="cuda")
+            lse_win = torch.empty((B, case.Hq, W), dtype=torch.float32, device="cuda")
+            for b_ in range(B):
+                n = int(case.seq_lens[b_])
+                vis = torch.arange(n, device="cuda")[None, :] <= (n - W + torch.arange(W, device="cuda"))[:, None]
+                for g_ in range(Hkv):
+                    qg = q[b_, g_ * G:(g_ + 1) * G].float()
+                    z = torch.einsum("gwd,nd->gwn", qg, k[b_, g_, :n].float()) * scale
+                    z = z.masked_fill(~vis[None], float("-inf"))
+                    lse_win[b_, g_ * G:(g_ + 1) * G] = torch.logsumexp(z, dim=-1)
+                    o_win[b_, g_ * G:(g_ + 1) * G] = (torch.softmax(z, dim=-1) @ v[b_, g_, :n].float()).to(torch.bfloat16)
+                    del z
+            given_dev.append((o_win, lse_win))
+        torch.cuda.synchronize()
+
+    def step_on(q, k, v, c, oi=idx, ok=k_out, ov=v_out):
+        if given:
+            api.obc_score_given(q, k, v, given_dev[c][0], given_dev[c][1], seq_lens=lens, variants=order, scores=scores,
+                                workspace=ws_score)
+        else:
+            api.obc_score(q, k, v, seq_lens=lens, variants=order, path=args.path, scores=scores, workspace=ws_score)
+        if adaptive:
+            api.obc_select_adaptive(scores[-1], budget=int(budgets[0]), safeguard=0.2, idx_stride=stride, seq_lens=lens,
+                                    n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
+                                    idx=oi, counts=counts, workspace=ws_sel)
+        else:
+            api.obc_select(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
+                           seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
+                           idx=oi, workspace=ws_sel)
+        api.obc_compact(k, v, oi, k_out=ok, v_out=ov)
+
+    def step(i):
+        c = i % n_copies
+        step_on(*dev[c], c)
 
     # One CUDA graph per input copy holds the whole step (the library only enqueues work on the
-    # current stream and allocates nothing, so a step can be captured); the timed loop replays
-    # them in rotation, which keeps the host out of the measurement.  --eager times plain calls.
-    for i in range(N_COPIES):
-        step(*dev[i])                               # first calls: function attributes, lazy module load
+    # current stream and allocates nothing, so a step can be captured); both ways of issuing a step
+    # are timed, plain library calls and graph replay; the job's figure is the faster one.
+    for i in range(n_copies):
+        step(i)                                     # first calls: function attributes, lazy module load
     torch.cuda.synchronize()
     graphs = []
     if not args.eager:
-        for i in range(N_COPIES):
+        for i in range(n_copies):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                step(*dev[i])
+                step(i)
             graphs.append(g)
 
-    # Both ways of issuing a step are timed over the same K steps, plain library calls and graph
-    # replay; the job's figure is the faster one (which one wins depends on the host).
     sampler = ClockSampler(local) if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
-    def timed(run):
-        for i in range(args.warmup):
-            run(i)
-        barrier()
-        e0.record()
-        for i in range(args.steps):
-            run(i)
-        e1.record()
-        torch.cuda.synchronize()
-        barrier()
-        return multirank.max_over_ranks(e0.elapsed_time(e1), "cuda")
-
     if sampler:
         sampler.mark("timed_begin")
-    ms_by_mode = {"plain library calls": timed(lambda i: step(*dev[i % N_COPIES]))}
+    by_mode = {"plain library calls": time_rounds(step, args.steps, args.warmup, barrier)}
     if graphs:
-        ms_by_mode["one captured CUDA graph per step, replayed"] = timed(lambda i: graphs[i % N_COPIES].replay())
+        by_mode["one captured CUDA graph per step, replayed"] = time_rounds(lambda i: graphs[i % n_copies].replay(),
+                                                                            args.steps, args.warmup, barrier)
     if sampler:
         sampler.mark("timed_end")
-    launch_mode, ms = min(ms_by_mode.items(), key=lambda kv: kv[1])
+    launch_mode, (ms_round, rounds) = min(by_mode.items(), key=lambda kv: kv[1][0])
 
     # ---- per-kernel times (same steps again, every kernel bracketed by CUDA events) -------------
-    prof_steps = min(args.steps, 200)
+    prof_steps = max(20, min(args.steps, 200))
     api.obc_profile_begin()
     for i in range(prof_steps):
-        step(*dev[i % N_COPIES])
+        step(i)
     torch.cuda.synchronize()
     prof = api.obc_profile_end()
     clocks = sampler.stop() if sampler else None
-    launches_per_step = sum(v[0] for v in prof.values()) // max(prof_steps, 1)
 
-    # ---- device-side extents of the two score kernels (first CTA start to last CTA end, read from the
-    # GPU's own timer by the kernels): plain calls, one step at a time, no events between the kernels ----
+    # ---- device-side extents of the two tensor-core score kernels (first CTA start to last CTA end, read from
+    # the GPU's own timer by the kernels): plain calls, one step at a time, no events between the kernels ----
     api.obc_score_kernel_spans(ws_score)                # zeroes the header words
-    spans = [0.0, 0.0]
-    span_steps = min(args.steps, 50)
+    spans = {"tc_pass1": 0.0, "tc_pass2": 0.0}
+    span_steps = 20
     for i in range(span_steps):
-        step(*dev[i % N_COPIES])
+        step(i)
         s1, s2 = api.obc_score_kernel_spans(ws_score)
-        spans[0] += s1 / span_steps; spans[1] += s2 / span_steps
+        spans["tc_pass1"] += s1 / span_steps; spans["tc_pass2"] += s2 / span_steps
 
-    # ---- end to end: host (pinned) inputs -> device, whole path, results back to the host -------
+    e2e = None
+    if headline:
+        e2e = run_e2e(args, world, barrier, dev, step_on, idx, k_out, v_out, tokens_per_step)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        if base == "llama32k":
+            v, desc, _ = cpu_prefill_sample(case, run, given=given, adaptive=adaptive)
+        elif base == "ragged":
+            v, desc, _ = cpu_prefill_sample(case, run, batch=1, budget_s=10.0, max_reps=2)
+        else:                                   # qwen128k, history4k: one KV head
+            v, desc, _ = cpu_prefill_sample(case, run, heads=1, given=given, budget_s=10.0, max_reps=2)
+        from oracle import reference as ref
+        cpu = {"value": v, "unit": UNIT, "cores": ref.host_threads(), "kind": "oracle", "sample": desc}
+
+    value = world * tokens_per_step * args.steps / (ms_round * 1e-3)
+    finish_line(name=name, world=world, args=args, metric=METRIC, unit=UNIT, value=value, ms_round=ms_round, rounds=rounds,
+                prof=prof, prof_steps=prof_steps, model=prefill_model(case, run, given), peaks=peaks, clocks=clocks, cpu=cpu,
+                e2e=e2e, headline_kernel="tc_pass2", spans=spans, launch=launch_mode,
+                extra={"ms_per_step_by_launch": {k: v[0] / args.steps for k, v in by_mode.items()}, "path": args.path})
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, world, barrier, dev, step_on, idx, k_out, v_out, tokens_per_step):
+    """End to end: host (pinned) inputs -> device, the whole path, results back to the host, every step.
+    The caller double-buffers, as a serving loop would: while step i runs, the inputs of step i + 1 travel to the
+    device on a copy stream and the results of step i - 1 travel back on another."""
+    import torch
+    import torch.distributed as dist
     pin = lambda t: t.cpu().pin_memory()
     host = [tuple(pin(t) for t in dev[c]) for c in range(2)]
-    dq, dk, dv = (torch.empty_like(t) for t in dev[0])
-    h_idx, h_k, h_v = pin(idx), pin(k_out), pin(v_out)
     h2d = sum(t.numel() * t.element_size() for t in host[0])
-    d2h = sum(t.numel() * t.element_size() for t in (h_idx, h_k, h_v))
-
-    # The caller double-buffers, as a serving loop would: while step i runs, the inputs of step i + 1 travel to the
-    # device on a copy stream and the results of step i - 1 travel back on another (PCIe carries both directions
-    # at once).  Every step's inputs are copied in and every step's results are copied out and waited for.
-    dins = [(dq, dk, dv), tuple(torch.empty_like(t) for t in dev[0])]
-    houts = [(h_idx, h_k, h_v), (pin(idx), pin(k_out), pin(v_out))]
+    d2h = sum(t.numel() * t.element_size() for t in (idx, k_out, v_out))
+    dins = [tuple(torch.empty_like(t) for t in dev[0]) for _ in range(2)]
+    houts = [(pin(idx), pin(k_out), pin(v_out)) for _ in range(2)]
     douts = [(idx, k_out, v_out), tuple(torch.empty_like(t) for t in (idx, k_out, v_out))]
     main = torch.cuda.current_stream()
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
@@ -293,13 +609,6 @@ def run_ours(args):
     ev_free = [torch.cuda.Event() for _ in range(2)]         # the step that read input buffer b has run
     ev_done = [torch.cuda.Event() for _ in range(2)]         # results of buffer b are complete on the device
     ev_back = [torch.cuda.Event() for _ in range(2)]         # results of buffer b are on the host
-
-    def e2e_step_buffers(b):
-        oi, ok, ov = douts[b]
-        api.obc_score(*dins[b], variants=run["variants"], path=args.path, scores=scores, workspace=ws_score)
-        api.obc_select(scores[0], budget=budget, n_recent=run["n_recent"], pool=run["pool_mode"],
-                       pool_kernel=run["pool_kernel"], idx=oi, workspace=ws_sel)
-        api.obc_compact(dins[b][1], dins[b][2], oi, k_out=ok, v_out=ov)
 
     def e2e_run(n):
         for b in range(2):
@@ -315,7 +624,7 @@ def run_ours(args):
             if i > 0:                                        # step i - 1 on the main stream, its results device -> host
                 pb = (i - 1) % 2
                 main.wait_event(ev_in[pb]); main.wait_event(ev_back[pb])
-                e2e_step_buffers(pb)
+                step_on(*dins[pb], pb, *douts[pb])
                 ev_free[pb].record(main); ev_done[pb].record(main)
                 s_out.wait_event(ev_done[pb])
                 with torch.cuda.stream(s_out):
@@ -326,6 +635,7 @@ def run_ours(args):
                 ev_back[i % 2].synchronize()                 # the caller reads the results of step i - 2
         ev_back[(n - 1) % 2].synchronize()
 
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2e_steps = max(3, min(args.steps, 20))
     e2e_run(2)
     barrier()
@@ -337,184 +647,93 @@ def run_ours(args):
     e2e_ms = torch.tensor([max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))], device="cuda")
     last = (e2e_steps - 1) % 2                              # what came back is what a plain step gives for those inputs
     got_idx, got_k = houts[last][0].clone(), houts[last][1].clone()
-    step(*dev[last])
+    step_on(*dev[last], last)
     torch.cuda.synchronize()
     if not (torch.equal(got_idx, idx.cpu()) and torch.equal(got_k.view(torch.int16), k_out.cpu().view(torch.int16))):
         raise RuntimeError("end-to-end run: the results copied back differ from a plain step on the same inputs")
     if world > 1:
         dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_value = world * tokens_per_step * e2e_steps / (float(e2e_ms.item()) * 1e-3)
-
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    # ---- roofline of the dominant kernel -----------------------------------------------------------
-    value = world * tokens_per_step * args.steps / (ms * 1e-3)
-    dom = max(prof.items(), key=lambda kv: kv[1][1])
-    dom_name, (dom_launches, dom_ms) = dom
-    dom_avg_s = dom_ms * 1e-3 / dom_launches
-    elem = 2
-    R = case.R
-    kv_bytes = B * Hkv * N * d * elem * 2                     # K and V read once
-    alg = {   # algorithmic bytes / flops per launch of each kernel on this workload
-        "pass1": (kv_bytes, 2 * 2 * R * N * d * B * Hkv),
-        "pass2": (kv_bytes + B * Hkv * N * 4, 2 * 2 * R * N * d * B * Hkv),
-    }
-    kind = "pass2" if "pass2" in dom_name else "pass1" if "pass1" in dom_name else None
-    roof = {"kernel": dom_name, "launches": dom_launches, "avg_us": dom_avg_s * 1e6, "traffic": None}
-    if kind and dom_name.startswith("simt"):
-        peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12      # fp32 FMA lanes x 2 flop x clock
-        ach = alg[kind][1] / dom_avg_s / 1e12
-        roof.update(bound="alu", achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
-                    peak_source="148 SMs x 128 fp32 lanes x 2 flop x max SM clock")
-    elif kind:
-        t_hbm = alg[kind][0] / (peaks["hbm_gbs"] * 1e9)
-        t_mma = alg[kind][1] / (peaks["bf16_tflops_sustained"] * 1e12)
-        if t_hbm >= t_mma:
-            ach = alg[kind][0] / dom_avg_s / 1e9
-            roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
-                        peak_source=f"{peaks['source']} STREAM-style copy")
-        else:
-            ach = alg[kind][1] / dom_avg_s / 1e12
-            roof.update(bound="tensor", achieved=ach, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
-                        frac=ach / peaks["bf16_tflops_sustained"], peak_source=f"{peaks['source']} cuBLAS bf16 sustained")
-    roof["traffic"] = ncu_traffic(dom_name)
-    # the two streaming score kernels take nearly equal time; the same figures for both, whichever dominates
-    by_kernel = {}
-    for name, (n_l, ms_k) in prof.items():
-        k2 = "pass2" if "pass2" in name else "pass1" if "pass1" in name else None
-        if k2 and name.startswith("tc"):
-            avg_s = ms_k * 1e-3 / n_l
-            by_kernel[name] = {"avg_us": avg_s * 1e6, "algorithmic_bytes": alg[k2][0],
-                               "achieved_gbs": alg[k2][0] / avg_s / 1e9, "frac": alg[k2][0] / avg_s / 1e9 / peaks["hbm_gbs"]}
-    kernels = {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}
-    # The event pair around a launch also times the launch latency that back-to-back kernels hide; the
-    # kernels' own clock readings give the extent on the device, reported beside the event figure.
-    for name, span in (("tc_pass1", spans[0]), ("tc_pass2", spans[1])):
-        if name in kernels and span > 0:
-            kernels[name]["device_span_us"] = span
-            if name in by_kernel:
-                by_kernel[name]["device_span_us"] = span
-                by_kernel[name]["frac_device_span"] = by_kernel[name]["frac"] * by_kernel[name]["avg_us"] / span
-            if name == dom_name and "achieved" in roof:
-                roof["device_span_us"] = span
-                roof["frac_device_span"] = roof["frac"] * roof["avg_us"] / span
-    if by_kernel:
-        roof["score_kernels"] = by_kernel
-
-    # ---- CPU baseline: the checker as it stands, on this machine's host cores ----------------------
-    cpu = None
-    if world == 1 and not args.no_cpu:
-        from oracle import reference as ref
-        ref.build()
-        c0 = cases[0]
-        reps, t0 = 0, time.time()
-        while reps < 1 or (time.time() - t0 < 10.0 and reps < 8):
-            s = ref.score(c0.q, c0.k, c0.v, want=("VK",))["VK"].astype(np.float32)
-            ridx = ref.select_pipeline(s, c0.seq_lens, [budget], 0, run["n_recent"], run["pool_mode"],
-                                       run["pool_kernel"], budget)
-            for h in range(Hkv):
-                ref.compact(c0.k_bits[0, h], ridx[0, h], budget)
-                ref.compact(c0.v_bits[0, h], ridx[0, h], budget)
-            reps += 1
-        dt = time.time() - t0
-        cpu = {"value": tokens_per_step * reps / dt, "unit": UNIT, "cores": ref.host_threads(), "kind": "oracle",
-               "sample": f"the full workload (8 KV heads x 32768 tokens), {reps} repetitions, {dt:.1f} s"}
-
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "path": args.path,
-                       "launch": launch_mode,
-                       "ms_per_step_by_launch": {k: v / args.steps for k, v in ms_by_mode.items()},
-                       "l2": f"{N_COPIES} distinct input copies rotated between steps ({N_COPIES} x 135 MB > 126 MB L2)",
-                       "parallelism": f"{world} independent layer caches, one per GPU, no collective"},
-            "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps},
-            "gpu_launches": launches_per_step * args.steps,
-            "roofline": roof, "kernels": kernels, "cpu_baseline": cpu}
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    return {"value": world * tokens_per_step * e2e_steps / (float(e2e_ms.item()) * 1e-3), "unit": UNIT,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
 
 
-def run_other(args):
-    """The other workloads (parity-test cases, not the headline): one JSON line each with the step
-    time from CUDA events and the per-kernel event times.  Single GPU."""
+def run_decode(args):
+    """Llama-3-8B shapes, batch 32: a 16384-token context already reduced to the 4096-token budget;
+    every step appends one token, rescores all 4097 live slots (W = 1) and evicts one."""
     import numpy as np
     import torch
-    from paper_2510_07651_b200 import api, build, synth
-
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    build.build()
-    api.lib()
+    from paper_2510_07651_b200 import api, synth
+    world, rank, local, barrier = setup_gpu()
+    peaks = load_peaks()
     bf = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    steps, warmup = args.steps, max(args.warmup, 3)
+    B, Hq, Hkv, n0, budget, n_sink, n_recent = 32, 32, 8, 4096, 4096, 4, 256
+    dc = synth.make_decode(B=B, Hq=Hq, Hkv=Hkv, d=128, n0=n0, steps=64, seed=1239)
+    cap = budget + 1
+    kc = torch.zeros((B, Hkv, cap, 128), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    kc[:, :, :n0] = bf(dc.k0_bits); vc[:, :, :n0] = bf(dc.v0_bits)
+    pos = torch.full((B, Hkv, cap), -1, dtype=torch.int32, device="cuda")
+    pos[:, :, :n0] = torch.arange(n0, dtype=torch.int32, device="cuda")
+    s_acc = torch.zeros((B, Hkv, cap), dtype=torch.float32, device="cuda")
+    state = torch.zeros((B, Hkv, 4), dtype=torch.int32, device="cuda")
+    state[..., 0] = n0; state[..., 1] = n0; state[..., 2] = n0
+    qd, kd, vd = bf(dc.q_t_bits), bf(dc.k_t_bits), bf(dc.v_t_bits)
+    ns = qd.shape[0]
+    q_t = [qd[t].unsqueeze(2) for t in range(ns)]; k_t = [kd[t].unsqueeze(2) for t in range(ns)]
+    v_t = [vd[t].unsqueeze(2) for t in range(ns)]
+    p = api.decode_params(q_t[0], kc, budget=budget, n_sink=n_sink, n_recent=n_recent)
+    ws = torch.empty(api.obc_decode_workspace(p), dtype=torch.uint8, device="cuda")
+    window = 16 if args.workload == "decode-window" else 0       # scores accumulated over the last 16 steps only
+    hist = torch.zeros((B, Hkv, window, cap), dtype=torch.float32, device="cuda") if window else None
 
-    if args.workload in ("decode", "decode-window"):
-        # Llama-3-8B shapes, batch 32: a 16384-token context already reduced to the 4096-token budget;
-        # every step appends one token, rescores all 4097 live slots (W = 1) and evicts one.
-        B, Hq, Hkv, n0, budget, n_sink, n_recent = 32, 32, 8, 4096, 4096, 4, 256
-        total = warmup + steps
-        dc = synth.make_decode(B=B, Hq=Hq, Hkv=Hkv, d=128, n0=n0, steps=min(total, 64), seed=1239)
-        cap = budget + 1
-        kc = torch.zeros((B, Hkv, cap, 128), dtype=torch.bfloat16, device="cuda")
-        vc = torch.zeros_like(kc)
-        kc[:, :, :n0] = bf(dc.k0_bits); vc[:, :, :n0] = bf(dc.v0_bits)
-        pos = torch.full((B, Hkv, cap), -1, dtype=torch.int32, device="cuda")
-        pos[:, :, :n0] = torch.arange(n0, dtype=torch.int32, device="cuda")
-        s_acc = torch.zeros((B, Hkv, cap), dtype=torch.float32, device="cuda")
-        state = torch.zeros((B, Hkv, 4), dtype=torch.int32, device="cuda")
-        state[..., 0] = n0; state[..., 1] = n0; state[..., 2] = n0
-        qd, kd, vd = bf(dc.q_t_bits), bf(dc.k_t_bits), bf(dc.v_t_bits)
-        ns = qd.shape[0]
-        q_t = [qd[t].unsqueeze(2) for t in range(ns)]; k_t = [kd[t].unsqueeze(2) for t in range(ns)]
-        v_t = [vd[t].unsqueeze(2) for t in range(ns)]
-        p = api.decode_params(q_t[0], kc, budget=budget, n_sink=n_sink, n_recent=n_recent)
-        ws = torch.empty(api.obc_decode_workspace(p), dtype=torch.uint8, device="cuda")
-        window = 16 if args.workload == "decode-window" else 0       # scores accumulated over the last 16 steps only
-        hist = torch.zeros((B, Hkv, window, cap), dtype=torch.float32, device="cuda") if window else None
+    def step(t):
+        api.obc_decode_step(q_t[t % ns], k_t[t % ns], v_t[t % ns], kc, vc, s_acc, pos, state, n0 + t,
+                            budget=budget, n_sink=n_sink, n_recent=n_recent, variant="VK", workspace=ws,
+                            acc_window=window, s_hist=hist)
+    sampler = ClockSampler(local)
+    sampler.mark("timed_begin")
+    ms_round, rounds = time_rounds(step, args.steps, args.warmup, barrier)
+    sampler.mark("timed_end")
+    prof_steps = max(20, min(args.steps, 100))
+    api.obc_profile_begin()
+    for t in range(10 ** 6, 10 ** 6 + prof_steps):
+        step(t)
+    torch.cuda.synchronize()
+    prof = api.obc_profile_end()
+    clocks = sampler.stop()
+    units, live = B * Hkv, n0 + 1
+    pairs = units * live * (Hq // Hkv)
+    kv = units * live * 128 * 2 * 2
+    model = {"pass1": dict(bytes=kv, pairs=pairs, fp32_per_pair=5, ex2_per_pair=1),
+             "step": dict(bytes=units * live * 520, flops=0, pairs=pairs, fp32_per_pair=15, ex2_per_pair=2)}
+    cpu = None
+    if not args.no_cpu:
+        from oracle import reference as ref
+        v, desc, _ = cpu_decode_sample(dc, n0=n0, budget=budget, n_sink=n_sink, n_recent=n_recent, steps=8, window=window)
+        cpu = {"value": v, "unit": "steps/s", "cores": ref.host_threads(), "kind": "oracle", "sample": desc}
+    finish_line(name=args.workload, world=1, args=args, metric="decode rescoring steps/sec", unit="steps/s",
+                value=args.steps / (ms_round * 1e-3), ms_round=ms_round, rounds=rounds, prof=prof, prof_steps=prof_steps,
+                model=model, peaks=peaks, clocks=clocks, cpu=cpu, launch="plain library calls",
+                extra={"note": "the step's algorithmic bytes are the floor (K and V of every live slot once, 8 bytes of "
+                               "accumulator and position traffic per slot); the kernels read V twice"})
 
-        def step(t):
-            api.obc_decode_step(q_t[t % ns], k_t[t % ns], v_t[t % ns], kc, vc, s_acc, pos, state, n0 + t,
-                                budget=budget, n_sink=n_sink, n_recent=n_recent, variant="VK", workspace=ws,
-                                acc_window=window, s_hist=hist)
-        for t in range(warmup):
-            step(t)
-        torch.cuda.synchronize()
-        e0.record()
-        for t in range(warmup, total):
-            step(t)
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        api.obc_profile_begin()
-        for t in range(total, total + min(steps, 100)):
-            step(t)
-        torch.cuda.synchronize()
-        prof = api.obc_profile_end()
-        live_bytes = B * Hkv * (n0 + 1) * 128 * 2 * 3            # K once, V twice per step
-        line = {"metric": "decode rescoring steps/sec", "value": steps / (ms * 1e-3), "unit": "steps/s",
-                "ms_per_step": ms / steps, "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": "decode: B32 Hq32 Hkv8 d128, live 4096 -> 4097 -> 4096 per step, W1, OBCache-V&K, "
-                                       "4 sinks, 256 recent, one eviction per head per step"
-                                       + (f", accumulator = the last {window} steps' scores" if window else "")},
-                "hbm_gbs_algorithmic": live_bytes / (ms / steps * 1e-3) / 1e9,
-                "kernels": {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}}
-        print(json.dumps(line))
-        return
 
-    if args.workload == "llama32k-sharded":
-        # One rank's share of the 32k Llama layer sharded by token range over two ranks (context parallelism):
-        # this rank holds the second half of the tokens (the window's own tokens are among them).  Per step:
-        # the shard's window attention, the merge with the other rank's (o, lse) (computed once during set-up;
-        # in a real job it arrives by all-gather: B*Hq*W*(d+1) floats = 0.5 MB), the scores of the local tokens,
-        # and the selection over the whole sequence's scores (the other half filled in once during set-up).
-        case, run = synth.config(2)
+def run_sharded(args):
+    """One rank's share of the 32k Llama layer sharded by token range over two ranks (context parallelism):
+    this rank holds the second half of the tokens (the window's own tokens are among them).  Per step: the shard's
+    window attention, the merge with the other rank's (o, lse) (computed once during set-up; in a real job it arrives
+    by all-gather: B*Hq*W*(d+1) floats = 0.5 MB), the scores of the local tokens, and the selection over the whole
+    sequence's scores (the other half filled in once during set-up)."""
+    import numpy as np
+    import torch
+    from paper_2510_07651_b200 import api, synth
+    world, rank, local, barrier = setup_gpu()
+    peaks = load_peaks()
+    bf = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    n_copies = 4
+    sets = []
+    for c in range(n_copies):
+        case, run = synth.config(2, seed=1236 + c)
         q, k, v = bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)
         N, half = case.Nmax, case.Nmax // 2
         m0 = torch.full((case.B,), N, dtype=torch.int32, device="cuda")
@@ -523,149 +742,60 @@ def run_other(args):
         o_parts = torch.empty((2, case.B, case.Hq, case.W, 128), dtype=torch.float32, device="cuda")
         lse_parts = torch.empty((2, case.B, case.Hq, case.W), dtype=torch.float32, device="cuda")
         api.obc_window_attention(q, k0, v0, mask_lens=m0, o_out=o_parts[0], lse_out=lse_parts[0])
-        o_all, lse_all = torch.empty_like(o_parts[0]), torch.empty_like(lse_parts[0])
-        sp = api.score_params(q, k1, variants=["VK"], mask_lens=m1)
-        ws = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
-        scores = torch.zeros((1, case.B, case.Hkv, N), dtype=torch.float32, device="cuda")
-        loc = torch.empty((1, case.B, case.Hkv, N - half), dtype=torch.float32, device="cuda")
-        api.obc_window_attention(q, k1, v1, mask_lens=m1, o_out=o_parts[1], lse_out=lse_parts[1], workspace=ws)
-        api.obc_merge_attention(o_parts, lse_parts, o_out=o_all, lse_out=lse_all)
-        sp0 = api.score_params(q, k0, variants=["VK"], mask_lens=m0)
-        ws0 = torch.empty(api.obc_score_workspace(sp0), dtype=torch.uint8, device="cuda")
-        scores[..., :half] = api.obc_score_given(q, k0, v0, o_all, lse_all, variants=["VK"], mask_lens=m0, workspace=ws0)
-        selp = api.select_params(scores[0], budget=run["budget"], n_recent=run["n_recent"], pool=run["pool_mode"],
-                                 pool_kernel=run["pool_kernel"])
-        ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
-        idx = torch.empty((case.B, case.Hkv, run["budget"]), dtype=torch.int32, device="cuda")
-
-        def step():
+        sets.append(dict(q=q, k1=k1, v1=v1, m1=m1, o_parts=o_parts, lse_parts=lse_parts))
+        if c == 0:
+            o_all, lse_all = torch.empty_like(o_parts[0]), torch.empty_like(lse_parts[0])
+            sp = api.score_params(q, k1, variants=["VK"], mask_lens=m1)
+            ws = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
+            scores = torch.zeros((1, case.B, case.Hkv, N), dtype=torch.float32, device="cuda")
+            loc = torch.empty((1, case.B, case.Hkv, N - half), dtype=torch.float32, device="cuda")
+            selp = api.select_params(scores[0], budget=run["budget"], n_recent=run["n_recent"], pool=run["pool_mode"],
+                                     pool_kernel=run["pool_kernel"])
+            ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
+            idx = torch.empty((case.B, case.Hkv, run["budget"]), dtype=torch.int32, device="cuda")
             api.obc_window_attention(q, k1, v1, mask_lens=m1, o_out=o_parts[1], lse_out=lse_parts[1], workspace=ws)
             api.obc_merge_attention(o_parts, lse_parts, o_out=o_all, lse_out=lse_all)
-            api.obc_score_given(q, k1, v1, o_all, lse_all, variants=["VK"], mask_lens=m1, scores=loc, workspace=ws)
-            scores[..., half:].copy_(loc)                       # stands for the all-gather of the scores
-            api.obc_select(scores[0], budget=run["budget"], n_recent=run["n_recent"], pool=run["pool_mode"],
-                           pool_kernel=run["pool_kernel"], idx=idx, workspace=ws_sel)
-        for _ in range(warmup):
-            step()
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(steps):
-            step()
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        api.obc_profile_begin()
-        for _ in range(min(steps, 50)):
-            step()
-        torch.cuda.synchronize()
-        prof = api.obc_profile_end()
-        line = {"metric": METRIC, "value": N * steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps,
-                "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": "one of two ranks of the 32k Llama layer sharded by token range (this rank: tokens "
-                                       f"{half}..{N - 1}), emulated on one GPU: window attention of the shard, merge with the "
-                                       "peer's (o, lse), local scores, selection over the gathered scores; no compaction",
-                           "l2": "single input copy (K+V of the shard = 67 MB)"},
-                "kernels": {k_: {"launches": v_[0], "avg_us": 1e3 * v_[1] / v_[0]} for k_, v_ in sorted(prof.items())}}
-        print(json.dumps(line))
-        return
-
-    given = args.workload.endswith("-given")     # the caller's attention outputs instead of a recompute
-    adaptive = args.workload.endswith("-adaptive")    # head-adaptive budgets (safeguard 0.2) instead of one budget per head
-    if args.workload == "history4k":             # the whole sequence as perturbation window (W = N = 4096)
-        case, run = synth.full_history(4096)
-    else:
-        idx_cfg = {"llama32k": 2, "qwen128k": 3, "ragged": 4}[args.workload.replace("-given", "").replace("-adaptive", "")]
-        case, run = synth.config(idx_cfg)
-    q, k, v = bf(case.q_bits), bf(case.k_bits), bf(case.v_bits)
-    lens = None if (case.seq_lens == case.Nmax).all() else torch.from_numpy(case.seq_lens).cuda()
-    order = [n for n in ("V", "K", "VK") if n in run["variants"]]
-    budgets = np.asarray(run["budget"] if isinstance(run["budget"], list) else [run["budget"]] * case.B, np.int32)
-    uniform = bool((budgets == budgets[0]).all())
-    bud_d = None if uniform else torch.from_numpy(budgets).cuda()
-    stride = int(budgets.max()) * (4 if adaptive else 1)      # adaptive: a head may keep up to four average budgets
-    sp = api.score_params(q, k, seq_lens=lens, variants=order)
-    ws_score = torch.empty(api.obc_score_workspace(sp), dtype=torch.uint8, device="cuda")
-    scores = torch.empty((len(order), case.B, case.Hkv, case.Nmax), dtype=torch.float32, device="cuda")
-    selp = api.select_params(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
-                             seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"])
-    ws_sel = torch.empty(api.obc_select_workspace(selp), dtype=torch.uint8, device="cuda")
-    if adaptive:
-        n_ws = api.C.c_size_t(0)
-        api._check(api.lib().obc_select_adaptive_workspace(api.C.byref(selp), 0.2, api.C.byref(n_ws)), "obc_select_adaptive_workspace")
-        ws_sel = torch.empty(n_ws.value, dtype=torch.uint8, device="cuda")
-    counts = torch.empty((case.B, case.Hkv), dtype=torch.int32, device="cuda")
-    idx = torch.empty((case.B, case.Hkv, stride), dtype=torch.int32, device="cuda")
-    k_out = torch.empty((case.B, case.Hkv, stride, 128), dtype=torch.bfloat16, device="cuda")
-    v_out = torch.empty_like(k_out)
-
-    o_win = lse_win = None
-    if given:
-        # what the model's attention kernel would hand over for the window rows, made here (untimed set-up)
-        # with plain tensor ops: O = softmax(scale * Q K^T) V and the natural-log LSE, causal over the window
-        G, W, scale = case.G, case.W, 1.0 / np.sqrt(128.0)
-        o_win = torch.empty((case.B, case.Hq, W, 128), dtype=torch.bfloat16, device="cuda")
-        lse_win = torch.empty((case.B, case.Hq, W), dtype=torch.float32, device="cuda")
-        for b_ in range(case.B):
-            n = int(case.seq_lens[b_])
-            vis = torch.arange(n, device="cuda")[None, :] <= (n - W + torch.arange(W, device="cuda"))[:, None]
-            for g_ in range(case.Hkv):
-                qg = q[b_, g_ * G:(g_ + 1) * G].float()                          # [G, W, d]
-                z = torch.einsum("gwd,nd->gwn", qg, k[b_, g_, :n].float()) * scale
-                z = z.masked_fill(~vis[None], float("-inf"))
-                lse_win[b_, g_ * G:(g_ + 1) * G] = torch.logsumexp(z, dim=-1)
-                o_win[b_, g_ * G:(g_ + 1) * G] = (torch.softmax(z, dim=-1) @ v[b_, g_, :n].float()).to(torch.bfloat16)
-                del z
-        torch.cuda.synchronize()
-
-    def step():
-        if given:
-            api.obc_score_given(q, k, v, o_win, lse_win, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
-        else:
-            api.obc_score(q, k, v, seq_lens=lens, variants=order, scores=scores, workspace=ws_score)
-        if adaptive:
-            api.obc_select_adaptive(scores[-1], budget=int(budgets[0]), safeguard=0.2, idx_stride=stride, seq_lens=lens,
-                                    n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
-                                    idx=idx, counts=counts, workspace=ws_sel)
-        else:
-            api.obc_select(scores[-1], budget=int(budgets[0]) if uniform else 0, budgets=bud_d, idx_stride=stride,
-                           seq_lens=lens, n_recent=run["n_recent"], pool=run["pool_mode"], pool_kernel=run["pool_kernel"],
-                           idx=idx, workspace=ws_sel)
-        api.obc_compact(k, v, idx, k_out=k_out, v_out=v_out)
-    for _ in range(3):
-        step()
+            sp0 = api.score_params(q, k0, variants=["VK"], mask_lens=m0)
+            ws0 = torch.empty(api.obc_score_workspace(sp0), dtype=torch.uint8, device="cuda")
+            scores[..., :half] = api.obc_score_given(q, k0, v0, o_all, lse_all, variants=["VK"], mask_lens=m0, workspace=ws0)
     torch.cuda.synchronize()
-    graph = torch.cuda.CUDAGraph()               # the library allocates nothing and only enqueues: a step can be captured
-    with torch.cuda.graph(graph):
-        step()
 
-    def timed(run):
-        for _ in range(warmup):
-            run()
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(steps):
-            run()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1)
-    ms_by_mode = {"plain library calls": timed(step), "one captured CUDA graph per step, replayed": timed(graph.replay)}
-    launch_mode, ms = min(ms_by_mode.items(), key=lambda kv: kv[1])
+    def step(i):
+        s = sets[i % n_copies]
+        api.obc_window_attention(s["q"], s["k1"], s["v1"], mask_lens=s["m1"], o_out=s["o_parts"][1], lse_out=s["lse_parts"][1], workspace=ws)
+        api.obc_merge_attention(s["o_parts"], s["lse_parts"], o_out=o_all, lse_out=lse_all)
+        api.obc_score_given(s["q"], s["k1"], s["v1"], o_all, lse_all, variants=["VK"], mask_lens=s["m1"], scores=loc, workspace=ws)
+        scores[..., half:].copy_(loc)                       # stands for the all-gather of the scores
+        api.obc_select(scores[0], budget=run["budget"], n_recent=run["n_recent"], pool=run["pool_mode"],
+                       pool_kernel=run["pool_kernel"], idx=idx, workspace=ws_sel)
+    sampler = ClockSampler(local)
+    sampler.mark("timed_begin")
+    ms_round, rounds = time_rounds(step, args.steps, args.warmup, barrier)
+    sampler.mark("timed_end")
+    prof_steps = max(20, min(args.steps, 50))
     api.obc_profile_begin()
-    for _ in range(min(steps, 50)):
-        step()
+    for i in range(prof_steps):
+        step(i)
     torch.cuda.synchronize()
     prof = api.obc_profile_end()
-    tokens = int(case.seq_lens.sum())
-    line = {"metric": METRIC, "value": tokens * steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / steps,
-            "steps": steps, "warmup": warmup, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{case.name}: B{case.B} Hq{case.Hq} Hkv{case.Hkv} d128 Nmax{case.Nmax} W{case.W} bf16, "
-                                   f"variants {order}, pool {run['pool_mode']} {run['pool_kernel']}, tokens/step {tokens}"
-                                   + (", window O and LSE supplied by the caller (no recompute)" if given else "")
-                                   + (", head-adaptive budgets (safeguard 0.2)" if adaptive else ""),
-                       "launch": launch_mode, "ms_per_step_by_launch": {k_: v_ / steps for k_, v_ in ms_by_mode.items()},
-                       "l2": "inputs (K+V) larger than L2" if tokens * case.Hkv * 512 > 126e6 else "single input copy"},
-            "kernels": {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}}
-    print(json.dumps(line))
+    clocks = sampler.stop()
+    tok_heads = (N - half) * case.Hkv
+    pairs = sum(N - half - case.W + i + 1 for i in range(case.W)) * case.G * case.Hkv
+    kv = tok_heads * 512
+    model = {"pass1": dict(bytes=kv, flops=4 * 128 * pairs, pairs=pairs, fp32_per_pair=5, ex2_per_pair=1),
+             "pass2": dict(bytes=kv + tok_heads * 4, flops=4 * 128 * pairs, pairs=pairs, fp32_per_pair=7, ex2_per_pair=1),
+             "step": dict(bytes=2 * kv + tok_heads * 12 + N * case.Hkv * 4, flops=8 * 128 * pairs, pairs=2 * pairs, fp32_per_pair=6, ex2_per_pair=1)}
+    cpu = None
+    if not args.no_cpu:
+        from oracle import reference as ref
+        v, desc, _ = cpu_prefill_sample(case, run)
+        cpu = {"value": v, "unit": UNIT, "cores": ref.host_threads(), "kind": "oracle",
+               "sample": "the unsharded layer: " + desc}
+    finish_line(name=args.workload, world=1, args=args, metric=METRIC, unit=UNIT, value=N * args.steps / (ms_round * 1e-3),
+                ms_round=ms_round, rounds=rounds, prof=prof, prof_steps=prof_steps, model=model, peaks=peaks, clocks=clocks,
+                cpu=cpu, launch="plain library calls",
+                extra={"note": "the step's algorithmic bytes count the shard's K and V twice: with the attention merged across "
+                               "ranks between the passes, the second read cannot be saved"})
 
 
 def main():
@@ -676,9 +806,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
-    ap.add_argument("--eager", action="store_true", help="time plain library calls instead of replaying CUDA graphs")
-    ap.add_argument("--workload", default="llama32k", choices=["llama32k", "qwen128k", "ragged", "decode", "llama32k-given", "qwen128k-given", "llama32k-adaptive", "history4k", "decode-window", "llama32k-sharded"],
-                    help="llama32k is the headline benchmark; the others print a shorter line (1 GPU)")
+    ap.add_argument("--eager", action="store_true", help="time plain library calls only (no CUDA graph replay)")
+    ap.add_argument("--workload", default="llama32k", choices=WORKLOADS,
+                    help="llama32k is the headline benchmark (the only one that runs on several GPUs)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"
     if args.steps is None:
@@ -687,12 +817,14 @@ def main():
         args.warmup = 1 if ref_arm else 20
     if not ref_arm:
         args.warmup = max(args.warmup, 3)
-    if args.impl == "reference":
+    if ref_arm:
         run_reference(args)
-    elif args.workload != "llama32k":
-        run_other(args)
+    elif args.workload.startswith("decode"):
+        run_decode(args)
+    elif args.workload == "llama32k-sharded":
+        run_sharded(args)
     else:
-        run_ours(args)
+        run_prefill(args)
 
 
 if __name__ == "__main__":

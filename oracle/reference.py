@@ -113,6 +113,29 @@ def score(q, k, v, *, seq_lens=None, scale=0.0, causal=True, formulation="eq",
     return outs
 
 
+def maskout_scores(q, k, v, *, scale=0.0, causal=True):
+    """Diagnostic, not one of the paper's scores: the exact output perturbation when token p is MASKED OUT of the
+    softmax (instead of having its row zeroed, as Def. 3.1 prunes).  Removing p rescales the other weights of row r
+    by 1/(1 - A_rp), which gives the closed form  sum_r (A_rp / (1 - A_rp))^2 ||v_p - o_r||^2.
+    q [G,W,d], k, v [N,d] (one KV head) -> float64 [N].  A and O come from the checker's own attention."""
+    q = np.asarray(q, np.float32); k = np.asarray(k, np.float32); v = np.asarray(v, np.float32)
+    G, W, d = q.shape
+    N = k.shape[0]
+    att = score(q[None], k[None, None], v[None, None], scale=scale, causal=causal, want=("ATTN",), return_attention=True)
+    O, m, l = att["O"][0, 0], att["m"][0, 0], att["l"][0, 0]                     # [R,d], [R], [R]
+    sc = scale if scale > 0 else 1.0 / np.sqrt(d)
+    out = np.zeros(N)
+    for r in range(G * W):
+        i = r % W
+        last = N - W + i if causal else N - 1
+        for p in range(last + 1):
+            z = sc * float(np.dot(q[r // W, i].astype(np.float64), k[p].astype(np.float64)))
+            a = np.exp(z - m[r]) / l[r]
+            diff = v[p].astype(np.float64) - O[r]
+            out[p] += (a / (1.0 - a)) ** 2 * float(np.dot(diff, diff))
+    return out
+
+
 def pool(s, lo, hi, mode, kernel):
     """fp32 pooling of one head's scores over [lo, hi).  mode: "none" | "avg" | "max"."""
     s, sp = _f(s)

@@ -175,15 +175,61 @@ constexpr int CL_NT = 512;                    // threads per CTA
 constexpr int CL_BINS = 2048;                 // 11-bit digits
 constexpr int CL_MAX_SEG = 20 * 1024;         // candidates per CTA (two 4-byte shared arrays of this size)
 
+constexpr int CL_GATHER = 8192;               // survivors of the first pass that every CTA can hold (all CTAs' lists together)
+
 struct ClusterShared {                        // fixed part of the CTA's shared memory
     uint32_t sum[3][CL_BINS];                 // per radix pass: histogram of the whole head (every CTA adds into every copy)
     uint32_t local[CL_BINS];                  // this CTA's histogram of the current pass
     uint32_t found[2];                        // result of a pass: prefix, remaining
     uint32_t n_list;                          // candidates of this CTA that survive the first pass
     uint32_t rank_gt[16], rank_eq[16];        // kept-candidate counts of every CTA of the cluster
+    uint32_t rank_list[16], rank_above[16];   // per CTA: survivors of the first pass, candidates in higher bins
+    uint32_t before[2];                       // kept candidates (greater, equal) in the CTAs before this one
     uint32_t warp_gt[CL_NT / 32], warp_eq[CL_NT / 32];
     uint32_t scan[CL_NT / 32];
+    uint32_t gathered[CL_GATHER];             // slot r: the survivors of CTA r (CL_GATHER / C keys each)
 };
+
+// The highest bin D of hist[0 .. CL_BINS) with count(bins > D) < remaining <= count(bins >= D), found by the
+// whole CTA (thread t owns bins [4t, 4t+4)); found[0] = D, found[1] = remaining - count(bins > D).
+__device__ __forceinline__ void find_bin(const uint32_t* hist, uint32_t remaining, uint32_t* scan, uint32_t* found) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t loc[4], tot = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { loc[j] = hist[tid * 4 + j]; tot += loc[j]; }
+    uint32_t incl = tot;                           // suffix sum over the lanes >= lane
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += t;
+    }
+    if (lane == 0) scan[warp] = incl;
+    __syncthreads();
+    uint32_t wsum = lane < CL_NT / 32 ? scan[lane] : 0u;          // suffix sum over the warps > warp
+#pragma unroll
+    for (int o = 1; o < CL_NT / 32; o <<= 1) {
+        const uint32_t t = __shfl_down_sync(0xffffffffu, wsum, o);
+        if (lane + o < CL_NT / 32) wsum += t;
+    }
+    const uint32_t above_warps = __shfl_sync(0xffffffffu, wsum, min(warp + 1, 31));
+    const uint32_t above = incl - tot + (warp + 1 < CL_NT / 32 ? above_warps : 0u);
+    if (above < remaining && remaining <= above + tot) {
+        uint32_t run = above;
+#pragma unroll
+        for (int j = 3; j >= 0; --j) {
+            if (run != 0xffffffffu) {
+                if (remaining <= run + loc[j]) {
+                    found[0] = (uint32_t)(tid * 4 + j);
+                    found[1] = remaining - run;
+                    run = 0xffffffffu;
+                } else {
+                    run += loc[j];
+                }
+            }
+        }
+    }
+    __syncthreads();
+}
 
 __global__ void __launch_bounds__(CL_NT)
 select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* __restrict__ idx_all, int seg_cap,
@@ -217,8 +263,8 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     // ---- this CTA's share of the candidates: [c0, c1) of [0, n) --------------------------------
     const int seg = ((n + C - 1) / C + 31) / 32 * 32;
     const int c0 = min(rank * seg, n), c1 = min(c0 + seg, n), m = c1 - c0;
-    for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;   // sum[3][] and local[]
     if (tid == 0) sh.n_list = 0;
+    if (keys_in) for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;   // sum[3][] and local[]
 
     if (keys_in) {                                 // the caller has the (pooled) keys already: [units][Nmax]
         const uint32_t* kin = keys_in + (size_t)unit * s.Nmax + lo + c0;
@@ -235,12 +281,16 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
                 const int i = base + u * CL_NT + tid, p = lo + c0 + i - half;
                 val[u] = (i < m + 2 * half && p >= lo && p < hi) ? sc[p] : pad;
             }
+            if (base == 0)                             // the histograms are cleared while the loads travel
+                for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;   // sum[3][] and local[]
     #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int i = base + u * CL_NT + tid;
                 if (i < m + 2 * half) stage[i] = val[u];
             }
         }
+        if (m + 2 * half <= 0)                         // a CTA without candidates issued no loads above
+            for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;
         __syncthreads();
         for (int i = tid; i < m; i += CL_NT) {
             float val;
@@ -274,13 +324,18 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     cluster.sync();                                // histograms zeroed and keys written everywhere
 
     // ---- radix search for the key T of the n_hh-th largest candidate ---------------------------
-    // Pass 0 histograms the top 11 bits of all keys of the CTA; the keys that fall into the bin
-    // of the n_hh-th largest are copied to a list (in the staging buffer, free by now), and passes
-    // 1 and 2 only walk that list.  Every CTA adds its non-empty bins into the `sum` copy of every
-    // CTA of the cluster, so that after one cluster barrier each CTA finds the bin by itself.
+    // Pass 0 histograms the top 11 bits of all keys of the CTA.  Every CTA adds its non-empty bins into the `sum`
+    // copy of every CTA of the cluster, so that after one cluster barrier each CTA finds by itself the bin D that
+    // holds the n_hh-th largest key.  The keys of bin D (a few hundred of a 32k-token head) are copied to a list,
+    // and every CTA hands its list, and how many of its candidates lie in the bins above D, to all the others:
+    // after a second barrier each CTA settles the remaining 21 bits on its own copy of all the lists and knows
+    // what the CTAs before it keep, without further exchanges.  Only when the lists do not fit their slots (keys
+    // that all but coincide) do passes 1 and 2 run across the cluster as pass 0 did.
     uint32_t* list = reinterpret_cast<uint32_t*>(stage);
     uint32_t prefix = 0, mask = 0, remaining = (uint32_t)n_hh;
-    for (int ps = 0; ps < 3; ++ps) {
+    const int slot_cap = CL_GATHER / C;
+    bool gathered_path = false;
+    for (int ps = 0; ps < 3 && !gathered_path; ++ps) {
         const int shift = ps == 0 ? 21 : ps == 1 ? 10 : 0;
         const uint32_t dmask = ps == 2 ? 1023u : 2047u;
         const uint32_t* src = ps == 0 ? keys : list;
@@ -293,65 +348,84 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
         __syncthreads();
         for (int bin = tid; bin < CL_BINS; bin += CL_NT) {
             const uint32_t c = sh.local[bin];
-            if (c) {
-                for (int r = 0; r < C; ++r) atomicAdd(cluster.map_shared_rank(&sh.sum[ps][bin], r), c);
-                sh.local[bin] = 0;
-            }
+            if (c) for (int r = 0; r < C; ++r) atomicAdd(cluster.map_shared_rank(&sh.sum[ps][bin], r), c);
         }
         cluster.sync();                            // every copy of sum[ps] holds the whole head
-        {
-            // thread t owns bins [4t, 4t+4); find the highest bin D with
-            // count(bins > D) < remaining <= count(bins >= D)
-            uint32_t loc[4], tot = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) { loc[j] = sh.sum[ps][tid * 4 + j]; tot += loc[j]; }
-            uint32_t incl = tot;                   // suffix sum over the lanes >= lane
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t t = __shfl_down_sync(0xffffffffu, incl, o);
-                if (lane + o < 32) incl += t;
+        find_bin(sh.sum[ps], remaining, sh.scan, sh.found);
+        const uint32_t digit = sh.found[0];
+        remaining = sh.found[1];
+        prefix |= digit << shift; mask |= dmask << shift;
+        if (ps == 0) {
+            // survivors of the first pass -> list (any order); candidates of this CTA in the bins above D
+            uint32_t above = 0;
+            for (int bin = (int)digit + 1 + tid; bin < CL_BINS; bin += CL_NT) above += sh.local[bin];
+            for (int i = tid; i < m; i += CL_NT) {        // survivors are few: one shared-memory atomic each
+                const uint32_t key = keys[i];
+                if ((key & mask) == prefix) list[atomicAdd(&sh.n_list, 1u)] = key;
             }
-            if (lane == 0) sh.scan[warp] = incl;
-            __syncthreads();
-            uint32_t wsum = lane < CL_NT / 32 ? sh.scan[lane] : 0u;      // suffix sum over the warps > warp
+            if (tid < 2) sh.before[tid] = 0;
 #pragma unroll
-            for (int o = 1; o < CL_NT / 32; o <<= 1) {
-                const uint32_t t = __shfl_down_sync(0xffffffffu, wsum, o);
-                if (lane + o < CL_NT / 32) wsum += t;
+            for (int o = 16; o > 0; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
+            if (lane == 0) sh.scan[warp] = above;
+            __syncthreads();                       // the list and its length are complete
+            const int nl = (int)sh.n_list;
+            if (tid < C) {                         // length and higher-bin count into every CTA
+                uint32_t ab = 0;
+                for (int w = 0; w < CL_NT / 32; ++w) ab += sh.scan[w];
+                cluster.map_shared_rank(&sh.rank_list[0], tid)[rank] = (uint32_t)nl;
+                cluster.map_shared_rank(&sh.rank_above[0], tid)[rank] = ab;
             }
-            const uint32_t above_warps = __shfl_sync(0xffffffffu, wsum, min(warp + 1, 31));
-            uint32_t above = incl - tot + (warp + 1 < CL_NT / 32 ? above_warps : 0u);
-            if (above < remaining && remaining <= above + tot) {
-                uint32_t run = above;
-#pragma unroll
-                for (int j = 3; j >= 0; --j) {
-                    if (run != 0xffffffffu) {
-                        if (remaining <= run + loc[j]) {
-                            sh.found[0] = prefix | ((uint32_t)(tid * 4 + j) << shift);
-                            sh.found[1] = remaining - run;
-                            run = 0xffffffffu;
-                        } else {
-                            run += loc[j];
-                        }
+            if (nl <= slot_cap)                    // the keys themselves, into slot `rank` of every CTA (warp w serves CTA w mod C)
+                for (int r = warp % C; r < C; r += CL_NT / 32) {
+                    uint32_t* dst = cluster.map_shared_rank(&sh.gathered[0], r) + rank * slot_cap;
+                    const int step = (CL_NT / 32 >= C ? CL_NT / 32 / C : 1) * 32;
+                    for (int i = (CL_NT / 32 >= C ? warp / C : 0) * 32 + lane; i < nl; i += step) dst[i] = list[i];
+                }
+            for (int bin = tid; bin < CL_BINS; bin += CL_NT) sh.local[bin] = 0;
+            cluster.sync();                        // lists and counts have arrived everywhere
+            bool fits = true;
+            for (int r = 0; r < C; ++r) fits = fits && (int)sh.rank_list[r] <= slot_cap;   // the same answer in every CTA
+            if (fits) {
+                // ---- the remaining 21 bits, on this CTA's copy of all lists (no cluster traffic) ----
+                for (int half_pass = 0; half_pass < 2; ++half_pass) {
+                    const int sh2 = half_pass == 0 ? 10 : 0;
+                    const uint32_t dm2 = half_pass == 0 ? 2047u : 1023u;
+                    for (int r = warp % C; r < C; r += CL_NT / 32) {          // warp w reads slot w mod C
+                        const int nr = (int)sh.rank_list[r];
+                        const uint32_t* g = sh.gathered + r * slot_cap;
+                        const int step = (CL_NT / 32 >= C ? CL_NT / 32 / C : 1) * 32;
+                        for (int i = (CL_NT / 32 >= C ? warp / C : 0) * 32 + lane; i < nr; i += step)
+                            if ((g[i] & mask) == prefix) atomicAdd(&sh.local[(g[i] >> sh2) & dm2], 1u);
+                    }
+                    __syncthreads();
+                    find_bin(sh.local, remaining, sh.scan, sh.found);
+                    prefix |= sh.found[0] << sh2; mask |= dm2 << sh2; remaining = sh.found[1];
+                    if (half_pass == 0) {
+                        for (int bin = tid; bin < CL_BINS; bin += CL_NT) sh.local[bin] = 0;
+                        __syncthreads();
                     }
                 }
+                // what the CTAs before this one keep: their candidates above bin D, and of their lists the keys > T, == T
+                uint32_t bg = 0, be = 0;
+                if (tid < rank) bg = sh.rank_above[tid];
+                for (int r = warp % C; r < rank; r += CL_NT / 32) {
+                    const int nr = (int)sh.rank_list[r];
+                    const uint32_t* g = sh.gathered + r * slot_cap;
+                    const int step = (CL_NT / 32 >= C ? CL_NT / 32 / C : 1) * 32;
+                    for (int i = (CL_NT / 32 >= C ? warp / C : 0) * 32 + lane; i < nr; i += step) { bg += g[i] > prefix; be += g[i] == prefix; }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    bg += __shfl_xor_sync(0xffffffffu, bg, o);
+                    be += __shfl_xor_sync(0xffffffffu, be, o);
+                }
+                if (lane == 0 && (bg | be)) { atomicAdd(&sh.before[0], bg); atomicAdd(&sh.before[1], be); }
+                gathered_path = true;              // leaves the pass loop; the barrier below publishes `before`
             }
-            __syncthreads();
+        } else {
+            for (int bin = tid; bin < CL_BINS; bin += CL_NT) sh.local[bin] = 0;
         }
-        prefix = sh.found[0]; remaining = sh.found[1]; mask |= dmask << shift;
-        if (ps == 0) {                             // survivors of the first pass -> list (any order)
-            for (int base = 0; base < m; base += CL_NT) {
-                const int i = base + tid;
-                const uint32_t key = i < m ? keys[i] : 0u;
-                const bool pred = i < m && (key & mask) == prefix;
-                const unsigned act = __ballot_sync(0xffffffffu, pred);
-                uint32_t at = 0;
-                if (lane == 0 && act) at = atomicAdd(&sh.n_list, (uint32_t)__popc(act));
-                at = __shfl_sync(0xffffffffu, at, 0);
-                if (pred) list[at + __popc(act & ((1u << lane) - 1u))] = key;
-            }
-        }
-        __syncthreads();                           // found[] may be rewritten, the list is complete
+        __syncthreads();
     }
     const uint32_t T = prefix, k_eq = remaining;   // keep all keys > T and the first k_eq keys == T
 
@@ -370,15 +444,22 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     }
     if (lane == 0) { sh.warp_gt[warp] = cgt; sh.warp_eq[warp] = ceq; }
     __syncthreads();
-    if (tid < C) {                                 // this CTA's totals into every CTA of the cluster
-        uint32_t tg = 0, te = 0;
-        for (int w = 0; w < CL_NT / 32; ++w) { tg += sh.warp_gt[w]; te += sh.warp_eq[w]; }
-        cluster.map_shared_rank(&sh.rank_gt[0], tid)[rank] = tg;
-        cluster.map_shared_rank(&sh.rank_eq[0], tid)[rank] = te;
+    if (!gathered_path) {                          // the CTAs' totals were not derived from the lists: exchange them
+        if (tid < C) {                             // this CTA's totals into every CTA of the cluster
+            uint32_t tg = 0, te = 0;
+            for (int w = 0; w < CL_NT / 32; ++w) { tg += sh.warp_gt[w]; te += sh.warp_eq[w]; }
+            cluster.map_shared_rank(&sh.rank_gt[0], tid)[rank] = tg;
+            cluster.map_shared_rank(&sh.rank_eq[0], tid)[rank] = te;
+        }
+        cluster.sync();
+        if (tid == 0) {
+            uint32_t bg = 0, be = 0;
+            for (int r = 0; r < rank; ++r) { bg += sh.rank_gt[r]; be += sh.rank_eq[r]; }
+            sh.before[0] = bg; sh.before[1] = be;
+        }
+        __syncthreads();
     }
-    cluster.sync();
-    uint32_t gt_before = 0, eq_before = 0;
-    for (int r = 0; r < rank; ++r) { gt_before += sh.rank_gt[r]; eq_before += sh.rank_eq[r]; }
+    uint32_t gt_before = sh.before[0], eq_before = sh.before[1];
     for (int w = 0; w < warp; ++w) { gt_before += sh.warp_gt[w]; eq_before += sh.warp_eq[w]; }
     uint32_t eq_run = eq_before;
     uint32_t out = s.n_sink + gt_before + min(eq_before, k_eq);

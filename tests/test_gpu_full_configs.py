@@ -49,6 +49,8 @@ def _prefill_full(idx):
     ref_idx = ref.select_pipeline(want[order[plane]].astype(np.float32), case.seq_lens, budgets, run["n_sink"],
                                   run["n_recent"], run["pool_mode"], run["pool_kernel"], stride)
     kb, vb = k_out.view(torch.int16).cpu().numpy(), v_out.view(torch.int16).cpu().numpy()
+    worst_overlap, worst_rel_top, worst_rel_max = 1.0, 0.0, 0.0
+    gp, wp = got[plane], want[order[plane]]
     for b in range(case.B):
         nb = int(budgets[b])
         for h in range(case.Hkv):
@@ -56,6 +58,15 @@ def _prefill_full(idx):
             assert np.array_equal(vb[b, h, :nb], ref.compact(case.v_bits[b, h].view(np.int16), want_idx[b, h], nb))
             kept, kept_ref = set(gi[b, h, :nb].tolist()), set(ref_idx[b, h, :nb].tolist())
             assert len(kept & kept_ref) >= 0.97 * nb, (b, h, len(kept & kept_ref), nb)
+            worst_overlap = min(worst_overlap, len(kept & kept_ref) / nb)
+            # relative error on the tokens the double-precision scores rank in the top budget (unpooled scores)
+            n = int(case.seq_lens[b])
+            top = np.argsort(-wp[b, h, :n], kind="stable")[:nb]
+            worst_rel_top = max(worst_rel_top, float(np.max(np.abs(gp[b, h, top] - wp[b, h, top]) / wp[b, h, top])))
+            worst_rel_max = max(worst_rel_max, float(np.abs(gp[b, h, :n] - wp[b, h, :n]).max() / wp[b, h, :n].max()))
+    # reported (the bound asserted above is the tolerance; these say how far inside it the kernels are)
+    print(f"\n[{case.name}] kept-set overlap with the double-precision selection >= {worst_overlap:.4f}; "
+          f"max relative error on the checker's top-budget tokens {worst_rel_top:.2e}; max error / max score {worst_rel_max:.2e}")
 
 
 def test_config2_llama_32k_full():

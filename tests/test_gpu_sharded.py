@@ -142,3 +142,47 @@ def test_llama_32k_layer_sharded_over_two_ranks_full():
             assert np.array_equal(vb[0, h, :n], case.v_bits[0, h].view(np.int16)[rows])
             filled[0, h] += n
     assert (filled == budget).all()
+
+
+@pytest.mark.parametrize("W,Hq,Hkv,path", [(32, 8, 2, "auto"), (64, 8, 2, "tc"), (16, 4, 2, "simt")])
+def test_context_parallel_scores_with_the_library_ops(W, Hq, Hkv, path):
+    """multirank.context_parallel_scores, the function every rank of a token-sharded job runs, with the library's own
+    calls and no process group (a job of one rank: the all-gather is skipped, everything else is the code the ranks
+    execute).  Once over the whole cache, and once per shard with the other shards' attention merged in by hand,
+    against the checker's scores of the unsharded cache."""
+    from paper_2510_07651_b200 import multirank
+    N = 2100
+    case = synth.make_prefill("cp", B=2, Hq=Hq, Hkv=Hkv, d=128, W=W, N=N, dtype="bf16", seed=77 + W, hh_frac=0.02)
+    q, k, v = H.upload(case)
+    variants = ["K", "VK", "ATTN"]
+    want = H.oracle_scores(case, variants)
+    mx = max(np.abs(want[n]).max() for n in ("K", "VK"))
+    s = multirank.context_parallel_scores(q, k, v, offset=0, total_len=N, variants=variants, path=path)
+    torch.cuda.synchronize()
+    s = s.cpu().numpy()
+    for i, n in enumerate(variants):
+        H.assert_scores_close(s[i], want[n], "bf16", tight=2e-2, what=f"one rank {n} {path}", mx=None if n == "ATTN" else mx)
+
+    # two shards: each rank's call, with an `ops` object whose merge folds in the peer's attention (what the
+    # all-gather would have delivered); window attention and scoring are the library's
+    cut = 1300
+    shards = [(0, cut), (cut, N)]
+    parts = [api.obc_window_attention(q, k[:, :, lo:hi], v[:, :, lo:hi],
+                                      mask_lens=torch.full((case.B,), N - lo, dtype=torch.int32, device="cuda"), path=path)
+             for lo, hi in shards]
+
+    class Ops:
+        def __init__(self, me): self.me = me
+        obc_window_attention = staticmethod(api.obc_window_attention)
+        obc_score_given = staticmethod(api.obc_score_given)
+        def obc_merge_attention(self, o_parts, lse_parts):
+            peer = parts[1 - self.me]
+            return api.obc_merge_attention(torch.cat([o_parts, peer[0].unsqueeze(0)]), torch.cat([lse_parts, peer[1].unsqueeze(0)]))
+    got = []
+    for r, (lo, hi) in enumerate(shards):
+        got.append(multirank.context_parallel_scores(q, k[:, :, lo:hi], v[:, :, lo:hi], offset=lo, total_len=N,
+                                                     variants=variants, path=path, ops=Ops(r)))
+    torch.cuda.synchronize()
+    s2 = torch.cat(got, dim=-1).cpu().numpy()
+    for i, n in enumerate(variants):
+        H.assert_scores_close(s2[i], want[n], "bf16", tight=2e-2, what=f"two ranks {n} {path}", mx=None if n == "ATTN" else mx)

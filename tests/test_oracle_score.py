@@ -303,3 +303,32 @@ def test_l1_value_aware_score():
     G, W, N = 2, 3, k.shape[0]
     u = run_oracle(np.zeros((G, W, k.shape[1]), np.float32), k, v, want=("VATP",), causal=False)
     np.testing.assert_allclose(u["VATP"], G * W / N * np.abs(v.astype(float)).sum(-1), rtol=1e-12)
+
+
+def test_maskout_diagnostic_equals_brute_force_removal():
+    """Masking token p out of the softmax (the other reading of "pruning", kept as a diagnostic): the closed form
+    sum_r (A/(1-A))^2 ||v_p - o_r||^2 must equal the output change of an attention recomputed without p."""
+    q, k, v = tiny(seed=21, G=2, W=4, N=20, d=8)
+    scale = 1.0 / np.sqrt(8.0)
+    got = ref.maskout_scores(q, k, v)
+    G, W, _ = q.shape
+    N = k.shape[0]
+    _, _, O = window_outputs(q.astype(np.float64), k.astype(np.float64), v.astype(np.float64), scale)
+    for p in range(N):
+        keep = [j for j in range(N) if j != p]
+        # the same window positions, token p absent: row i still sees original tokens <= N - W + i
+        Z = scale * np.einsum("gwd,nd->gwn", q.astype(np.float64), k[keep].astype(np.float64))
+        vis = np.array([[j <= N - W + i for j in keep] for i in range(W)])
+        Zm = np.where(vis[None], Z, -np.inf)
+        E = np.exp(Zm - Zm.max(-1, keepdims=True))
+        O2 = (E / E.sum(-1, keepdims=True)) @ v[keep].astype(np.float64)
+        want = float(((O2 - O) ** 2).sum())
+        assert abs(got[p] - want) <= 1e-12 * max(1.0, want), (p, got[p], want)
+
+
+def test_rank_agreement_fixture_is_what_the_script_writes():
+    """tests/golden/rank_agreement.txt (reported in the results table, nothing is asserted about its values) is
+    reproducible from tests/golden/make_rank_agreement.py, which calls only the checker."""
+    from tests.golden import make_rank_agreement as mk
+    stored = open(os.path.join(GOLD, "rank_agreement.txt")).read()
+    assert mk.render(mk.compute()) == stored
