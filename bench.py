@@ -160,12 +160,13 @@ def workload_config(name, world=1):
             "parallelism": f"{world} independent layer caches, one per GPU, no collective"}
 
 
-def time_rounds(run_step, steps, warmup, barrier, min_total_s=MIN_TIMED_S, max_rounds=2000):
+def time_rounds(run_step, steps, warmup, barrier, min_total_s=None, max_rounds=2000):
     """Median over rounds of exactly `steps` steps; each round has a barrier + synchronise on both sides.
     Returns (median ms per round, number of rounds)."""
     import torch
     from paper_2510_07651_b200 import multirank
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    min_total_s = MIN_TIMED_S if min_total_s is None else min_total_s
     for i in range(warmup):
         run_step(i)
     rounds, total, it = [], 0.0, warmup
@@ -181,6 +182,7 @@ def time_rounds(run_step, steps, warmup, barrier, min_total_s=MIN_TIMED_S, max_r
         rounds.append(ms); total += ms * 1e-3
         if total >= min_total_s or len(rounds) >= max_rounds:
             break
+    time_rounds.last = {"first_round_ms": rounds[0], "fastest_round_ms": min(rounds), "slowest_round_ms": max(rounds)}
     return statistics.median(rounds), len(rounds)
 
 
@@ -246,7 +248,7 @@ def kernel_kind(name):
 
 
 def finish_line(*, name, world, args, metric, unit, value, ms_round, rounds, prof, prof_steps, model, peaks, clocks,
-                cpu, e2e=None, headline_kernel=None, spans=None, extra=None, launch=None):
+                cpu, e2e=None, headline_kernel=None, spans=None, extra=None, launch=None, timing_detail=None):
     ms_step = ms_round / args.steps
     clock = clocks.get("sm_mhz") if clocks else None
     kernels = {k: {"launches": v[0], "avg_us": 1e3 * v[1] / v[0]} for k, v in sorted(prof.items())}
@@ -275,7 +277,9 @@ def finish_line(*, name, world, args, metric, unit, value, ms_round, rounds, pro
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic", "config": workload_config(name, world),
             "timing": {"rounds": rounds, "steps_per_round": args.steps, "reported": "median round",
-                       "min_timed_s": MIN_TIMED_S, "launch": launch},
+                       "min_timed_s": MIN_TIMED_S, "launch": launch,
+                       # the first rounds run at boost clocks; under a long run the power cap lowers them (see `clocks`)
+                       "ms_per_step_of_rounds": {k: v / args.steps for k, v in (timing_detail or {}).items()}},
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": (sum(v[0] for v in prof.values()) // max(prof_steps, 1)) * args.steps,
             "roofline": roof, "kernels": kernels, "cpu_baseline": cpu}
@@ -535,9 +539,11 @@ def run_prefill(args):
     if sampler:
         sampler.mark("timed_begin")
     by_mode = {"plain library calls": time_rounds(step, args.steps, args.warmup, barrier)}
+    detail = {"plain library calls": dict(time_rounds.last)}
     if graphs:
         by_mode["one captured CUDA graph per step, replayed"] = time_rounds(lambda i: graphs[i % n_copies].replay(),
                                                                             args.steps, args.warmup, barrier)
+        detail["one captured CUDA graph per step, replayed"] = dict(time_rounds.last)
     if sampler:
         sampler.mark("timed_end")
     launch_mode, (ms_round, rounds) = min(by_mode.items(), key=lambda kv: kv[1][0])
@@ -584,7 +590,7 @@ def run_prefill(args):
     value = world * tokens_per_step * args.steps / (ms_round * 1e-3)
     finish_line(name=name, world=world, args=args, metric=METRIC, unit=UNIT, value=value, ms_round=ms_round, rounds=rounds,
                 prof=prof, prof_steps=prof_steps, model=prefill_model(case, run, given), peaks=peaks, clocks=clocks, cpu=cpu,
-                e2e=e2e, headline_kernel="tc_pass2", spans=spans, launch=launch_mode,
+                e2e=e2e, headline_kernel="tc_pass2", spans=spans, launch=launch_mode, timing_detail=detail[launch_mode],
                 extra={"ms_per_step_by_launch": {k: v[0] / args.steps for k, v in by_mode.items()}, "path": args.path})
     if world > 1:
         dist.destroy_process_group()
@@ -693,6 +699,7 @@ def run_decode(args):
     sampler = ClockSampler(local)
     sampler.mark("timed_begin")
     ms_round, rounds = time_rounds(step, args.steps, args.warmup, barrier)
+    detail = dict(time_rounds.last)
     sampler.mark("timed_end")
     prof_steps = max(20, min(args.steps, 100))
     api.obc_profile_begin()
@@ -713,7 +720,7 @@ def run_decode(args):
         cpu = {"value": v, "unit": "steps/s", "cores": ref.host_threads(), "kind": "oracle", "sample": desc}
     finish_line(name=args.workload, world=1, args=args, metric="decode rescoring steps/sec", unit="steps/s",
                 value=args.steps / (ms_round * 1e-3), ms_round=ms_round, rounds=rounds, prof=prof, prof_steps=prof_steps,
-                model=model, peaks=peaks, clocks=clocks, cpu=cpu, launch="plain library calls",
+                model=model, peaks=peaks, clocks=clocks, cpu=cpu, launch="plain library calls", timing_detail=detail,
                 extra={"note": "the step's algorithmic bytes are the floor (K and V of every live slot once, 8 bytes of "
                                "accumulator and position traffic per slot); the kernels read V twice"})
 
@@ -771,6 +778,7 @@ def run_sharded(args):
     sampler = ClockSampler(local)
     sampler.mark("timed_begin")
     ms_round, rounds = time_rounds(step, args.steps, args.warmup, barrier)
+    detail = dict(time_rounds.last)
     sampler.mark("timed_end")
     prof_steps = max(20, min(args.steps, 50))
     api.obc_profile_begin()
@@ -793,7 +801,7 @@ def run_sharded(args):
                "sample": "the unsharded layer: " + desc}
     finish_line(name=args.workload, world=1, args=args, metric=METRIC, unit=UNIT, value=N * args.steps / (ms_round * 1e-3),
                 ms_round=ms_round, rounds=rounds, prof=prof, prof_steps=prof_steps, model=model, peaks=peaks, clocks=clocks,
-                cpu=cpu, launch="plain library calls",
+                cpu=cpu, launch="plain library calls", timing_detail=detail,
                 extra={"note": "the step's algorithmic bytes count the shard's K and V twice: with the attention merged across "
                                "ranks between the passes, the second read cannot be saved"})
 
@@ -807,10 +815,15 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--eager", action="store_true", help="time plain library calls only (no CUDA graph replay)")
+    ap.add_argument("--min-timed-s", type=float, default=None,
+                    help="timed rounds are repeated until this many seconds are timed (default 0.5; 0 = one round, for profiler runs)")
     ap.add_argument("--workload", default="llama32k", choices=WORKLOADS,
                     help="llama32k is the headline benchmark (the only one that runs on several GPUs)")
     args = ap.parse_args()
     ref_arm = args.impl == "reference"
+    if args.min_timed_s is not None:
+        global MIN_TIMED_S
+        MIN_TIMED_S = max(0.0, args.min_timed_s)
     if args.steps is None:
         args.steps = 3 if ref_arm else (2000 if args.workload == "llama32k" else 200)
     if args.warmup is None:

@@ -348,30 +348,11 @@ __device__ __forceinline__ void score_rows16(const uint32_t (&zr)[16], const uin
     }
 }
 
-// one (tile, chunk) item of one token: all rows of the chunk, TMEM loads one batch ahead of the math
+// One (tile, chunk) item of one token: all rows of the chunk, one batch of 16 rows in registers at a time.  (Loading
+// the next batch ahead of the math, which doubles the registers, was slower in both kernels: the other epilogue
+// warps of the SM sub-partition cover the wait for a batch.)
 template <unsigned VARS, bool MASKED>
 __device__ __forceinline__ void score_chunk(uint32_t zt, uint32_t tt, int chunk_rows, const float4* cst,
-                                            float2 sl2, float2 sc, RowSums& S, int ptok, int mask_base, int W, int wi) {
-    uint32_t z0[16], t0[16], z1[16], t1[16];
-    tc_ld16(zt, z0);
-    tc_ld16(tt, t0);
-    for (int c0 = 0; c0 < chunk_rows; c0 += 32) {
-        tc_wait_ld16x2(z0, t0);
-        const bool second = c0 + 16 < chunk_rows;
-        if (second) { tc_ld16(zt + c0 + 16, z1); tc_ld16(tt + c0 + 16, t1); }
-        score_rows16<VARS, MASKED>(z0, t0, cst + (c0 >> 1), sl2, sc, S, ptok, mask_base, W, wi);
-        if (second) {
-            tc_wait_ld16x2(z1, t1);
-            if (c0 + 32 < chunk_rows) { tc_ld16(zt + c0 + 32, z0); tc_ld16(tt + c0 + 32, t0); }
-            score_rows16<VARS, MASKED>(z1, t1, cst + (c0 >> 1) + 8, sl2, sc, S, ptok, mask_base, W, wi);
-        }
-    }
-}
-
-// The same item with one batch of 16 rows in registers at a time (half the registers): for kernels whose SM
-// sub-partitions run four epilogue warps, where the other warps cover the wait for the next batch.
-template <unsigned VARS, bool MASKED>
-__device__ __forceinline__ void score_chunk_lean(uint32_t zt, uint32_t tt, int chunk_rows, const float4* cst,
                                                  float2 sl2, float2 sc, RowSums& S, int ptok, int mask_base, int W, int wi) {
     uint32_t z0[16], t0[16];
 #pragma unroll 1
@@ -597,9 +578,9 @@ tc_pass2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 256u + (uint32_t)r_begin, tt = zt + 128u;
             if (r_count > 0) {
                 if (masked_tile)
-                    score_chunk_lean<VARS, true>(zt, tt, r_count, cst, sl2, sc, S, ptok, Nm - p.W, p.W, r_begin % p.W);
+                    score_chunk<VARS, true>(zt, tt, r_count, cst, sl2, sc, S, ptok, Nm - p.W, p.W, r_begin % p.W);
                 else
-                    score_chunk_lean<VARS, false>(zt, tt, r_count, cst, sl2, sc, S, ptok, 0, 0, 0);
+                    score_chunk<VARS, false>(zt, tt, r_count, cst, sl2, sc, S, ptok, 0, 0, 0);
             }
             tc_fence_before();
             __syncwarp();
