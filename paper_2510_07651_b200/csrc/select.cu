@@ -236,7 +236,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
                       const uint32_t* __restrict__ keys_in) {
     extern __shared__ __align__(16) uint8_t sel_smem[];
     ClusterShared& sh = *reinterpret_cast<ClusterShared*>(sel_smem);
-    uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(ClusterShared));
+    uint32_t* keys = reinterpret_cast<uint32_t*>(sel_smem + ((sizeof(ClusterShared) + 15) & ~(size_t)15));   // 16-byte aligned
     float* stage = reinterpret_cast<float*>(keys + seg_cap);          // seg_cap + pool_kernel - 1 floats
 
     pdl_wait();
@@ -269,6 +269,8 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     if (keys_in) {                                 // the caller has the (pooled) keys already: [units][Nmax]
         const uint32_t* kin = keys_in + (size_t)unit * s.Nmax + lo + c0;
         for (int i = tid; i < m; i += CL_NT) keys[i] = kin[i];
+        __syncthreads();
+        cluster.barrier_arrive();
     } else {
         // pooled keys: stage the scores with their halo, then pool out of shared memory
         const float* sc = scores + (size_t)unit * s.Nmax;
@@ -292,6 +294,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
         if (m + 2 * half <= 0)                         // a CTA without candidates issued no loads above
             for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;
         __syncthreads();
+        cluster.barrier_arrive();                      // this CTA's histograms are clear: others may add to them after their wait
         for (int i = tid; i < m; i += CL_NT) {
             float val;
             if (half == 0) {
@@ -321,7 +324,8 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
             keys[i] = float_key(val);
         }
     }
-    cluster.sync();                                // histograms zeroed and keys written everywhere
+    // (the first cluster barrier is split: arrival above, once this CTA's histograms were clear; the wait comes just
+    // before the first remote additions, behind the pooling and the first local histogram)
 
     // ---- radix search for the key T of the n_hh-th largest candidate ---------------------------
     // Pass 0 histograms the top 11 bits of all keys of the CTA.  Every CTA adds its non-empty bins into the `sum`
@@ -346,6 +350,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
             if (pred) atomicAdd(&sh.local[(src[i] >> shift) & dmask], 1u);
         }
         __syncthreads();
+        if (ps == 0) cluster.barrier_wait();       // every CTA of the cluster runs and has cleared its histograms
         for (int bin = tid; bin < CL_BINS; bin += CL_NT) {
             const uint32_t c = sh.local[bin];
             if (c) for (int r = 0; r < C; ++r) atomicAdd(cluster.map_shared_rank(&sh.sum[ps][bin], r), c);
@@ -429,13 +434,27 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
     }
     const uint32_t T = prefix, k_eq = remaining;   // keep all keys > T and the first k_eq keys == T
 
-    // ---- ordered emission: each warp owns a contiguous run of this CTA's candidates --------------
-    const int wseg = ((m + CL_NT / 32 - 1) / (CL_NT / 32) + 31) / 32 * 32;
+    // ---- ordered emission: each warp owns a contiguous run of this CTA's candidates, in blocks of 256 keys of
+    // which a lane holds eight consecutive ones (two 16-byte reads) ------------------------------------------------
+    const int wseg = ((m + CL_NT / 32 - 1) / (CL_NT / 32) + 255) / 256 * 256;
     const int s0 = min(warp * wseg, m), s1 = min(s0 + wseg, m);
+    auto load8 = [&](int i, uint32_t (&k8)[8]) -> unsigned {           // returns the mask of keys that exist
+        if (i + 8 <= s1) {
+            const uint4 a = *reinterpret_cast<const uint4*>(keys + i), b = *reinterpret_cast<const uint4*>(keys + i + 4);
+            k8[0] = a.x; k8[1] = a.y; k8[2] = a.z; k8[3] = a.w; k8[4] = b.x; k8[5] = b.y; k8[6] = b.z; k8[7] = b.w;
+            return 0xffu;
+        }
+        unsigned have = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { const bool in = i + j < s1; k8[j] = in ? keys[i + j] : 0u; have |= (unsigned)in << j; }
+        return have;
+    };
     uint32_t cgt = 0, ceq = 0;
-    for (int i = s0 + lane; i < s1; i += 32) {
-        const uint32_t key = keys[i];
-        cgt += key > T; ceq += key == T;
+    for (int base = s0; base < s1; base += 256) {
+        uint32_t k8[8];
+        const unsigned have = load8(base + lane * 8, k8);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { cgt += ((have >> j) & 1u) && k8[j] > T; ceq += ((have >> j) & 1u) && k8[j] == T; }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -459,21 +478,31 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
         }
         __syncthreads();
     }
-    uint32_t gt_before = sh.before[0], eq_before = sh.before[1];
-    for (int w = 0; w < warp; ++w) { gt_before += sh.warp_gt[w]; eq_before += sh.warp_eq[w]; }
-    uint32_t eq_run = eq_before;
-    uint32_t out = s.n_sink + gt_before + min(eq_before, k_eq);
-    const unsigned lt_mask = (1u << lane) - 1u;
-    for (int base = s0; base < s1; base += 32) {
-        const int i = base + lane;
-        const uint32_t key = i < s1 ? keys[i] : 0u;
-        const bool is_eq = i < s1 && key == T;
-        const unsigned beq = __ballot_sync(0xffffffffu, is_eq);
-        const bool sel = i < s1 && (key > T || (is_eq && eq_run + __popc(beq & lt_mask) < k_eq));
-        const unsigned bsel = __ballot_sync(0xffffffffu, sel);
-        if (sel) idx[out + __popc(bsel & lt_mask)] = lo + c0 + i;
-        out += __popc(bsel);
-        eq_run += __popc(beq);
+    uint32_t gt_run = sh.before[0], eq_run = sh.before[1];             // kept candidates before the block at hand
+    for (int w = 0; w < warp; ++w) { gt_run += sh.warp_gt[w]; eq_run += sh.warp_eq[w]; }
+    for (int base = s0; base < s1; base += 256) {
+        uint32_t k8[8];
+        const int i = base + lane * 8;
+        const unsigned have = load8(i, k8);
+        uint32_t g = 0, e = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { g += ((have >> j) & 1u) && k8[j] > T; e += ((have >> j) & 1u) && k8[j] == T; }
+        uint32_t gi = g, ei = e;                   // inclusive scans over the lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t tg = __shfl_up_sync(0xffffffffu, gi, o), te = __shfl_up_sync(0xffffffffu, ei, o);
+            if (lane >= o) { gi += tg; ei += te; }
+        }
+        uint32_t eq_at = eq_run + ei - e;          // equal keys before this lane's first key: the first k_eq of them are kept
+        uint32_t out = s.n_sink + gt_run + (gi - g) + min(eq_at, k_eq);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (!((have >> j) & 1u)) continue;
+            if (k8[j] > T) idx[out++] = lo + c0 + i + j;
+            else if (k8[j] == T) { if (eq_at < k_eq) idx[out++] = lo + c0 + i + j; ++eq_at; }
+        }
+        gt_run += __shfl_sync(0xffffffffu, gi, 31);
+        eq_run += __shfl_sync(0xffffffffu, ei, 31);
     }
 }
 
