@@ -50,6 +50,22 @@ def test_select_ties_keep_lowest_index_and_all_equal_scores():
     assert (g[..., 777:] == -1).all()
 
 
+@pytest.mark.parametrize("N,budget", [(40000, 3000), (33000, 2048)])
+def test_select_when_the_first_radix_pass_leaves_too_many_survivors(N, budget):
+    """Scores that share their top 11 key bits (all equal; five distinct values; a narrow range with distinct low
+    bits): the survivor lists of the first pass do not fit their slots, and the cluster settles the remaining bits
+    with two more exchanged passes instead of on gathered lists."""
+    rng = np.random.default_rng(N)
+    scores = np.empty((1, 4, N), np.float32)
+    scores[0, 0] = 0.25                                                     # all equal: ties -> lowest indices
+    scores[0, 1] = (1.0 + rng.integers(0, 5, N) * 2.0 ** -20).astype(np.float32)   # five values in one bin, heavy ties
+    scores[0, 2] = (1.0 + rng.random(N) * 2.0 ** -12).astype(np.float32)    # one bin, distinct low bits
+    scores[0, 3] = (rng.random(N, dtype=np.float32) ** 8 * 1e-3)            # an ordinary head beside them
+    for pool, kern in (("none", 1), ("max", 7)):
+        got, want = _select_both(scores, [N], [budget], 4, 32, pool, kern)
+        assert np.array_equal(got.cpu().numpy(), want), (pool, kern)
+
+
 def test_select_ragged_lengths_and_per_sequence_budgets():
     rng = np.random.default_rng(1)
     lens = np.array([4096, 517, 2300], np.int32)
