@@ -995,7 +995,7 @@ struct P1Params {
     int n_splits, tiles_per_split;                         // CTAs per (unit, chunk); each writes one partial
     int l2_stream;                                         // K/V copies carry the "evict first" L2 hint
     float* part_m; float* part_l; float* part_o;           // [units][n_splits][R] (x d for part_o)
-    float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the CTAs of the last row chunk
+    float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the CTAs of the last row chunk; null: not wanted
     unsigned int* status;
     unsigned long long* span;                              // [2]: ~(earliest CTA start), latest CTA end, in globaltimer ns
 };
@@ -1055,6 +1055,23 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return r;
 }
 
+// Row chunk of a block.  Under a causal window a chunk of rows visits the tiles up to its last row's position;
+// with more CTAs than SMs the chunks that visit most tiles are handed out first.  When the chunks do not
+// straddle heads (cph chunks per head), blocks are ordered by the chunk's place within its head, last place
+// first; otherwise by chunk, last first.
+__device__ __forceinline__ void p1_chunk_of_block(const P1Params& p, int vu, int& unit, int& c) {
+    const int cph = p.W / p.chunk_rows;
+    if (p.causal && p.n_chunks > 1 && p.W % p.chunk_rows == 0 && p.G * cph == p.n_chunks) {
+        const int per_place = p.B * p.Hkv * p.G;
+        const int place = cph - 1 - vu / per_place, rest = vu % per_place;
+        unit = rest / p.G;
+        c = (rest % p.G) * cph + place;
+        return;
+    }
+    unit = vu / p.n_chunks;
+    c = p.n_chunks - 1 - vu % p.n_chunks;
+}
+
 __global__ void __launch_bounds__(kThreadsP1, 1)
 tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ P1Params p) {
@@ -1067,15 +1084,15 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     span_begin(p.span);
 
-    const int split = blockIdx.x, vu = blockIdx.y;
-    // row chunks are taken last to first: under a causal window the later chunks see more of the cache, and
-    // with more CTAs than SMs the long ones should start first
-    const int unit = vu / p.n_chunks, c = p.n_chunks - 1 - vu % p.n_chunks;
+    const int split = blockIdx.x;
+    int unit, c;
+    p1_chunk_of_block(p, blockIdx.y, unit, c);
     const int b = unit / p.Hkv, g = unit % p.Hkv;
+    const bool nv_job = p.nv != nullptr && c == p.n_chunks - 1;     // this CTA also writes ||v_p||^2 of the tiles it visits
     if (threadIdx.x == 0) {
         prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
-        // a K/V stage is released by the MMA commit and, in the CTAs of the last row chunk, by the two ||v||^2 warps
-        for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), c == p.n_chunks - 1 ? 3 : 1); }
+        // a K/V stage is released by the MMA commit and, where they are at work, by the two ||v||^2 warps
+        for (int i = 0; i < P1_NSTAGE; ++i) { mbar_init(bar(P1_FULL + i), 1); mbar_init(bar(P1_EMPTY + i), nv_job ? 3 : 1); }
         mbar_init(bar(P1_QFULL), 1); mbar_init(bar(P1_ODONE), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(bar(P1_SFULL + i), 1); mbar_init(bar(P1_PFULL + i), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1179,8 +1196,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // ============ ||v_p||^2 of every cached token (CTAs of the last row chunk) ===============
         // Pass 2 needs it per token; the V tile is in shared memory here anyway, and these two warps
         // have nothing else to do, whereas in pass 2 every issue slot next to the epilogue counts.
-        // (The last chunk holds the last window row, which sees every token, so its CTAs visit every tile.)
-        if (c == p.n_chunks - 1) {
+        // (The last chunk holds the last window row, which sees every token, so its CTAs visit every tile.  The
+        // pass-2 kernel for more than 128 window rows computes the norms itself: p.nv is null then.)
+        if (nv_job) {
             const int t64 = threadIdx.x - 64;                                // 0..63
             for (int i = 0; i < n_tiles && !failed; ++i) {
                 const uint32_t st = i % P1_NSTAGE;
@@ -1562,7 +1580,9 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.l2_stream = l2_stream ? 1 : 0;
         p1.part_m = (float*)(wsb + plan.off_part_m); p1.part_l = (float*)(wsb + plan.off_part_l);
         p1.part_o = (float*)(wsb + plan.off_part_o);
-        p1.nv = (float*)(wsb + plan.off_nv);
+        // only the single-chunk pass 2 without the l1 plane reads the norms that pass 1 leaves
+        const bool want_nv = ch.n_chunks == 1 && !attention_only && !(s.variants & OBC_VAR_VATP);
+        p1.nv = want_nv ? (float*)(wsb + plan.off_nv) : nullptr;
         p1.status = (unsigned int*)(wsb + plan.off_flag);
         p1.span = (unsigned long long*)(wsb + plan.off_flag + kSpanOffset);
         OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
