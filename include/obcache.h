@@ -279,8 +279,11 @@ obc_status obc_compact(int32_t batch, int32_t n_kv_heads, int32_t head_dim, int3
  * window are protected, one eviction per step once over budget).
  *
  * The cache of each (b, g) is a set of `capacity` slots.  pos[slot] is the token position held
- * by the slot (-1 = free); state[b,g] = {live, next_slot, hi, reserved}: live slots, the slot the
- * next token goes to, and one past the highest slot ever used.  One call:
+ * by the slot (-1 = free); state[b,g] = {live, next_slot, hi, flag}: live slots, the slot the
+ * next token goes to, one past the highest slot ever used, and a word the caller zeroes and the
+ * step raises: 1 = the step was not applied (no free slot), 2 = a device-side wait for a copy of
+ * cache rows gave up after its time limit (the step's results for that (b, g) are undefined).
+ * One call:
  *   1. writes (k_t, v_t) into next_slot with pos = step_pos and accumulator 0;
  *   2. with the newest query of each of the G heads, recomputes attention over the live slots
  *      and the chosen variant's score of every live slot (W = 1);

@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units (not part of the C ABI).
 #pragma once
 #include <cuda_runtime.h>
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <utility>
@@ -131,6 +132,12 @@ size_t tc_workspace_bytes(const ScoreShape& s);
 obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, TensorView v,
                            float* scores, void* ws, cudaStream_t stream, const GivenAttention* given = nullptr,
                            SimtPlan* attention_only = nullptr);   // non-null: stop after pass 1 + combine, return the plan
+
+// ---- tensor maps ----------------------------------------------------------------------------------
+// bf16 tensor map of rank 2 or 4 with 128-byte swizzle, innermost dimension = head_dim (128), box
+// {64, box_rows, 1, 1}; strides in bytes for dimensions 1..rank-1.  Maps are cached per host thread.
+bool make_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+              uint32_t box_rows);
 
 // ---- programmatic dependent launch ------------------------------------------------------------
 // Every kernel of the library is launched with programmatic stream serialization: its CTAs may

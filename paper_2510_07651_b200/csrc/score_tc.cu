@@ -1415,31 +1415,6 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 }
 
 // ---- host side ----------------------------------------------------------------------------------
-PFN_cuTensorMapEncodeTiled get_encode() {
-    static PFN_cuTensorMapEncodeTiled fn = nullptr;
-    if (!fn) {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (PFN_cuTensorMapEncodeTiled)ptr;
-    }
-    return fn;
-}
-
-// bf16 tensor map, rank 2 or 4, innermost dimension = head_dim (128), box {64, box_rows, 1, 1}
-bool make_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-              uint32_t box_rows) {
-    PFN_cuTensorMapEncodeTiled enc = get_encode();
-    if (!enc) return false;
-    cuuint64_t gdim[4]; cuuint64_t gstr[3]; cuuint32_t box[4] = {64, box_rows, 1, 1}; cuuint32_t estr[4] = {1, 1, 1, 1};
-    for (int i = 0; i < rank; ++i) gdim[i] = dims[i];
-    for (int i = 0; i < rank - 1; ++i) gstr[i] = strides_bytes[i];
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // Row chunks.  Pass 1 cuts the R window rows into n_chunks pieces of chunk_rows <= 128 (its MMA M
 // dimension).  Pass 2 takes the rows whole when R <= 128 and in pieces of 64 otherwise; rows_out is
 // the padded row count of the combined arrays it reads.
