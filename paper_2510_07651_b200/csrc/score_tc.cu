@@ -998,6 +998,10 @@ struct P1Params {
     float* nv;                                             // [units][Nmax]: ||v_p||^2, written by the CTAs of the last row chunk; null: not wanted
     unsigned int* status;
     unsigned long long* span;                              // [2]: ~(earliest CTA start), latest CTA end, in globaltimer ns
+    // One CTA per (unit, row chunk) and no padding rows: the CTA writes the merged results itself (what the combine
+    // kernel would make of its single partial) and no combine kernel runs.  Null out_o: partial results as above.
+    float* out_o; __nv_bfloat16* out_obf;                  // [units][R][d]: O and -2 O
+    float* out_lse2; float* out_onorm; float* out_cpair;   // [units][R]; row-pair constants as float4 per pair
 };
 
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
@@ -1364,7 +1368,13 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const float f0 = m0 == -INFINITY ? 0.f : fast_exp2(m0 - M), f1 = m1 == -INFINITY ? 0.f : fast_exp2(m1 - M);
             const uint32_t tO0 = tmem_base + lane_addr + 256u + w * 64u, tO1 = tO0 + 128u;   // this half of O_0 and O_1
             const size_t prow0 = ((size_t)unit * p.n_splits + split) * p.R + (size_t)c * p.chunk_rows;   // row 0 of the chunk
-            if (w == 0 && valid) { p.part_m[prow0 + row] = M; p.part_l[prow0 + row] = fmaf(xl[row], f0, xl[128 + row] * f1); }
+            const bool fin = p.out_o != nullptr;
+            const float Lrow = fmaf(xl[row], f0, xl[128 + row] * f1);
+            // (L = 0: the row saw no token, which only a shard of a longer sequence can show)
+            const float o_scale = fin ? (Lrow > 0.f ? 1.f / Lrow : 0.f) : 1.f;
+            const float g0 = f0 * o_scale, g1 = f1 * o_scale;
+            float sq = 0.f;                                                  // squared norm of this thread's 64 output columns
+            if (w == 0 && valid && !fin) { p.part_m[prow0 + row] = M; p.part_l[prow0 + row] = Lrow; }
 #pragma unroll 1
             for (int q = 0; q < 2; ++q) {
                 // CTA-uniform: warpgroup 0 owns tiles iff the split has any, warpgroup 1 iff it has two or more
@@ -1376,16 +1386,22 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 for (int j = 0; j < 8; ++j) {
                     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (n_tiles > 0)
-                        o = make_float4(__uint_as_float(oa[4 * j]) * f0, __uint_as_float(oa[4 * j + 1]) * f0,
-                                        __uint_as_float(oa[4 * j + 2]) * f0, __uint_as_float(oa[4 * j + 3]) * f0);
+                        o = make_float4(__uint_as_float(oa[4 * j]) * g0, __uint_as_float(oa[4 * j + 1]) * g0,
+                                        __uint_as_float(oa[4 * j + 2]) * g0, __uint_as_float(oa[4 * j + 3]) * g0);
                     if (n_tiles > 1) {
-                        o.x = fmaf(__uint_as_float(ob[4 * j]), f1, o.x);     o.y = fmaf(__uint_as_float(ob[4 * j + 1]), f1, o.y);
-                        o.z = fmaf(__uint_as_float(ob[4 * j + 2]), f1, o.z); o.w = fmaf(__uint_as_float(ob[4 * j + 3]), f1, o.w);
+                        o.x = fmaf(__uint_as_float(ob[4 * j]), g1, o.x);     o.y = fmaf(__uint_as_float(ob[4 * j + 1]), g1, o.y);
+                        o.z = fmaf(__uint_as_float(ob[4 * j + 2]), g1, o.z); o.w = fmaf(__uint_as_float(ob[4 * j + 3]), g1, o.w);
                     }
+                    sq = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, sq))));
                     const int chunk = w * 16 + q * 8 + j;
                     *reinterpret_cast<uint4*>(xo + row * 512 + ((chunk ^ (row & 31)) << 4)) =
                         make_uint4(__float_as_uint(o.x), __float_as_uint(o.y), __float_as_uint(o.z), __float_as_uint(o.w));
                 }
+            }
+            float* xs = xl + 256;                                            // [2][128]: the two halves of ||o||^2; then [128] log2-sum-exp
+            if (fin) {
+                xs[w * 128 + row] = sq;
+                if (w == 0) xs[256 + row] = M + log2f(Lrow);
             }
             asm volatile("bar.sync 2, 256;" ::: "memory");                   // the merged tile is complete
             const int row_lo = (warp - 4) * 16;                              // 8 warps x 16 rows
@@ -1395,10 +1411,33 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const int orow = row_lo + rr;
                 rowv[rr] = *reinterpret_cast<const uint4*>(xo + orow * 512 + ((lane ^ (orow & 31)) << 4));
             }
+            if (fin) {
+                // rows of the unit are rows of the outputs (one split, no padding rows): O, -2 O in bf16, and per row
+                // the log2-sum-exp, ||o||^2 and the row's half of its pair's constants
 #pragma unroll
-            for (int rr = 0; rr < 16; ++rr) {                                // one coalesced 512-byte row per instruction
-                const int orow = row_lo + rr;
-                if (orow < rows_valid) *reinterpret_cast<uint4*>(p.part_o + (prow0 + orow) * kD + lane * 4) = rowv[rr];
+                for (int rr = 0; rr < 16; ++rr) {
+                    const int orow = row_lo + rr;
+                    if (orow < rows_valid) {
+                        *reinterpret_cast<uint4*>(p.out_o + (prow0 + orow) * kD + lane * 4) = rowv[rr];
+                        const uint32_t b0 = pack_bf16x2(-2.f * __uint_as_float(rowv[rr].x), -2.f * __uint_as_float(rowv[rr].y));
+                        const uint32_t b1 = pack_bf16x2(-2.f * __uint_as_float(rowv[rr].z), -2.f * __uint_as_float(rowv[rr].w));
+                        *reinterpret_cast<uint2*>(p.out_obf + (prow0 + orow) * kD + lane * 4) = make_uint2(b0, b1);
+                    }
+                }
+                if (lane < 16 && row_lo + lane < rows_valid) {
+                    const int orow = row_lo + lane;
+                    const size_t gr = prow0 + orow;
+                    const float lse2 = xs[256 + orow], on = xs[orow] + xs[128 + orow];
+                    p.out_lse2[gr] = lse2; p.out_onorm[gr] = on;
+                    float* cp = p.out_cpair + (gr >> 1) * 4 + (gr & 1);
+                    cp[0] = -lse2; cp[2] = on;
+                }
+            } else {
+#pragma unroll
+                for (int rr = 0; rr < 16; ++rr) {                            // one coalesced 512-byte row per instruction
+                    const int orow = row_lo + rr;
+                    if (orow < rows_valid) *reinterpret_cast<uint4*>(p.part_o + (prow0 + orow) * kD + lane * 4) = rowv[rr];
+                }
             }
         }
         tc_fence_before();
@@ -1560,11 +1599,20 @@ obc_status launch_score_tc(const ScoreShape& s, TensorView q, TensorView k, Tens
         p1.nv = want_nv ? (float*)(wsb + plan.off_nv) : nullptr;
         p1.status = (unsigned int*)(wsb + plan.off_flag);
         p1.span = (unsigned long long*)(wsb + plan.off_flag + kSpanOffset);
+        // with one CTA per (unit, row chunk) and no padding rows there is nothing to merge: pass 1 writes the results itself
+        const bool direct = plan.n_splits == 1 && ch.rows_out == s.R;
+        if (direct) {
+            p1.out_o = (float*)(wsb + plan.off_o); p1.out_obf = (__nv_bfloat16*)(wsb + plan.off_obf);
+            p1.out_lse2 = (float*)(wsb + plan.off_lse2); p1.out_onorm = (float*)(wsb + plan.off_onorm);
+            p1.out_cpair = (float*)(wsb + plan.off_cpair);
+        }
         OBC_CUDA_TRY(cudaFuncSetAttribute(tc_pass1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP1));
         { ProfScope ps("tc_pass1", stream);
           OBC_CUDA_TRY(launch_pdl(tc_pass1_kernel, dim3(plan.n_splits, units * ch.n_chunks), dim3(kThreadsP1), kSmemP1, stream, 1, mq, mk, mv, p1)); }
-        obc_status st = launch_combine(s, plan, ws, stream);
-        if (st != OBC_OK) return st;
+        if (!direct) {
+            obc_status st = launch_combine(s, plan, ws, stream);
+            if (st != OBC_OK) return st;
+        }
     }
     if (attention_only) { *attention_only = plan; return OBC_OK; }      // the workspace holds the window attention
     TcParams p{};
