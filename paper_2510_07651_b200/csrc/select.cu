@@ -175,7 +175,8 @@ constexpr int CL_NT = 512;                    // threads per CTA
 constexpr int CL_BINS = 2048;                 // 11-bit digits
 constexpr int CL_MAX_SEG = 20 * 1024;         // candidates per CTA (two 4-byte shared arrays of this size)
 
-constexpr int CL_GATHER = 8192;               // survivors of the first pass that every CTA can hold (all CTAs' lists together)
+constexpr int CL_GATHER = 2 * CL_BINS;        // survivors of the first pass that every CTA can hold (all CTAs' lists together):
+                                              // they lie over the histograms of passes 1 and 2, which are used only when the lists do not fit
 
 struct ClusterShared {                        // fixed part of the CTA's shared memory
     uint32_t sum[3][CL_BINS];                 // per radix pass: histogram of the whole head (every CTA adds into every copy)
@@ -187,7 +188,8 @@ struct ClusterShared {                        // fixed part of the CTA's shared 
     uint32_t before[2];                       // kept candidates (greater, equal) in the CTAs before this one
     uint32_t warp_gt[CL_NT / 32], warp_eq[CL_NT / 32];
     uint32_t scan[CL_NT / 32];
-    uint32_t gathered[CL_GATHER];             // slot r: the survivors of CTA r (CL_GATHER / C keys each)
+    // slot r of the gathered lists: the survivors of CTA r (CL_GATHER / C keys each), in the space of sum[1] and sum[2]
+    __device__ __forceinline__ uint32_t* gathered() { return &sum[1][0]; }
 };
 
 // The highest bin D of hist[0 .. CL_BINS) with count(bins > D) < remaining <= count(bins >= D), found by the
@@ -382,7 +384,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
             }
             if (nl <= slot_cap)                    // the keys themselves, into slot `rank` of every CTA (warp w serves CTA w mod C)
                 for (int r = warp % C; r < C; r += CL_NT / 32) {
-                    uint32_t* dst = cluster.map_shared_rank(&sh.gathered[0], r) + rank * slot_cap;
+                    uint32_t* dst = cluster.map_shared_rank(sh.gathered(), r) + rank * slot_cap;
                     const int step = (CL_NT / 32 >= C ? CL_NT / 32 / C : 1) * 32;
                     for (int i = (CL_NT / 32 >= C ? warp / C : 0) * 32 + lane; i < nl; i += step) dst[i] = list[i];
                 }
@@ -397,7 +399,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
                     const uint32_t dm2 = half_pass == 0 ? 2047u : 1023u;
                     for (int r = warp % C; r < C; r += CL_NT / 32) {          // warp w reads slot w mod C
                         const int nr = (int)sh.rank_list[r];
-                        const uint32_t* g = sh.gathered + r * slot_cap;
+                        const uint32_t* g = sh.gathered() + r * slot_cap;
                         const int step = (CL_NT / 32 >= C ? CL_NT / 32 / C : 1) * 32;
                         for (int i = (CL_NT / 32 >= C ? warp / C : 0) * 32 + lane; i < nr; i += step)
                             if ((g[i] & mask) == prefix) atomicAdd(&sh.local[(g[i] >> sh2) & dm2], 1u);
@@ -415,7 +417,7 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
                 if (tid < rank) bg = sh.rank_above[tid];
                 for (int r = warp % C; r < rank; r += CL_NT / 32) {
                     const int nr = (int)sh.rank_list[r];
-                    const uint32_t* g = sh.gathered + r * slot_cap;
+                    const uint32_t* g = sh.gathered() + r * slot_cap;
                     const int step = (CL_NT / 32 >= C ? CL_NT / 32 / C : 1) * 32;
                     for (int i = (CL_NT / 32 >= C ? warp / C : 0) * 32 + lane; i < nr; i += step) { bg += g[i] > prefix; be += g[i] == prefix; }
                 }
@@ -426,6 +428,11 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
                 }
                 if (lane == 0 && (bg | be)) { atomicAdd(&sh.before[0], bg); atomicAdd(&sh.before[1], be); }
                 gathered_path = true;              // leaves the pass loop; the barrier below publishes `before`
+            } else {
+                // the exchanged passes 1 and 2 add into the histograms that the lists have overwritten: clear them
+                // everywhere before any CTA adds to another's copy
+                for (int i = tid; i < 2 * CL_BINS; i += CL_NT) sh.gathered()[i] = 0;
+                cluster.sync();
             }
         } else {
             for (int bin = tid; bin < CL_BINS; bin += CL_NT) sh.local[bin] = 0;
@@ -654,8 +661,19 @@ static obc_status launch_select_impl(const SelectShape& s, const float* scores, 
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, select_cluster_kernel, &cfg) == cudaSuccess && max_clusters > 0) {
+        // whether the device can host such a cluster depends on the cluster size and the shared memory alone: asked once
+        // per (device, size, bytes) and remembered (the query costs as much host time as the launch)
+        thread_local struct { int dev, C; size_t smem; int max_clusters; } seen[4] = {};
+        thread_local int seen_next = 0;
+        int dev = -1, max_clusters = -1;
+        (void)cudaGetDevice(&dev);
+        for (const auto& e : seen) if (e.C == C && e.smem == smem && e.dev == dev) max_clusters = e.max_clusters;
+        if (max_clusters < 0) {
+            if (cudaOccupancyMaxActiveClusters(&max_clusters, select_cluster_kernel, &cfg) != cudaSuccess) { max_clusters = 0; (void)cudaGetLastError(); }
+            seen[seen_next] = {dev, C, smem, max_clusters};
+            seen_next = (seen_next + 1) % 4;
+        }
+        if (max_clusters > 0) {
             { ProfScope ps("select_cluster", stream);
               OBC_CUDA_TRY(launch_pdl(select_cluster_kernel, dim3((unsigned)(units * C)), dim3(CL_NT), smem, stream, C, s, scores, idx, seg_cap, keys_in)); }
             return OBC_OK;
