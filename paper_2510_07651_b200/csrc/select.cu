@@ -570,6 +570,22 @@ adaptive_boost_kernel(int units, int Nmax, int n_sink, int n_safe, int safe_stri
 // per (b, h) finds its head's stretch by binary search and writes the head's row of idx: sinks, chosen
 // tokens, recent tail, -1 padding; counts[b, h] = tokens kept (or -1, with a row of -1, when the row does
 // not fit idx_stride or the budget does not fit the sequence).
+// First position of the ascending array a[0, n) whose value is >= v (n if none), found by the whole block: every
+// round the threads probe evenly spaced positions of the remaining range at once, so 16384 entries take three
+// round trips to memory where a binary search by one thread takes fourteen.  Called by all threads of the block.
+template <typename Less>
+__device__ __forceinline__ int block_lower_bound(int n, Less value_below) {
+    int lo = 0, hi = n;
+    while (hi > lo) {
+        const int step = (hi - lo + (int)blockDim.x - 1) / (int)blockDim.x;
+        const int pos = lo + (int)threadIdx.x * step;
+        const int cnt = __syncthreads_count(pos < hi && value_below(pos));   // the probes below v are a prefix
+        if (cnt == 0) { hi = lo; }
+        else { const int last = lo + (cnt - 1) * step; lo = last + 1; hi = min(last + step, hi); }
+    }
+    return lo;
+}
+
 __global__ void __launch_bounds__(256)
 adaptive_split_kernel(SelectShape s, int total, const int32_t* __restrict__ vidx_all,
                       int32_t* __restrict__ idx_all, int32_t* __restrict__ counts) {
@@ -580,9 +596,7 @@ adaptive_split_kernel(SelectShape s, int total, const int32_t* __restrict__ vidx
     const int32_t* vidx = vidx_all + (size_t)b * total;
     int32_t* idx = idx_all + (size_t)unit * s.idx_stride;
     auto lower_bound = [&](int v) {                       // first position whose virtual index is >= v
-        int a = 0, z = total;
-        while (a < z) { const int m = (a + z) >> 1; if (vidx[m] < v) a = m + 1; else z = m; }
-        return a;
+        return block_lower_bound(total, [&](int i) { return vidx[i] < v; });
     };
     const int seg0 = lower_bound(h * s.Nmax), seg1 = lower_bound((h + 1) * s.Nmax), c = seg1 - seg0;
     const int kept = s.n_sink + c + s.n_recent;
@@ -609,9 +623,7 @@ shard_indices_kernel(int idx_stride, int t0, int n, const int32_t* __restrict__ 
     const int32_t* idx = idx_all + (size_t)unit * idx_stride;
     int32_t* local = local_all + (size_t)unit * idx_stride;
     auto lower_bound = [&](int v) {                       // first entry >= v; the -1 padding counts as past every token
-        int a = 0, z = idx_stride;
-        while (a < z) { const int m = (a + z) >> 1; const int x = idx[m]; if (x >= 0 && x < v) a = m + 1; else z = m; }
-        return a;
+        return block_lower_bound(idx_stride, [&](int i) { const int x = idx[i]; return x >= 0 && x < v; });
     };
     const int seg0 = lower_bound(t0), seg1 = lower_bound(t0 + n), c = seg1 - seg0;
     for (int j = threadIdx.x; j < idx_stride; j += blockDim.x) local[j] = j < c ? idx[seg0 + j] - t0 : -1;
