@@ -882,7 +882,14 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 tc_fence_after();
                 const float4* cst = reinterpret_cast<const float4*>(sConst + cs * 128);
                 const uint32_t zt = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + buf * 128u, tt = zt + 64u;
-                if (masked_tile)
+                // a chunk whose rows lie in one head sees the whole tile as soon as its first row does (with the whole
+                // sequence as the window that is every item off the diagonal)
+                bool use_mask = masked_tile;
+                if (use_mask) {
+                    const int wfirst = (c * MC_ROWS) % p.W;
+                    if (wfirst + MC_ROWS <= p.W && t0 + TILE - 1 <= Nm - p.W + wfirst) use_mask = false;
+                }
+                if (use_mask)
                     score_chunk<VARS, true>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, Nm - p.W, p.W, (c * MC_ROWS) % p.W);
                 else
                     score_chunk<VARS, false>(zt, tt, MC_ROWS, cst, sl2, sc, S, ptok, 0, 0, 0);
@@ -1250,8 +1257,9 @@ tc_pass1_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const int t0 = (tile_lo + i) * TILE;
             if (!mbar_wait(bar(P1_SFULL + w), my_tiles & 1)) { failed = true; fail_site = __LINE__; break; }
             tc_fence_after();
-            const bool masked = t0 + TILE > first_masked;
             const int nvis = last - t0 + 1;                                  // columns j < nvis are visible
+            // (a warp whose rows all see the whole tile skips the mask: under a whole-sequence window that is every tile off the diagonal)
+            const bool masked = t0 + TILE > first_masked && __any_sync(0xffffffffu, nvis < TILE);
 
             // sweep 1: tile maximum of the row (raw logits; the scale is positive)
             float mt = -INFINITY;
