@@ -5,9 +5,8 @@
 // With G <= 8 score rows per KV head the contractions are thin (slots x heads x 128 channels) and
 // the step is bound by HBM traffic.  A CTA takes one chunk of 128 slots of one KV head: the 256-byte
 // K and V rows travel into shared memory as one tiled bulk copy per chunk (TMA, two 64-channel halves
-// with the 128-byte swizzle; per-thread 16-byte asynchronous copies where the cache's strides rule a
-// tensor map out) and the contractions run as warp-level m16n8k16 MMAs fed by ldmatrix; one thread per
-// slot does the softmax and score arithmetic, and reductions over slots use warp shuffles.
+// with the 128-byte swizzle) and the contractions run as warp-level m16n8k16 MMAs fed by ldmatrix; one
+// thread per slot does the softmax and score arithmetic, and reductions over slots use warp shuffles.
 //
 //   decode_pass1   append (k_t, v_t); logits of every live slot (kept in the workspace so K is
 //                  read once); per-chunk softmax statistics and partial outputs
@@ -16,7 +15,6 @@
 //                  the evictable slots
 //   decode_final   per (b, g): pick the slot to free, update pos / state
 #include "obc_common.cuh"
-#include <string.h>
 
 namespace obc {
 namespace {
@@ -55,30 +53,7 @@ __device__ __forceinline__ const __nv_bfloat16* bf_row(const TensorView& t, int 
     return reinterpret_cast<const __nv_bfloat16*>(t.ptr) + b * t.sb + h * t.sh + tok * t.st;
 }
 
-// The 256-byte rows [c0, c0 + CH) of one cache travel into shared memory by asynchronous 16-byte copies
-// (cp.async: no registers hold them on the way, and a CTA has its K and its V rows under way together).
-// A warp copies two whole rows per instruction, coalesced; rows at or beyond `hi` are not read and are
-// zeroed.  The 16-byte piece c of row r lands at piece c ^ (r & 15), so that the eight rows of an 8x8
-// tile fall into distinct banks when ldmatrix reads them.
-__device__ __forceinline__ void copy_rows_async(uint4* dst, const TensorView& t, int b, int g, int c0, int hi) {
-    // thread t copies piece c = t % 16 of rows t / 16, t / 16 + 8, ...: one source pointer that advances by eight
-    // rows, and a destination whose swizzle (r & 15) alternates between two values
-    const int c = threadIdx.x & 15, r0 = threadIdx.x >> 4;
-    const char* src = reinterpret_cast<const char*>(bf_row(t, b, g, c0 + r0)) + c * 16;
-    const size_t step = (size_t)t.st * 2 * (CH / 16);                  // bytes between rows CH / 16 apart
-    const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(dst);
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
-        const int r = r0 + k * (CH / 16);
-        const uint32_t d = d0 + (uint32_t)(r * 16 + (c ^ (r & 15))) * 16u;
-        if (c0 + r < hi) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + k * step) : "memory");
-        else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(d), "r"(0u) : "memory");
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-}
-template <int N> __device__ __forceinline__ void copy_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// ---- the same chunk as one tiled bulk copy ------------------------------------------------------------
+// ---- a chunk of cache rows as one tiled bulk copy ------------------------------------------------------
 // Layout in shared memory: two halves of [CH rows][128 bytes] (channels 0-63, 64-127); the 16-byte piece c of a
 // half's row r lands at piece c ^ (r & 7) (the 128-byte swizzle), so the eight rows of an 8x8 ldmatrix tile fall
 // into distinct banks.  Rows past the cache's capacity arrive as zeros; rows past the live extent hold whatever
@@ -123,9 +98,8 @@ __device__ __forceinline__ bool chunk_wait(uint64_t* bar, uint32_t parity) {
     }
 }
 // piece `piece` (0..15) of staged row `row`
-template <bool TMA>
 __device__ __forceinline__ int staged_piece(int row, int piece) {
-    return TMA ? (piece >> 3) * (CH * 8) + row * 8 + ((piece & 7) ^ (row & 7)) : row * 16 + (piece ^ (row & 15));
+    return (piece >> 3) * (CH * 8) + row * 8 + ((piece & 7) ^ (row & 7));
 }
 
 // ---- warp-level tensor-core pieces ------------------------------------------------------------------
@@ -150,12 +124,11 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
 // address of the 8x8 tile that lane `lane` names for an x4 load covering 16 staged rows from `row0` and the two
 // 16-byte pieces `piece0`, `piece0 + 1`.  rows_major: tiles ordered (rows 0-7, p0), (rows 8-15, p0), (rows 0-7, p1),
 // (rows 8-15, p1), the A operand of slots x channels; otherwise (rows 0-7, p0), (rows 0-7, p1), (rows 8-15, p0), ...
-template <bool TMA>
 __device__ __forceinline__ const uint4* tile_addr(const uint4* sRows, int row0, int piece0, int lane, bool rows_major) {
     const int mi = lane >> 3, rr = lane & 7;
     const int row = row0 + (rows_major ? (mi & 1) : (mi >> 1)) * 8 + rr;
     const int piece = piece0 + (rows_major ? (mi >> 1) : (mi & 1));
-    return sRows + staged_piece<TMA>(row, piece);
+    return sRows + staged_piece(row, piece);
 }
 // x = hi + lo with both halves bf16: two MMAs then carry an fp32 operand to about 16 bits
 __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
@@ -165,26 +138,24 @@ __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, u
     lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-// TMA: the chunks arrive as tiled bulk copies through the two tensor maps (else by per-thread asynchronous copies).
-// A bulk copy that does not complete within its time limit is reported in the unit's state word 3 (value 2).
-template <int G, bool TMA>
+// The chunks arrive as tiled bulk copies through the two tensor maps.  A bulk copy that does not complete within its
+// time limit is reported in the unit's state word 3 (value 2).
+template <int G>
 __global__ void __launch_bounds__(CH)
 decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     DecodeShape s, DecodePlan plan, TensorView q, TensorView kt, TensorView vt,
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
                     int step_pos, char* ws) {
     extern __shared__ __align__(16) uint4 sStageRaw[];                  // [CH][16]: the chunk's K rows, later its V rows
-    uint4* sStage = TMA ? reinterpret_cast<uint4*>(((uintptr_t)sStageRaw + 1023) & ~(uintptr_t)1023) : sStageRaw;
+    uint4* sStage = reinterpret_cast<uint4*>(((uintptr_t)sStageRaw + 1023) & ~(uintptr_t)1023);   // the swizzle's 1024-byte frame
     __shared__ uint64_t sBar;
-    if (TMA) {
-        // the chunk's K rows were last written four kernels back (the preceding step's new token), so they are
-        // requested before the wait on the preceding kernel
-        if (threadIdx.x == 0) {
-            chunk_bar_init(&sBar);
-            copy_chunk_tma(sStage, &map_k, &sBar, blockIdx.y / s.Hkv, blockIdx.y % s.Hkv, blockIdx.x * CH, 1);          // K is read once per step
-        }
-        __syncthreads();                                       // the barrier is initialised for every waiter
+    // the chunk's K rows were last written four kernels back (the preceding step's new token), so they are
+    // requested before the wait on the preceding kernel
+    if (threadIdx.x == 0) {
+        chunk_bar_init(&sBar);
+        copy_chunk_tma(sStage, &map_k, &sBar, blockIdx.y / s.Hkv, blockIdx.y % s.Hkv, blockIdx.x * CH, 1);              // K is read once per step
     }
+    __syncthreads();                                           // the barrier is initialised for every waiter
     pdl_wait();
     __shared__ float sP[G][CH];
     __shared__ __align__(16) float sO[NWARP][G][kD];
@@ -203,7 +174,7 @@ decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     bool copy_failed = false;
     if (c0 >= hi) {
         if (tid < G) { part_m[tid] = -INFINITY; part_l[tid] = 0.f; }
-        if (TMA && tid == 0 && !chunk_wait(&sBar, 0)) atomicMax(&state[unit * 4 + 3], 2);   // no copy may be under way when the CTA leaves
+        if (tid == 0 && !chunk_wait(&sBar, 0)) atomicMax(&state[unit * 4 + 3], 2);   // no copy may be under way when the CTA leaves
         return;
     }
     // B operand of the logits: lane (n = lane / 4, t = lane % 4) holds q_n[16 ks + 2t .. +1] and [.. + 8 .. +9]
@@ -231,18 +202,13 @@ decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     // the softmax arithmetic.  (Half the shared memory per CTA lets more CTAs of the SM overlap their round trips.)
     const uint4* sRows = sStage;
     const uint4* sVrows = sStage;
-    if (!TMA) copy_rows_async(sStage, kc, b, g, c0, hi);
     const int slot = c0 + tid;
     const bool live = slot < hi && ((valid && slot == next) || pos[(size_t)unit * s.cap + slot] >= 0);
     const bool owns_new = valid && next >= c0 && next < c0 + CH;
-    if (TMA) {
-        copy_failed = !chunk_wait(&sBar, 0);
-        // the bulk copy was asked for before the new token's row was written: put that row in place here
-        if (owns_new && tid < 16)
-            sStage[staged_piece<true>(next - c0, tid)] = reinterpret_cast<const uint4*>(bf_row(kt, b, g, 0))[tid];
-    } else {
-        copy_wait<0>();                                    // this thread's K pieces have landed
-    }
+    copy_failed = !chunk_wait(&sBar, 0);
+    // the bulk copy was asked for before the new token's row was written: put that row in place here
+    if (owns_new && tid < 16)
+        sStage[staged_piece(next - c0, tid)] = reinterpret_cast<const uint4*>(bf_row(kt, b, g, 0))[tid];
     __syncthreads();
     const float sl2 = s.scale * kLog2e;
     // logits of the warp's 32 slots: two 16-slot tiles, eight 16-channel steps each
@@ -253,7 +219,7 @@ decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             uint32_t a[4];
-            ldsm_x4(a, tile_addr<TMA>(sRows, row0, 2 * ks, lane, true));
+            ldsm_x4(a, tile_addr(sRows, row0, 2 * ks, lane, true));
             mma_bf16(acc, a, qf[ks][0], qf[ks][1]);
         }
         // acc[0], acc[1]: slot row0 + lane / 4, heads 2 (lane % 4), + 1; acc[2], acc[3]: slot + 8
@@ -261,10 +227,9 @@ decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         if (h0 < G) { sP[h0][sl] = acc[0]; sP[h0][sl + 8] = acc[2]; }
         if (h0 + 1 < G) { sP[h0 + 1][sl] = acc[1]; sP[h0 + 1][sl + 8] = acc[3]; }
     }
-    if (TMA) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // this thread's writes to the buffer precede the bulk copy into it
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // this thread's writes to the buffer precede the bulk copy into it
     __syncthreads();                                       // the K rows are no longer read
-    if (TMA) { if (tid == 0) copy_chunk_tma(sStage, &map_v, &sBar, b, g, c0, 2); }   // V is read again by the score kernel
-    else copy_rows_async(sStage, vc, b, g, c0, hi);
+    if (tid == 0) copy_chunk_tma(sStage, &map_v, &sBar, b, g, c0, 2);   // V is read again by the score kernel
     float z2[G];
 #pragma unroll
     for (int r = 0; r < G; ++r) z2[r] = sP[r][tid];        // this thread's slot; sP[.][tid] is rewritten below by this thread only
@@ -290,17 +255,13 @@ decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         sP[r][tid] = p;
         lsum[r] = warp_sum(p);
     }
-    if (TMA) {
-        copy_failed |= !chunk_wait(&sBar, 1);
-        if (owns_new && tid < 16)
-            sStage[staged_piece<true>(next - c0, tid)] = reinterpret_cast<const uint4*>(bf_row(vt, b, g, 0))[tid];
-        // rows at or beyond the live extent may hold anything, and 0 x NaN would spoil the outputs: zero them
-        if (c0 + CH > hi)
-            for (int i = tid; i < CH * 16; i += CH) if (c0 + (i >> 4) >= hi) sStage[staged_piece<true>(i >> 4, i & 15)] = make_uint4(0, 0, 0, 0);
-        if (copy_failed) atomicMax(&state[unit * 4 + 3], 2);
-    } else {
-        copy_wait<0>();                                    // this thread's V pieces have landed
-    }
+    copy_failed |= !chunk_wait(&sBar, 1);
+    if (owns_new && tid < 16)
+        sStage[staged_piece(next - c0, tid)] = reinterpret_cast<const uint4*>(bf_row(vt, b, g, 0))[tid];
+    // rows at or beyond the live extent may hold anything, and 0 x NaN would spoil the outputs: zero them
+    if (c0 + CH > hi)
+        for (int i = tid; i < CH * 16; i += CH) if (c0 + (i >> 4) >= hi) sStage[staged_piece(i >> 4, i & 15)] = make_uint4(0, 0, 0, 0);
+    if (copy_failed) atomicMax(&state[unit * 4 + 3], 2);
     __syncthreads();                                       // sRed reads done, sP complete, V rows staged
 #pragma unroll
     for (int r = 0; r < G; ++r) if (lane == 0) sRed[warp][r] = lsum[r];
@@ -324,7 +285,7 @@ decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk) {
                 uint32_t a[4];
-                ldsm_x4_trans(a, tile_addr<TMA>(sVrows, warp * 32 + kk * 16, 2 * j, lane, false));
+                ldsm_x4_trans(a, tile_addr(sVrows, warp * 32 + kk * 16, 2 * j, lane, false));
                 mma_bf16(acc, a, ph[kk][0], ph[kk][1]);
                 mma_bf16(acc, a, pl[kk][0], pl[kk][1]);
             }
@@ -422,12 +383,12 @@ decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
     }
 }
 
-template <int G, bool TMA>
+template <int G>
 __global__ void __launch_bounds__(CH)
 decode_score_kernel(const __grid_constant__ CUtensorMap map_v, DecodeShape s, DecodePlan plan, TensorView vc, float* s_acc,
                     const int32_t* pos, int32_t* state, int step_pos, char* ws) {
     extern __shared__ __align__(16) uint4 sRowsRaw[];                   // [CH][16]: the chunk's V rows
-    uint4* sRows = TMA ? reinterpret_cast<uint4*>(((uintptr_t)sRowsRaw + 1023) & ~(uintptr_t)1023) : sRowsRaw;
+    uint4* sRows = reinterpret_cast<uint4*>(((uintptr_t)sRowsRaw + 1023) & ~(uintptr_t)1023);
     __shared__ uint64_t sBar;
     __shared__ float sLse[G], sNo[G];
     __shared__ float sT[G + 1][CH];                                     // v_slot . o_r (r < G) and ||v_slot||^2
@@ -440,12 +401,8 @@ decode_score_kernel(const __grid_constant__ CUtensorMap map_v, DecodeShape s, De
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // The V rows are requested before anything else, and before the wait on the preceding kernel: the cache
     // was last written two kernels back (the new token's row), and which rows are live is sorted out below.
-    if (TMA) {
-        if (tid == 0) { chunk_bar_init(&sBar); copy_chunk_tma(sRows, &map_v, &sBar, b, g, c0, 1); }
-        __syncthreads();                                   // the barrier is initialised for every waiter
-    } else {
-        copy_rows_async(sRows, vc, b, g, c0, s.cap);
-    }
+    if (tid == 0) { chunk_bar_init(&sBar); copy_chunk_tma(sRows, &map_v, &sBar, b, g, c0, 1); }
+    __syncthreads();                                       // the barrier is initialised for every waiter
     // Likewise this slot's position, logits and accumulator, all written two kernels back or earlier: asked for
     // whether or not the slot turns out to be live, so that no later load has to wait for an earlier one.
     const int slot = c0 + tid;
@@ -464,8 +421,7 @@ decode_score_kernel(const __grid_constant__ CUtensorMap map_v, DecodeShape s, De
     if (c0 >= hi) {
         if (tid == 0) *part_min = MinCand{INFINITY, -1, -1, 0};
         // no copy may be under way when the CTA leaves
-        if (TMA) { if (tid == 0 && !chunk_wait(&sBar, 0)) atomicMax(&state[unit * 4 + 3], 2); }
-        else copy_wait<0>();
+        if (tid == 0 && !chunk_wait(&sBar, 0)) atomicMax(&state[unit * 4 + 3], 2);
         return;
     }
     if (tid < G) {
@@ -489,11 +445,10 @@ decode_score_kernel(const __grid_constant__ CUtensorMap map_v, DecodeShape s, De
             }
     }
     const int my_pos = slot < hi ? pos_in : -1;
-    if (TMA) { if (!chunk_wait(&sBar, 0)) atomicMax(&state[unit * 4 + 3], 2); }
-    else copy_wait<0>();
+    if (!chunk_wait(&sBar, 0)) atomicMax(&state[unit * 4 + 3], 2);
     __syncthreads();
     if (c0 + CH > hi) {                                    // rows beyond the live extent may hold anything: zero them
-        for (int i = tid; i < CH * 16; i += CH) if (c0 + (i >> 4) >= hi) sRows[staged_piece<TMA>(i >> 4, i & 15)] = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < CH * 16; i += CH) if (c0 + (i >> 4) >= hi) sRows[staged_piece(i >> 4, i & 15)] = make_uint4(0, 0, 0, 0);
         __syncthreads();
     }
     const bool live = my_pos >= 0;
@@ -507,7 +462,7 @@ decode_score_kernel(const __grid_constant__ CUtensorMap map_v, DecodeShape s, De
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             uint32_t a[4];
-            ldsm_x4(a, tile_addr<TMA>(sRows, row0, 2 * ks, lane, true));
+            ldsm_x4(a, tile_addr(sRows, row0, 2 * ks, lane, true));
             mma_bf16(acc, a, oh[ks][0], oh[ks][1]);
             mma_bf16(acc, a, ol[ks][0], ol[ks][1]);
             mma_bf16(n_lo, a, a[0], a[2]);                 // columns = slots row0 .. + 7
@@ -631,18 +586,18 @@ bool cache_map(CUtensorMap* map, const TensorView& t, const DecodeShape& s) {
     return make_map(map, t.ptr, 4, dims, strides, CH);
 }
 
-template <int G, bool TMA>
+template <int G>
 obc_status launch_g(const DecodeShape& s, const DecodePlan& plan, const CUtensorMap& mk, const CUtensorMap& mv,
                     TensorView q, TensorView kt, TensorView vt,
                     TensorView kc, TensorView vc, float* s_acc, int32_t* pos, int32_t* state,
                     int step_pos, char* ws, cudaStream_t stream) {
     const int units = s.B * s.Hkv;
-    const size_t stage = kStageBytes + (TMA ? 1024 : 0);                // + room to align the swizzled tile
-    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_pass1_kernel<G, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage));
-      OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G, TMA>, dim3(plan.chunks, units), dim3(CH), stage, stream, 1, mk, mv, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
+    const size_t stage = kStageBytes + 1024;                            // + room to align the swizzled tile
+    { ProfScope ps("decode_pass1", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_pass1_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage));
+      OBC_CUDA_TRY(launch_pdl(decode_pass1_kernel<G>, dim3(plan.chunks, units), dim3(CH), stage, stream, 1, mk, mv, s, plan, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, ws)); }
     { ProfScope ps("decode_combine", stream); OBC_CUDA_TRY(launch_pdl(decode_combine_kernel, dim3(units * s.G), dim3(kD), 0, stream, 1, s, plan, ws)); }
-    { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_score_kernel<G, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage));
-      OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G, TMA>, dim3(plan.chunks, units), dim3(CH), stage, stream, 1, mv, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
+    { ProfScope ps("decode_score", stream); OBC_CUDA_TRY(cudaFuncSetAttribute(decode_score_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage));
+      OBC_CUDA_TRY(launch_pdl(decode_score_kernel<G>, dim3(plan.chunks, units), dim3(CH), stage, stream, 1, mv, s, plan, vc, s_acc, pos, state, step_pos, ws)); }
     { ProfScope ps("decode_final", stream); OBC_CUDA_TRY(launch_pdl(decode_final_kernel, dim3((units + 3) / 4), dim3(128), 0, stream, 1, s, plan, pos, state, ws)); }
     return OBC_OK;
 }
@@ -656,11 +611,10 @@ obc_status launch_decode(const DecodeShape& s, TensorView q, TensorView kt, Tens
                          int step_pos, void* ws, cudaStream_t stream) {
     const DecodePlan plan = make_plan(s);
     char* w = (char*)ws;
+    // (the entry point has checked what a tensor map asks of the caches: 16-byte aligned base, strides whole 16-byte units)
     CUtensorMap mk, mv;
-    const bool tma = cache_map(&mk, kc, s) && cache_map(&mv, vc, s);
-    if (!tma) { memset(&mk, 0, sizeof(mk)); memset(&mv, 0, sizeof(mv)); }
-#define OBC_DECODE_CASE(Gv) case Gv: return tma ? launch_g<Gv, true>(s, plan, mk, mv, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, w, stream) \
-                                                : launch_g<Gv, false>(s, plan, mk, mv, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, w, stream)
+    if (!cache_map(&mk, kc, s) || !cache_map(&mv, vc, s)) { set_last_cuda_error((int)cudaErrorInvalidValue); return OBC_ERR_CUDA; }
+#define OBC_DECODE_CASE(Gv) case Gv: return launch_g<Gv>(s, plan, mk, mv, q, kt, vt, kc, vc, s_acc, pos, state, step_pos, w, stream)
     switch (s.G) {
         OBC_DECODE_CASE(1); OBC_DECODE_CASE(2); OBC_DECODE_CASE(3); OBC_DECODE_CASE(4);
         OBC_DECODE_CASE(5); OBC_DECODE_CASE(6); OBC_DECODE_CASE(7); OBC_DECODE_CASE(8);
