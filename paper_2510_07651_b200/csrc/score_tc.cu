@@ -816,30 +816,35 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
         }
     } else if (warp < 4) {
         // ==================== ||v_p||^2 per tile, per-row constants per chunk ===================
+        // At a new position the constants of the first chunk go out before the norms are computed: the epilogue needs
+        // them as soon as the first accumulators are ready, the norms only when the position's last chunk is summed.
         const int t64 = threadIdx.x - 64;                          // 0..63
         uint32_t pitem = 0, citem = 0;
         for (; !tw.done() && !failed; tw.next(), ++pitem) {
             const int unit = tw.unit;
-            for (int j = 0; j < 2 && !failed; ++j) {
-                if (!mbar_wait(bar(MC_FULL + j), pitem & 1)) { failed = true; fail_site = __LINE__; break; }
-                const uint8_t* vt = smem + MC_OFF_V + j * kOperandBytes;
-                float2* nvdst = sNv + ((pitem & 1) * 2 + j) * TILE;
+            auto norms = [&]() -> bool {
+                for (int j = 0; j < 2; ++j) {
+                    if (!mbar_wait(bar(MC_FULL + j), pitem & 1)) { fail_site = __LINE__; return false; }
+                    const uint8_t* vt = smem + MC_OFF_V + j * kOperandBytes;
+                    float2* nvdst = sNv + ((pitem & 1) * 2 + j) * TILE;
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
-                    const int tok = t64 + 64 * jj;
-                    float l2, l1;
-                    value_norms<(VARS & OBC_VAR_VATP) != 0>(vt, tok, l2, l1);
-                    nvdst[tok] = make_float2(l2, l1);
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int tok = t64 + 64 * jj;
+                        float l2, l1;
+                        value_norms<(VARS & OBC_VAR_VATP) != 0>(vt, tok, l2, l1);
+                        nvdst[tok] = make_float2(l2, l1);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(MC_EMPTY + j));
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(MC_EMPTY + j));
-            }
-            if (failed) break;
-            if (lane == 0) mbar_arrive(bar(MC_NV + (pitem & 1)));
+                if (lane == 0) mbar_arrive(bar(MC_NV + (pitem & 1)));
+                return true;
+            };
+            bool norms_done = false;
             int pair, cs;
             if (SPLIT) split_position(tw.tile, tw.tiles_in_unit, cstep, pair, cs); else { pair = tw.tile; cs = 0; }
             const int pair_first = pair * 2 * TILE, Nu = tc_mask_len(p, unit / p.Hkv);
-            for (int c = cs; c < nc; c += cstep) {
+            for (int c = cs; c < nc && !failed; c += cstep) {
                 if (may_skip && rows_last_token(c * MC_ROWS, min(c * MC_ROWS + MC_ROWS, p.R) - 1, p.W, Nu, 1) < pair_first) continue;
                 const uint32_t cs = citem & 3;
                 const size_t crow = (size_t)unit * p.rows_out + (size_t)c * MC_ROWS + t64;
@@ -854,7 +859,9 @@ tc_pass2_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_co
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(MC_CONST + cs));
                 ++citem;
+                if (!norms_done) { norms_done = true; if (!norms()) { failed = true; break; } }
             }
+            if (!failed && !norms_done && !norms()) failed = true;
         }
     } else if (warp < 12) {
         // ======================================= epilogue =======================================
