@@ -107,18 +107,22 @@ class ClockSampler:
                 "window": where}
 
 
-def ncu_traffic(kernel):
-    """DRAM bytes per launch of `kernel` from the committed ncu summary, or None when there is no
-    capture or the kernel source has changed since it was taken."""
+def ncu_traffic(workload, kernel):
+    """DRAM bytes per launch of `kernel` on `workload` from the committed ncu summaries, or None when there is
+    no capture for that pair or the kernel's source file has changed since it was taken."""
     import hashlib
     path = os.path.join(ROOT, "profiles", "traffic.txt")
     if not os.path.exists(path):
         return None
     rec = dict(l.split() for l in open(path) if l.strip() and not l.startswith("#"))
-    src = os.path.join(ROOT, "paper_2510_07651_b200", "csrc", "score_tc.cu")
-    if rec.get("source_sha256") != hashlib.sha256(open(src, "rb").read()).hexdigest():
+    key = f"{workload}.{kernel}"
+    if key not in rec:
         return None
-    return float(rec[kernel]) if kernel in rec else None
+    source = "decode.cu" if kernel.startswith("decode") else "score_tc.cu"
+    src = os.path.join(ROOT, "paper_2510_07651_b200", "csrc", source)
+    if rec.get("sha256." + source) != hashlib.sha256(open(src, "rb").read()).hexdigest():
+        return None
+    return float(rec[key])
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -270,7 +274,7 @@ def finish_line(*, name, world, args, metric, unit, value, ms_round, rounds, pro
     roof = {"kernel": dom, "launches": kernels[dom]["launches"] if dom else None, "traffic": None}
     if dom:
         roof.update(by_kernel[dom])
-        roof["traffic"] = ncu_traffic(dom)
+        roof["traffic"] = ncu_traffic(name, dom)
     roof["kernels"] = by_kernel
     roof["step"] = dict(us=ms_step * 1e3, **bounds_of(model["step"], ms_step * 1e-3, peaks, clock))
     line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
