@@ -149,14 +149,13 @@ decode_pass1_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     extern __shared__ __align__(16) uint4 sStageRaw[];                  // [CH][16]: the chunk's K rows, later its V rows
     uint4* sStage = reinterpret_cast<uint4*>(((uintptr_t)sStageRaw + 1023) & ~(uintptr_t)1023);   // the swizzle's 1024-byte frame
     __shared__ uint64_t sBar;
-    // the chunk's K rows were last written four kernels back (the preceding step's new token), so they are
-    // requested before the wait on the preceding kernel
-    if (threadIdx.x == 0) {
-        chunk_bar_init(&sBar);
-        copy_chunk_tma(sStage, &map_k, &sBar, blockIdx.y / s.Hkv, blockIdx.y % s.Hkv, blockIdx.x * CH, 1);              // K is read once per step
-    }
+    if (threadIdx.x == 0) chunk_bar_init(&sBar);
     __syncthreads();                                           // the barrier is initialised for every waiter
+    // this is the step's first kernel: the kernel before it in the stream may be the caller's and may have written the
+    // cache (the compaction that fills it, for one), so nothing is read before the wait
     pdl_wait();
+    if (threadIdx.x == 0)
+        copy_chunk_tma(sStage, &map_k, &sBar, blockIdx.y / s.Hkv, blockIdx.y % s.Hkv, blockIdx.x * CH, 1);              // K is read once per step
     __shared__ float sP[G][CH];
     __shared__ __align__(16) float sO[NWARP][G][kD];
     __shared__ float sRed[NWARP][G];
