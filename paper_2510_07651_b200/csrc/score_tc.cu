@@ -1517,7 +1517,9 @@ static int tc_chunk_split(const ScoreShape& s, const TcChunks& ch) {
     const long long pairs = (long long)s.B * s.Hkv * (((s.Nmax + TILE - 1) / TILE + 1) / 2);
     const int nc = ch.rows_out / MC_ROWS, sms = sm_count();
     if (pairs >= 2LL * sms) return 1;
-    int c = (int)((3LL * sms + pairs - 1) / pairs);
+    // about seven positions per SM: on the 4k whole-sequence window 8 CTAs per pair took 272 us, 4 took 305, 3 took 326,
+    // 12 took 270 and 16 took 282 (every position loads its tile pair again and adds a copy of the score planes)
+    int c = (int)((7LL * sms + pairs - 1) / pairs);
     if (c > 8) c = 8;
     if (c > nc) c = nc;
     return c < 1 ? 1 : c;
