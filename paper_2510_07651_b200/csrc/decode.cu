@@ -373,8 +373,12 @@ decode_combine_kernel(DecodeShape s, DecodePlan plan, char* ws) {
     ((float*)(ws + plan.off_o))[((size_t)unit * G + r) * kD + c] = oc;
     {   // the score kernel's MMA operand: o to about 16 bits as two bf16 halves
         const __nv_bfloat16 hi = __float2bfloat16_rn(oc);
-        ((__nv_bfloat16*)(ws + plan.off_ohi))[((size_t)unit * G + r) * kD + c] = hi;
-        ((__nv_bfloat16*)(ws + plan.off_olo))[((size_t)unit * G + r) * kD + c] = __float2bfloat16_rn(oc - __bfloat162float(hi));
+        // stored in the order the score kernel's MMA lanes take them: the 32-bit word w = 8 ks + 4 hf + t (channels 2w, 2w + 1;
+        // k step ks, half hf, lane-in-group t) goes to word 16 t + 2 ks + hf, so that a lane's sixteen words are four 16-byte loads
+        const int w = c >> 1, wpos = (w & 3) * 16 + (w >> 3) * 2 + ((w >> 2) & 1);
+        const size_t at = ((size_t)unit * G + r) * kD + wpos * 2 + (c & 1);
+        ((__nv_bfloat16*)(ws + plan.off_ohi))[at] = hi;
+        ((__nv_bfloat16*)(ws + plan.off_olo))[at] = __float2bfloat16_rn(oc - __bfloat162float(hi));
     }
     if (c == 0) {
         ((float*)(ws + plan.off_lse))[(size_t)unit * G + r] = M + log2f(L);
@@ -412,8 +416,8 @@ decode_score_kernel(const __grid_constant__ CUtensorMap map_v, DecodeShape s, De
 #pragma unroll
     for (int r = 0; r < G; ++r) zin[r] = in_cache ? zbuf[(size_t)r * s.cap + slot] : 0.f;
     const float acc_in = in_cache ? s_acc[(size_t)unit * s.cap + slot] : 0.f;
+    const int next = state[unit * 4 + 1], hi_old = state[unit * 4 + 2];   // written by the preceding step's last kernel
     pdl_wait();
-    const int next = state[unit * 4 + 1], hi_old = state[unit * 4 + 2];
     const bool valid = next >= 0 && next < s.cap;
     const int hi = valid ? max(hi_old, next + 1) : hi_old;
     MinCand* part_min = (MinCand*)(ws + plan.off_min) + (size_t)unit * plan.chunks + chunk;
@@ -432,16 +436,15 @@ decode_score_kernel(const __grid_constant__ CUtensorMap map_v, DecodeShape s, De
     uint32_t oh[8][2], ol[8][2];
     {
         const int n = lane >> 2, t = lane & 3;
-        const size_t row = ((size_t)unit * G + (n < G ? n : 0)) * (kD / 2);
-        const uint32_t* hrow = reinterpret_cast<const uint32_t*>(ws + plan.off_ohi) + row;
-        const uint32_t* lrow = reinterpret_cast<const uint32_t*>(ws + plan.off_olo) + row;
+        const size_t row = ((size_t)unit * G + (n < G ? n : 0)) * (kD / 2) + t * 16;   // the lane's sixteen words, in (ks, hf) order
+        const uint4* hrow = reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(ws + plan.off_ohi) + row);
+        const uint4* lrow = reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(ws + plan.off_olo) + row);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                oh[ks][hf] = n < G ? hrow[ks * 8 + hf * 4 + t] : 0u;
-                ol[ks][hf] = n < G ? lrow[ks * 8 + hf * 4 + t] : 0u;
-            }
+        for (int q4 = 0; q4 < 4; ++q4) {
+            const uint4 h4 = n < G ? hrow[q4] : make_uint4(0, 0, 0, 0), l4 = n < G ? lrow[q4] : make_uint4(0, 0, 0, 0);
+            oh[2 * q4][0] = h4.x; oh[2 * q4][1] = h4.y; oh[2 * q4 + 1][0] = h4.z; oh[2 * q4 + 1][1] = h4.w;
+            ol[2 * q4][0] = l4.x; ol[2 * q4][1] = l4.y; ol[2 * q4 + 1][0] = l4.z; ol[2 * q4 + 1][1] = l4.w;
+        }
     }
     const int my_pos = slot < hi ? pos_in : -1;
     if (!chunk_wait(&sBar, 0)) atomicMax(&state[unit * 4 + 3], 2);
