@@ -278,17 +278,19 @@ select_cluster_kernel(SelectShape s, const float* __restrict__ scores, int32_t* 
         const float* sc = scores + (size_t)unit * s.Nmax;
         const int half = (s.pool_mode == OBC_POOL_NONE) ? 0 : s.pool_kernel / 2;
         const float pad = s.pool_mode == OBC_POOL_MAX ? -INFINITY : 0.f;
-        for (int base = 0; base < m + 2 * half; base += 8 * CL_NT) {      // eight loads in flight per thread
-            float val[8];
+        // nine loads in flight per thread: a share of 4096 candidates and its halo travel in one round trip
+        constexpr int LD = 9;
+        for (int base = 0; base < m + 2 * half; base += LD * CL_NT) {
+            float val[LD];
     #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < LD; ++u) {
                 const int i = base + u * CL_NT + tid, p = lo + c0 + i - half;
                 val[u] = (i < m + 2 * half && p >= lo && p < hi) ? sc[p] : pad;
             }
             if (base == 0)                             // the histograms are cleared while the loads travel
                 for (int i = tid; i < 4 * CL_BINS; i += CL_NT) (&sh.sum[0][0])[i] = 0;   // sum[3][] and local[]
     #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < LD; ++u) {
                 const int i = base + u * CL_NT + tid;
                 if (i < m + 2 * half) stage[i] = val[u];
             }
