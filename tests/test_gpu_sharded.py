@@ -60,6 +60,34 @@ def test_token_sharded_cache_scores_like_the_whole(N, W, Hq, Hkv, dtype, path, c
     assert np.abs(o_all.cpu().numpy() - o_ref).max() <= tol * max(1.0, np.abs(o_ref).max())
 
 
+def test_window_attention_with_one_cta_per_row_chunk():
+    """2560 window rows per KV head in 20 chunks: pass 1 has one CTA per (unit, chunk), writes the merged results
+    itself and no merge kernel runs; in the second shard the early rows see no token at all (their output is 0 and
+    their log-sum-exp -inf, which the merge of the shards must weigh as nothing)."""
+    N, W, Hq, Hkv = 1024, 640, 32, 8
+    case = synth.make_prefill("direct", B=1, Hq=Hq, Hkv=Hkv, d=128, W=W, N=N, dtype="bf16", seed=77, hh_frac=0.02)
+    q, k, v = H.upload(case)
+    shards = [(0, 700), (700, N)]
+    parts = [api.obc_window_attention(q, k[:, :, lo:hi], v[:, :, lo:hi],
+                                      mask_lens=torch.full((1,), N - lo, dtype=torch.int32, device="cuda"), path="tc")
+             for lo, hi in shards]
+    lse1 = parts[1][1].cpu().numpy()
+    assert np.isneginf(lse1[0, :, : 700 - (N - W)]).all() and np.isfinite(lse1[0, :, 700 - (N - W):]).all()
+    o_all, lse_all = api.obc_merge_attention(torch.stack([p[0] for p in parts]), torch.stack([p[1] for p in parts]))
+    torch.cuda.synchronize()
+    from oracle import reference as ref
+    att = ref.score(case.q, case.k, case.v, want=("ATTN",), return_attention=True)
+    o_ref = att["O"].reshape(1, Hq, W, 128)
+    lse_ref = (att["m"] + np.log(att["l"])).reshape(1, Hq, W)
+    assert np.abs(lse_all.cpu().numpy() - lse_ref).max() <= 2e-2
+    assert np.abs(o_all.cpu().numpy() - o_ref).max() <= 2e-2 * max(1.0, np.abs(o_ref).max())
+    # the unsharded call takes the same path
+    o_one, lse_one = api.obc_window_attention(q, k, v, path="tc")
+    torch.cuda.synchronize()
+    assert np.abs(lse_one.cpu().numpy() - lse_ref).max() <= 2e-2
+    assert np.abs(o_one.cpu().numpy() - o_ref).max() <= 2e-2 * max(1.0, np.abs(o_ref).max())
+
+
 def test_merge_attention_weights_and_empty_shards():
     """lse = log sum exp(lse_s), o = sum exp(lse_s - lse) o_s; a shard that saw nothing (lse = -inf) weighs 0."""
     g = torch.Generator(device="cpu").manual_seed(3)
