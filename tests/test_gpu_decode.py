@@ -13,12 +13,19 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", seed=55, s_acc0=False, window=0):
+def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", seed=55, s_acc0=False, window=0,
+         strided=False):
     G = Hq // Hkv
     dc = synth.make_decode(B=B, Hq=Hq, Hkv=Hkv, d=128, n0=n0, steps=steps, seed=seed)
     dev = "cuda"
-    kc = torch.zeros((B, Hkv, cap, 128), dtype=torch.bfloat16, device=dev)
-    vc = torch.zeros_like(kc)
+    if strided:      # caches that are views of larger allocations: rows 272 bytes apart, spare slots after every head, NaN between
+        kbig = torch.full((B, Hkv + 1, cap + 5, 136), float("nan"), dtype=torch.bfloat16, device=dev)
+        vbig = torch.full((B, Hkv + 1, cap + 5, 136), float("nan"), dtype=torch.bfloat16, device=dev)
+        kc, vc = kbig[:, :Hkv, :cap, :128], vbig[:, :Hkv, :cap, :128]
+        kc.zero_(); vc.zero_()
+    else:
+        kc = torch.zeros((B, Hkv, cap, 128), dtype=torch.bfloat16, device=dev)
+        vc = torch.zeros_like(kc)
     kc[:, :, :n0] = H.dev_bf16(dc.k0_bits)
     vc[:, :, :n0] = H.dev_bf16(dc.v0_bits)
     pos = torch.full((B, Hkv, cap), -1, dtype=torch.int32, device=dev)
@@ -58,7 +65,10 @@ def _run(B, Hq, Hkv, n0, budget, cap, n_sink, n_recent, steps, variant="VK", see
                 assert np.array_equal(g_pos[b, h], st.pos), f"step {t} unit {b},{h}"
                 assert tuple(g_state[b, h][:3]) == (st.live, st.next_slot, st.hi)
                 assert g_state[b, h][3] == 0
-    kb, vb = kc.view(torch.int16).cpu().numpy(), vc.view(torch.int16).cpu().numpy()
+    kb, vb = kc.contiguous().view(torch.int16).cpu().numpy(), vc.contiguous().view(torch.int16).cpu().numpy()
+    if strided:      # nothing outside the views was written
+        assert torch.isnan(kbig[:, Hkv]).all() and torch.isnan(kbig[:, :, cap:]).all() and torch.isnan(kbig[..., 128:]).all()
+        assert torch.isnan(vbig[:, Hkv]).all() and torch.isnan(vbig[:, :, cap:]).all() and torch.isnan(vbig[..., 128:]).all()
     for b in range(B):
         for h in range(Hkv):
             st = sts[b][h]
@@ -96,3 +106,10 @@ def test_decode_accumulation_window(window):
     chunks, a window shorter and longer than a token's usual stay beyond the protected recents."""
     ev = _run(B=2, Hq=8, Hkv=2, n0=280, budget=290, cap=291, n_sink=4, n_recent=12, steps=40, window=window)
     assert ev == 2 * 2 * 30
+
+
+def test_decode_caches_that_are_views_of_larger_buffers():
+    """Strided caches (the tensor maps of the bulk copies carry the strides); capacity not a multiple of the chunk, so the
+    last chunk's rows beyond it must read as zeros although the memory behind them holds NaN."""
+    assert _run(B=2, Hq=8, Hkv=2, n0=300, budget=280, cap=333, n_sink=4, n_recent=8, steps=6, strided=True) > 0
+
